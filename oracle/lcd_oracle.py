@@ -1,0 +1,370 @@
+"""CPU oracle for the LUT-based inference matmul of the LCD paper (Section 4,
+"Inference with Table Lookup").
+
+TEST INFRASTRUCTURE ONLY.  Plain, slow, double-precision numpy written from the paper;
+it shares no code with the CUDA path and must never be imported by the product package.
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may call it.
+
+What is implemented, and which passage each part follows:
+
+* ``smooth_quantize``      Section 4.1 "Input Transformation Stage", both equations:
+                           smoothing and uniform symmetric quantisation fused into a single
+                           multiply, round to nearest, clip.  (An *encoding*: taken step by
+                           step in a fixed binary32 operation order, see the function.)
+* ``lut_linear_dequant``   the plain definition the method reaches exactly: dequantise the
+                           clustered weights and the quantised activations and multiply
+                           (Section 4.2: the looked-up values are "pre-computed" products
+                           that are then summed; no dequantisation pass changes the value).
+* ``lut_linear_product``   Section 4.2 first paragraph: a table of pre-computed
+                           (activation level x weight centroid) products, read by index pair
+                           and accumulated.
+* ``lut_linear_signfold``  Section 4.2 third paragraph, last sentence: only non-negative
+                           activation levels are stored, the sign is applied when accumulating.
+* ``lut_linear_bucket``    Section 4.2 third paragraph: centroid-stationary buckets - per
+                           weight centroid, gather what belongs to it, then combine with the
+                           centroid values.
+* ``pack_weights`` / ``unpack_weights``  Section 4.2 last paragraph (fewer than 16
+                           centroids => low-bit index representation); the byte layout is this
+                           library's own and is specified in the function docstrings.
+
+Parity pins (tests/test_oracle_pins.py): the four linear forms agree with each other and
+with a brute-force triple loop, with a float64 library matmul on the dequantised matrix,
+with closed forms for one-centroid and affine codebooks and with exhaustive enumeration on
+tiny inputs.  The paper prints no numeric example of this path, so the quantiser's tie rule
+(half to even) and the absmax/7 scale are pinned by invariants only (sign symmetry,
+power-of-two scale invariance, monotonicity, exact ties): "parity unpinned" against paper
+values for those two choices of ``smooth_quantize``.
+"""
+from __future__ import annotations
+
+import struct
+import numpy as np
+
+QMIN, QMAX = -8, 7            # 4-bit symmetric range [-2^(b-1), 2^(b-1)-1], b = 4
+LEVELS = 16
+MAGIC = 0x5744434C            # "LCDW"
+VERSION = 1
+LAYOUT_TILE8X256 = 1
+HEADER_BYTES = 64
+INDEX_OFFSET = 256
+TILE_ROWS = 8
+TILE_K = 256
+KBLOCK = 128
+
+
+def _f32(v):
+    """Round a float64 array to binary32 and return it as float64 (one IEEE rounding)."""
+    return np.asarray(v, dtype=np.float64).astype(np.float32).astype(np.float64)
+
+
+def round_up(v: int, m: int) -> int:
+    return (v + m - 1) // m * m
+
+
+# --------------------------------------------------------------------------------------
+# Section 4.1 - input transformation
+# --------------------------------------------------------------------------------------
+def smooth_quantize(x_fp16: np.ndarray, inv_s: np.ndarray | None, static_scale: float | None = None):
+    """Activation index assignment, Section 4.1.
+
+    q = Clip(round(X / (s_m * s_q))): the smoothing divide and the quantisation divide are one
+    multiply.  Per token m (dynamic mode, static_scale is None):
+        t_k = fl32(x_k * inv_s_k)            inv_s_k = 1/s_k given as binary32
+        A   = max_k |t_k|
+        A == 0:  s_q = 1, q = 0
+        else     s_q = fl32(A / 7),  r = fl32(7 / A),  u_k = fl32(t_k * r)
+        q_k = clip(round_half_even(u_k), -8, 7)
+    Static mode (the paper's literal form: s_q fixed offline): the caller passes
+    f_k = 1/(s_k*s_q) as ``inv_s`` and s_q as ``static_scale``;  q_k = clip(rhe(fl32(x_k*f_k))).
+    Every product of two binary32 values is exact in binary64 and a binary32 quotient obtained
+    through one binary64 division rounds identically (53 >= 2*24+2), so casting to binary32 after
+    each step reproduces IEEE binary32 arithmetic exactly.
+
+    Returns (q int8 [M,K], s_q float32 [M]).
+    """
+    x = np.asarray(x_fp16, dtype=np.float16).astype(np.float64)
+    M, K = x.shape
+    f = np.ones(K) if inv_s is None else np.asarray(inv_s, dtype=np.float32).astype(np.float64)
+    t = _f32(x * f[None, :])
+    if static_scale is not None:
+        q = np.clip(np.rint(t), QMIN, QMAX).astype(np.int8)
+        return q, np.full(M, np.float32(static_scale), dtype=np.float32)
+    A = np.abs(t).max(axis=1) if K else np.zeros(M)
+    s_q = np.ones(M, dtype=np.float64)
+    r = np.zeros(M, dtype=np.float64)
+    nz = A > 0
+    s_q[nz] = _f32(A[nz] / 7.0)
+    r[nz] = _f32(7.0 / A[nz])
+    u = _f32(t * r[:, None])
+    q = np.clip(np.rint(u), QMIN, QMAX).astype(np.int8)   # np.rint rounds half to even
+    return q, s_q.astype(np.float32)
+
+
+def smooth_quantize_ideal(x_fp16, inv_s):
+    """The same assignment in unrounded real arithmetic (binary64): x/(s_k*s_q) with s_q = A/7.
+    Differs from ``smooth_quantize`` only where the pre-rounding value sits within a few binary32
+    ulps of a half-integer; used to count such positions, never as an expected value."""
+    x = np.asarray(x_fp16, dtype=np.float16).astype(np.float64)
+    f = np.ones(x.shape[1]) if inv_s is None else np.asarray(inv_s, dtype=np.float32).astype(np.float64)
+    t = x * f[None, :]
+    A = np.abs(t).max(axis=1)
+    u = np.where(A[:, None] > 0, t * 7.0 / np.where(A > 0, A, 1.0)[:, None], 0.0)
+    return np.clip(np.rint(u), QMIN, QMAX).astype(np.int8)
+
+
+def pack_act(q: np.ndarray, K_pad: int | None = None) -> np.ndarray:
+    """Activation indices a = q + 8 in [0,15], two per byte (even k in the low nibble), row padded
+    to K_pad (multiple of 256) with a = 8 (q = 0)."""
+    M, K = q.shape
+    K_pad = round_up(K, TILE_K) if K_pad is None else K_pad
+    a = np.full((M, K_pad), 8, dtype=np.uint8)
+    a[:, :K] = (q.astype(np.int16) + 8).astype(np.uint8)
+    return (a[:, 0::2] | (a[:, 1::2] << 4)).astype(np.uint8)
+
+
+def unpack_act(packed: np.ndarray, K: int) -> np.ndarray:
+    M = packed.shape[0]
+    a = np.empty((M, packed.shape[1] * 2), dtype=np.int16)
+    a[:, 0::2] = packed & 0xF
+    a[:, 1::2] = packed >> 4
+    return (a[:, :K] - 8).astype(np.int8)
+
+
+# --------------------------------------------------------------------------------------
+# Section 4.2 - lookup and accumulation, four equivalent statements
+# --------------------------------------------------------------------------------------
+def dequantize(idx: np.ndarray, codebook_fp16: np.ndarray) -> np.ndarray:
+    """W_q[n][k] = codebook[n][idx[n][k]] as float64."""
+    cb = np.asarray(codebook_fp16, dtype=np.float16).astype(np.float64)
+    return np.take_along_axis(cb, idx.astype(np.int64), axis=1)
+
+
+def lut_linear_dequant(idx, codebook_fp16, q, s_q) -> np.ndarray:
+    """y[m][n] = s_q[m] * sum_k q[m][k] * cb[n][idx[n][k]]   (float64, library matmul as the sum)."""
+    Wq = dequantize(idx, codebook_fp16)
+    acc = q.astype(np.float64) @ Wq.T
+    return np.asarray(s_q, dtype=np.float64)[:, None] * acc
+
+
+def lut_linear_loops(idx, codebook_fp16, q, s_q) -> np.ndarray:
+    """The same definition as an explicit triple loop, k ascending (tiny inputs only)."""
+    cb = np.asarray(codebook_fp16, dtype=np.float16).astype(np.float64)
+    M, K = q.shape
+    N = idx.shape[0]
+    y = np.zeros((M, N))
+    for m in range(M):
+        for n in range(N):
+            acc = 0.0
+            for k in range(K):
+                acc += float(q[m, k]) * cb[n, idx[n, k]]
+            y[m, n] = float(s_q[m]) * acc
+    return y
+
+
+def lut_linear_product(idx, codebook_fp16, q, s_q) -> np.ndarray:
+    """Product table: T_{m,n}[a][w] = ((a-8) * s_q[m]) * cb[n][w];  y[m][n] = sum_k T[a_k][idx_k]."""
+    cb = np.asarray(codebook_fp16, dtype=np.float16).astype(np.float64)
+    M, K = q.shape
+    N, C = cb.shape
+    a = q.astype(np.int64) + 8
+    levels = np.arange(LEVELS, dtype=np.float64) - 8.0
+    y = np.zeros((M, N))
+    ii = idx.astype(np.int64)
+    for m in range(M):
+        act_val = levels * float(s_q[m])                  # 16 activation values of this token
+        for n in range(N):
+            T = act_val[:, None] * cb[n][None, :]         # 16 x C table
+            y[m, n] = T[a[m], ii[n]].sum()
+    return y
+
+
+def lut_linear_signfold(idx, codebook_fp16, q, s_q) -> np.ndarray:
+    """Only |q| in [0,8] is tabulated: T+[|q|][w] = (|q| * s_q) * cb[w]; y = sum_k sgn(q_k) * T+[|q_k|][idx_k]."""
+    cb = np.asarray(codebook_fp16, dtype=np.float16).astype(np.float64)
+    M, K = q.shape
+    N, C = cb.shape
+    mag = np.abs(q.astype(np.int64))
+    sgn = np.sign(q.astype(np.int64)).astype(np.float64)
+    y = np.zeros((M, N))
+    ii = idx.astype(np.int64)
+    for m in range(M):
+        lev = np.arange(9, dtype=np.float64) * float(s_q[m])
+        for n in range(N):
+            Tp = lev[:, None] * cb[n][None, :]            # 9 x C
+            y[m, n] = (sgn[m] * Tp[mag[m], ii[n]]).sum()
+    return y
+
+
+def bucket_sums(idx, q, C: int) -> np.ndarray:
+    """S[m][n][w] = sum over {k : idx[n][k] == w} of q[m][k]   (exact int64)."""
+    M, K = q.shape
+    N = idx.shape[0]
+    S = np.zeros((M, N, C), dtype=np.int64)
+    q64 = q.astype(np.int64)
+    for w in range(C):
+        mask = (idx == w).astype(np.int64)                # N x K
+        S[:, :, w] = q64 @ mask.T
+    return S
+
+
+def lut_linear_bucket(idx, codebook_fp16, q, s_q) -> np.ndarray:
+    """Centroid-stationary form: y[m][n] = s_q[m] * sum_w cb[n][w] * S[m][n][w]."""
+    cb = np.asarray(codebook_fp16, dtype=np.float16).astype(np.float64)
+    S = bucket_sums(idx, q, cb.shape[1]).astype(np.float64)
+    return np.asarray(s_q, dtype=np.float64)[:, None] * np.einsum("mnw,nw->mn", S, cb)
+
+
+def lut_linear_rows(idx, codebook_fp16, q, s_q, rows: np.ndarray) -> np.ndarray:
+    """Dequant form restricted to a sample of output rows (for spot checks at full size)."""
+    return lut_linear_dequant(idx[rows], np.asarray(codebook_fp16)[rows], q, s_q)
+
+
+# --------------------------------------------------------------------------------------
+# Packed-weight blob (layout id 1, "tile8x256")
+# --------------------------------------------------------------------------------------
+def packed_weights_bytes(N: int, K: int, bits: int) -> int:
+    N_pad, K_pad = round_up(N, TILE_ROWS), round_up(K, TILE_K)
+    idx_bytes = N_pad * K_pad * bits // 8
+    cb_off = round_up(INDEX_OFFSET + idx_bytes, 256)
+    return cb_off + round_up(N_pad * (1 << bits) * 2, 256)
+
+
+def _tile_lane_bytes_2bit(rows_idx: np.ndarray, g: int, t: int) -> np.ndarray:
+    """16 bytes of lane (g,t) of one 2-bit tile.  rows_idx: [8][256] indices of the tile."""
+    out = np.zeros(16, dtype=np.uint8)
+    for half in range(2):                 # k-block 0 / 1 of the tile
+        for p in range(8):                # byte position inside the 8-byte quarter record
+            G = 8 * t + ((p + g) % 8)     # k-group (4 consecutive k) inside the k-block, rotated by g
+            b = 0
+            for i in range(4):
+                k = KBLOCK * half + 4 * G + i
+                b |= int(rows_idx[g, k]) << (2 * i)
+            out[8 * half + p] = b
+    return out
+
+
+def _record_3bit(v32: np.ndarray) -> np.ndarray:
+    """12-byte record of 32 three-bit indices v32[0..31]: words 0..2 carry indices 8i+j in bits
+    [4j,4j+3); index 24+j has bit b stored at bit 4j+3 of word b."""
+    words = [0, 0, 0]
+    for i in range(3):
+        for j in range(8):
+            words[i] |= int(v32[8 * i + j]) << (4 * j)
+    for j in range(8):
+        v = int(v32[24 + j])
+        for b in range(3):
+            words[b] |= ((v >> b) & 1) << (4 * j + 3)
+    return np.frombuffer(struct.pack("<3I", *words), dtype=np.uint8)
+
+
+def pack_weights(idx: np.ndarray, codebook_fp16: np.ndarray, bits: int, C: int | None = None) -> np.ndarray:
+    """Build the blob (uint8 array).
+
+    Header, 64 bytes little-endian:  u32 magic "LCDW", u32 version=1, u64 N, u64 K, u64 K_pad,
+    u32 bits, u32 C, u32 layout=1, u32 checksum (sum of all payload bytes mod 2^32),
+    u64 index_offset (=256), u64 codebook_offset.  Bytes 64..255 are zero.
+
+    Index area: rows padded to N_pad = 8*ceil(N/8), columns to K_pad = 256*ceil(K/256), padding
+    index 0.  Tiles of 8 rows x 256 columns, tile (rg, kt) at index_offset + (rg*(K_pad/256)+kt)*T,
+    T = 512 bytes (2 bit) or 768 bytes (3 bit).  Lane l = 4*g + t (g = 0..7 row inside the tile,
+    t = 0..3 quarter) owns, for each of the tile's two 128-column k-blocks h, the 32 columns
+    128*h + 32*t .. +31 of row g.
+      2 bit: lane record = 16 bytes at tile + 16*l: bytes [8h, 8h+8) are k-block h.  Byte p of those
+             holds k-group G = 8t + ((p+g) mod 8): columns 128h + 4G + i at bits [2i, 2i+2).
+      3 bit: the tile is three 256-byte planes; plane b holds, at plane + 8*l, word b of the lane's
+             record for k-block 0 then word b of its record for k-block 1.  A record packs the 32
+             columns 128h + 32t + m: m = 8i+j (i<3) in bits [4j,4j+3) of word i; m = 24+j has its bit b
+             at bit 4j+3 of word b.
+    Codebook area: N_pad rows of 2^bits fp16 values (entries >= C and padded rows are zero).
+    """
+    idx = np.asarray(idx, dtype=np.uint8)
+    N, K = idx.shape
+    C = (1 << bits) if C is None else C
+    if bits not in (2, 3) or not (1 <= C <= (1 << bits)):
+        raise ValueError("bits/C")
+    if idx.size and int(idx.max()) >= C:
+        raise ValueError("index out of range")
+    cb = np.asarray(codebook_fp16, dtype=np.float16)
+    assert cb.shape == (N, C)
+    N_pad, K_pad = round_up(N, TILE_ROWS), round_up(K, TILE_K)
+    total = packed_weights_bytes(N, K, bits)
+    blob = np.zeros(total, dtype=np.uint8)
+    P = np.zeros((N_pad, K_pad), dtype=np.uint8)
+    P[:N, :K] = idx
+    tile_bytes = TILE_ROWS * TILE_K * bits // 8
+    n_kt = K_pad // TILE_K
+    for rg in range(N_pad // TILE_ROWS):
+        for kt in range(n_kt):
+            sub = P[rg * 8:(rg + 1) * 8, kt * TILE_K:(kt + 1) * TILE_K]
+            base = INDEX_OFFSET + (rg * n_kt + kt) * tile_bytes
+            for g in range(8):
+                for t in range(4):
+                    lane = 4 * g + t
+                    if bits == 2:
+                        blob[base + 16 * lane: base + 16 * lane + 16] = _tile_lane_bytes_2bit(sub, g, t)
+                    else:
+                        for h in range(2):
+                            rec = _record_3bit(sub[g, KBLOCK * h + 32 * t: KBLOCK * h + 32 * t + 32])
+                            for b in range(3):
+                                o = base + 256 * b + 8 * lane + 4 * h
+                                blob[o:o + 4] = rec[4 * b:4 * b + 4]
+    cb_off = round_up(INDEX_OFFSET + N_pad * K_pad * bits // 8, 256)
+    cbp = np.zeros((N_pad, 1 << bits), dtype=np.float16)
+    cbp[:N, :C] = cb
+    blob[cb_off:cb_off + cbp.size * 2] = cbp.view(np.uint8).reshape(-1)
+    checksum = int(blob[HEADER_BYTES:].astype(np.uint64).sum()) & 0xFFFFFFFF
+    hdr = struct.pack("<IIQQQIIIIQQ", MAGIC, VERSION, N, K, K_pad, bits, C, LAYOUT_TILE8X256, checksum,
+                      INDEX_OFFSET, cb_off)
+    assert len(hdr) == HEADER_BYTES
+    blob[:HEADER_BYTES] = np.frombuffer(hdr, dtype=np.uint8)
+    return blob
+
+
+def parse_header(blob: np.ndarray) -> dict:
+    f = struct.unpack("<IIQQQIIIIQQ", bytes(blob[:HEADER_BYTES]))
+    keys = ("magic", "version", "N", "K", "K_pad", "bits", "C", "layout", "checksum", "index_offset",
+            "codebook_offset")
+    return dict(zip(keys, f))
+
+
+def unpack_weights(blob: np.ndarray):
+    """Exact inverse of ``pack_weights``: returns (idx uint8 [N,K], codebook fp16 [N,C], bits, C)."""
+    h = parse_header(blob)
+    if h["magic"] != MAGIC or h["version"] != VERSION or h["layout"] != LAYOUT_TILE8X256:
+        raise ValueError("bad blob header")
+    if (int(blob[HEADER_BYTES:].astype(np.uint64).sum()) & 0xFFFFFFFF) != h["checksum"]:
+        raise ValueError("bad blob checksum")
+    N, K, K_pad, bits, C = h["N"], h["K"], h["K_pad"], h["bits"], h["C"]
+    N_pad = round_up(N, TILE_ROWS)
+    tile_bytes = TILE_ROWS * TILE_K * bits // 8
+    n_kt = K_pad // TILE_K
+    P = np.zeros((N_pad, K_pad), dtype=np.uint8)
+    for rg in range(N_pad // TILE_ROWS):
+        for kt in range(n_kt):
+            base = h["index_offset"] + (rg * n_kt + kt) * tile_bytes
+            for g in range(8):
+                for t in range(4):
+                    lane = 4 * g + t
+                    for hb in range(2):
+                        k0 = kt * TILE_K + KBLOCK * hb
+                        if bits == 2:
+                            for p in range(8):
+                                G = 8 * t + ((p + g) % 8)
+                                b = int(blob[base + 16 * lane + 8 * hb + p])
+                                for i in range(4):
+                                    P[rg * 8 + g, k0 + 4 * G + i] = (b >> (2 * i)) & 3
+                        else:
+                            words = []
+                            for b in range(3):
+                                o = base + 256 * b + 8 * lane + 4 * hb
+                                words.append(struct.unpack("<I", bytes(blob[o:o + 4]))[0])
+                            for m in range(32):
+                                if m < 24:
+                                    v = (words[m // 8] >> (4 * (m % 8))) & 7
+                                else:
+                                    j = m - 24
+                                    v = sum(((words[b] >> (4 * j + 3)) & 1) << b for b in range(3))
+                                P[rg * 8 + g, k0 + 32 * t + m] = v
+    cbp = blob[h["codebook_offset"]:h["codebook_offset"] + N_pad * (1 << bits) * 2].view(np.float16)
+    cbp = cbp.reshape(N_pad, 1 << bits)
+    return P[:N, :K].copy(), cbp[:N, :C].copy(), bits, C

@@ -1,0 +1,284 @@
+"""Pins for the CPU oracle: each test fixes it to something other than itself - a closed form, an
+invariant, a library routine, brute force, or a hand-worked example under tests/golden/.  The paper
+(Section 4) prints no numeric example of the LUT path, so none of the pins is a paper-printed value."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+from oracle import lcd_oracle as O
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+
+def rnd_case(seed, N, K, C, M):
+    rng = np.random.default_rng(seed)
+    idx = rng.integers(0, C, size=(N, K), dtype=np.uint8)
+    cb = (rng.standard_normal((N, C)) * 0.1).astype(np.float16)
+    q = rng.integers(-8, 8, size=(M, K), dtype=np.int8)
+    s_q = (rng.random(M) + 0.1).astype(np.float32)
+    return idx, cb, q, s_q
+
+
+# ---------------------------------------------------------------- linear forms (Section 4.2)
+@pytest.mark.parametrize("bits", [2, 3])
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_four_forms_and_loops_agree(bits, seed):
+    C = 1 << bits
+    idx, cb, q, s_q = rnd_case(seed, N=7, K=61, C=C, M=3)
+    ref = O.lut_linear_loops(idx, cb, q, s_q)
+    scale = (np.abs(q.astype(float)).sum(axis=1)[:, None] * np.abs(cb.astype(float)).max(axis=1)[None, :]
+             * s_q[:, None].astype(float))
+    for f in (O.lut_linear_dequant, O.lut_linear_product, O.lut_linear_signfold, O.lut_linear_bucket):
+        y = f(idx, cb, q, s_q)
+        assert np.all(np.abs(y - ref) <= 1e-12 * scale + 1e-300), f.__name__
+
+
+def test_matches_library_matmul_on_dequantised_matrix():
+    idx, cb, q, s_q = rnd_case(5, N=33, K=200, C=8, M=4)
+    Wq = np.empty((33, 200))
+    for n in range(33):
+        for k in range(200):
+            Wq[n, k] = float(cb[n, idx[n, k]])
+    xq = s_q[:, None].astype(np.float64) * q.astype(np.float64)
+    ref = np.matmul(xq, Wq.T)
+    y = O.lut_linear_bucket(idx, cb, q, s_q)
+    assert np.allclose(y, ref, rtol=1e-12, atol=1e-12)
+    assert np.allclose(O.lut_linear_dequant(idx, cb, q, s_q), ref, rtol=1e-12, atol=1e-12)
+
+
+def test_one_centroid_codebook_gives_c_times_sum_x():
+    rng = np.random.default_rng(3)
+    N, K, M = 5, 40, 2
+    idx = np.zeros((N, K), dtype=np.uint8)
+    cb = (rng.standard_normal((N, 1))).astype(np.float16)
+    q = rng.integers(-8, 8, size=(M, K), dtype=np.int8)
+    s_q = np.array([0.25, 1.5], dtype=np.float32)
+    expect = (s_q.astype(float)[:, None] * q.astype(float).sum(axis=1)[:, None]) * cb.astype(float)[:, 0][None, :]
+    for f in (O.lut_linear_dequant, O.lut_linear_product, O.lut_linear_signfold, O.lut_linear_bucket):
+        assert np.allclose(f(idx, cb, q, s_q), expect, rtol=1e-13, atol=0), f.__name__
+
+
+def test_affine_codebook_closed_form_hand_case():
+    # hand-worked example, see tests/golden/affine_k4.txt
+    g = [l for l in open(os.path.join(HERE, "golden", "affine_k4.txt")) if not l.startswith("#")]
+    vals = [float(v) for v in g[0].split()]
+    idx = np.array([[0, 3, 1, 2]], dtype=np.uint8)
+    cb = np.array([[0.5 * w - 0.25 for w in range(4)]], dtype=np.float16)        # alpha=.5, beta=-.25
+    q = np.array([[3, -2, 7, -8]], dtype=np.int8)
+    s_q = np.array([0.5], dtype=np.float32)
+    # sum q*idx = 0 - 6 + 7 - 16 = -15 ; sum q = 0 ; y = 0.5 * (0.5 * -15 + -0.25 * 0) = -3.75
+    for f in (O.lut_linear_dequant, O.lut_linear_product, O.lut_linear_signfold, O.lut_linear_bucket,
+              O.lut_linear_loops):
+        assert f(idx, cb, q, s_q)[0, 0] == vals[0] == -3.75
+
+
+@pytest.mark.parametrize("seed", [0, 1])
+def test_affine_codebook_closed_form_random(seed):
+    rng = np.random.default_rng(seed)
+    N, K, M, C = 6, 50, 3, 8
+    idx = rng.integers(0, C, size=(N, K), dtype=np.uint8)
+    alpha = rng.integers(-4, 5, size=N) / 8.0
+    beta = rng.integers(-8, 9, size=N) / 16.0
+    cb = (alpha[:, None] * np.arange(C)[None, :] + beta[:, None]).astype(np.float16)   # exact in fp16
+    q = rng.integers(-8, 8, size=(M, K), dtype=np.int8)
+    s_q = np.array([0.5, 2.0, 0.125], dtype=np.float32)
+    sqi = (q.astype(np.int64) @ idx.astype(np.int64).T)
+    sq = q.astype(np.int64).sum(axis=1)
+    expect = s_q.astype(float)[:, None] * (alpha[None, :] * sqi + beta[None, :] * sq[:, None])
+    for f in (O.lut_linear_dequant, O.lut_linear_bucket, O.lut_linear_product, O.lut_linear_signfold):
+        assert np.allclose(f(idx, cb, q, s_q), expect, rtol=1e-13, atol=1e-13)
+
+
+def test_brute_force_all_index_patterns_k6_c2():
+    K = 6
+    cb = np.array([[-0.75, 1.25]], dtype=np.float16)
+    acts = np.array([[1, -2, 3, -4, 5, -6], [7, 7, -8, 0, 0, 1]], dtype=np.int8)
+    s_q = np.array([1.0, 0.5], dtype=np.float32)
+    for pattern in itertools.product([0, 1], repeat=K):
+        idx = np.array([pattern], dtype=np.uint8)
+        expect = [[s * sum(int(a[k]) * (1.25 if pattern[k] else -0.75) for k in range(K))] for a, s in
+                  zip(acts, [1.0, 0.5])]
+        for f in (O.lut_linear_dequant, O.lut_linear_bucket, O.lut_linear_product, O.lut_linear_signfold):
+            assert np.array_equal(f(idx, cb, acts, s_q), np.array(expect))
+
+
+def test_bucket_sums_partition_the_activation_sum():
+    idx, cb, q, s_q = rnd_case(9, N=4, K=97, C=4, M=2)
+    S = O.bucket_sums(idx, q, 4)
+    assert np.array_equal(S.sum(axis=2), np.repeat(q.astype(np.int64).sum(axis=1)[:, None], 4, axis=1))
+    # a transposed operand or swapped index would break this one-hot case
+    idx1 = np.zeros((2, 5), dtype=np.uint8); idx1[1, 3] = 2
+    q1 = np.array([[1, 2, 3, 4, 5]], dtype=np.int8)
+    S1 = O.bucket_sums(idx1, q1, 4)
+    assert S1.tolist() == [[[15, 0, 0, 0], [11, 0, 4, 0]]]
+
+
+# ---------------------------------------------------------------- quantiser (Section 4.1)
+def test_quantiser_hand_example():
+    # x = [7, -3.5, 0.5, 1.5, 2.5, -7] with inv_s = 1: A = 7, s_q = 1, r = 1 -> ties go to even
+    x = np.array([[7, -3.5, 0.5, 1.5, 2.5, -7]], dtype=np.float16)
+    q, s = O.smooth_quantize(x, None)
+    assert q.tolist() == [[7, -4, 0, 2, 2, -7]] and s[0] == 1.0
+    # smoothing is a multiply by 1/s_k: halving channel 0 moves the max to channel 5
+    q2, s2 = O.smooth_quantize(x, np.array([0.5, 1, 1, 1, 1, 1], dtype=np.float32))
+    assert q2.tolist() == [[4, -4, 0, 2, 2, -7]] and s2[0] == 1.0   # 3.5 -> 4 (even), A still 7
+
+
+def test_quantiser_max_maps_to_pm7_and_sign_symmetry():
+    rng = np.random.default_rng(0)
+    x = rng.standard_normal((5, 300)).astype(np.float16)
+    inv_s = (rng.random(300) + 0.5).astype(np.float32)
+    q, s = O.smooth_quantize(x, inv_s)
+    assert np.all(np.abs(q).max(axis=1) == 7) and q.min() >= -7
+    qn, sn = O.smooth_quantize(-x, inv_s)
+    assert np.array_equal(qn, -q) and np.array_equal(sn, s)
+
+
+def test_quantiser_power_of_two_scale_invariance():
+    rng = np.random.default_rng(1)
+    x = (rng.standard_normal((3, 128))).astype(np.float16)
+    inv_s = (rng.random(128) + 0.5).astype(np.float32)
+    q, s = O.smooth_quantize(x, inv_s)
+    for j in (-3, 2, 5):
+        q2, s2 = O.smooth_quantize((x.astype(np.float32) * 2.0 ** j).astype(np.float16), inv_s)
+        assert np.array_equal(q2, q)
+        assert np.array_equal(s2, (s * np.float32(2.0 ** j)).astype(np.float32))
+
+
+def test_quantiser_monotone_and_zero_row_and_static_mode():
+    xs = np.linspace(-3, 3, 193).astype(np.float16)
+    x = np.concatenate([xs, [4.0]]).astype(np.float16)[None, :]        # fixed maximum 4 -> fixed scale
+    q, s = O.smooth_quantize(x, None)
+    assert np.all(np.diff(q[0, :-1].astype(int)) >= 0)
+    z, sz = O.smooth_quantize(np.zeros((2, 8), dtype=np.float16), None)
+    assert not z.any() and np.all(sz == 1.0)
+    # static mode: f = 1/(s*s_q) and every level -8..7 is reachable, values beyond are clipped
+    xv = np.arange(-10, 10, dtype=np.float16)[None, :]
+    qs, ss = O.smooth_quantize(xv, np.full(20, 1.0, dtype=np.float32), static_scale=1.0)
+    assert qs.tolist() == [[-8, -8, -8, -7, -6, -5, -4, -3, -2, -1, 0, 1, 2, 3, 4, 5, 6, 7, 7, 7]]
+    qt, _ = O.smooth_quantize(np.array([[0.5, 1.5, 2.5, -0.5, -1.5, 6.5, -6.5]], dtype=np.float16),
+                              np.ones(7, dtype=np.float32), static_scale=1.0)
+    assert qt.tolist() == [[0, 2, 2, 0, -2, 6, -6]]
+
+
+def test_quantiser_is_binary32_arithmetic():
+    # the double-with-casts sequence must equal native float32 arithmetic step by step
+    rng = np.random.default_rng(2)
+    x = (rng.standard_normal((4, 512)) * 3).astype(np.float16)
+    inv_s = (rng.random(512) * 3 + 0.01).astype(np.float32)
+    q, s = O.smooth_quantize(x, inv_s)
+    t = x.astype(np.float32) * inv_s[None, :]
+    A = np.abs(t).max(axis=1)
+    s32 = A / np.float32(7.0)
+    r = np.float32(7.0) / A
+    u = t * r[:, None]
+    q32 = np.clip(np.rint(u), -8, 7).astype(np.int8)
+    assert np.array_equal(q, q32) and np.array_equal(s, s32.astype(np.float32))
+    ideal = O.smooth_quantize_ideal(x, inv_s)
+    assert (ideal != q).mean() < 1e-3
+
+
+def test_quantisation_error_bound():
+    # |x/s - s_q*q| <= s_q/2 (+ rounding slack): the encoding is a uniform quantiser of step s_q
+    rng = np.random.default_rng(4)
+    x = rng.standard_normal((3, 256)).astype(np.float16)
+    q, s = O.smooth_quantize(x, None)
+    err = np.abs(x.astype(np.float64) - s.astype(np.float64)[:, None] * q)
+    assert np.all(err <= 0.5 * s[:, None] * (1 + 1e-5))
+
+
+def test_act_pack_roundtrip_and_padding():
+    rng = np.random.default_rng(0)
+    q = rng.integers(-8, 8, size=(3, 300), dtype=np.int8)
+    p = O.pack_act(q)
+    assert p.shape == (3, 256) and np.array_equal(O.unpack_act(p, 300), q)
+    assert np.all(p[:, 150:] == 0x88)
+    assert p[0, 0] == ((int(q[0, 0]) + 8) | ((int(q[0, 1]) + 8) << 4))
+
+
+# ---------------------------------------------------------------- packing
+@pytest.mark.parametrize("bits,C", [(2, 4), (3, 8), (3, 5), (2, 3)])
+def test_pack_roundtrip_random(bits, C):
+    rng = np.random.default_rng(bits * 10 + C)
+    N, K = 19, 300
+    idx = rng.integers(0, C, size=(N, K), dtype=np.uint8)
+    cb = rng.standard_normal((N, C)).astype(np.float16)
+    blob = O.pack_weights(idx, cb, bits, C)
+    assert blob.size == O.packed_weights_bytes(N, K, bits)
+    N_pad, K_pad = 24, 512
+    assert blob.size == 256 + N_pad * K_pad * bits // 8 + ((N_pad * (1 << bits) * 2 + 255) // 256) * 256
+    i2, c2, b2, C2 = O.unpack_weights(blob)
+    assert np.array_equal(i2, idx) and np.array_equal(c2.view(np.uint16), cb.view(np.uint16)) and (b2, C2) == (bits, C)
+
+
+@pytest.mark.parametrize("bits", [2, 3])
+def test_pack_one_hot_positions_hit_distinct_bits(bits):
+    # each (row, column) of one tile maps to its own bit field: one-hot inputs give disjoint blobs whose
+    # union is the all-ones blob, and every payload bit is covered exactly once (exactly `bits` bits/weight)
+    C = 1 << bits
+    N, K = 8, 256
+    cb = np.zeros((N, C), dtype=np.float16)
+    full = O.pack_weights(np.full((N, K), C - 1, dtype=np.uint8), cb, bits)
+    body = slice(256, 256 + N * K * bits // 8)
+    assert np.all(full[body] == 0xFF)
+    acc = np.zeros(N * K * bits // 8, dtype=np.uint16)
+    for n in (0, 3, 7):
+        for k in range(K):
+            idx = np.zeros((N, K), dtype=np.uint8)
+            idx[n, k] = C - 1
+            b = O.pack_weights(idx, cb, bits)[body]
+            assert int(np.unpackbits(b).sum()) == bits
+            assert not np.any(acc.astype(np.uint8) & b)
+            acc |= b
+    assert int(np.unpackbits(acc.astype(np.uint8)).sum()) == 3 * K * bits
+
+
+def test_pack_2bit_layout_spot_bytes():
+    # written out by hand from the layout text: tile 0, lane l = 4g+t, byte p of k-block h holds k-group
+    # G = 8t + (p+g)%8; column 128h+4G+i sits at bits [2i,2i+2)
+    N, K = 8, 256
+    idx = np.zeros((N, K), dtype=np.uint8)
+    idx[0, 0] = 3          # g=0,t=0,h=0,G=0,i=0 -> p=0        -> byte 256+0,       value 0b11
+    idx[1, 5] = 2          # g=1,t=0,h=0,G=1,i=1 -> p=(1-1)%8=0 -> byte 256+16*4+0,  value 2<<2
+    idx[2, 128 + 37] = 1   # g=2,h=1,G=9 -> t=1, (p+2)%8=1 -> p=7, i=1 -> byte 256+16*(8+1)+8+7, value 1<<2
+    idx[7, 255] = 3        # g=7,h=1,G=31,t=3,(p+7)%8=7 -> p=0, i=3 -> byte 256+16*31+8+0, value 3<<6
+    blob = O.pack_weights(idx, np.zeros((N, 4), dtype=np.float16), 2)
+    body = blob[256:256 + 512]
+    expect = np.zeros(512, dtype=np.uint8)
+    expect[0] = 3
+    expect[16 * 4 + 0] = 2 << 2
+    expect[16 * 9 + 8 + 7] = 1 << 2
+    expect[16 * 31 + 8 + 0] = 3 << 6
+    assert np.array_equal(body, expect)
+
+
+def test_pack_3bit_layout_spot_bytes():
+    N, K = 8, 256
+    idx = np.zeros((N, K), dtype=np.uint8)
+    idx[0, 0] = 5            # g=0,t=0,h=0,m=0  -> word0 bits[0,3) = 5        -> plane0 byte 0 = 5
+    idx[0, 9] = 7            # m=9 -> word1, j=1 -> bits [4,7)                 -> plane1 byte 0 = 0x70
+    idx[0, 24] = 6           # m=24 (j=0): bit1 -> word1 bit3, bit2 -> word2 bit3
+    idx[3, 128 + 32 * 2 + 31] = 1   # g=3,t=2,h=1,m=31 (j=7): bit0 -> word0 bit 31 -> lane 14, byte offset 8*14+4+3
+    blob = O.pack_weights(idx, np.zeros((N, 8), dtype=np.float16), 3)
+    body = blob[256:256 + 768]
+    expect = np.zeros(768, dtype=np.uint8)
+    expect[0] = 5
+    expect[256 + 0] = 0x70 | 0x08
+    expect[512 + 0] = 0x08
+    expect[8 * 14 + 4 + 3] = 0x80
+    assert np.array_equal(body, expect)
+
+
+def test_pack_rejects_bad_indices_and_corruption():
+    cb = np.zeros((2, 3), dtype=np.float16)
+    with pytest.raises(ValueError):
+        O.pack_weights(np.full((2, 4), 3, dtype=np.uint8), cb, 2, 3)
+    blob = O.pack_weights(np.zeros((2, 4), dtype=np.uint8), cb, 2, 3)
+    bad = blob.copy(); bad[300] ^= 1
+    with pytest.raises(ValueError):
+        O.unpack_weights(bad)
+    bad = blob.copy(); bad[0] ^= 1
+    with pytest.raises(ValueError):
+        O.unpack_weights(bad)
