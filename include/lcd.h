@@ -1,0 +1,164 @@
+/*
+ * lcd.h - C ABI of the B200 (sm_100a) LUT-based inference matmul of the LCD paper
+ *         ("Inference with Table Lookup", Section 4).
+ *
+ * A linear layer y = x W^T (W is N x K) whose clustered weights are stored as packed 2- or 3-bit
+ * centroid indices idx[n][k] plus a per-output-row fp16 codebook cb[n][w].  Activations are
+ * smoothed per input channel, mapped to 4-bit indices a = q + 8 (q in [-8,7]) with one fp32 scale
+ * per token, and every output is formed by table lookup and accumulation:
+ *
+ *      y[m][n] = s_q[m] * sum_k q[m][k] * cb[n][idx[n][k]]          (fp32)
+ *
+ * Conventions for every function:
+ *   - returns an lcd_status; never aborts, traps or throws;
+ *   - "host" / "device" in a parameter comment says where the pointer must point;
+ *   - the caller owns every buffer; the library keeps no state except lazily set kernel attributes;
+ *   - device entry points are stream-ordered on `cuda_stream` (a cudaStream_t passed as void*;
+ *     NULL = legacy default stream), do not synchronise and do not allocate;
+ *   - argument errors are reported before anything is launched; an asynchronous problem (a bounded
+ *     wait inside a kernel that expired) is written to `*status_word_dev` when that pointer is given.
+ */
+#ifndef LCD_H_
+#define LCD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LCD_OK = 0,
+  LCD_ERR_INVALID_ARG = 1,      /* null pointer, non-positive size, bad alignment, bad enum          */
+  LCD_ERR_UNSUPPORTED = 2,      /* valid request this build has no kernel for                       */
+  LCD_ERR_BUFFER_TOO_SMALL = 3, /* an output / workspace / scratch buffer is smaller than required  */
+  LCD_ERR_INDEX_RANGE = 4,      /* a weight index >= C                                              */
+  LCD_ERR_BAD_BLOB = 5,         /* header magic / version / layout / checksum / size mismatch       */
+  LCD_ERR_CUDA = 6,             /* a CUDA runtime call or a launch failed (see lcd_last_cuda_error) */
+  LCD_ERR_TIMEOUT = 7           /* value written to the status word when a device-side wait expired */
+} lcd_status;
+
+/* Which kernel family lcd_lut_linear uses.  Every family computes the same y. */
+typedef enum {
+  LCD_ALGO_AUTO = 0,        /* choose by (M, bits): see lcd_lut_linear                                        */
+  LCD_ALGO_REFERENCE = 1,   /* plain per-weight lookup cb[n][idx] and multiply-accumulate; any M, slow        */
+  LCD_ALGO_BUCKET_LUT = 2,  /* Section 4.2 centroid-stationary buckets: shared-memory tables built from the   */
+                            /* token's activation levels return, per byte of four weight indices, the partial */
+                            /* per-centroid activation sums; exact int32 bucket sums dotted with the codebook  */
+                            /* at the end.  M == 1, bits == 2.                                                 */
+  LCD_ALGO_REGISTER_LUT = 3,/* Section 4.2 lookup with the row codebook held as a byte table in registers      */
+                            /* (fixed-point, 16 bit), four weights looked up per instruction, accumulated as    */
+                            /* integer dot products with the activation levels.  M <= 16.                      */
+  LCD_ALGO_DENSE_TC = 4     /* batched prefill: indices decoded through the codebook into fp16 shared-memory   */
+                            /* tiles feeding tcgen05 tensor cores with fp32 accumulators in tensor memory.      */
+} lcd_algo;
+
+#define LCD_HEADER_BYTES 64
+#define LCD_ACT_BITS 4
+
+const char* lcd_status_string(lcd_status s);
+/* Text of the last CUDA error this library saw on the calling thread ("" if none). */
+const char* lcd_last_cuda_error(void);
+
+/* ----------------------------------------------------------------------------------------------
+ * Offline: index packing (Section 4.2, last paragraph: fewer than 16 centroids per layer allow a
+ * compact low-bit index representation; Section 4.1: everything the lookup needs is fixed ahead of
+ * time).  Host functions, bit-exact, no CUDA calls.
+ *
+ * Blob = 64-byte header | zero padding to 256 | index area | codebook area.
+ *   header (little endian): u32 magic 'LCDW', u32 version 1, u64 N, u64 K, u64 K_pad, u32 bits, u32 C,
+ *     u32 layout (1), u32 checksum (sum of all bytes after the header, mod 2^32), u64 index_offset (256),
+ *     u64 codebook_offset.
+ *   index area: rows padded to N_pad = 8*ceil(N/8), columns to K_pad = 256*ceil(K/256) with index 0,
+ *     cut into tiles of 8 rows x 256 columns stored row-group major: tile (rg, kt) starts at
+ *     index_offset + (rg*(K_pad/256) + kt)*T with T = 512 (2 bit) or 768 (3 bit) bytes.  Inside a tile,
+ *     lane l = 4*g + t (g = row 0..7, t = quarter 0..3) owns columns 128*h + 32*t .. +31 of row g for
+ *     both 128-column k-blocks h = 0,1 of the tile:
+ *       2 bit: 16 bytes at tile + 16*l; bytes [8h, 8h+8) belong to k-block h; byte p of those holds the
+ *              four columns 128h + 4G + i (i = 0..3, at bits [2i,2i+2)) of k-group G = 8t + ((p+g) mod 8).
+ *              (The rotation by g lets 32 lanes read 32 different shared-memory banks of the bucket tables.)
+ *       3 bit: three 256-byte planes; plane b has, at plane + 8*l + 4*h, word b of the lane's 12-byte
+ *              record of k-block h.  A record packs columns 128h + 32t + m: m = 8i+j (i < 3) at bits
+ *              [4j, 4j+3) of word i; m = 24+j has bit b of its index at bit 4j+3 of word b.
+ *   codebook area: N_pad rows of 2^bits fp16 values; entries >= C and padding rows are zero.
+ * -------------------------------------------------------------------------------------------- */
+
+/* Size in bytes of the blob for an N x K layer.  bits in {2,3}.  *bytes is written on LCD_OK. */
+lcd_status lcd_packed_weights_bytes(int64_t N, int64_t K, int bits, size_t* bytes);
+
+/* idx: host, uint8 [N][K] row-major (ld = K), every value < C else LCD_ERR_INDEX_RANGE
+ *      (bad_n/bad_k, if non-NULL, receive the first offending position);
+ * codebook_fp16: host, raw IEEE binary16 bits [N][C]; 1 <= C <= 2^bits;
+ * out: host buffer of out_bytes >= lcd_packed_weights_bytes(...), written completely.
+ * The caller copies the blob to the device (base address aligned to 256 bytes) and keeps the first
+ * 64 bytes on the host: device entry points take both. */
+lcd_status lcd_pack_weights(const uint8_t* idx, const uint16_t* codebook_fp16, int64_t N, int64_t K,
+                            int bits, int C, void* out, size_t out_bytes, int64_t* bad_n, int64_t* bad_k);
+
+/* Exact inverse.  blob: host.  Any of idx / codebook_fp16 may be NULL to only read the sizes; otherwise
+ * idx must hold N*K bytes and codebook_fp16 N*C values.  Verifies magic, version, layout, sizes, checksum. */
+lcd_status lcd_unpack_weights(const void* blob, size_t blob_bytes, uint8_t* idx, uint16_t* codebook_fp16,
+                              int64_t* N, int64_t* K, int* bits, int* C);
+
+/* ----------------------------------------------------------------------------------------------
+ * Online step 1: input transformation (Section 4.1, both equations).  Smoothing and uniform symmetric
+ * quantisation are one multiply followed by round-to-nearest(-even) and clip to [-8, 7]:
+ *     dynamic (static_scale == NULL), per token:  t_k = x_k * inv_smooth_k ; A = max_k |t_k| ;
+ *         A == 0: s_q = 1, q = 0 ; else s_q = A / 7, r = 7 / A, q_k = clip(rint(t_k * r)) ;
+ *     static (the paper's literal form, scale fixed offline): inv_smooth_k must already hold
+ *         1/(s_k * s_q) and *static_scale = s_q;  q_k = clip(rint(x_k * inv_smooth_k)).
+ * All arithmetic is IEEE binary32, one rounding per written operation, so the indices are reproducible
+ * bit for bit.
+ *   x_fp16:      device, binary16 [M][ldx], ldx >= K;
+ *   inv_smooth:  device, fp32 [K], or NULL for all ones;
+ *   static_scale device, fp32 scalar, or NULL;
+ *   act_bits:    must be 4;
+ *   act_idx:     device out, uint8 [M][K_pad/2], K_pad = 256*ceil(K/256): a = q + 8, column k even in the
+ *                low nibble; columns K..K_pad-1 are written as a = 8 (q = 0);
+ *   act_scale:   device out, fp32 [M] (s_q).
+ * -------------------------------------------------------------------------------------------- */
+lcd_status lcd_smooth_quantize_act(const void* x_fp16, int64_t M, int64_t K, int64_t ldx,
+                                   const float* inv_smooth, const float* static_scale, int act_bits,
+                                   uint8_t* act_idx, float* act_scale, void* cuda_stream);
+
+/* ----------------------------------------------------------------------------------------------
+ * Online steps 2+3: table lookup and accumulation (Section 4.2).
+ *   packed_weights_dev: device, the blob, 256-byte aligned;
+ *   header_host:        host, the blob's first 64 bytes;
+ *   act_idx, act_scale: device, as written by lcd_smooth_quantize_act for the same K;
+ *   y:                  device out, fp32 [M][ldy], ldy >= N;
+ *   algo:               LCD_ALGO_AUTO picks BUCKET_LUT for (M == 1, 2 bit), REGISTER_LUT for other M <= 16,
+ *                       DENSE_TC for M > 16; a family asked for outside its range => LCD_ERR_UNSUPPORTED;
+ *   workspace:          device scratch of at least lcd_lut_linear_workspace_bytes(...) bytes, 256-byte
+ *                       aligned, contents undefined before and after (may be NULL when that size is 0);
+ *   status_word_dev:    device int32 or NULL; receives LCD_ERR_TIMEOUT if a bounded device-side wait
+ *                       expired (the output is then invalid); never written otherwise.
+ * -------------------------------------------------------------------------------------------- */
+lcd_status lcd_lut_linear_workspace_bytes(const void* header_host, int64_t M, lcd_algo algo, size_t* bytes);
+
+lcd_status lcd_lut_linear(const void* packed_weights_dev, const void* header_host, const uint8_t* act_idx,
+                          const float* act_scale, int64_t M, float* y, int64_t ldy, lcd_algo algo,
+                          void* workspace, size_t workspace_bytes, int32_t* status_word_dev,
+                          void* cuda_stream);
+
+/* ----------------------------------------------------------------------------------------------
+ * The whole online path (Section 4: input transformation -> bucket table lookup -> accumulation) from
+ * HOST activations to HOST outputs, for callers that keep activations on the host: copies x to the
+ * device, runs lcd_smooth_quantize_act (dynamic mode) and lcd_lut_linear (LCD_ALGO_AUTO), copies y back.
+ * All copies and kernels are enqueued on cuda_stream; the call returns without synchronising, y_host is
+ * valid after the stream is synchronised.  x_host / y_host should be pinned for the copies to be async.
+ *   x_host_fp16: host, binary16 [M][K] dense;   y_host: host out, fp32 [M][N] dense;
+ *   inv_smooth:  device fp32 [K] or NULL;
+ *   scratch:     device, >= lcd_linear_host_scratch_bytes(...) bytes, 256-byte aligned.
+ * -------------------------------------------------------------------------------------------- */
+lcd_status lcd_linear_host_scratch_bytes(const void* header_host, int64_t M, size_t* bytes);
+
+lcd_status lcd_linear_host(const void* packed_weights_dev, const void* header_host, const void* x_host_fp16,
+                           int64_t M, const float* inv_smooth, float* y_host, void* scratch,
+                           size_t scratch_bytes, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LCD_H_ */

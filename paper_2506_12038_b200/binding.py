@@ -1,0 +1,198 @@
+"""Thin ctypes binding of the C ABI in include/lcd.h: argument marshalling only.
+
+Every step of the path (index packing, input transformation, table lookup and accumulation) runs inside
+liblcd_b200.so; torch is used for device memory and streams.  There is no CPU fallback: if the shared
+library is missing, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import c_char_p, c_int, c_int32, c_int64, c_size_t, c_void_p, POINTER, byref
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblcd_b200.so")
+
+LCD_OK = 0
+STATUS_NAMES = {0: "LCD_OK", 1: "LCD_ERR_INVALID_ARG", 2: "LCD_ERR_UNSUPPORTED", 3: "LCD_ERR_BUFFER_TOO_SMALL",
+                4: "LCD_ERR_INDEX_RANGE", 5: "LCD_ERR_BAD_BLOB", 6: "LCD_ERR_CUDA", 7: "LCD_ERR_TIMEOUT"}
+ALGO_AUTO, ALGO_REFERENCE, ALGO_BUCKET_LUT, ALGO_REGISTER_LUT, ALGO_DENSE_TC = 0, 1, 2, 3, 4
+HEADER_BYTES = 64
+
+EXPORTS = ["lcd_status_string", "lcd_last_cuda_error", "lcd_packed_weights_bytes", "lcd_pack_weights",
+           "lcd_unpack_weights", "lcd_smooth_quantize_act", "lcd_lut_linear_workspace_bytes", "lcd_lut_linear",
+           "lcd_linear_host_scratch_bytes", "lcd_linear_host"]
+
+
+class LcdError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} {detail}".strip())
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} not built: run `python -m paper_2506_12038_b200.build` "
+                          "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    lib.lcd_status_string.restype = c_char_p
+    lib.lcd_status_string.argtypes = [c_int]
+    lib.lcd_last_cuda_error.restype = c_char_p
+    lib.lcd_packed_weights_bytes.argtypes = [c_int64, c_int64, c_int, POINTER(c_size_t)]
+    lib.lcd_pack_weights.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int, c_int, c_void_p, c_size_t,
+                                     POINTER(c_int64), POINTER(c_int64)]
+    lib.lcd_unpack_weights.argtypes = [c_void_p, c_size_t, c_void_p, c_void_p, POINTER(c_int64), POINTER(c_int64),
+                                       POINTER(c_int), POINTER(c_int)]
+    lib.lcd_smooth_quantize_act.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_int,
+                                            c_void_p, c_void_p, c_void_p]
+    lib.lcd_lut_linear_workspace_bytes.argtypes = [c_void_p, c_int64, c_int, POINTER(c_size_t)]
+    lib.lcd_lut_linear.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_int64, c_int,
+                                   c_void_p, c_size_t, c_void_p, c_void_p]
+    lib.lcd_linear_host_scratch_bytes.argtypes = [c_void_p, c_int64, POINTER(c_size_t)]
+    lib.lcd_linear_host.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_size_t,
+                                    c_void_p]
+    for name in EXPORTS:
+        if name not in ("lcd_status_string", "lcd_last_cuda_error"):
+            getattr(lib, name).restype = c_int
+    return lib
+
+
+lib = _load()
+
+
+def _check(st: int, where: str):
+    if st != LCD_OK:
+        detail = lib.lcd_last_cuda_error().decode() if st == 6 else ""
+        raise LcdError(st, where, detail)
+
+
+def _np_ptr(a: np.ndarray) -> c_void_p:
+    return c_void_p(a.ctypes.data)
+
+
+# ------------------------------------------------------------------------------------------- host: packing
+def packed_weights_bytes(N: int, K: int, bits: int) -> int:
+    out = c_size_t(0)
+    _check(lib.lcd_packed_weights_bytes(N, K, bits, byref(out)), "lcd_packed_weights_bytes")
+    return out.value
+
+
+def pack_weights(idx: np.ndarray, codebook_fp16: np.ndarray, bits: int, C: int | None = None) -> np.ndarray:
+    """idx uint8 [N,K], codebook fp16 [N,C] (host numpy) -> blob (host numpy uint8)."""
+    idx = np.ascontiguousarray(idx, dtype=np.uint8)
+    N, K = idx.shape
+    C = (1 << bits) if C is None else C
+    cb = np.ascontiguousarray(codebook_fp16, dtype=np.float16)
+    if cb.shape != (N, C):
+        raise ValueError("codebook shape")
+    size = packed_weights_bytes(N, K, bits)
+    out = np.empty(size, dtype=np.uint8)
+    bn, bk = c_int64(-1), c_int64(-1)
+    st = lib.lcd_pack_weights(_np_ptr(idx), _np_ptr(cb), N, K, bits, C, _np_ptr(out), size, byref(bn), byref(bk))
+    if st == 4:
+        raise LcdError(st, "lcd_pack_weights", f"at n={bn.value} k={bk.value}")
+    _check(st, "lcd_pack_weights")
+    return out
+
+
+def unpack_weights(blob: np.ndarray):
+    blob = np.ascontiguousarray(blob, dtype=np.uint8)
+    N, K, bits, C = c_int64(), c_int64(), c_int(), c_int()
+    _check(lib.lcd_unpack_weights(_np_ptr(blob), blob.size, None, None, byref(N), byref(K), byref(bits), byref(C)),
+           "lcd_unpack_weights")
+    idx = np.empty((N.value, K.value), dtype=np.uint8)
+    cb = np.empty((N.value, C.value), dtype=np.float16)
+    _check(lib.lcd_unpack_weights(_np_ptr(blob), blob.size, _np_ptr(idx), _np_ptr(cb), byref(N), byref(K),
+                                  byref(bits), byref(C)), "lcd_unpack_weights")
+    return idx, cb, bits.value, C.value
+
+
+# ------------------------------------------------------------------------------------------- device calls
+def _stream_ptr(stream=None) -> c_void_p:
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return c_void_p(s.cuda_stream)
+
+
+class PackedWeights:
+    """A blob resident on the device plus the host copy of its 64-byte header."""
+
+    def __init__(self, blob: np.ndarray, device="cuda"):
+        import torch
+        self.header = bytes(blob[:HEADER_BYTES])
+        self._hdr_buf = ctypes.create_string_buffer(self.header, HEADER_BYTES)
+        f = np.frombuffer(self.header, dtype="<u8")
+        self.N, self.K, self.K_pad = int(f[1]), int(f[2]), int(f[3])
+        u = np.frombuffer(self.header, dtype="<u4")
+        self.bits, self.C = int(u[8]), int(u[9])
+        self.nbytes = int(blob.size)
+        self.dev = torch.from_numpy(np.ascontiguousarray(blob)).to(device)
+        assert self.dev.data_ptr() % 256 == 0
+
+    @property
+    def header_ptr(self) -> c_void_p:
+        return ctypes.cast(self._hdr_buf, c_void_p)
+
+
+def smooth_quantize_act(x, inv_smooth=None, static_scale=None, act_idx=None, act_scale=None, stream=None):
+    """x: CUDA fp16 [M,K] (row stride may exceed K) -> (act_idx uint8 [M,K_pad/2], act_scale fp32 [M])."""
+    import torch
+    assert x.is_cuda and x.dtype == torch.float16 and x.dim() == 2 and x.stride(1) == 1
+    M, K = x.shape
+    K_pad = (K + 255) // 256 * 256
+    if act_idx is None:
+        act_idx = torch.empty((M, K_pad // 2), dtype=torch.uint8, device=x.device)
+    if act_scale is None:
+        act_scale = torch.empty((M,), dtype=torch.float32, device=x.device)
+    st = lib.lcd_smooth_quantize_act(c_void_p(x.data_ptr()), M, K, x.stride(0),
+                                     c_void_p(inv_smooth.data_ptr()) if inv_smooth is not None else None,
+                                     c_void_p(static_scale.data_ptr()) if static_scale is not None else None,
+                                     4, c_void_p(act_idx.data_ptr()), c_void_p(act_scale.data_ptr()),
+                                     _stream_ptr(stream))
+    _check(st, "lcd_smooth_quantize_act")
+    return act_idx, act_scale
+
+
+def lut_linear_workspace_bytes(w: PackedWeights, M: int, algo: int = ALGO_AUTO) -> int:
+    out = c_size_t(0)
+    _check(lib.lcd_lut_linear_workspace_bytes(w.header_ptr, M, algo, byref(out)), "lcd_lut_linear_workspace_bytes")
+    return out.value
+
+
+def lut_linear(w: PackedWeights, act_idx, act_scale, y=None, algo: int = ALGO_AUTO, workspace=None,
+               status_word=None, stream=None):
+    """y[m][n] = s_q[m] * sum_k q[m][k] * cb[n][idx[n][k]]  (CUDA fp32 [M,N])."""
+    import torch
+    M = act_idx.shape[0]
+    if y is None:
+        y = torch.empty((M, w.N), dtype=torch.float32, device=act_idx.device)
+    need = lut_linear_workspace_bytes(w, M, algo)
+    if need and (workspace is None or workspace.numel() * workspace.element_size() < need):
+        workspace = torch.empty(need, dtype=torch.uint8, device=act_idx.device)
+    st = lib.lcd_lut_linear(c_void_p(w.dev.data_ptr()), w.header_ptr, c_void_p(act_idx.data_ptr()),
+                            c_void_p(act_scale.data_ptr()), M, c_void_p(y.data_ptr()), y.stride(0), algo,
+                            c_void_p(workspace.data_ptr()) if workspace is not None else None,
+                            workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                            c_void_p(status_word.data_ptr()) if status_word is not None else None,
+                            _stream_ptr(stream))
+    _check(st, "lcd_lut_linear")
+    return y
+
+
+def linear_host_scratch_bytes(w: PackedWeights, M: int) -> int:
+    out = c_size_t(0)
+    _check(lib.lcd_linear_host_scratch_bytes(w.header_ptr, M, byref(out)), "lcd_linear_host_scratch_bytes")
+    return out.value
+
+
+def linear_host(w: PackedWeights, x_host, inv_smooth, y_host, scratch, stream=None):
+    """x_host: pinned CPU fp16 [M,K]; y_host: pinned CPU fp32 [M,N]; enqueues copies + kernels, no sync."""
+    M = x_host.shape[0]
+    st = lib.lcd_linear_host(c_void_p(w.dev.data_ptr()), w.header_ptr, c_void_p(x_host.data_ptr()), M,
+                             c_void_p(inv_smooth.data_ptr()) if inv_smooth is not None else None,
+                             c_void_p(y_host.data_ptr()), c_void_p(scratch.data_ptr()),
+                             scratch.numel() * scratch.element_size(), _stream_ptr(stream))
+    _check(st, "lcd_linear_host")
+    return y_host

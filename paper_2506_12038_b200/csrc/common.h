@@ -1,0 +1,64 @@
+// Shared declarations of the library's translation units (host side).
+#ifndef LCD_COMMON_H_
+#define LCD_COMMON_H_
+
+#include <cstddef>
+#include <cstdint>
+
+#include "lcd.h"
+
+namespace lcd {
+
+constexpr uint32_t kMagic = 0x5744434Cu;  // "LCDW"
+constexpr uint32_t kVersion = 1;
+constexpr uint32_t kLayoutTile8x256 = 1;
+constexpr uint64_t kIndexOffset = 256;
+constexpr int kTileRows = 8;
+constexpr int kTileK = 256;
+constexpr int kKBlock = 128;
+constexpr bool kHaveBucketLut = false;  // kernels that are not built yet are skipped by LCD_ALGO_AUTO
+constexpr bool kHaveDenseTc = false;
+
+#pragma pack(push, 1)
+struct Header {
+  uint32_t magic, version;
+  uint64_t N, K, K_pad;
+  uint32_t bits, C, layout, checksum;
+  uint64_t index_offset, codebook_offset;
+};
+#pragma pack(pop)
+static_assert(sizeof(Header) == LCD_HEADER_BYTES, "header is 64 bytes");
+
+inline uint64_t round_up_u64(uint64_t v, uint64_t m) { return (v + m - 1) / m * m; }
+
+bool parse_header(const void* header_host, Header* h);
+size_t blob_bytes(uint64_t N, uint64_t K, int bits);
+
+// A resolved view of a problem handed to the kernel launchers.
+struct Problem {
+  const uint8_t* tiles;     // device: index area
+  const uint16_t* codebook; // device: [N_pad][2^bits] fp16 bits
+  int64_t N, K, K_pad, N_pad;
+  int bits, C;
+  const uint8_t* act_idx;   // device [M][K_pad/2]
+  const float* act_scale;   // device [M]
+  int64_t M;
+  float* y;
+  int64_t ldy;
+};
+
+void set_cuda_error(int err);  // records cudaGetErrorString for lcd_last_cuda_error
+
+// kernel launchers (each returns LCD_OK or LCD_ERR_CUDA / LCD_ERR_UNSUPPORTED)
+lcd_status launch_smooth_quantize(const void* x, int64_t M, int64_t K, int64_t ldx, const float* inv_smooth,
+                                  const float* static_scale, uint8_t* act_idx, float* act_scale, void* stream);
+lcd_status launch_reference(const Problem& p, void* stream);
+size_t bucket_lut_workspace_bytes(int64_t N, int64_t K_pad);
+lcd_status launch_bucket_lut(const Problem& p, void* workspace, size_t workspace_bytes, void* stream);
+lcd_status launch_register_lut(const Problem& p, void* stream);
+size_t dense_tc_workspace_bytes(int64_t M, int64_t K_pad);
+lcd_status launch_dense_tc(const Problem& p, void* workspace, size_t workspace_bytes, int32_t* status_word,
+                           void* stream);
+
+}  // namespace lcd
+#endif
