@@ -1,0 +1,373 @@
+#!/usr/bin/env python
+"""Benchmark of the LUT-linear hot path (input transformation -> table lookup -> accumulation) on B200.
+
+One "step" is one pass of the whole hot path over one decoder layer's projections: for every matrix,
+`lcd_smooth_quantize_act` on its input tokens followed by `lcd_lut_linear`.  The default workload is the
+LLaMA-7B-shaped layer at M = 1 with 2-bit weights; the metric is microseconds per layer (lower is better)
+with the matching HBM GB/s on index + codebook + activation bytes.  Weights rotate over several device copies
+(> 256 MB in total) so that L2 cannot serve them.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+
+With --impl reference the CPU oracle is timed instead (a deliberately slow double-precision program).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from synth import gen  # noqa: E402
+
+L2_BYTES = 126e6
+ROTATE_BYTES = 300e6          # total size of the weight copies the timed loop rotates over
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--config", type=int, default=1, help="index into BASELINE.json configs (default 1)")
+    ap.add_argument("--M", type=int, default=None, help="token count (default: first M of the config)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def algorithmic_bytes(N, K, bits, M):
+    """index + codebook + activation-index bytes the method must read for one matrix (no padding, no output)."""
+    return N * K * bits / 8 + N * (1 << bits) * 2 + M * (K / 2 + 4)
+
+
+def build_layers(cfg_id, M):
+    cfg = gen.CONFIGS[cfg_id]
+    layers = []
+    for mi, (name, N, K) in enumerate(cfg["shapes"]):
+        L = gen.make_layer(cfg_id, mi, N, K, cfg["bits"], M, outlier_frac=cfg["frac"], outlier_scale=cfg["scale"])
+        layers.append((name, L))
+    return cfg, layers
+
+
+# ----------------------------------------------------------------------------------------------- oracle
+def oracle_layer_pass(layers):
+    from oracle import lcd_oracle as O
+    outs = []
+    for _, L in layers:
+        q, s = O.smooth_quantize(L.x, L.inv_s)
+        outs.append(O.lut_linear_dequant(L.idx, L.codebook, q, s))
+    return outs
+
+
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        return int(n)
+    except Exception:
+        return 1
+
+
+def oracle_sample(cfg_id, layers, M):
+    """Bounded sample for the CPU legs: whole layer at small M; at large M the first matrix restricted to
+    256 output rows and 64 tokens, scaled to the layer by multiply-accumulate count."""
+    total_macs = sum(L.N * L.K * M for _, L in layers)
+    if M * sum(L.N * L.K for _, L in layers) <= 4e9:
+        return layers, 1.0, f"all {len(layers)} matrices of one layer, M={M}, dequant form"
+    name, L = layers[0]
+    rows, toks = min(256, L.N), min(64, M)
+    import copy
+    S = copy.copy(L)
+    S.idx, S.codebook, S.x, S.N, S.M = L.idx[:rows], L.codebook[:rows], L.x[:toks], rows, toks
+    scale = total_macs / (rows * L.K * toks)
+    return [(name, S)], scale, f"{name}: {rows} output rows x {toks} tokens, scaled x{scale:.0f} by MAC count"
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = gen.CONFIGS[args.config]
+    M = args.M or cfg["Ms"][0]
+    _, layers = build_layers(args.config, M)
+    sample, scale, desc = oracle_sample(args.config, layers, M)
+    for _ in range(min(args.warmup, 1)):
+        oracle_layer_pass(sample)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_layer_pass(sample)
+    dt = (time.perf_counter() - t0) / args.steps * scale
+    us = dt * 1e6
+    cores = oracle_threads()
+    line = {"impl": "reference", "metric": metric_name(M), "value": us, "unit": "us/layer", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(args.config, M, 1),
+            "cpu_baseline": {"value": us, "unit": "us/layer", "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": us, "unit": "us/layer", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def metric_name(M):
+    return "lut_linear_us_per_layer_m%d" % M
+
+
+def workload_config(cfg_id, M, copies):
+    cfg = gen.CONFIGS[cfg_id]
+    return {"workload": f"BASELINE configs[{cfg_id}] {cfg['name']}: " +
+                        ", ".join(f"{n} {N}x{K}" for n, N, K in cfg["shapes"]),
+            "bits": cfg["bits"], "M": M, "act_bits": 4, "outliers": f"{cfg['frac'] * 100:g}% x{cfg['scale']:g}",
+            "l2": f"weights rotate over {copies} device copies (> {int(L2_BYTES / 1e6)} MB L2)"}
+
+
+# ----------------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in out.strip().splitlines():
+            f = [v.strip() for v in ln.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------------- ours
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2506_12038_b200 as lcd
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+
+    cfg = gen.CONFIGS[args.config]
+    M = args.M or cfg["Ms"][0]
+    bits = cfg["bits"]
+    _, layers = build_layers(args.config, M)       # every rank: its own replica of the layer (weak scaling)
+    layer_bytes = sum(lcd.packed_weights_bytes(L.N, L.K, bits) for _, L in layers)
+    copies = max(2, int(np.ceil(ROTATE_BYTES / layer_bytes)))
+
+    mats = []
+    for name, L in layers:
+        blob = lcd.pack_weights(L.idx, L.codebook, bits)
+        ws = [lcd.PackedWeights(blob, dev) for _ in range(copies)]
+        x = torch.from_numpy(L.x).to(dev)
+        inv_s = torch.from_numpy(L.inv_s).to(dev)
+        K_pad = ws[0].K_pad
+        a = torch.empty((M, K_pad // 2), dtype=torch.uint8, device=dev)
+        s = torch.empty((M,), dtype=torch.float32, device=dev)
+        y = torch.empty((M, L.N), dtype=torch.float32, device=dev)
+        wsb = lcd.lut_linear_workspace_bytes(ws[0], M)
+        work = torch.empty(max(wsb, 256), dtype=torch.uint8, device=dev)
+        mats.append(dict(name=name, L=L, w=ws, x=x, inv_s=inv_s, a=a, s=s, y=y, work=work,
+                         bytes=algorithmic_bytes(L.N, L.K, bits, M), flop=2.0 * M * L.N * L.K))
+
+    def step(c):
+        for mt in mats:
+            lcd.smooth_quantize_act(mt["x"], mt["inv_s"], act_idx=mt["a"], act_scale=mt["s"])
+            lcd.lut_linear(mt["w"][c], mt["a"], mt["s"], y=mt["y"], workspace=mt["work"])
+
+    launches_per_step = 2 * len(mats)
+    stream = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(stream):
+        for c in range(copies):
+            step(c)
+        torch.cuda.synchronize()
+        # one CUDA graph per weight copy: the layer's launches back to back, no host gaps
+        graphs = []
+        for c in range(copies):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                step(c)
+            graphs.append(g)
+        for i in range(max(args.warmup, 3)):
+            graphs[i % copies].replay()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        sampler = ClockSampler(local)
+        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(args.steps):
+            graphs[i % copies].replay()
+        e1.record()
+        torch.cuda.synchronize()
+        ms_total = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms_total], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_total = float(t.item())
+            dist.barrier()
+
+        # dominant kernel: lookup+accumulate launches only, per matrix, back to back inside a graph
+        kern_ms, kern_bytes, kern_flop, per_matrix = 0.0, 0.0, 0.0, []
+        reps = 4
+        for mt in mats:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for r in range(reps):
+                    for c in range(copies):
+                        lcd.lut_linear(mt["w"][c], mt["a"], mt["s"], y=mt["y"], workspace=mt["work"])
+            g.replay()
+            torch.cuda.synchronize()
+            k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n_rep = max(3, min(args.steps, 20))
+            k0.record()
+            for _ in range(n_rep):
+                g.replay()
+            k1.record()
+            torch.cuda.synchronize()
+            ms = k0.elapsed_time(k1) / (n_rep * reps * copies)
+            kern_ms += ms
+            kern_bytes += mt["bytes"]
+            kern_flop += mt["flop"]
+            per_matrix.append({"matrix": mt["name"], "N": mt["L"].N, "K": mt["L"].K, "us": ms * 1e3,
+                               "GBps": mt["bytes"] / ms / 1e6, "TFLOPs_equiv": mt["flop"] / ms / 1e9})
+        clocks = sampler.stop()
+
+        # end to end through the host-buffer entry point: pinned host x -> device -> kernels -> pinned host y
+        e2e_ms, h2d, d2h = None, 0, 0
+        host = []
+        for mt in mats:
+            L = mt["L"]
+            xh = torch.from_numpy(L.x).pin_memory()
+            yh = torch.empty((M, L.N), dtype=torch.float32).pin_memory()
+            sc = torch.empty(lcd.linear_host_scratch_bytes(mt["w"][0], M), dtype=torch.uint8, device=dev)
+            host.append((xh, yh, sc))
+            h2d += xh.numel() * 2
+            d2h += yh.numel() * 4
+
+        def e2e_step(c):
+            for mt, (xh, yh, sc) in zip(mats, host):
+                lcd.linear_host(mt["w"][c], xh, mt["inv_s"], yh, sc)
+            torch.cuda.current_stream().synchronize()
+
+        n_e2e = max(3, min(args.steps, 50))
+        for c in range(min(copies, 3)):
+            e2e_step(c)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for i in range(n_e2e):
+            e2e_step(i % copies)
+        g1.record()
+        torch.cuda.synchronize()
+        e2e_ms = max(g0.elapsed_time(g1), (time.perf_counter() - t0) * 1e3) / n_e2e
+        if world > 1:
+            t = torch.tensor([e2e_ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+
+    ms_step = ms_total / args.steps
+    us_per_layer = ms_step * 1e3 / world             # `world` replicas each finish one layer per step
+    layer_alg_bytes = sum(mt["bytes"] for mt in mats)
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    tensor_bound = M > 16
+    if tensor_bound:
+        peak = peaks.get("bf16_tflops", 1590.0)
+        achieved = kern_flop / kern_ms / 1e9
+        roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                "traffic": None, "peak_source": "measured (cuBLAS bf16 burst)" if peaks else "fallback"}
+    else:
+        peak = peaks.get("hbm_gbs", 6650.0)
+        achieved = kern_bytes / kern_ms / 1e6
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "peak_source": "measured (copy)" if peaks else "fallback",
+                "frac_of_8TBps_nominal": achieved / 8000.0}
+    roof["kernel"] = "lcd_lut_linear launches of one layer (sum of bytes / sum of durations)"
+    roof["per_matrix"] = per_matrix
+
+    if rank != 0:
+        return
+    line = {"metric": metric_name(M), "value": us_per_layer, "unit": "us/layer", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "s8 lookups, s32 accumulate, f32 epilogue" if not tensor_bound else "f16 x f16 -> f32",
+            "data": "synthetic", "config": workload_config(args.config, M, copies),
+            "layer_GBps": layer_alg_bytes * world / (ms_step * 1e-3) / 1e9,
+            "layer_algorithmic_bytes": layer_alg_bytes,
+            "TFLOPs_equiv": sum(mt["flop"] for mt in mats) * world / (ms_step * 1e-3) / 1e12,
+            "clocks": clocks, "gpu_launches": launches_per_step * args.steps,
+            "e2e": {"value": e2e_ms * 1e3 / world, "unit": "us/layer", "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h},
+            "roofline": roof}
+    if not args.no_cpu_baseline and world == 1:
+        sample, scale, desc = oracle_sample(args.config, layers, M)
+        t0 = time.perf_counter()
+        n = 0
+        while True:
+            oracle_layer_pass(sample)
+            n += 1
+            if time.perf_counter() - t0 > 10.0 or n >= 5:
+                break
+        us = (time.perf_counter() - t0) / n * scale * 1e6
+        line["cpu_baseline"] = {"value": us, "unit": "us/layer", "cores": oracle_threads(), "kind": "oracle",
+                                "sample": desc + f", mean of {n} passes"}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -188,9 +188,34 @@ __device__ __forceinline__ void kblock(const Tables<BITS>& T, const uint32_t* r,
   }
 }
 
-// grid: persistent CTAs over "rounds"; one round = RGC row groups.  KS * RGC == 8 warps.
+// Persistent CTAs of 8 warps.  Work unit = (row group, column slice); a CTA iteration takes 8 consecutive units,
+// i.e. 8/KS row groups x KS slices, so the slices of a row group meet in the same CTA and are combined through
+// shared memory.  A warp first issues the loads of up to kBatch tiles of its slice (memory-level parallelism),
+// then consumes them.
+constexpr int kBatch = 8;
+
+template <int BITS>
+struct TileRegs {
+  uint32_t w[BITS * 2];   // 2 bit: 4 words (16 B); 3 bit: 6 words (3 x 8 B)
+};
+
+template <int BITS>
+__device__ __forceinline__ TileRegs<BITS> load_tile(const uint8_t* tile, int lane) {
+  TileRegs<BITS> r;
+  if (BITS == 2) {
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(tile + 16 * lane));
+    r.w[0] = v.x; r.w[1] = v.y; r.w[2] = v.z; r.w[3] = v.w;
+  } else {
+    const uint2 a = __ldg(reinterpret_cast<const uint2*>(tile + 8 * lane));
+    const uint2 b = __ldg(reinterpret_cast<const uint2*>(tile + 256 + 8 * lane));
+    const uint2 c = __ldg(reinterpret_cast<const uint2*>(tile + 512 + 8 * lane));
+    r.w[0] = a.x; r.w[1] = b.x; r.w[2] = c.x; r.w[3] = a.y; r.w[4] = b.y; r.w[5] = c.y;
+  }
+  return r;
+}
+
 template <int BITS, int MT>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 2)
 register_lut_kernel(const uint8_t* __restrict__ tiles, const uint16_t* __restrict__ codebook, int64_t N,
                     int64_t n_rg, int n_kt, const uint8_t* __restrict__ act_idx,
                     const float* __restrict__ act_scale, int M, float* __restrict__ y, int64_t ldy, int KS,
@@ -211,19 +236,34 @@ register_lut_kernel(const uint8_t* __restrict__ tiles, const uint16_t* __restric
     selU0 |= (uint32_t)((j - g) & 7) << (4 * j);
     selU1 |= (uint32_t)((4 + j - g) & 7) << (4 * j);
   }
+  const int slice_tiles = (n_kt + KS - 1) / KS;
   const int64_t n_rounds = (n_rg + RGC - 1) / RGC;
   bool staged = false;
   for (int64_t round = blockIdx.x; round < n_rounds; round += gridDim.x) {
     const int64_t rg = round * RGC + rgi;
     const bool active = rg < n_rg;
-    Tables<BITS> T;
-    if (active) T = build_tables<BITS>(codebook + (rg * 8 + g) * (1 << BITS));
+    const uint8_t* row_tiles = tiles + (size_t)(active ? rg : 0) * n_kt * TILE_BYTES;
     int accH[MT], accL[MT];
 #pragma unroll
     for (int m = 0; m < MT; ++m) accH[m] = accL[m] = 0;
+    Tables<BITS> T;
+    bool have_tables = false;
     for (int c = 0; c < n_chunks; ++c) {
       const int kt0 = c * chunk_tiles;
       const int kt1 = min(n_kt, kt0 + chunk_tiles);
+      // this warp's tiles inside the chunk
+      const int my0 = max(kt0, ks * slice_tiles), my1 = min(kt1, min(n_kt, (ks + 1) * slice_tiles));
+      TileRegs<BITS> buf[kBatch];
+      int kt = my0;
+      if (active) {
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b)
+          if (kt + b < my1) buf[b] = load_tile<BITS>(row_tiles + (size_t)(kt + b) * TILE_BYTES, lane);
+      }
+      if (active && !have_tables) {
+        T = build_tables<BITS>(codebook + (rg * 8 + g) * (1 << BITS));
+        have_tables = true;
+      }
       if (n_chunks > 1 || !staged) {
         __syncthreads();
 #pragma unroll
@@ -234,22 +274,25 @@ register_lut_kernel(const uint8_t* __restrict__ tiles, const uint16_t* __restric
         staged = true;
       }
       if (active) {
-        const uint8_t* row_tiles = tiles + (size_t)rg * n_kt * TILE_BYTES;
-        for (int kt = kt0 + ks; kt < kt1; kt += KS) {
-          const uint8_t* tile = row_tiles + (size_t)kt * TILE_BYTES;
-          const uint32_t* q_tile = q_s + (size_t)(kt - kt0) * (kTileK / 4) + t * 8;
-          if (BITS == 2) {
-            const uint4 w = *reinterpret_cast<const uint4*>(tile + 16 * lane);
-            const uint32_t r0[2] = {w.x, w.y}, r1[2] = {w.z, w.w};
-            kblock<BITS, MT>(T, r0, q_tile, chunk_words, selU0, selU1, accH, accL);
-            kblock<BITS, MT>(T, r1, q_tile + kKBlock / 4, chunk_words, selU0, selU1, accH, accL);
-          } else {
-            const uint2 w0 = *reinterpret_cast<const uint2*>(tile + 8 * lane);
-            const uint2 w1 = *reinterpret_cast<const uint2*>(tile + 256 + 8 * lane);
-            const uint2 w2 = *reinterpret_cast<const uint2*>(tile + 512 + 8 * lane);
-            const uint32_t r0[3] = {w0.x, w1.x, w2.x}, r1[3] = {w0.y, w1.y, w2.y};
-            kblock<BITS, MT>(T, r0, q_tile, chunk_words, selU0, selU1, accH, accL);
-            kblock<BITS, MT>(T, r1, q_tile + kKBlock / 4, chunk_words, selU0, selU1, accH, accL);
+        while (kt < my1) {
+#pragma unroll
+          for (int b = 0; b < kBatch; ++b) {
+            if (kt + b < my1) {
+              const uint32_t* q_tile = q_s + (size_t)(kt + b - kt0) * (kTileK / 4) + t * 8;
+              if (BITS == 2) {
+                kblock<BITS, MT>(T, &buf[b].w[0], q_tile, chunk_words, selU0, selU1, accH, accL);
+                kblock<BITS, MT>(T, &buf[b].w[2], q_tile + kKBlock / 4, chunk_words, selU0, selU1, accH, accL);
+              } else {
+                kblock<BITS, MT>(T, &buf[b].w[0], q_tile, chunk_words, selU0, selU1, accH, accL);
+                kblock<BITS, MT>(T, &buf[b].w[3], q_tile + kKBlock / 4, chunk_words, selU0, selU1, accH, accL);
+              }
+            }
+          }
+          kt += kBatch;
+          if (kt < my1) {
+#pragma unroll
+            for (int b = 0; b < kBatch; ++b)
+              if (kt + b < my1) buf[b] = load_tile<BITS>(row_tiles + (size_t)(kt + b) * TILE_BYTES, lane);
           }
         }
       }
@@ -262,25 +305,33 @@ register_lut_kernel(const uint8_t* __restrict__ tiles, const uint16_t* __restric
       accH[m] += __shfl_xor_sync(0xffffffffu, accH[m], 2);
       accL[m] += __shfl_xor_sync(0xffffffffu, accL[m], 2);
     }
-    __syncthreads();   // red_s free again (previous round's readers are done)
-    if (t == 0) {
+    if (KS > 1) {
+      __syncthreads();   // red_s free again (previous round's readers are done)
+      if (t == 0) {
 #pragma unroll
-      for (int m = 0; m < MT; ++m) {
-        red_s[((warp * MT + m) * 8 + g) * 2 + 0] = active ? accH[m] : 0;
-        red_s[((warp * MT + m) * 8 + g) * 2 + 1] = active ? accL[m] : 0;
+        for (int m = 0; m < MT; ++m) {
+          red_s[((warp * MT + m) * 8 + g) * 2 + 0] = active ? accH[m] : 0;
+          red_s[((warp * MT + m) * 8 + g) * 2 + 1] = active ? accL[m] : 0;
+        }
       }
+      __syncthreads();
     }
-    __syncthreads();
     // warps with ks == 0 finish their row group: lane (g,t) handles tokens t, t+4, ...
     if (ks == 0 && active) {
       const int64_t n = rg * 8 + g;
-      for (int m = t; m < M; m += 4) {
-        int h = 0, l = 0;
-        for (int s = 0; s < KS; ++s) {
-          h += red_s[(((rgi * KS + s) * MT + m) * 8 + g) * 2 + 0];
-          l += red_s[(((rgi * KS + s) * MT + m) * 8 + g) * 2 + 1];
+#pragma unroll
+      for (int m = 0; m < MT; ++m) {
+        if ((m & 3) == t && m < M) {
+          int h = accH[m], l = accL[m];
+          if (KS > 1) {
+            h = 0; l = 0;
+            for (int s = 0; s < KS; ++s) {
+              h += red_s[(((rgi * KS + s) * MT + m) * 8 + g) * 2 + 0];
+              l += red_s[(((rgi * KS + s) * MT + m) * 8 + g) * 2 + 1];
+            }
+          }
+          if (n < N) y[(size_t)m * ldy + n] = act_scale[m] * T.scale * ((float)h * 256.0f + (float)l);
         }
-        if (n < N) y[(size_t)m * ldy + n] = act_scale[m] * T.scale * ((float)h * 256.0f + (float)l);
       }
     }
   }
@@ -290,9 +341,18 @@ template <int BITS, int MT>
 lcd_status launch_t(const Problem& p, cudaStream_t stream) {
   const int n_kt = (int)(p.K_pad / kTileK);
   const int64_t n_rg = p.N_pad / kTileRows;
-  // column slices per CTA: enough CTAs to fill the machine, at least ~4 tiles per warp when possible
+  // column slices per row group: minimise (waves of CTAs) x (tiles per slice + one tile of fixed cost)
   int KS = 1;
-  while (KS < 8 && (n_rg / (kWarps / KS)) < 2 * 148 && n_kt / (KS * 2) >= 2) KS *= 2;
+  {
+    int64_t best = -1;
+    for (int cand = 1; cand <= 8; cand *= 2) {
+      const int slice = (n_kt + cand - 1) / cand;
+      if (cand > 1 && slice < 2) break;
+      const int64_t rounds = (n_rg + kWarps / cand - 1) / (kWarps / cand);
+      const int64_t cost = ((rounds + 295) / 296) * (slice + 1);
+      if (best < 0 || cost < best) { best = cost; KS = cand; }
+    }
+  }
   const size_t red_bytes = (size_t)kWarps * MT * 8 * 2 * sizeof(int);
   int chunk_tiles = n_kt;
   const size_t per_tile = (size_t)MT * kTileK;
@@ -309,7 +369,7 @@ lcd_status launch_t(const Problem& p, cudaStream_t stream) {
   const int RGC = kWarps / KS;
   const int64_t n_rounds = (n_rg + RGC - 1) / RGC;
   int per_sm = (int)((size_t)(220 * 1024) / (smem + 1024));
-  per_sm = per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm);
+  per_sm = per_sm < 1 ? 1 : (per_sm > 2 ? 2 : per_sm);
   const int64_t grid = n_rounds < (int64_t)148 * per_sm ? n_rounds : (int64_t)148 * per_sm;
   kern<<<(unsigned)grid, kThreads, smem, stream>>>(p.tiles, p.codebook, p.N, n_rg, n_kt, p.act_idx, p.act_scale,
                                                    (int)p.M, p.y, p.ldy, KS, chunk_tiles, n_chunks);
