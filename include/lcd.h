@@ -41,21 +41,22 @@ typedef enum {
 
 /* Which kernel family lcd_lut_linear uses.  Every family computes the same y. */
 typedef enum {
-  LCD_ALGO_AUTO = 0,        /* choose by (M, bits): see lcd_lut_linear                                        */
+  LCD_ALGO_AUTO = 0,        /* REGISTER_LUT for M <= 16, DENSE_TC above                                        */
   LCD_ALGO_REFERENCE = 1,   /* plain per-weight lookup cb[n][idx] and multiply-accumulate; any M, slow        */
-  LCD_ALGO_BUCKET_LUT = 2,  /* Section 4.2 centroid-stationary buckets: shared-memory tables built from the   */
-                            /* token's activation levels return, per byte of four weight indices, the partial */
-                            /* per-centroid activation sums; exact int32 bucket sums dotted with the codebook  */
-                            /* at the end.  M == 1, bits == 2.                                                 */
-  LCD_ALGO_REGISTER_LUT = 3,/* Section 4.2 lookup with the row codebook held as a byte table in registers      */
-                            /* (fixed-point, 16 bit), four weights looked up per instruction, accumulated as    */
-                            /* integer dot products with the activation levels.  M <= 16.                      */
+  LCD_ALGO_BUCKET_LUT = 2,  /* Section 4.2 centroid-stationary buckets: per output and per centroid w the exact */
+                            /* integer sum S_w of the activation levels whose weight index is w (one-hot byte   */
+                            /* tables looked up four weights at a time, accumulated by int8 tensor-core MMAs),   */
+                            /* then y = s_q * sum_w cb[w] * S_w: 2^bits multiplies per output.  M <= 16.         */
+  LCD_ALGO_REGISTER_LUT = 3,/* Section 4.2 lookup with the row codebook held as byte tables in registers        */
+                            /* (16-bit fixed point, high and low byte), four weights looked up per instruction,  */
+                            /* accumulated by int8 tensor-core MMAs against the activation levels.  M <= 16.     */
   LCD_ALGO_DENSE_TC = 4     /* batched prefill: indices decoded through the codebook into fp16 shared-memory   */
                             /* tiles feeding tcgen05 tensor cores with fp32 accumulators in tensor memory.      */
 } lcd_algo;
 
 #define LCD_HEADER_BYTES 64
 #define LCD_ACT_BITS 4
+#define LCD_MAX_BATCH 8   /* problems per grouped call */
 
 const char* lcd_status_string(lcd_status s);
 /* Text of the last CUDA error this library saw on the calling thread ("" if none). */
@@ -68,16 +69,15 @@ const char* lcd_last_cuda_error(void);
  *
  * Blob = 64-byte header | zero padding to 256 | index area | codebook area.
  *   header (little endian): u32 magic 'LCDW', u32 version 1, u64 N, u64 K, u64 K_pad, u32 bits, u32 C,
- *     u32 layout (1), u32 checksum (sum of all bytes after the header, mod 2^32), u64 index_offset (256),
+ *     u32 layout (2), u32 checksum (sum of all bytes after the header, mod 2^32), u64 index_offset (256),
  *     u64 codebook_offset.
- *   index area: rows padded to N_pad = 8*ceil(N/8), columns to K_pad = 256*ceil(K/256) with index 0,
- *     cut into tiles of 8 rows x 256 columns stored row-group major: tile (rg, kt) starts at
- *     index_offset + (rg*(K_pad/256) + kt)*T with T = 512 (2 bit) or 768 (3 bit) bytes.  Inside a tile,
- *     lane l = 4*g + t (g = row 0..7, t = quarter 0..3) owns columns 128*h + 32*t .. +31 of row g for
- *     both 128-column k-blocks h = 0,1 of the tile:
+ *   index area: rows padded to N_pad = 16*ceil(N/16), columns to K_pad = 256*ceil(K/256) with index 0,
+ *     cut into items of 16 rows x 256 columns stored row-group major: item (rp, kt) starts at
+ *     index_offset + (rp*(K_pad/256) + kt)*2T and is two tiles of T = 512 (2 bit) or 768 (3 bit) bytes, rows
+ *     16rp..16rp+7 then rows 16rp+8..16rp+15.  Inside a tile, lane l = 4*g + t (g = row 0..7, t = quarter
+ *     0..3) owns columns 128*h + 32*t .. +31 of row g for both 128-column k-blocks h = 0,1 of the tile:
  *       2 bit: 16 bytes at tile + 16*l; bytes [8h, 8h+8) belong to k-block h; byte p of those holds the
- *              four columns 128h + 4G + i (i = 0..3, at bits [2i,2i+2)) of k-group G = 8t + ((p+g) mod 8).
- *              (The rotation by g lets 32 lanes read 32 different shared-memory banks of the bucket tables.)
+ *              four columns 128h + 32t + 4p + i (i = 0..3, at bits [2i,2i+2)).
  *       3 bit: three 256-byte planes; plane b has, at plane + 8*l + 4*h, word b of the lane's 12-byte
  *              record of k-block h.  A record packs columns 128h + 32t + m: m = 8i+j (i < 3) at bits
  *              [4j, 4j+3) of word i; m = 24+j has bit b of its index at bit 4j+3 of word b.
@@ -122,18 +122,39 @@ lcd_status lcd_smooth_quantize_act(const void* x_fp16, int64_t M, int64_t K, int
                                    const float* inv_smooth, const float* static_scale, int act_bits,
                                    uint8_t* act_idx, float* act_scale, void* cuda_stream);
 
+/* The same transformation for up to LCD_MAX_BATCH independent activation matrices (the inputs of the
+ * projections of one decoder layer) in one launch.  Fields as the arguments of lcd_smooth_quantize_act. */
+typedef struct {
+  const void* x_fp16;        /* device */
+  int64_t M, K, ldx;
+  const float* inv_smooth;   /* device or NULL */
+  const float* static_scale; /* device or NULL */
+  uint8_t* act_idx;          /* device out */
+  float* act_scale;          /* device out */
+} lcd_act_problem;
+
+lcd_status lcd_smooth_quantize_act_batch(const lcd_act_problem* problems /* host */, int count, int act_bits,
+                                         void* cuda_stream);
+
 /* ----------------------------------------------------------------------------------------------
  * Online steps 2+3: table lookup and accumulation (Section 4.2).
  *   packed_weights_dev: device, the blob, 256-byte aligned;
  *   header_host:        host, the blob's first 64 bytes;
  *   act_idx, act_scale: device, as written by lcd_smooth_quantize_act for the same K;
  *   y:                  device out, fp32 [M][ldy], ldy >= N;
- *   algo:               LCD_ALGO_AUTO picks BUCKET_LUT for (M == 1, 2 bit), REGISTER_LUT for other M <= 16,
- *                       DENSE_TC for M > 16; a family asked for outside its range => LCD_ERR_UNSUPPORTED;
+ *   algo:               LCD_ALGO_AUTO picks REGISTER_LUT for M <= 16 and DENSE_TC above; a family asked for
+ *                       outside its range => LCD_ERR_UNSUPPORTED;
  *   workspace:          device scratch of at least lcd_lut_linear_workspace_bytes(...) bytes, 256-byte
- *                       aligned, contents undefined before and after (may be NULL when that size is 0);
+ *                       aligned (may be NULL when that size is 0).  REGISTER_LUT and BUCKET_LUT keep integer
+ *                       partial sums and arrival counters there: the caller zero-fills it once before its
+ *                       first use, every call that completes leaves it zero-filled again, and two calls that
+ *                       may overlap on the device need separate workspaces.  The other families do not care
+ *                       about its contents;
  *   status_word_dev:    device int32 or NULL; receives LCD_ERR_TIMEOUT if a bounded device-side wait
- *                       expired (the output is then invalid); never written otherwise.
+ *                       expired (the output is then invalid and the workspace must be zero-filled again);
+ *                       never written otherwise.
+ * The M <= 16 kernels are launched with programmatic stream serialization: they begin streaming weights
+ * while the previous kernel of the stream finishes and wait for it before reading act_idx / act_scale.
  * -------------------------------------------------------------------------------------------- */
 lcd_status lcd_lut_linear_workspace_bytes(const void* header_host, int64_t M, lcd_algo algo, size_t* bytes);
 
@@ -141,6 +162,27 @@ lcd_status lcd_lut_linear(const void* packed_weights_dev, const void* header_hos
                           const float* act_scale, int64_t M, float* y, int64_t ldy, lcd_algo algo,
                           void* workspace, size_t workspace_bytes, int32_t* status_word_dev,
                           void* cuda_stream);
+
+/* Up to LCD_MAX_BATCH independent problems with M <= 16 (e.g. the q/k/v or gate/up projections of a decoder
+ * layer, or all projections of a layer when their inputs are independent) in ONE launch: the SMs are divided
+ * among the problems in proportion to their index bytes.  All problems must have the same index width.
+ * algo: AUTO, REGISTER_LUT or BUCKET_LUT.  Workspace rules as for lcd_lut_linear. */
+typedef struct {
+  const void* packed_weights_dev; /* device, 256-byte aligned */
+  const void* header_host;        /* host */
+  const uint8_t* act_idx;         /* device */
+  const float* act_scale;         /* device */
+  int64_t M;
+  float* y;                       /* device out, fp32 [M][ldy] */
+  int64_t ldy;
+} lcd_linear_problem;
+
+lcd_status lcd_lut_linear_batch_workspace_bytes(const lcd_linear_problem* problems /* host */, int count,
+                                                lcd_algo algo, size_t* bytes);
+
+lcd_status lcd_lut_linear_batch(const lcd_linear_problem* problems /* host */, int count, lcd_algo algo,
+                                void* workspace, size_t workspace_bytes, int32_t* status_word_dev,
+                                void* cuda_stream);
 
 /* ----------------------------------------------------------------------------------------------
  * The whole online path (Section 4: input transformation -> bucket table lookup -> accumulation) from
@@ -150,7 +192,8 @@ lcd_status lcd_lut_linear(const void* packed_weights_dev, const void* header_hos
  * valid after the stream is synchronised.  x_host / y_host should be pinned for the copies to be async.
  *   x_host_fp16: host, binary16 [M][K] dense;   y_host: host out, fp32 [M][N] dense;
  *   inv_smooth:  device fp32 [K] or NULL;
- *   scratch:     device, >= lcd_linear_host_scratch_bytes(...) bytes, 256-byte aligned.
+ *   scratch:     device, >= lcd_linear_host_scratch_bytes(...) bytes, 256-byte aligned, contents undefined
+ *                (the call clears the part the lookup kernel needs zeroed).
  * -------------------------------------------------------------------------------------------- */
 lcd_status lcd_linear_host_scratch_bytes(const void* header_host, int64_t M, size_t* bytes);
 

@@ -44,10 +44,11 @@ QMIN, QMAX = -8, 7            # 4-bit symmetric range [-2^(b-1), 2^(b-1)-1], b =
 LEVELS = 16
 MAGIC = 0x5744434C            # "LCDW"
 VERSION = 1
-LAYOUT_TILE8X256 = 1
+LAYOUT_PAIR16X256 = 2
 HEADER_BYTES = 64
 INDEX_OFFSET = 256
-TILE_ROWS = 8
+TILE_ROWS = 8              # rows of one tile
+PAIR_ROWS = 16             # two tiles (rows 0-7, rows 8-15) form one 16-row item
 TILE_K = 256
 KBLOCK = 128
 
@@ -220,10 +221,10 @@ def lut_linear_rows(idx, codebook_fp16, q, s_q, rows: np.ndarray) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------------------
-# Packed-weight blob (layout id 1, "tile8x256")
+# Packed-weight blob (layout id 2, "pair16x256")
 # --------------------------------------------------------------------------------------
 def packed_weights_bytes(N: int, K: int, bits: int) -> int:
-    N_pad, K_pad = round_up(N, TILE_ROWS), round_up(K, TILE_K)
+    N_pad, K_pad = round_up(N, PAIR_ROWS), round_up(K, TILE_K)
     idx_bytes = N_pad * K_pad * bits // 8
     cb_off = round_up(INDEX_OFFSET + idx_bytes, 256)
     return cb_off + round_up(N_pad * (1 << bits) * 2, 256)
@@ -234,7 +235,7 @@ def _tile_lane_bytes_2bit(rows_idx: np.ndarray, g: int, t: int) -> np.ndarray:
     out = np.zeros(16, dtype=np.uint8)
     for half in range(2):                 # k-block 0 / 1 of the tile
         for p in range(8):                # byte position inside the 8-byte quarter record
-            G = 8 * t + ((p + g) % 8)     # k-group (4 consecutive k) inside the k-block, rotated by g
+            G = 8 * t + p                 # k-group (4 consecutive k) inside the k-block
             b = 0
             for i in range(4):
                 k = KBLOCK * half + 4 * G + i
@@ -261,16 +262,17 @@ def pack_weights(idx: np.ndarray, codebook_fp16: np.ndarray, bits: int, C: int |
     """Build the blob (uint8 array).
 
     Header, 64 bytes little-endian:  u32 magic "LCDW", u32 version=1, u64 N, u64 K, u64 K_pad,
-    u32 bits, u32 C, u32 layout=1, u32 checksum (sum of all payload bytes mod 2^32),
+    u32 bits, u32 C, u32 layout=2, u32 checksum (sum of all payload bytes mod 2^32),
     u64 index_offset (=256), u64 codebook_offset.  Bytes 64..255 are zero.
 
-    Index area: rows padded to N_pad = 8*ceil(N/8), columns to K_pad = 256*ceil(K/256), padding
-    index 0.  Tiles of 8 rows x 256 columns, tile (rg, kt) at index_offset + (rg*(K_pad/256)+kt)*T,
-    T = 512 bytes (2 bit) or 768 bytes (3 bit).  Lane l = 4*g + t (g = 0..7 row inside the tile,
-    t = 0..3 quarter) owns, for each of the tile's two 128-column k-blocks h, the 32 columns
-    128*h + 32*t .. +31 of row g.
+    Index area: rows padded to N_pad = 16*ceil(N/16), columns to K_pad = 256*ceil(K/256), padding
+    index 0.  Tiles of 8 rows x 256 columns of T = 512 bytes (2 bit) or 768 bytes (3 bit); the two
+    tiles of a 16-row group rp (rows 16rp..16rp+7, then 16rp+8..16rp+15) are adjacent and form one
+    item: tile (rg, kt), rg = 2*rp + u, is at index_offset + (rp*(K_pad/256) + kt)*2T + u*T.
+    Lane l = 4*g + t (g = 0..7 row inside the tile, t = 0..3 quarter) owns, for each of the tile's
+    two 128-column k-blocks h, the 32 columns 128*h + 32*t .. +31 of row g.
       2 bit: lane record = 16 bytes at tile + 16*l: bytes [8h, 8h+8) are k-block h.  Byte p of those
-             holds k-group G = 8t + ((p+g) mod 8): columns 128h + 4G + i at bits [2i, 2i+2).
+             holds columns 128h + 32t + 4p + i at bits [2i, 2i+2) (plain little-endian packing).
       3 bit: the tile is three 256-byte planes; plane b holds, at plane + 8*l, word b of the lane's
              record for k-block 0 then word b of its record for k-block 1.  A record packs the 32
              columns 128h + 32t + m: m = 8i+j (i<3) in bits [4j,4j+3) of word i; m = 24+j has its bit b
@@ -286,7 +288,7 @@ def pack_weights(idx: np.ndarray, codebook_fp16: np.ndarray, bits: int, C: int |
         raise ValueError("index out of range")
     cb = np.asarray(codebook_fp16, dtype=np.float16)
     assert cb.shape == (N, C)
-    N_pad, K_pad = round_up(N, TILE_ROWS), round_up(K, TILE_K)
+    N_pad, K_pad = round_up(N, PAIR_ROWS), round_up(K, TILE_K)
     total = packed_weights_bytes(N, K, bits)
     blob = np.zeros(total, dtype=np.uint8)
     P = np.zeros((N_pad, K_pad), dtype=np.uint8)
@@ -296,7 +298,7 @@ def pack_weights(idx: np.ndarray, codebook_fp16: np.ndarray, bits: int, C: int |
     for rg in range(N_pad // TILE_ROWS):
         for kt in range(n_kt):
             sub = P[rg * 8:(rg + 1) * 8, kt * TILE_K:(kt + 1) * TILE_K]
-            base = INDEX_OFFSET + (rg * n_kt + kt) * tile_bytes
+            base = INDEX_OFFSET + ((rg // 2) * n_kt + kt) * 2 * tile_bytes + (rg % 2) * tile_bytes
             for g in range(8):
                 for t in range(4):
                     lane = 4 * g + t
@@ -313,7 +315,7 @@ def pack_weights(idx: np.ndarray, codebook_fp16: np.ndarray, bits: int, C: int |
     cbp[:N, :C] = cb
     blob[cb_off:cb_off + cbp.size * 2] = cbp.view(np.uint8).reshape(-1)
     checksum = int(blob[HEADER_BYTES:].astype(np.uint64).sum()) & 0xFFFFFFFF
-    hdr = struct.pack("<IIQQQIIIIQQ", MAGIC, VERSION, N, K, K_pad, bits, C, LAYOUT_TILE8X256, checksum,
+    hdr = struct.pack("<IIQQQIIIIQQ", MAGIC, VERSION, N, K, K_pad, bits, C, LAYOUT_PAIR16X256, checksum,
                       INDEX_OFFSET, cb_off)
     assert len(hdr) == HEADER_BYTES
     blob[:HEADER_BYTES] = np.frombuffer(hdr, dtype=np.uint8)
@@ -330,18 +332,18 @@ def parse_header(blob: np.ndarray) -> dict:
 def unpack_weights(blob: np.ndarray):
     """Exact inverse of ``pack_weights``: returns (idx uint8 [N,K], codebook fp16 [N,C], bits, C)."""
     h = parse_header(blob)
-    if h["magic"] != MAGIC or h["version"] != VERSION or h["layout"] != LAYOUT_TILE8X256:
+    if h["magic"] != MAGIC or h["version"] != VERSION or h["layout"] != LAYOUT_PAIR16X256:
         raise ValueError("bad blob header")
     if (int(blob[HEADER_BYTES:].astype(np.uint64).sum()) & 0xFFFFFFFF) != h["checksum"]:
         raise ValueError("bad blob checksum")
     N, K, K_pad, bits, C = h["N"], h["K"], h["K_pad"], h["bits"], h["C"]
-    N_pad = round_up(N, TILE_ROWS)
+    N_pad = round_up(N, PAIR_ROWS)
     tile_bytes = TILE_ROWS * TILE_K * bits // 8
     n_kt = K_pad // TILE_K
     P = np.zeros((N_pad, K_pad), dtype=np.uint8)
     for rg in range(N_pad // TILE_ROWS):
         for kt in range(n_kt):
-            base = h["index_offset"] + (rg * n_kt + kt) * tile_bytes
+            base = h["index_offset"] + ((rg // 2) * n_kt + kt) * 2 * tile_bytes + (rg % 2) * tile_bytes
             for g in range(8):
                 for t in range(4):
                     lane = 4 * g + t
@@ -349,7 +351,7 @@ def unpack_weights(blob: np.ndarray):
                         k0 = kt * TILE_K + KBLOCK * hb
                         if bits == 2:
                             for p in range(8):
-                                G = 8 * t + ((p + g) % 8)
+                                G = 8 * t + p
                                 b = int(blob[base + 16 * lane + 8 * hb + p])
                                 for i in range(4):
                                     P[rg * 8 + g, k0 + 4 * G + i] = (b >> (2 * i)) & 3

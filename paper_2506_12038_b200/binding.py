@@ -8,7 +8,7 @@ from __future__ import annotations
 
 import ctypes
 import os
-from ctypes import c_char_p, c_int, c_int32, c_int64, c_size_t, c_void_p, POINTER, byref
+from ctypes import c_char_p, c_int, c_int64, c_size_t, c_void_p, POINTER, Structure, byref
 
 import numpy as np
 
@@ -20,10 +20,24 @@ STATUS_NAMES = {0: "LCD_OK", 1: "LCD_ERR_INVALID_ARG", 2: "LCD_ERR_UNSUPPORTED",
                 4: "LCD_ERR_INDEX_RANGE", 5: "LCD_ERR_BAD_BLOB", 6: "LCD_ERR_CUDA", 7: "LCD_ERR_TIMEOUT"}
 ALGO_AUTO, ALGO_REFERENCE, ALGO_BUCKET_LUT, ALGO_REGISTER_LUT, ALGO_DENSE_TC = 0, 1, 2, 3, 4
 HEADER_BYTES = 64
+MAX_BATCH = 8
 
 EXPORTS = ["lcd_status_string", "lcd_last_cuda_error", "lcd_packed_weights_bytes", "lcd_pack_weights",
            "lcd_unpack_weights", "lcd_smooth_quantize_act", "lcd_lut_linear_workspace_bytes", "lcd_lut_linear",
-           "lcd_linear_host_scratch_bytes", "lcd_linear_host"]
+           "lcd_linear_host_scratch_bytes", "lcd_linear_host", "lcd_smooth_quantize_act_batch",
+           "lcd_lut_linear_batch_workspace_bytes", "lcd_lut_linear_batch"]
+
+
+class ActProblem(Structure):
+    """lcd_act_problem"""
+    _fields_ = [("x_fp16", c_void_p), ("M", c_int64), ("K", c_int64), ("ldx", c_int64), ("inv_smooth", c_void_p),
+                ("static_scale", c_void_p), ("act_idx", c_void_p), ("act_scale", c_void_p)]
+
+
+class LinearProblem(Structure):
+    """lcd_linear_problem"""
+    _fields_ = [("packed_weights_dev", c_void_p), ("header_host", c_void_p), ("act_idx", c_void_p),
+                ("act_scale", c_void_p), ("M", c_int64), ("y", c_void_p), ("ldy", c_int64)]
 
 
 class LcdError(RuntimeError):
@@ -53,6 +67,9 @@ def _load() -> ctypes.CDLL:
     lib.lcd_linear_host_scratch_bytes.argtypes = [c_void_p, c_int64, POINTER(c_size_t)]
     lib.lcd_linear_host.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_size_t,
                                     c_void_p]
+    lib.lcd_smooth_quantize_act_batch.argtypes = [POINTER(ActProblem), c_int, c_int, c_void_p]
+    lib.lcd_lut_linear_batch_workspace_bytes.argtypes = [POINTER(LinearProblem), c_int, c_int, POINTER(c_size_t)]
+    lib.lcd_lut_linear_batch.argtypes = [POINTER(LinearProblem), c_int, c_int, c_void_p, c_size_t, c_void_p, c_void_p]
     for name in EXPORTS:
         if name not in ("lcd_status_string", "lcd_last_cuda_error"):
             getattr(lib, name).restype = c_int
@@ -170,7 +187,7 @@ def lut_linear(w: PackedWeights, act_idx, act_scale, y=None, algo: int = ALGO_AU
         y = torch.empty((M, w.N), dtype=torch.float32, device=act_idx.device)
     need = lut_linear_workspace_bytes(w, M, algo)
     if need and (workspace is None or workspace.numel() * workspace.element_size() < need):
-        workspace = torch.empty(need, dtype=torch.uint8, device=act_idx.device)
+        workspace = torch.zeros(need, dtype=torch.uint8, device=act_idx.device)   # must start zero-filled
     st = lib.lcd_lut_linear(c_void_p(w.dev.data_ptr()), w.header_ptr, c_void_p(act_idx.data_ptr()),
                             c_void_p(act_scale.data_ptr()), M, c_void_p(y.data_ptr()), y.stride(0), algo,
                             c_void_p(workspace.data_ptr()) if workspace is not None else None,
@@ -179,6 +196,52 @@ def lut_linear(w: PackedWeights, act_idx, act_scale, y=None, algo: int = ALGO_AU
                             _stream_ptr(stream))
     _check(st, "lcd_lut_linear")
     return y
+
+
+class ActBatch:
+    """Up to MAX_BATCH activation matrices quantised by one launch.  items: (x, inv_smooth, act_idx, act_scale)
+    CUDA tensors (inv_smooth may be None); the argument array is built once and reused by run()."""
+
+    def __init__(self, items):
+        self._keep = list(items)
+        self.count = len(self._keep)
+        self.arr = (ActProblem * self.count)()
+        for a, (x, inv_s, idx, scale) in zip(self.arr, self._keep):
+            a.x_fp16, a.M, a.K, a.ldx = x.data_ptr(), x.shape[0], x.shape[1], x.stride(0)
+            a.inv_smooth = inv_s.data_ptr() if inv_s is not None else None
+            a.static_scale = None
+            a.act_idx, a.act_scale = idx.data_ptr(), scale.data_ptr()
+
+    def run(self, stream=None):
+        _check(lib.lcd_smooth_quantize_act_batch(self.arr, self.count, 4, _stream_ptr(stream)),
+               "lcd_smooth_quantize_act_batch")
+
+
+class LinearBatch:
+    """Up to MAX_BATCH independent lookup problems (M <= 16, same index width) run by one launch.
+    items: (PackedWeights, act_idx, act_scale, y) with CUDA tensors; the zero-filled workspace is owned here."""
+
+    def __init__(self, items, algo: int = ALGO_AUTO, status_word=None):
+        import torch
+        self._keep = list(items)
+        self.count = len(self._keep)
+        self.algo = algo
+        self.arr = (LinearProblem * self.count)()
+        for a, (w, idx, scale, y) in zip(self.arr, self._keep):
+            a.packed_weights_dev, a.header_host = w.dev.data_ptr(), w.header_ptr
+            a.act_idx, a.act_scale, a.M = idx.data_ptr(), scale.data_ptr(), idx.shape[0]
+            a.y, a.ldy = y.data_ptr(), y.stride(0)
+        need = c_size_t(0)
+        _check(lib.lcd_lut_linear_batch_workspace_bytes(self.arr, self.count, algo, byref(need)),
+               "lcd_lut_linear_batch_workspace_bytes")
+        self.workspace = torch.zeros(max(need.value, 256), dtype=torch.uint8, device=self._keep[0][1].device)
+        self.status_word = status_word
+
+    def run(self, stream=None):
+        _check(lib.lcd_lut_linear_batch(self.arr, self.count, self.algo, c_void_p(self.workspace.data_ptr()),
+                                        self.workspace.numel(),
+                                        c_void_p(self.status_word.data_ptr()) if self.status_word is not None else None,
+                                        _stream_ptr(stream)), "lcd_lut_linear_batch")
 
 
 def linear_host_scratch_bytes(w: PackedWeights, M: int) -> int:

@@ -15,25 +15,65 @@ void set_cuda_error(int err) { g_cuda_error = cudaGetErrorString(static_cast<cud
 
 static bool aligned(const void* p, size_t a) { return reinterpret_cast<uintptr_t>(p) % a == 0; }
 
-static lcd_algo resolve_algo(const Header& h, int64_t M, lcd_algo algo) {
+static lcd_algo resolve_algo(int64_t M, lcd_algo algo) {
   if (algo != LCD_ALGO_AUTO) return algo;
-  if (M == 1 && h.bits == 2 && kHaveBucketLut) return LCD_ALGO_BUCKET_LUT;
   if (M <= 16) return LCD_ALGO_REGISTER_LUT;
   return kHaveDenseTc ? LCD_ALGO_DENSE_TC : LCD_ALGO_REFERENCE;
 }
 
-static lcd_status workspace_for(const Header& h, int64_t M, lcd_algo algo, size_t* bytes) {
-  const int64_t n_pad = (int64_t)round_up_u64(h.N, kTileRows);
-  switch (resolve_algo(h, M, algo)) {
+// Fills everything of a Problem that follows from the blob header and the call's pointers.
+static lcd_status make_problem(const void* packed_weights_dev, const void* header_host, const uint8_t* act_idx,
+                               const float* act_scale, int64_t M, float* y, int64_t ldy, Problem* p) {
+  if (!packed_weights_dev || !header_host || !act_idx || !act_scale || !y || M < 1) return LCD_ERR_INVALID_ARG;
+  Header h;
+  if (!parse_header(header_host, &h)) return LCD_ERR_BAD_BLOB;
+  if (ldy < (int64_t)h.N || M > (1LL << 21)) return LCD_ERR_INVALID_ARG;
+  if (!aligned(packed_weights_dev, 256) || !aligned(act_idx, 16) || !aligned(act_scale, 4) || !aligned(y, 4))
+    return LCD_ERR_INVALID_ARG;
+  const uint8_t* blob = static_cast<const uint8_t*>(packed_weights_dev);
+  p->tiles = blob + h.index_offset;
+  p->codebook = reinterpret_cast<const uint16_t*>(blob + h.codebook_offset);
+  p->N = (int64_t)h.N;
+  p->K = (int64_t)h.K;
+  p->K_pad = (int64_t)h.K_pad;
+  p->N_pad = (int64_t)round_up_u64(h.N, kPairRows);
+  p->bits = (int)h.bits;
+  p->C = (int)h.C;
+  p->act_idx = act_idx;
+  p->act_scale = act_scale;
+  p->M = M;
+  p->y = y;
+  p->ldy = ldy;
+  return LCD_OK;
+}
+
+// Sizes only (no pointers needed): the Problem a header and a token count describe.
+static bool shape_problem(const void* header_host, int64_t M, Problem* p) {
+  Header h;
+  if (!parse_header(header_host, &h)) return false;
+  *p = Problem{};
+  p->N = (int64_t)h.N;
+  p->K = (int64_t)h.K;
+  p->K_pad = (int64_t)h.K_pad;
+  p->N_pad = (int64_t)round_up_u64(h.N, kPairRows);
+  p->bits = (int)h.bits;
+  p->C = (int)h.C;
+  p->M = M;
+  return true;
+}
+
+static lcd_status workspace_for(const Problem& p, lcd_algo algo, size_t* bytes) {
+  switch (resolve_algo(p.M, algo)) {
     case LCD_ALGO_REFERENCE:
-    case LCD_ALGO_REGISTER_LUT:
       *bytes = 0;
       return LCD_OK;
+    case LCD_ALGO_REGISTER_LUT:
     case LCD_ALGO_BUCKET_LUT:
-      *bytes = bucket_lut_workspace_bytes(n_pad, (int64_t)h.K_pad);
+      if (p.M > 16) return LCD_ERR_UNSUPPORTED;
+      *bytes = lut_gemv_workspace_bytes(&p, 1, resolve_algo(p.M, algo));
       return LCD_OK;
     case LCD_ALGO_DENSE_TC:
-      *bytes = dense_tc_workspace_bytes(M, (int64_t)h.K_pad);
+      *bytes = dense_tc_workspace_bytes(p.M, p.K_pad);
       return LCD_OK;
     default:
       return LCD_ERR_INVALID_ARG;
@@ -71,60 +111,96 @@ extern "C" lcd_status lcd_smooth_quantize_act(const void* x_fp16, int64_t M, int
   return launch_smooth_quantize(x_fp16, M, K, ldx, inv_smooth, static_scale, act_idx, act_scale, cuda_stream);
 }
 
+extern "C" lcd_status lcd_smooth_quantize_act_batch(const lcd_act_problem* problems, int count, int act_bits,
+                                                    void* cuda_stream) {
+  if (!problems || count < 1 || count > LCD_MAX_BATCH) return LCD_ERR_INVALID_ARG;
+  if (act_bits != LCD_ACT_BITS) return LCD_ERR_UNSUPPORTED;
+  for (int i = 0; i < count; ++i) {
+    const lcd_act_problem& q = problems[i];
+    if (!q.x_fp16 || !q.act_idx || !q.act_scale || q.M < 1 || q.K < 1 || q.ldx < q.K || q.M > 0x7fffffffLL)
+      return LCD_ERR_INVALID_ARG;
+    if (!aligned(q.x_fp16, 2) || !aligned(q.act_scale, 4) || (q.inv_smooth && !aligned(q.inv_smooth, 4)))
+      return LCD_ERR_INVALID_ARG;
+  }
+  return launch_smooth_quantize_batch(problems, count, cuda_stream);
+}
+
 extern "C" lcd_status lcd_lut_linear_workspace_bytes(const void* header_host, int64_t M, lcd_algo algo,
                                                      size_t* bytes) {
   if (!header_host || !bytes || M < 1) return LCD_ERR_INVALID_ARG;
-  Header h;
-  if (!parse_header(header_host, &h)) return LCD_ERR_BAD_BLOB;
-  return workspace_for(h, M, algo, bytes);
+  Problem p;
+  if (!shape_problem(header_host, M, &p)) return LCD_ERR_BAD_BLOB;
+  return workspace_for(p, algo, bytes);
 }
 
 extern "C" lcd_status lcd_lut_linear(const void* packed_weights_dev, const void* header_host,
                                      const uint8_t* act_idx, const float* act_scale, int64_t M, float* y,
                                      int64_t ldy, lcd_algo algo, void* workspace, size_t workspace_bytes,
                                      int32_t* status_word_dev, void* cuda_stream) {
-  if (!packed_weights_dev || !header_host || !act_idx || !act_scale || !y || M < 1) return LCD_ERR_INVALID_ARG;
-  Header h;
-  if (!parse_header(header_host, &h)) return LCD_ERR_BAD_BLOB;
-  if (ldy < (int64_t)h.N || M > (1LL << 21)) return LCD_ERR_INVALID_ARG;
-  if (!aligned(packed_weights_dev, 256) || !aligned(act_idx, 16) || !aligned(act_scale, 4) || !aligned(y, 4))
-    return LCD_ERR_INVALID_ARG;
+  Problem p;
+  lcd_status st = make_problem(packed_weights_dev, header_host, act_idx, act_scale, M, y, ldy, &p);
+  if (st != LCD_OK) return st;
   size_t need = 0;
-  lcd_status st = workspace_for(h, M, algo, &need);
+  st = workspace_for(p, algo, &need);
   if (st != LCD_OK) return st;
   if (need > 0 && (!workspace || workspace_bytes < need)) return LCD_ERR_BUFFER_TOO_SMALL;
   if (need > 0 && !aligned(workspace, 256)) return LCD_ERR_INVALID_ARG;
-
-  Problem p;
-  const uint8_t* blob = static_cast<const uint8_t*>(packed_weights_dev);
-  p.tiles = blob + h.index_offset;
-  p.codebook = reinterpret_cast<const uint16_t*>(blob + h.codebook_offset);
-  p.N = (int64_t)h.N;
-  p.K = (int64_t)h.K;
-  p.K_pad = (int64_t)h.K_pad;
-  p.N_pad = (int64_t)round_up_u64(h.N, kTileRows);
-  p.bits = (int)h.bits;
-  p.C = (int)h.C;
-  p.act_idx = act_idx;
-  p.act_scale = act_scale;
-  p.M = M;
-  p.y = y;
-  p.ldy = ldy;
-
-  switch (resolve_algo(h, M, algo)) {
+  const lcd_algo resolved = resolve_algo(M, algo);
+  switch (resolved) {
     case LCD_ALGO_REFERENCE:
       return launch_reference(p, cuda_stream);
-    case LCD_ALGO_BUCKET_LUT:
-      if (M != 1 || h.bits != 2) return LCD_ERR_UNSUPPORTED;
-      return launch_bucket_lut(p, workspace, workspace_bytes, cuda_stream);
     case LCD_ALGO_REGISTER_LUT:
-      if (M > 16) return LCD_ERR_UNSUPPORTED;
-      return launch_register_lut(p, cuda_stream);
+    case LCD_ALGO_BUCKET_LUT:
+      return launch_lut_gemv(&p, 1, resolved, workspace, workspace_bytes, status_word_dev, cuda_stream);
     case LCD_ALGO_DENSE_TC:
       return launch_dense_tc(p, workspace, workspace_bytes, status_word_dev, cuda_stream);
     default:
       return LCD_ERR_INVALID_ARG;
   }
+}
+
+static lcd_status batch_algo(const lcd_linear_problem* problems, int count, lcd_algo algo, lcd_algo* resolved) {
+  if (!problems || count < 1 || count > LCD_MAX_BATCH) return LCD_ERR_INVALID_ARG;
+  if (algo != LCD_ALGO_AUTO && algo != LCD_ALGO_REGISTER_LUT && algo != LCD_ALGO_BUCKET_LUT) return LCD_ERR_UNSUPPORTED;
+  for (int i = 0; i < count; ++i)
+    if (problems[i].M < 1 || problems[i].M > 16) return problems[i].M < 1 ? LCD_ERR_INVALID_ARG : LCD_ERR_UNSUPPORTED;
+  *resolved = algo == LCD_ALGO_AUTO ? LCD_ALGO_REGISTER_LUT : algo;
+  return LCD_OK;
+}
+
+extern "C" lcd_status lcd_lut_linear_batch_workspace_bytes(const lcd_linear_problem* problems, int count,
+                                                           lcd_algo algo, size_t* bytes) {
+  lcd_algo resolved;
+  lcd_status st = batch_algo(problems, count, algo, &resolved);
+  if (st != LCD_OK) return st;
+  if (!bytes) return LCD_ERR_INVALID_ARG;
+  Problem p[LCD_MAX_BATCH];
+  for (int i = 0; i < count; ++i) {
+    if (!problems[i].header_host) return LCD_ERR_INVALID_ARG;
+    if (!shape_problem(problems[i].header_host, problems[i].M, &p[i])) return LCD_ERR_BAD_BLOB;
+    if (p[i].bits != p[0].bits) return LCD_ERR_UNSUPPORTED;
+  }
+  *bytes = lut_gemv_workspace_bytes(p, count, resolved);
+  return LCD_OK;
+}
+
+extern "C" lcd_status lcd_lut_linear_batch(const lcd_linear_problem* problems, int count, lcd_algo algo,
+                                           void* workspace, size_t workspace_bytes, int32_t* status_word_dev,
+                                           void* cuda_stream) {
+  lcd_algo resolved;
+  lcd_status st = batch_algo(problems, count, algo, &resolved);
+  if (st != LCD_OK) return st;
+  Problem p[LCD_MAX_BATCH];
+  for (int i = 0; i < count; ++i) {
+    const lcd_linear_problem& q = problems[i];
+    st = make_problem(q.packed_weights_dev, q.header_host, q.act_idx, q.act_scale, q.M, q.y, q.ldy, &p[i]);
+    if (st != LCD_OK) return st;
+    if (p[i].bits != p[0].bits) return LCD_ERR_UNSUPPORTED;
+  }
+  const size_t need = lut_gemv_workspace_bytes(p, count, resolved);
+  if (!workspace || workspace_bytes < need) return LCD_ERR_BUFFER_TOO_SMALL;
+  if (!aligned(workspace, 256)) return LCD_ERR_INVALID_ARG;
+  return launch_lut_gemv(p, count, resolved, workspace, workspace_bytes, status_word_dev, cuda_stream);
 }
 
 // ---- host-buffer path -------------------------------------------------------------------------------
@@ -134,7 +210,9 @@ struct HostScratch {
 };
 lcd_status host_scratch_layout(const Header& h, int64_t M, HostScratch* s) {
   size_t ws = 0;
-  lcd_status st = workspace_for(h, M, LCD_ALGO_AUTO, &ws);
+  Problem shape;
+  if (!shape_problem(&h, M, &shape)) return LCD_ERR_BAD_BLOB;
+  lcd_status st = workspace_for(shape, LCD_ALGO_AUTO, &ws);
   if (st != LCD_OK) return st;
   size_t o = 0;
   s->x_off = o;      o += round_up_u64((uint64_t)M * h.K * 2, 256);
@@ -180,6 +258,10 @@ extern "C" lcd_status lcd_linear_host(const void* packed_weights_dev, const void
   st = lcd_smooth_quantize_act(base + s.x_off, M, (int64_t)h.K, (int64_t)h.K, inv_smooth, nullptr, LCD_ACT_BITS,
                                idx, scale, cuda_stream);
   if (st != LCD_OK) return st;
+  if (s.ws_bytes) {   // the lookup kernels want their scratch zero-filled
+    e = cudaMemsetAsync(base + s.ws_off, 0, s.ws_bytes, stream);
+    if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
+  }
   st = lcd_lut_linear(packed_weights_dev, header_host, idx, scale, M, y, (int64_t)h.N, LCD_ALGO_AUTO,
                       s.ws_bytes ? base + s.ws_off : nullptr, s.ws_bytes, nullptr, cuda_stream);
   if (st != LCD_OK) return st;

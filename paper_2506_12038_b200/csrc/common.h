@@ -11,13 +11,13 @@ namespace lcd {
 
 constexpr uint32_t kMagic = 0x5744434Cu;  // "LCDW"
 constexpr uint32_t kVersion = 1;
-constexpr uint32_t kLayoutTile8x256 = 1;
+constexpr uint32_t kLayoutPair16x256 = 2;
 constexpr uint64_t kIndexOffset = 256;
-constexpr int kTileRows = 8;
+constexpr int kTileRows = 8;    // rows of one tile
+constexpr int kPairRows = 16;   // two adjacent tiles form one 16-row item
 constexpr int kTileK = 256;
 constexpr int kKBlock = 128;
-constexpr bool kHaveBucketLut = false;  // kernels that are not built yet are skipped by LCD_ALGO_AUTO
-constexpr bool kHaveDenseTc = false;
+constexpr bool kHaveDenseTc = false;  // a kernel that is not built yet is skipped by LCD_ALGO_AUTO
 
 #pragma pack(push, 1)
 struct Header {
@@ -53,9 +53,11 @@ void set_cuda_error(int err);  // records cudaGetErrorString for lcd_last_cuda_e
 lcd_status launch_smooth_quantize(const void* x, int64_t M, int64_t K, int64_t ldx, const float* inv_smooth,
                                   const float* static_scale, uint8_t* act_idx, float* act_scale, void* stream);
 lcd_status launch_reference(const Problem& p, void* stream);
-size_t bucket_lut_workspace_bytes(int64_t N, int64_t K_pad);
-lcd_status launch_bucket_lut(const Problem& p, void* workspace, size_t workspace_bytes, void* stream);
-lcd_status launch_register_lut(const Problem& p, void* stream);
+lcd_status launch_smooth_quantize_batch(const lcd_act_problem* probs, int count, void* stream);
+// LCD_ALGO_REGISTER_LUT / LCD_ALGO_BUCKET_LUT for up to LCD_MAX_BATCH problems of equal index width in one launch
+size_t lut_gemv_workspace_bytes(const Problem* probs, int count, lcd_algo algo);
+lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void* workspace, size_t workspace_bytes,
+                           int32_t* status_word, void* stream);
 size_t dense_tc_workspace_bytes(int64_t M, int64_t K_pad);
 lcd_status launch_dense_tc(const Problem& p, void* workspace, size_t workspace_bytes, int32_t* status_word,
                            void* stream);

@@ -8,7 +8,7 @@ namespace lcd {
 
 // Index of column kk (0..255) of row g (0..7) inside one 512-byte 2-bit tile.
 __device__ __forceinline__ uint32_t tile_index_2bit(const uint8_t* tile, int g, int kk) {
-  const int h = kk >> 7, r = kk & 127, G = r >> 2, t = G >> 3, p = ((G & 7) - g) & 7;
+  const int h = kk >> 7, r = kk & 127, G = r >> 2, t = G >> 3, p = G & 7;
   return (tile[16 * (4 * g + t) + 8 * h + p] >> (2 * (r & 3))) & 3u;
 }
 

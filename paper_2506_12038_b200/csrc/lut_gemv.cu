@@ -1,0 +1,754 @@
+// LUT-GEMV for M <= 16 tokens (Section 4.2 of the LCD paper: values are fetched from a small per-row table by
+// weight index and accumulated; no weight is dequantised to floating point and multiplied).
+//
+// Lookup.  Per output row the 2^bits centroids live in registers as byte tables; one PRMT instruction, whose
+// selector nibbles are four weight indices, looks four weights up at once.  Two table sets exist:
+//   kFixed16  - the fp16 centroids as 16-bit fixed point, a signed high-byte table and an unsigned low-byte
+//               table; y = s_q * 2^e_n * (256 * sumH + sumL).
+//   kBuckets  - Section 4.2, third paragraph (centroid-stationary buckets): one-hot tables, one per centroid
+//               w >= 1, so that the accumulated value is the exact bucket sum S_w = sum_{k: idx = w} q_k;
+//               S_0 is the token's sum of levels (an all-ones plane) minus the others, and
+//               y = s_q * sum_w cb[w] * S_w in fp32: 2^bits multiplies per output.
+// Accumulation.  The looked-up bytes are the A fragments of warp-level int8 tensor-core MMAs (m16n8k32), whose B
+// fragments are the tokens' activation levels (int8, staged in shared memory in lookup order): 16 rows x 8
+// tokens per instruction, exact int32 sums, so the result does not depend on the order of summation.
+//
+// Streaming.  The index area is a sequence of 16-row x 256-column items.  The items of one problem are split
+// evenly (stream-K) over the warps of the CTAs that work on it; each warp streams its items through its own
+// shared-memory ring filled by bulk asynchronous copies (cp.async.bulk + mbarrier), so many kilobytes per warp
+// are in flight without holding registers.  A 16-row group whose columns are shared by several warps is summed
+// with integer atomics in global scratch; the warp that arrives last (ticket counter) converts the total to
+// fp32, writes y and leaves the scratch zero again.
+//
+// Several independent problems (the projections of a decoder layer) can run in one launch: CTAs are divided
+// among the problems in proportion to their index bytes.
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include "common.h"
+
+namespace lcd {
+
+namespace {
+
+constexpr int kWarps = 16;
+constexpr int kThreads = kWarps * 32;
+constexpr int kDepth = 3;            // ring slots per warp
+constexpr int kStageItems = 2;       // items per slot
+constexpr int kBarBytes = 512;       // mbarriers: kWarps * kDepth * 8 = 384 bytes, padded
+constexpr int kMaxSmem = 227 * 1024;
+constexpr unsigned long long kTimeoutNs = 2000000000ull;   // bounded wait on a bulk copy: 2 s
+
+struct GemvProblem {
+  const uint8_t* items;       // index area
+  const uint16_t* codebook;   // [N_pad][2^bits]
+  const uint8_t* act_idx;     // [M][K_pad/2]
+  const float* act_scale;     // [M]
+  float* y;
+  int* acc;                   // scratch: [n_rp][MG][planes][4][32] int32, zero on entry and on exit
+  int* ticket;                // scratch: [n_rp] int32, zero on entry and on exit
+  long long ldy;
+  int N, n_rp, n_kt, M;
+  int pw;                     // columns are walked in panels of pw items (pw == n_kt: a single panel)
+  int n_panels;
+  int cta0, n_cta;            // CTAs [cta0, cta0 + n_cta) of the grid work on this problem
+  int n_warps;                // active warps of this problem, <= 16 * n_cta and <= number of items
+  int tstride;                // bytes between tokens inside a staged activation window
+};
+
+struct GemvBatch {
+  int count;
+  GemvProblem p[LCD_MAX_BATCH];
+};
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+  return d;
+}
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long globaltimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mma_s8(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_u8(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: false when the phase did not complete within kTimeoutNs.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try(bar, parity)) return true;
+    if ((it & 1023u) == 0 && globaltimer() - t0 > kTimeoutNs) return false;
+  }
+}
+
+enum TableKind { kFixed16 = 0, kBuckets = 1 };
+
+template <int BITS, int KIND>
+struct Planes {
+  static constexpr int value = KIND == kFixed16 ? 2 : (1 << BITS);
+};
+
+// Byte tables of one row.  kFixed16: plane 0 = high bytes (signed), plane 1 = low bytes (unsigned); entries
+// w = 0..3 in lo[], 4..7 in hi[] (3 bit).  kBuckets: the tables are the same for every row (one-hot) and are
+// generated on the fly, only the centroid values are kept.
+template <int BITS, int KIND>
+struct RowTables {
+  uint32_t lo[KIND == kFixed16 ? 2 : 1], hi[KIND == kFixed16 ? 2 : 1];   // [plane]
+  float scale;                                                          // kFixed16: 2^(e-15)
+  float c[KIND == kBuckets ? (1 << BITS) : 1];                           // kBuckets: centroid values
+};
+
+template <int BITS>
+struct RawCodebook {
+  uint32_t w[BITS == 2 ? 2 : 4];
+};
+
+template <int BITS>
+__device__ __forceinline__ RawCodebook<BITS> load_codebook(const uint16_t* cb_row) {
+  RawCodebook<BITS> r;
+  if (BITS == 2) {
+    const uint2 v = __ldg(reinterpret_cast<const uint2*>(cb_row));
+    r.w[0] = v.x; r.w[1] = v.y;
+  } else {
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(cb_row));
+    r.w[0] = v.x; r.w[1] = v.y; r.w[2] = v.z; r.w[3] = v.w;
+  }
+  return r;
+}
+
+template <int BITS, int KIND>
+__device__ __forceinline__ RowTables<BITS, KIND> build_tables(const RawCodebook<BITS>& raw) {
+  constexpr int C = 1 << BITS;
+  float v[C];
+#pragma unroll
+  for (int i = 0; i < C / 2; ++i) {
+    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&raw.w[i]));
+    v[2 * i] = a.x; v[2 * i + 1] = a.y;
+  }
+  RowTables<BITS, KIND> T;
+  if (KIND == kBuckets) {
+#pragma unroll
+    for (int i = 0; i < C; ++i) T.c[i] = v[i];
+    T.scale = 1.0f;
+    T.lo[0] = T.hi[0] = 0;
+  } else {
+    float mx = 0.0f;
+#pragma unroll
+    for (int i = 0; i < C; ++i) mx = fmaxf(mx, fabsf(v[i]));
+    int ex = 0;
+    (void)frexpf(mx, &ex);                       // mx < 2^ex
+    const float up = scalbnf(1.0f, 15 - ex);     // |v| * up < 32768
+    T.scale = scalbnf(1.0f, ex - 15);
+    uint32_t hb[2] = {0, 0}, lb[2] = {0, 0};
+#pragma unroll
+    for (int i = 0; i < C; ++i) {
+      const int f = __float2int_rn(v[i] * up);
+      hb[i >> 2] |= ((uint32_t)(f >> 8) & 0xffu) << (8 * (i & 3));
+      lb[i >> 2] |= ((uint32_t)f & 0xffu) << (8 * (i & 3));
+    }
+    T.lo[0] = hb[0]; T.lo[1] = lb[0];
+    if (BITS == 3) { T.hi[0] = hb[1]; T.hi[1] = lb[1]; } else { T.hi[0] = hb[0]; T.hi[1] = lb[0]; }
+  }
+  return T;
+}
+
+// Four weights (selector nibbles of sel, low 16 bits) looked up in plane p of a row's tables.  p is a constant
+// after unrolling.  kBuckets: plane p < C - 1 is the one-hot table of centroid p + 1 (byte w is 1 iff
+// w == p + 1), the last plane is all ones.
+template <int BITS, int KIND>
+__device__ __forceinline__ uint32_t pick_lookup(const RowTables<BITS, KIND>& T, uint32_t sel, int p) {
+  if (KIND == kFixed16) return prmt(T.lo[p], T.hi[p], sel);
+  if (p == (1 << BITS) - 1) return 0x01010101u;
+  const int w = p + 1;
+  const uint32_t t_lo = w < 4 ? (1u << (8 * w)) : 0u;
+  const uint32_t t_hi = BITS == 2 ? t_lo : (w >= 4 ? (1u << (8 * (w - 4))) : 0u);
+  return prmt(t_lo, t_hi, sel);
+}
+
+// Activation levels of `n_words` source words (8 columns each, packed 4-bit a = q + 8, even column in the low
+// nibble) as signed bytes, ordered the way the lookups emit weights.  Per 32-column quarter (4 source words):
+//   2 bit: staged words [E(w0) E(w1) O(w0) O(w1) E(w2) E(w3) O(w2) O(w3)], E/O = even/odd columns of a word;
+//   3 bit: natural column order.
+template <int BITS>
+__device__ __forceinline__ void stage_window(uint32_t* dst, const uint32_t* src, int n_words, int tid) {
+  for (int j = tid; j < n_words; j += kThreads) {
+    const uint32_t a = __ldcg(src + j);
+    uint32_t e = a & 0x0f0f0f0fu, o = (a >> 4) & 0x0f0f0f0fu;
+    e = (e + 0x78787878u) ^ 0x80808080u;   // per byte a - 8, no carry between bytes
+    o = (o + 0x78787878u) ^ 0x80808080u;
+    const int quarter = j >> 2, w = j & 3;
+    if (BITS == 2) {
+      dst[quarter * 8 + (w & 1) + 4 * (w >> 1)] = e;
+      dst[quarter * 8 + 2 + (w & 1) + 4 * (w >> 1)] = o;
+    } else {
+      dst[quarter * 8 + 2 * w] = prmt(e, o, 0x5140u);
+      dst[quarter * 8 + 2 * w + 1] = prmt(e, o, 0x7362u);
+    }
+  }
+}
+
+// Position inside a problem's item sequence, walked panel by panel: all 16-row groups of the first pw item
+// columns, then of the next pw, ...
+struct Cursor {
+  uint32_t x, pn, rp, kk, pw;
+};
+__device__ __forceinline__ void cursor_set(Cursor& c, uint32_t x, const GemvProblem& P) {
+  const uint32_t panel_items = (uint32_t)P.n_rp * (uint32_t)P.pw;
+  c.x = x;
+  c.pn = x / panel_items;
+  const uint32_t r = x - c.pn * panel_items;
+  const int left = P.n_kt - (int)c.pn * P.pw;
+  c.pw = (uint32_t)(left < P.pw ? (left > 0 ? left : 1) : P.pw);
+  c.rp = r / c.pw;
+  c.kk = r - c.rp * c.pw;
+}
+__device__ __forceinline__ uint32_t stage_len(const Cursor& c, uint32_t x_end) {
+  uint32_t n = x_end - c.x;
+  n = n < (uint32_t)kStageItems ? n : (uint32_t)kStageItems;
+  const uint32_t row_left = c.pw - c.kk;
+  return n < row_left ? n : row_left;
+}
+__device__ __forceinline__ void cursor_advance(Cursor& c, uint32_t n, const GemvProblem& P) {
+  c.x += n;
+  c.kk += n;
+  if (c.kk == c.pw) {
+    c.kk = 0;
+    if (++c.rp == (uint32_t)P.n_rp) {
+      c.rp = 0;
+      ++c.pn;
+      const int left = P.n_kt - (int)c.pn * P.pw;
+      c.pw = (uint32_t)(left < P.pw ? (left > 0 ? left : 1) : P.pw);
+    }
+  }
+}
+// First item of warp W (of n_warps) and the warp that owns item x, for an even split of n_items.
+__device__ __forceinline__ uint32_t warp_begin(uint32_t W, uint32_t n_items, uint32_t n_warps) {
+  return (uint32_t)(((unsigned long long)W * n_items) / n_warps);
+}
+__device__ __forceinline__ uint32_t warp_of(uint32_t x, uint32_t n_items, uint32_t n_warps) {
+  return (uint32_t)((((unsigned long long)(x + 1)) * n_warps + n_items - 1) / n_items) - 1;
+}
+
+template <int BITS, int KIND, int MG>
+__global__ void __launch_bounds__(kThreads, 1)
+lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ status) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  constexpr int ITEM = 512 * BITS;
+  constexpr int HALF = ITEM / 2;                 // bytes of one 8-row tile
+  constexpr int SLOT = kStageItems * ITEM;
+  constexpr int PL = Planes<BITS, KIND>::value;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, t = lane & 3;
+
+  // which problem this CTA works on
+  int pi = 0;
+#pragma unroll 1
+  for (int i = 1; i < batch.count; ++i)
+    if ((int)blockIdx.x >= batch.p[i].cta0) pi = i;
+  const GemvProblem& P = batch.p[pi];
+  const uint32_t cta = blockIdx.x - P.cta0;
+  const uint32_t n_items = (uint32_t)P.n_rp * (uint32_t)P.n_kt;
+  const uint32_t n_warps = (uint32_t)P.n_warps;
+  if (cta * kWarps >= n_warps) return;            // whole CTA idle (uniform)
+
+  uint8_t* ring = smem + kBarBytes + (size_t)warp * kDepth * SLOT;
+  const uint32_t bar0 = smem_u32(smem) + 8u * (uint32_t)(warp * kDepth);
+  uint8_t* act_s = smem + kBarBytes + (size_t)kWarps * kDepth * SLOT;
+  const int win_bytes = (P.M < 8 * MG ? P.M : 8 * MG) * P.tstride;
+
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < kDepth; ++s)
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0 + 8u * s));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncwarp();
+
+  // this warp's items
+  const uint32_t W = cta * kWarps + warp;
+  const bool warp_active = W < n_warps;
+  const uint32_t wx0 = warp_active ? warp_begin(W, n_items, n_warps) : 0;
+  const uint32_t wx1 = warp_active ? warp_begin(W + 1, n_items, n_warps) : 0;
+  // the CTA's items and the panels they touch
+  const uint32_t last_w = (cta + 1) * kWarps < n_warps ? (cta + 1) * kWarps : n_warps;
+  const uint32_t cx0 = warp_begin(cta * kWarps, n_items, n_warps), cx1 = warp_begin(last_w, n_items, n_warps);
+  const uint32_t panel_items = (uint32_t)P.n_rp * (uint32_t)P.pw;
+  const uint32_t pA = cx0 / panel_items, pB = (cx1 - 1) / panel_items;
+
+  uint32_t stage_c = 0, stage_f = 0;    // consumed / fetched stages of this warp (ring position and parity)
+  bool aborted = false;
+
+  auto issue = [&](Cursor& fc, uint32_t x_end) {
+    const uint32_t n = stage_len(fc, x_end);
+    if (lane == 0) {
+      const uint32_t slot = stage_f % kDepth;
+      const uint32_t bar = bar0 + 8u * slot;
+      const uint32_t bytes = n * ITEM;
+      const uint8_t* src = P.items + ((size_t)fc.rp * P.n_kt + (size_t)fc.pn * P.pw + fc.kk) * ITEM;
+      const uint32_t dst = smem_u32(ring + slot * SLOT);
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+      asm volatile(
+          "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+          ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+    }
+    cursor_advance(fc, n, P);
+    ++stage_f;
+  };
+
+  // The weights do not depend on the kernel that produced the activation indices: start streaming them
+  // before waiting for it.
+  Cursor fc, cc;
+  uint32_t round_lo = 0, round_hi = 0;
+  {
+    const uint32_t lo = pA * panel_items, hi = (pA + 2) * panel_items;
+    round_lo = wx0 > lo ? wx0 : lo;
+    round_hi = wx1 < hi ? wx1 : hi;
+    if (round_hi < round_lo) round_hi = round_lo;
+    cursor_set(fc, round_lo, P);
+    cc = fc;
+    while (fc.x < round_hi && stage_f - stage_c < (uint32_t)kDepth) issue(fc, round_hi);
+  }
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  RowTables<BITS, KIND> Ta, Tb;           // rows 16*rp + g and 16*rp + 8 + g
+  RawCodebook<BITS> next_a, next_b;
+  uint32_t tables_rp = 0xffffffffu, next_rp = 0xffffffffu;
+  int acc[MG][PL][4];
+#pragma unroll
+  for (int G = 0; G < MG; ++G)
+#pragma unroll
+    for (int p = 0; p < PL; ++p)
+#pragma unroll
+      for (int r = 0; r < 4; ++r) acc[G][p][r] = 0;
+  uint32_t seg_kk0 = 0;
+  bool seg_open = false;
+
+  // Writes the finished sums of 16-row group rp (this warp's share [seg_kk0, kk_end) of panel pn).
+  auto flush = [&](uint32_t rp, uint32_t pn, uint32_t pw_n, uint32_t kk_end) {
+    const bool direct = P.n_panels == 1 && seg_kk0 == 0 && kk_end == pw_n;
+    bool finish = direct;
+    if (!direct) {
+      int* a = P.acc + (size_t)rp * (MG * PL * 128) + lane;
+#pragma unroll
+      for (int G = 0; G < MG; ++G)
+#pragma unroll
+        for (int p = 0; p < PL; ++p)
+#pragma unroll
+          for (int r = 0; r < 4; ++r)
+            if (8 * G + 2 * t + (r & 1) < P.M) atomicAdd(a + ((G * PL + p) * 4 + r) * 32, acc[G][p][r]);
+      __threadfence();
+      __syncwarp();
+      // how many warps contribute to this 16-row group: per panel, the warps whose items meet its run
+      uint32_t part = 0;
+      if (lane < P.n_panels) {
+        const int left = P.n_kt - lane * P.pw;
+        const uint32_t w_l = (uint32_t)(left < P.pw ? left : P.pw);
+        const uint32_t r0 = (uint32_t)lane * panel_items + rp * w_l;
+        part = warp_of(r0 + w_l - 1, n_items, n_warps) - warp_of(r0, n_items, n_warps) + 1;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+      int old = 0;
+      if (lane == 0) old = atomicAdd(P.ticket + rp, 1);
+      old = __shfl_sync(0xffffffffu, old, 0);
+      finish = (uint32_t)old + 1 == part;
+      if (finish) {
+        __threadfence();
+#pragma unroll
+        for (int G = 0; G < MG; ++G)
+#pragma unroll
+          for (int p = 0; p < PL; ++p)
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+              if (8 * G + 2 * t + (r & 1) < P.M) acc[G][p][r] = atomicExch(a + ((G * PL + p) * 4 + r) * 32, 0);
+        if (lane == 0) atomicExch(P.ticket + rp, 0);
+      }
+    }
+    if (finish) {
+#pragma unroll
+      for (int G = 0; G < MG; ++G)
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          const int m = 8 * G + 2 * t + (r & 1);
+          const int n = 16 * (int)rp + g + ((r & 2) ? 8 : 0);
+          if (m < P.M && n < P.N) {
+            const RowTables<BITS, KIND>& T = (r & 2) ? Tb : Ta;
+            float v;
+            if (KIND == kFixed16) {
+              v = T.scale * ((float)acc[G][0][r] * 256.0f + (float)acc[G][1][r]);
+            } else {
+              // planes 0..C-2 hold the exact bucket sums S_1..S_{C-1}, the last one the token's sum of levels
+              int s0 = acc[G][PL - 1][r];
+#pragma unroll
+              for (int p = 0; p < PL - 1; ++p) s0 -= acc[G][p][r];
+              v = T.c[0] * (float)s0;
+#pragma unroll
+              for (int p = 0; p < PL - 1; ++p) v = fmaf(T.c[p + 1], (float)acc[G][p][r], v);
+            }
+            v *= __ldg(P.act_scale + m);
+            P.y[(size_t)m * P.ldy + n] = v;
+          }
+        }
+    }
+#pragma unroll
+    for (int G = 0; G < MG; ++G)
+#pragma unroll
+      for (int p = 0; p < PL; ++p)
+#pragma unroll
+        for (int r = 0; r < 4; ++r) acc[G][p][r] = 0;
+  };
+
+#pragma unroll 1
+  for (uint32_t pbase = pA; pbase <= pB; pbase += 2) {
+    if (pbase != pA) {
+      const uint32_t lo = pbase * panel_items, hi = (pbase + 2) * panel_items;
+      round_lo = wx0 > lo ? wx0 : lo;
+      round_hi = wx1 < hi ? wx1 : hi;
+      if (round_hi < round_lo) round_hi = round_lo;
+      cursor_set(fc, round_lo, P);
+      cc = fc;
+      if (!aborted)
+        while (fc.x < round_hi && stage_f - stage_c < (uint32_t)kDepth) issue(fc, round_hi);
+      __syncthreads();     // every warp is done with the previous windows
+    }
+    // stage the activation windows of panels pbase and pbase + 1
+#pragma unroll 1
+    for (uint32_t wdw = 0; wdw < 2 && pbase + wdw <= pB; ++wdw) {
+      const uint32_t pn = pbase + wdw;
+      const int left = P.n_kt - (int)pn * P.pw;
+      const int pw_n = left < P.pw ? left : P.pw;
+      const int n_words = pw_n * 32;
+      const int n_tok = P.M < 8 * MG ? P.M : 8 * MG;
+      for (int m = 0; m < n_tok; ++m)
+        stage_window<BITS>(reinterpret_cast<uint32_t*>(act_s + wdw * win_bytes + m * P.tstride),
+                           reinterpret_cast<const uint32_t*>(P.act_idx + (size_t)m * P.n_kt * 128 +
+                                                             (size_t)pn * P.pw * 128),
+                           n_words, tid);
+    }
+    __syncthreads();
+
+    if (warp_active && !aborted) {
+#pragma unroll 1
+      while (cc.x < round_hi) {
+        const uint32_t n = stage_len(cc, round_hi);
+        const uint32_t slot = stage_c % kDepth;
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(bar0 + 8u * slot, (stage_c / kDepth) & 1u));
+        if (!ok) {
+          aborted = true;
+          if (lane == 0 && status) atomicExch(status, (int)LCD_ERR_TIMEOUT);
+          break;
+        }
+        // row tables of this 16-row group
+        if (cc.rp != tables_rp) {
+          if (next_rp != cc.rp) {
+            next_a = load_codebook<BITS>(P.codebook + ((size_t)cc.rp * 16 + g) * (1 << BITS));
+            next_b = load_codebook<BITS>(P.codebook + ((size_t)cc.rp * 16 + 8 + g) * (1 << BITS));
+          }
+          Ta = build_tables<BITS, KIND>(next_a);
+          Tb = build_tables<BITS, KIND>(next_b);
+          tables_rp = cc.rp;
+          next_rp = cc.rp + 1 < (uint32_t)P.n_rp ? cc.rp + 1 : 0;
+          next_a = load_codebook<BITS>(P.codebook + ((size_t)next_rp * 16 + g) * (1 << BITS));
+          next_b = load_codebook<BITS>(P.codebook + ((size_t)next_rp * 16 + 8 + g) * (1 << BITS));
+        }
+        if (!seg_open) { seg_kk0 = cc.kk; seg_open = true; }
+        const uint8_t* slot_p = ring + slot * SLOT;
+        const uint8_t* win = act_s + (cc.pn - pbase) * win_bytes;
+#pragma unroll 1
+        for (uint32_t i = 0; i < n; ++i) {
+          const uint8_t* item = slot_p + i * ITEM;
+          const uint8_t* qbase = win + (size_t)(cc.kk + i) * 256 + t * 32;
+          // the lane's indices of rows g and g + 8 for both 128-column blocks of the item
+          uint32_t raw_a[BITS * 2], raw_b[BITS * 2];
+          if (BITS == 2) {
+            const uint4 wa = *reinterpret_cast<const uint4*>(item + 16 * lane);
+            const uint4 wb = *reinterpret_cast<const uint4*>(item + HALF + 16 * lane);
+            raw_a[0] = wa.x; raw_a[1] = wa.y; raw_a[2] = wa.z; raw_a[3] = wa.w;
+            raw_b[0] = wb.x; raw_b[1] = wb.y; raw_b[2] = wb.z; raw_b[3] = wb.w;
+          } else {
+#pragma unroll
+            for (int b = 0; b < 3; ++b) {
+              const uint2 va = *reinterpret_cast<const uint2*>(item + 256 * b + 8 * lane);
+              const uint2 vb = *reinterpret_cast<const uint2*>(item + HALF + 256 * b + 8 * lane);
+              raw_a[b] = va.x; raw_a[3 + b] = va.y;
+              raw_b[b] = vb.x; raw_b[3 + b] = vb.y;
+            }
+          }
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            // activation levels of this quarter: words 0..3 and 4..7 of the staged order, per token group
+            uint4 qa[MG], qb[MG];
+#pragma unroll
+            for (int G = 0; G < MG; ++G) {
+              const int tok = 8 * G + g < P.M ? 8 * G + g : P.M - 1;
+              const uint8_t* q = qbase + (size_t)tok * P.tstride + h * 128;
+              qa[G] = *reinterpret_cast<const uint4*>(q);
+              qb[G] = *reinterpret_cast<const uint4*>(q + 16);
+            }
+            uint32_t sel_a[8], sel_b[8];    // selector words of rows g and g + 8: lookup l uses sel[l]
+            if (BITS == 2) {
+              const uint32_t ua[2] = {raw_a[2 * h], raw_a[2 * h + 1]}, ub[2] = {raw_b[2 * h], raw_b[2 * h + 1]};
+#pragma unroll
+              for (int w = 0; w < 2; ++w) {
+                const uint32_t a0 = ua[w] & 0x33333333u, a1 = (ua[w] >> 2) & 0x33333333u;
+                const uint32_t b0 = ub[w] & 0x33333333u, b1 = (ub[w] >> 2) & 0x33333333u;
+                sel_a[4 * w] = a0; sel_a[4 * w + 1] = a0 >> 16; sel_a[4 * w + 2] = a1; sel_a[4 * w + 3] = a1 >> 16;
+                sel_b[4 * w] = b0; sel_b[4 * w + 1] = b0 >> 16; sel_b[4 * w + 2] = b1; sel_b[4 * w + 3] = b1 >> 16;
+              }
+            } else {
+              uint32_t ra[3], rb[3];
+#pragma unroll
+              for (int b = 0; b < 3; ++b) {
+                ra[b] = raw_a[3 * h + b];
+                rb[b] = raw_b[3 * h + b];
+              }
+              const uint32_t xa = ((ra[0] & 0x88888888u) >> 3) | ((ra[1] & 0x88888888u) >> 2) |
+                                  ((ra[2] & 0x88888888u) >> 1);
+              const uint32_t xb = ((rb[0] & 0x88888888u) >> 3) | ((rb[1] & 0x88888888u) >> 2) |
+                                  ((rb[2] & 0x88888888u) >> 1);
+#pragma unroll
+              for (int b = 0; b < 3; ++b) {
+                const uint32_t da = ra[b] & 0x77777777u, db = rb[b] & 0x77777777u;
+                sel_a[2 * b] = da; sel_a[2 * b + 1] = da >> 16;
+                sel_b[2 * b] = db; sel_b[2 * b + 1] = db >> 16;
+              }
+              sel_a[6] = xa; sel_a[7] = xa >> 16;
+              sel_b[6] = xb; sel_b[7] = xb >> 16;
+            }
+            // four MMAs per plane: MMA j takes lookups 2j and 2j + 1 and staged words 2j, 2j + 1
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              uint32_t b0[MG], b1[MG];
+#pragma unroll
+              for (int G = 0; G < MG; ++G) {
+                const uint4& q = j < 2 ? qa[G] : qb[G];
+                b0[G] = (j & 1) ? q.z : q.x;
+                b1[G] = (j & 1) ? q.w : q.y;
+              }
+#pragma unroll
+              for (int p = 0; p < PL; ++p) {
+                uint32_t a[4];
+                a[0] = pick_lookup<BITS, KIND>(Ta, sel_a[2 * j], p);
+                a[1] = pick_lookup<BITS, KIND>(Tb, sel_b[2 * j], p);
+                a[2] = pick_lookup<BITS, KIND>(Ta, sel_a[2 * j + 1], p);
+                a[3] = pick_lookup<BITS, KIND>(Tb, sel_b[2 * j + 1], p);
+#pragma unroll
+                for (int G = 0; G < MG; ++G) {
+                  if (KIND == kFixed16 && p == 1) mma_u8(acc[G][p], a, b0[G], b1[G]);
+                  else mma_s8(acc[G][p], a, b0[G], b1[G]);
+                }
+              }
+            }
+          }
+        }
+        const uint32_t rp_done = cc.rp, pn_done = cc.pn, pw_done = cc.pw, kk_end = cc.kk + n;
+        cursor_advance(cc, n, P);
+        if (kk_end == pw_done || cc.x == round_hi) {
+          flush(rp_done, pn_done, pw_done, kk_end);
+          seg_open = false;
+        }
+        __syncwarp();
+        ++stage_c;
+        if (fc.x < round_hi) issue(fc, round_hi);
+      }
+    }
+    if (aborted) {
+      // copies already issued must land before the CTA may exit
+      while (stage_c < stage_f) {
+        (void)mbar_wait(bar0 + 8u * (stage_c % kDepth), (stage_c / kDepth) & 1u);
+        ++stage_c;
+      }
+    }
+  }
+}
+
+
+int sm_count() {
+  static int cached = 0;
+  if (cached == 0) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
+      n = 148;
+    cached = n;
+  }
+  return cached;
+}
+
+int planes_of(int bits, int kind) { return kind == kFixed16 ? 2 : (1 << bits); }
+
+struct ScratchLayout {
+  size_t acc_off, ticket_off, end;
+};
+ScratchLayout scratch_layout(size_t begin, int64_t n_rp, int MG, int planes) {
+  ScratchLayout s;
+  s.acc_off = begin;
+  s.ticket_off = s.acc_off + (size_t)n_rp * MG * planes * 128 * sizeof(int);
+  s.end = (size_t)round_up_u64(s.ticket_off + (size_t)n_rp * sizeof(int), 256);
+  return s;
+}
+
+template <int BITS, int KIND, int MG>
+lcd_status launch_t(const GemvBatch& batch, int grid, size_t smem, int32_t* status, cudaStream_t stream) {
+  auto kern = lut_gemv_kernel<BITS, KIND, MG>;
+  static bool attr_set = false;   // per template instance
+  if (!attr_set) {
+    const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+    if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
+    attr_set = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  // The kernel may start while the previous kernel of the stream drains: it streams weights first and waits
+  // (griddepcontrol.wait) before it touches the activation indices.
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, batch, status);
+  if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
+  return LCD_OK;
+}
+
+}  // namespace
+
+size_t lut_gemv_workspace_bytes(const Problem* probs, int count, lcd_algo algo) {
+  const int kind = algo == LCD_ALGO_BUCKET_LUT ? kBuckets : kFixed16;
+  int64_t max_m = 1;
+  for (int i = 0; i < count; ++i) max_m = probs[i].M > max_m ? probs[i].M : max_m;
+  const int MG = max_m > 8 ? 2 : 1;
+  size_t off = 0;
+  for (int i = 0; i < count; ++i)
+    off = scratch_layout(off, probs[i].N_pad / kPairRows, MG, planes_of(probs[i].bits, kind)).end;
+  return off;
+}
+
+lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void* workspace, size_t workspace_bytes,
+                           int32_t* status_word, void* stream) {
+  if (count < 1 || count > LCD_MAX_BATCH) return LCD_ERR_INVALID_ARG;
+  const int kind = algo == LCD_ALGO_BUCKET_LUT ? kBuckets : kFixed16;
+  const int bits = probs[0].bits;
+  int64_t max_m = 1;
+  for (int i = 0; i < count; ++i) {
+    if (probs[i].bits != bits || probs[i].M > 16 || probs[i].M < 1) return LCD_ERR_UNSUPPORTED;
+    max_m = probs[i].M > max_m ? probs[i].M : max_m;
+  }
+  const int MG = max_m > 8 ? 2 : 1;
+  const int planes = planes_of(bits, kind);
+  if (workspace_bytes < lut_gemv_workspace_bytes(probs, count, algo) || !workspace) return LCD_ERR_BUFFER_TOO_SMALL;
+
+  const int item_bytes = 512 * bits;
+  const size_t ring_bytes = (size_t)kWarps * kDepth * kStageItems * item_bytes;
+  const size_t act_budget = (size_t)kMaxSmem - kBarBytes - ring_bytes;
+
+  GemvBatch batch;
+  batch.count = count;
+  size_t act_bytes = 0, off = 0;
+  for (int i = 0; i < count; ++i) {
+    const Problem& p = probs[i];
+    GemvProblem& g = batch.p[i];
+    g.items = p.tiles;
+    g.codebook = p.codebook;
+    g.act_idx = p.act_idx;
+    g.act_scale = p.act_scale;
+    g.y = p.y;
+    g.ldy = p.ldy;
+    g.N = (int)p.N;
+    g.n_rp = (int)(p.N_pad / kPairRows);
+    g.n_kt = (int)(p.K_pad / kTileK);
+    g.M = (int)p.M;
+    if ((int64_t)g.n_rp * g.n_kt > (1LL << 30) / 16) return LCD_ERR_UNSUPPORTED;
+    const ScratchLayout sl = scratch_layout(off, g.n_rp, MG, planes);
+    g.acc = reinterpret_cast<int*>(static_cast<uint8_t*>(workspace) + sl.acc_off);
+    g.ticket = reinterpret_cast<int*>(static_cast<uint8_t*>(workspace) + sl.ticket_off);
+    off = sl.end;
+    // panels: a single one when all tokens' levels of the whole row fit, else the fewest that let two
+    // panel windows fit
+    const size_t m_eff = (size_t)(g.M < 8 * MG ? g.M : 8 * MG);
+    int n_panels = 1, pw = g.n_kt;
+    if (m_eff * ((size_t)g.n_kt * 256 + 16) > act_budget) {
+      for (n_panels = 2;; ++n_panels) {
+        pw = (g.n_kt + n_panels - 1) / n_panels;
+        if (2 * m_eff * ((size_t)pw * 256 + 16) <= act_budget) break;
+        if (pw == 1) return LCD_ERR_UNSUPPORTED;
+      }
+      n_panels = (g.n_kt + pw - 1) / pw;
+      if (n_panels > 32) return LCD_ERR_UNSUPPORTED;
+    }
+    g.pw = pw;
+    g.n_panels = n_panels;
+    g.tstride = pw * 256 + 16;
+    const size_t need = (n_panels == 1 ? 1 : 2) * m_eff * (size_t)g.tstride;
+    act_bytes = need > act_bytes ? need : act_bytes;
+  }
+  // CTAs per problem: one each, then one more at a time to the problem with the most items per CTA (at most
+  // one CTA per 16 items), until every SM has one
+  const int n_sm = sm_count();
+  int grid = 0;
+  {
+    int given[LCD_MAX_BATCH], cap[LCD_MAX_BATCH];
+    int used = 0;
+    for (int i = 0; i < count; ++i) {
+      const long long items = (long long)batch.p[i].n_rp * batch.p[i].n_kt;
+      cap[i] = (int)((items + kWarps - 1) / kWarps);
+      given[i] = 1;
+      ++used;
+    }
+    while (used < n_sm) {
+      int best = -1;
+      double best_load = 0.0;
+      for (int i = 0; i < count; ++i) {
+        const double load = (double)batch.p[i].n_rp * batch.p[i].n_kt / given[i];
+        if (given[i] < cap[i] && (best < 0 || load > best_load)) { best = i; best_load = load; }
+      }
+      if (best < 0) break;
+      ++given[best];
+      ++used;
+    }
+    for (int i = 0; i < count; ++i) {
+      batch.p[i].cta0 = grid;
+      batch.p[i].n_cta = given[i];
+      const long long items = (long long)batch.p[i].n_rp * batch.p[i].n_kt;
+      const long long w = (long long)given[i] * kWarps;
+      batch.p[i].n_warps = (int)(w < items ? w : items);
+      grid += given[i];
+    }
+  }
+  for (int i = count; i < LCD_MAX_BATCH; ++i) batch.p[i] = batch.p[0];
+  const size_t smem = kBarBytes + ring_bytes + act_bytes;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (bits == 2) {
+    if (kind == kFixed16) return MG == 1 ? launch_t<2, kFixed16, 1>(batch, grid, smem, status_word, s)
+                                         : launch_t<2, kFixed16, 2>(batch, grid, smem, status_word, s);
+    return MG == 1 ? launch_t<2, kBuckets, 1>(batch, grid, smem, status_word, s)
+                   : launch_t<2, kBuckets, 2>(batch, grid, smem, status_word, s);
+  }
+  if (kind == kFixed16) return MG == 1 ? launch_t<3, kFixed16, 1>(batch, grid, smem, status_word, s)
+                                       : launch_t<3, kFixed16, 2>(batch, grid, smem, status_word, s);
+  return MG == 1 ? launch_t<3, kBuckets, 1>(batch, grid, smem, status_word, s)
+                 : launch_t<3, kBuckets, 2>(batch, grid, smem, status_word, s);
+}
+
+}  // namespace lcd

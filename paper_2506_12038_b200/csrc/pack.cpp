@@ -16,26 +16,32 @@ static inline uint32_t payload_checksum(const uint8_t* p, size_t n) {
 
 bool parse_header(const void* header_host, Header* h) {
   std::memcpy(h, header_host, sizeof(Header));
-  if (h->magic != kMagic || h->version != kVersion || h->layout != kLayoutTile8x256) return false;
+  if (h->magic != kMagic || h->version != kVersion || h->layout != kLayoutPair16x256) return false;
   if (h->bits != 2 && h->bits != 3) return false;
   if (h->C < 1 || h->C > (1u << h->bits)) return false;
   if (h->N < 1 || h->K < 1) return false;
   if (h->K_pad != round_up_u64(h->K, kTileK)) return false;
   if (h->index_offset != kIndexOffset) return false;
-  const uint64_t n_pad = round_up_u64(h->N, kTileRows);
+  const uint64_t n_pad = round_up_u64(h->N, kPairRows);
   if (h->codebook_offset != round_up_u64(kIndexOffset + n_pad * h->K_pad * h->bits / 8, 256)) return false;
   return true;
 }
 
 size_t blob_bytes(uint64_t N, uint64_t K, int bits) {
-  const uint64_t n_pad = round_up_u64(N, kTileRows), k_pad = round_up_u64(K, kTileK);
+  const uint64_t n_pad = round_up_u64(N, kPairRows), k_pad = round_up_u64(K, kTileK);
   const uint64_t cb_off = round_up_u64(kIndexOffset + n_pad * k_pad * bits / 8, 256);
   return cb_off + round_up_u64(n_pad * (2ull << bits), 256);
 }
 
+// Byte offset (inside the index area) of tile (rg, kt): the tiles of rows 16rp..16rp+7 and 16rp+8..16rp+15
+// are adjacent and form one 16-row item.
+static inline uint64_t tile_offset(uint64_t rg, uint64_t kt, uint64_t n_kt, size_t tile_bytes) {
+  return ((rg >> 1) * n_kt + kt) * 2 * tile_bytes + (rg & 1) * tile_bytes;
+}
+
 // Position of column kk (0..255) of tile row g inside a 2-bit tile: byte offset and bit shift.
 static inline void locate2(int g, int kk, int* byte, int* shift) {
-  const int h = kk >> 7, r = kk & 127, G = r >> 2, t = G >> 3, p = ((G & 7) - g) & 7;
+  const int h = kk >> 7, r = kk & 127, G = r >> 2, t = G >> 3, p = G & 7;
   *byte = 16 * (4 * g + t) + 8 * h + p;
   *shift = 2 * (r & 3);
 }
@@ -86,12 +92,12 @@ extern "C" lcd_status lcd_pack_weights(const uint8_t* idx, const uint16_t* codeb
       }
   uint8_t* blob = static_cast<uint8_t*>(out);
   std::memset(blob, 0, total);
-  const uint64_t n_pad = round_up_u64(N, kTileRows), k_pad = round_up_u64(K, kTileK);
+  const uint64_t n_pad = round_up_u64(N, kPairRows), k_pad = round_up_u64(K, kTileK);
   const uint64_t n_kt = k_pad / kTileK;
   const size_t tile_bytes = kTileRows * kTileK * bits / 8;
   for (uint64_t rg = 0; rg < n_pad / kTileRows; ++rg) {
     for (uint64_t kt = 0; kt < n_kt; ++kt) {
-      uint8_t* tile = blob + kIndexOffset + (rg * n_kt + kt) * tile_bytes;
+      uint8_t* tile = blob + kIndexOffset + tile_offset(rg, kt, n_kt, tile_bytes);
       for (int g = 0; g < kTileRows; ++g) {
         const uint64_t n = rg * kTileRows + g;
         if (n >= (uint64_t)N) break;
@@ -131,7 +137,7 @@ extern "C" lcd_status lcd_pack_weights(const uint8_t* idx, const uint16_t* codeb
   h.K_pad = k_pad;
   h.bits = (uint32_t)bits;
   h.C = (uint32_t)C;
-  h.layout = kLayoutTile8x256;
+  h.layout = kLayoutPair16x256;
   h.index_offset = kIndexOffset;
   h.codebook_offset = cb_off;
   h.checksum = payload_checksum(blob + sizeof(Header), total - sizeof(Header));
@@ -160,7 +166,7 @@ extern "C" lcd_status lcd_unpack_weights(const void* blob_v, size_t blob_bytes_i
       const uint64_t rg = n / kTileRows;
       const int g = (int)(n % kTileRows);
       for (uint64_t k = 0; k < h.K; ++k) {
-        const uint8_t* tile = blob + h.index_offset + (rg * n_kt + k / kTileK) * tile_bytes;
+        const uint8_t* tile = blob + h.index_offset + tile_offset(rg, k / kTileK, n_kt, tile_bytes);
         const int kk = (int)(k % kTileK);
         uint32_t v;
         if (h.bits == 2) {

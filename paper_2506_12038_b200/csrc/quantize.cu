@@ -18,16 +18,16 @@ __device__ __forceinline__ int quant_level(float v) {
   return (int)r;
 }
 
-// One CTA per token.  VEC: rows are 16-byte aligned and K is a multiple of 8, so each thread handles 8
+// One token per CTA.  VEC: rows are 16-byte aligned and K is a multiple of 8, so each thread handles 8
 // consecutive columns per step (one 16-byte load of x, two of inv_smooth, one 4-byte store).
 template <bool VEC>
-__global__ void __launch_bounds__(kQThreads)
-smooth_quantize_kernel(const __half* __restrict__ x, int64_t K, int64_t K_pad, int64_t ldx,
-                       const float* __restrict__ inv_smooth, const float* __restrict__ static_scale,
-                       uint8_t* __restrict__ act_idx, float* __restrict__ act_scale) {
+__device__ __forceinline__ void smooth_quantize_token(const __half* __restrict__ x, int64_t m, int64_t K,
+                                                      int64_t K_pad, int64_t ldx,
+                                                      const float* __restrict__ inv_smooth,
+                                                      const float* __restrict__ static_scale,
+                                                      uint8_t* __restrict__ act_idx, float* __restrict__ act_scale) {
   __shared__ float s_red[kQThreads / 32];
   __shared__ float s_mult;
-  const int64_t m = blockIdx.x;
   const __half* xr = x + m * ldx;
   uint8_t* out = act_idx + m * (K_pad / 2);
   const int tid = threadIdx.x;
@@ -129,26 +129,82 @@ smooth_quantize_kernel(const __half* __restrict__ x, int64_t K, int64_t K_pad, i
   }
 }
 
-lcd_status launch_smooth_quantize(const void* x, int64_t M, int64_t K, int64_t ldx, const float* inv_smooth,
-                                  const float* static_scale, uint8_t* act_idx, float* act_scale, void* stream) {
-  const int64_t K_pad = (int64_t)round_up_u64((uint64_t)K, kTileK);
-  const bool vec = (reinterpret_cast<uintptr_t>(x) % 16 == 0) && (ldx % 8 == 0) && (K % 8 == 0) &&
-                   (inv_smooth == nullptr || reinterpret_cast<uintptr_t>(inv_smooth) % 16 == 0) &&
-                   (reinterpret_cast<uintptr_t>(act_idx) % 4 == 0);
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const __half* xh = static_cast<const __half*>(x);
-  if (vec)
-    smooth_quantize_kernel<true><<<(unsigned)M, kQThreads, 0, s>>>(xh, K, K_pad, ldx, inv_smooth, static_scale,
-                                                                   act_idx, act_scale);
+struct QuantProblem {
+  const __half* x;
+  const float* inv_smooth;
+  const float* static_scale;
+  uint8_t* act_idx;
+  float* act_scale;
+  long long K, K_pad, ldx;
+  int cta0;    // tokens of this problem are CTAs [cta0, cta0 + M)
+  int vec;
+};
+struct QuantBatch {
+  int count;
+  QuantProblem p[LCD_MAX_BATCH];
+};
+
+// One CTA per token of every problem of the batch.
+__global__ void __launch_bounds__(kQThreads) smooth_quantize_kernel(const __grid_constant__ QuantBatch batch) {
+  // let a dependent kernel (launched with programmatic stream serialization) start its own prologue now; it
+  // still waits for this grid to finish before it reads the indices
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  int pi = 0;
+#pragma unroll 1
+  for (int i = 1; i < batch.count; ++i)
+    if ((int)blockIdx.x >= batch.p[i].cta0) pi = i;
+  const QuantProblem& q = batch.p[pi];
+  const int64_t m = (int64_t)blockIdx.x - q.cta0;
+  if (q.vec)
+    smooth_quantize_token<true>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx, q.act_scale);
   else
-    smooth_quantize_kernel<false><<<(unsigned)M, kQThreads, 0, s>>>(xh, K, K_pad, ldx, inv_smooth, static_scale,
-                                                                    act_idx, act_scale);
+    smooth_quantize_token<false>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx, q.act_scale);
+}
+
+lcd_status launch_smooth_quantize_batch(const lcd_act_problem* probs, int count, void* stream) {
+  QuantBatch batch;
+  batch.count = count;
+  long long grid = 0;
+  for (int i = 0; i < count; ++i) {
+    const lcd_act_problem& a = probs[i];
+    QuantProblem& q = batch.p[i];
+    q.x = static_cast<const __half*>(a.x_fp16);
+    q.inv_smooth = a.inv_smooth;
+    q.static_scale = a.static_scale;
+    q.act_idx = a.act_idx;
+    q.act_scale = a.act_scale;
+    q.K = a.K;
+    q.K_pad = (long long)round_up_u64((uint64_t)a.K, kTileK);
+    q.ldx = a.ldx;
+    q.cta0 = (int)grid;
+    q.vec = (reinterpret_cast<uintptr_t>(a.x_fp16) % 16 == 0) && (a.ldx % 8 == 0) && (a.K % 8 == 0) &&
+            (a.inv_smooth == nullptr || reinterpret_cast<uintptr_t>(a.inv_smooth) % 16 == 0) &&
+            (reinterpret_cast<uintptr_t>(a.act_idx) % 4 == 0);
+    grid += a.M;
+    if (grid > 0x7fffffffLL) return LCD_ERR_INVALID_ARG;
+  }
+  for (int i = count; i < LCD_MAX_BATCH; ++i) batch.p[i] = batch.p[0];
+  smooth_quantize_kernel<<<(unsigned)grid, kQThreads, 0, static_cast<cudaStream_t>(stream)>>>(batch);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
     set_cuda_error((int)e);
     return LCD_ERR_CUDA;
   }
   return LCD_OK;
+}
+
+lcd_status launch_smooth_quantize(const void* x, int64_t M, int64_t K, int64_t ldx, const float* inv_smooth,
+                                  const float* static_scale, uint8_t* act_idx, float* act_scale, void* stream) {
+  lcd_act_problem a;
+  a.x_fp16 = x;
+  a.M = M;
+  a.K = K;
+  a.ldx = ldx;
+  a.inv_smooth = inv_smooth;
+  a.static_scale = static_scale;
+  a.act_idx = act_idx;
+  a.act_scale = act_scale;
+  return launch_smooth_quantize_batch(&a, 1, stream);
 }
 
 }  // namespace lcd

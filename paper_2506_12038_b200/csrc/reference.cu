@@ -28,7 +28,7 @@ reference_kernel(const uint8_t* __restrict__ tiles, const uint16_t* __restrict__
   const uint8_t* act_row = act_idx + (m < M ? m : 0) * (K_pad / 2);
   float acc = 0.0f;
   for (int64_t k = 0; k < K; ++k) {
-    const uint8_t* tile = tiles + (rg * n_kt + k / kTileK) * tile_bytes;
+    const uint8_t* tile = tiles + (((rg >> 1) * n_kt + k / kTileK) * 2 + (rg & 1)) * tile_bytes;
     const uint32_t w = bits == 2 ? tile_index_2bit(tile, g, (int)(k % kTileK)) : tile_index_3bit(tile, g, (int)(k % kTileK));
     const uint32_t byte = act_row[k >> 1];
     const int q = (int)((byte >> (4 * (k & 1))) & 15u) - 8;

@@ -94,6 +94,60 @@ def test_register_lut_matches_oracle(bits, N, K, M):
 
 
 @pytest.mark.parametrize("bits", [2, 3])
+@pytest.mark.parametrize("N,K,M", [(8, 256, 1), (200, 1000, 2), (1031, 520, 5), (64, 4096, 8), (24, 11008, 16),
+                                   (520, 2304, 11)])
+def test_bucket_lut_matches_oracle(bits, N, K, M):
+    # exact integer bucket sums dotted with the fp16 codebook in fp32: no fixed-point step at all
+    run_case(gen.random_case(seed=N + K + M + bits, N=N, K=K, bits=bits, M=M), lcd.ALGO_BUCKET_LUT)
+
+
+@pytest.mark.parametrize("bits,N,K,M", [(3, 40, 11008, 16), (2, 48, 28672, 8), (3, 16, 28672, 16), (2, 2064, 28672, 16),
+                                        (3, 4096, 4096, 16)])
+def test_lookup_with_column_panels(bits, N, K, M):
+    # token count x row length too large for one shared-memory window: the columns are walked in panels and
+    # every 16-row group is finished through the integer scratch
+    L = gen.random_case(seed=N + K + M + bits, N=N, K=K, bits=bits, M=M)
+    run_case(L, lcd.ALGO_REGISTER_LUT)
+
+
+def test_grouped_launch_matches_oracle_and_leaves_scratch_zero():
+    shapes = [(2, 200, 1000, 1), (2, 4096, 512, 3), (2, 24, 11008, 5), (2, 1031, 520, 1), (2, 8, 256, 8)]
+    for bits in (2, 3):
+        cases = [gen.random_case(seed=31 * i + bits, N=N, K=K, bits=bits, M=M) for i, (_, N, K, M) in enumerate(shapes)]
+        acts, items, refs = [], [], []
+        for L in cases:
+            w = lcd.PackedWeights(lcd.pack_weights(L.idx, L.codebook, bits))
+            x, inv_s = torch.from_numpy(L.x).cuda(), torch.from_numpy(L.inv_s).cuda()
+            a = torch.empty((L.M, w.K_pad // 2), dtype=torch.uint8, device="cuda")
+            sc = torch.empty((L.M,), dtype=torch.float32, device="cuda")
+            y = torch.full((L.M, L.N), float("nan"), dtype=torch.float32, device="cuda")
+            acts.append((x, inv_s, a, sc))
+            items.append((w, a, sc, y))
+            q_ref, s_ref = O.smooth_quantize(L.x, L.inv_s)
+            refs.append((q_ref, s_ref, O.lut_linear_dequant(L.idx, L.codebook, q_ref, s_ref)))
+        qb, lb = lcd.ActBatch(acts), lcd.LinearBatch(items)
+        for _ in range(3):          # repeated calls reuse the scratch the previous call left
+            qb.run()
+            lb.run()
+        torch.cuda.synchronize()
+        assert not lb.workspace.any()
+        for (w, a, sc, y), (q_ref, s_ref, y_ref) in zip(items, refs):
+            assert np.array_equal(a.cpu().numpy(), O.pack_act(q_ref))
+            assert np.array_equal(sc.cpu().numpy(), s_ref)
+            check_y(y, y_ref)
+
+
+def test_status_word_untouched_on_success():
+    L = gen.random_case(seed=3, N=100, K=600, bits=2, M=2)
+    w = lcd.PackedWeights(lcd.pack_weights(L.idx, L.codebook, 2))
+    a, s = lcd.smooth_quantize_act(torch.from_numpy(L.x).cuda(), torch.from_numpy(L.inv_s).cuda())
+    word = torch.full((1,), 12345, dtype=torch.int32, device="cuda")
+    lcd.lut_linear(w, a, s, status_word=word)
+    torch.cuda.synchronize()
+    assert int(word.item()) == 12345
+
+
+@pytest.mark.parametrize("bits", [2, 3])
 @pytest.mark.parametrize("N,K,M", [(8, 256, 1), (200, 1000, 3), (1031, 520, 17), (64, 4096, 40), (24, 700, 33)])
 def test_reference_kernel_matches_oracle(bits, N, K, M):
     run_case(gen.random_case(seed=N + K + M + bits, N=N, K=K, bits=bits, M=M), lcd.ALGO_REFERENCE)

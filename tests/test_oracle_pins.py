@@ -207,7 +207,7 @@ def test_pack_roundtrip_random(bits, C):
     cb = rng.standard_normal((N, C)).astype(np.float16)
     blob = O.pack_weights(idx, cb, bits, C)
     assert blob.size == O.packed_weights_bytes(N, K, bits)
-    N_pad, K_pad = 24, 512
+    N_pad, K_pad = 32, 512
     assert blob.size == 256 + N_pad * K_pad * bits // 8 + ((N_pad * (1 << bits) * 2 + 255) // 256) * 256
     i2, c2, b2, C2 = O.unpack_weights(blob)
     assert np.array_equal(i2, idx) and np.array_equal(c2.view(np.uint16), cb.view(np.uint16)) and (b2, C2) == (bits, C)
@@ -236,21 +236,37 @@ def test_pack_one_hot_positions_hit_distinct_bits(bits):
 
 
 def test_pack_2bit_layout_spot_bytes():
-    # written out by hand from the layout text: tile 0, lane l = 4g+t, byte p of k-block h holds k-group
-    # G = 8t + (p+g)%8; column 128h+4G+i sits at bits [2i,2i+2)
-    N, K = 8, 256
+    # written out by hand from the layout text: item 0 = tile of rows 0-7 (512 bytes) then tile of rows 8-15;
+    # in a tile, lane l = 4g+t, byte p of k-block h holds columns 128h + 32t + 4p + i at bits [2i,2i+2)
+    N, K = 16, 256
     idx = np.zeros((N, K), dtype=np.uint8)
-    idx[0, 0] = 3          # g=0,t=0,h=0,G=0,i=0 -> p=0        -> byte 256+0,       value 0b11
-    idx[1, 5] = 2          # g=1,t=0,h=0,G=1,i=1 -> p=(1-1)%8=0 -> byte 256+16*4+0,  value 2<<2
-    idx[2, 128 + 37] = 1   # g=2,h=1,G=9 -> t=1, (p+2)%8=1 -> p=7, i=1 -> byte 256+16*(8+1)+8+7, value 1<<2
-    idx[7, 255] = 3        # g=7,h=1,G=31,t=3,(p+7)%8=7 -> p=0, i=3 -> byte 256+16*31+8+0, value 3<<6
+    idx[0, 0] = 3          # g=0,t=0,h=0,p=0,i=0            -> byte 0,                  value 0b11
+    idx[1, 5] = 2          # g=1,t=0,h=0,p=1,i=1            -> byte 16*4 + 1,           value 2<<2
+    idx[2, 128 + 37] = 1   # g=2,h=1,r=37: t=1,p=1,i=1      -> byte 16*(8+1) + 8 + 1,   value 1<<2
+    idx[7, 255] = 3        # g=7,h=1,r=127: t=3,p=7,i=3     -> byte 16*31 + 8 + 7,      value 3<<6
+    idx[9, 4] = 1          # second tile, g=1,t=0,h=0,p=1,i=0 -> byte 512 + 16*4 + 1,   value 1
     blob = O.pack_weights(idx, np.zeros((N, 4), dtype=np.float16), 2)
-    body = blob[256:256 + 512]
-    expect = np.zeros(512, dtype=np.uint8)
+    body = blob[256:256 + 1024]
+    expect = np.zeros(1024, dtype=np.uint8)
     expect[0] = 3
-    expect[16 * 4 + 0] = 2 << 2
-    expect[16 * 9 + 8 + 7] = 1 << 2
-    expect[16 * 31 + 8 + 0] = 3 << 6
+    expect[16 * 4 + 1] = 2 << 2
+    expect[16 * 9 + 8 + 1] = 1 << 2
+    expect[16 * 31 + 8 + 7] = 3 << 6
+    expect[512 + 16 * 4 + 1] = 1
+    assert np.array_equal(body, expect)
+
+
+def test_pack_item_order_two_row_groups_two_column_tiles():
+    # item (rp, kt) sits at 256 + (rp * n_kt + kt) * 1024 (2 bit): rows 16..31, columns 256..511 -> item 3
+    N, K = 32, 512
+    idx = np.zeros((N, K), dtype=np.uint8)
+    idx[16, 256] = 2       # rp=1, kt=1, first tile, g=0,t=0,h=0,p=0,i=0
+    idx[31, 0] = 1         # rp=1, kt=0, second tile, g=7,t=0,h=0,p=0,i=0 -> lane 28
+    blob = O.pack_weights(idx, np.zeros((N, 4), dtype=np.float16), 2)
+    body = blob[256:256 + 4 * 1024]
+    expect = np.zeros(4 * 1024, dtype=np.uint8)
+    expect[3 * 1024] = 2
+    expect[2 * 1024 + 512 + 16 * 28] = 1
     assert np.array_equal(body, expect)
 
 
