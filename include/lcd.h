@@ -185,6 +185,34 @@ lcd_status lcd_lut_linear_batch(const lcd_linear_problem* problems /* host */, i
                                 void* cuda_stream);
 
 /* ----------------------------------------------------------------------------------------------
+ * lcd_lut_linear for M <= 16 without a caller-provided workspace.  (No counterpart in the paper: this is a
+ * convenience of the library.)
+ *
+ * Who needs it: code that is not in a position to allocate device memory when it wants to run a layer.  A
+ * plug-in running inside a host application that owns the GPU's memory pool, a serving loop that promised
+ * its scheduler never to call cudaMalloc after start-up (the call synchronises the whole device and can fail
+ * when memory is fragmented), or a component that only ever sees buffers handed to it, cannot obtain the
+ * zero-filled workspace lcd_lut_linear asks for.  Here the integer partial sums and arrival counters live in a
+ * fixed array of LCD_STATIC_SCRATCH_BYTES that is part of the library's device image: every GPU on which the
+ * library is loaded holds that much memory until the process ends, and nothing is allocated or freed by this
+ * call (no cudaMalloc / cudaFree, no allocating library routine).
+ *
+ * Arguments as lcd_lut_linear (inputs and outputs are still the caller's); algo is AUTO, REGISTER_LUT or
+ * BUCKET_LUT.  A layer whose scratch need (lcd_lut_linear_workspace_bytes) exceeds LCD_STATIC_SCRATCH_BYTES
+ * is refused with LCD_ERR_BUFFER_TOO_SMALL before anything is enqueued; M > 16 gives LCD_ERR_UNSUPPORTED.
+ * The first call on each device looks up the array's device address (with that device current) and keeps
+ * it; make that first call outside any stream capture.  Every call uses the same array and finds what the
+ * previous call left in it, so each call first clears the part it needs (a memset enqueued on cuda_stream).
+ * Two calls that can overlap on the GPU - different streams, or different host threads on different streams -
+ * race on the array and give wrong results: serialise them, or use lcd_lut_linear with separate workspaces.
+ * -------------------------------------------------------------------------------------------- */
+#define LCD_STATIC_SCRATCH_BYTES (4u << 20)
+
+lcd_status lcd_lut_linear_static(const void* packed_weights_dev, const void* header_host, const uint8_t* act_idx,
+                                 const float* act_scale, int64_t M, float* y, int64_t ldy, lcd_algo algo,
+                                 int32_t* status_word_dev, void* cuda_stream);
+
+/* ----------------------------------------------------------------------------------------------
  * The whole online path (Section 4: input transformation -> bucket table lookup -> accumulation) from
  * HOST activations to HOST outputs, for callers that keep activations on the host: copies x to the
  * device, runs lcd_smooth_quantize_act (dynamic mode) and lcd_lut_linear (LCD_ALGO_AUTO), copies y back.

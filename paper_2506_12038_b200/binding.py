@@ -25,7 +25,8 @@ MAX_BATCH = 8
 EXPORTS = ["lcd_status_string", "lcd_last_cuda_error", "lcd_packed_weights_bytes", "lcd_pack_weights",
            "lcd_unpack_weights", "lcd_smooth_quantize_act", "lcd_lut_linear_workspace_bytes", "lcd_lut_linear",
            "lcd_linear_host_scratch_bytes", "lcd_linear_host", "lcd_smooth_quantize_act_batch",
-           "lcd_lut_linear_batch_workspace_bytes", "lcd_lut_linear_batch"]
+           "lcd_lut_linear_batch_workspace_bytes", "lcd_lut_linear_batch", "lcd_lut_linear_static"]
+STATIC_SCRATCH_BYTES = 4 << 20
 
 
 class ActProblem(Structure):
@@ -48,7 +49,7 @@ class LcdError(RuntimeError):
 
 def _load() -> ctypes.CDLL:
     if not os.path.exists(LIB_PATH):
-        raise ImportError(f"{LIB_PATH} not built: run `python -m paper_2506_12038_b200.build` "
+        raise ImportError(f"{LIB_PATH} not built: run `python paper_2506_12038_b200/build.py` "
                           "(there is no fallback path)")
     lib = ctypes.CDLL(LIB_PATH)
     lib.lcd_status_string.restype = c_char_p
@@ -70,6 +71,8 @@ def _load() -> ctypes.CDLL:
     lib.lcd_smooth_quantize_act_batch.argtypes = [POINTER(ActProblem), c_int, c_int, c_void_p]
     lib.lcd_lut_linear_batch_workspace_bytes.argtypes = [POINTER(LinearProblem), c_int, c_int, POINTER(c_size_t)]
     lib.lcd_lut_linear_batch.argtypes = [POINTER(LinearProblem), c_int, c_int, c_void_p, c_size_t, c_void_p, c_void_p]
+    lib.lcd_lut_linear_static.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_int64, c_int,
+                                          c_void_p, c_void_p]
     for name in EXPORTS:
         if name not in ("lcd_status_string", "lcd_last_cuda_error"):
             getattr(lib, name).restype = c_int
@@ -195,6 +198,18 @@ def lut_linear(w: PackedWeights, act_idx, act_scale, y=None, algo: int = ALGO_AU
                             c_void_p(status_word.data_ptr()) if status_word is not None else None,
                             _stream_ptr(stream))
     _check(st, "lcd_lut_linear")
+    return y
+
+
+def lut_linear_static(w: PackedWeights, act_idx, act_scale, y, algo: int = ALGO_AUTO, status_word=None, stream=None):
+    """lcd_lut_linear_static: M <= 16 lookup whose scratch is the library's built-in device array.  Nothing is
+    allocated here either: the caller passes y (CUDA fp32 [M, >= N]).  Calls must not overlap on the GPU."""
+    M = act_idx.shape[0]
+    st = lib.lcd_lut_linear_static(c_void_p(w.dev.data_ptr()), w.header_ptr, c_void_p(act_idx.data_ptr()),
+                                   c_void_p(act_scale.data_ptr()), M, c_void_p(y.data_ptr()), y.stride(0), algo,
+                                   c_void_p(status_word.data_ptr()) if status_word is not None else None,
+                                   _stream_ptr(stream))
+    _check(st, "lcd_lut_linear_static")
     return y
 
 
