@@ -51,8 +51,7 @@ struct GemvProblem {
   int N, n_rp, n_kt, M;
   int pw;                     // columns are walked in panels of pw items (pw == n_kt: a single panel)
   int n_panels;
-  int cta0, n_cta;            // CTAs [cta0, cta0 + n_cta) of the grid work on this problem
-  int n_warps;                // active warps of this problem, <= 16 * n_cta and <= number of items
+  int cta0, n_cta;            // CTAs [cta0, cta0 + n_cta) of the grid work on this problem, n_cta <= runs
   int tstride;                // bytes between tokens inside a staged activation window
 };
 
@@ -73,12 +72,12 @@ __device__ __forceinline__ unsigned long long globaltimer() {
   return t;
 }
 __device__ __forceinline__ void mma_s8(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ void mma_u8(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
@@ -153,10 +152,11 @@ __device__ __forceinline__ RowTables<BITS, KIND> build_tables(const RawCodebook<
     float mx = 0.0f;
 #pragma unroll
     for (int i = 0; i < C; ++i) mx = fmaxf(mx, fabsf(v[i]));
-    int ex = 0;
-    (void)frexpf(mx, &ex);                       // mx < 2^ex
-    const float up = scalbnf(1.0f, 15 - ex);     // |v| * up < 32768
-    T.scale = scalbnf(1.0f, ex - 15);
+    // mx < 2^ex from the exponent field (fp16 inputs are normal as floats); ex >= -30 keeps both powers finite
+    int ex = (int)((__float_as_uint(mx) >> 23) & 0xffu) - 126;
+    ex = ex < -30 ? -30 : ex;
+    const float up = __uint_as_float((uint32_t)(15 - ex + 127) << 23);   // 2^(15-ex): |v| * up < 32768
+    T.scale = __uint_as_float((uint32_t)(ex - 15 + 127) << 23);          // 2^(ex-15)
     uint32_t hb[2] = {0, 0}, lb[2] = {0, 0};
 #pragma unroll
     for (int i = 0; i < C; ++i) {
@@ -239,12 +239,116 @@ __device__ __forceinline__ void cursor_advance(Cursor& c, uint32_t n, const Gemv
     }
   }
 }
-// First item of warp W (of n_warps) and the warp that owns item x, for an even split of n_items.
-__device__ __forceinline__ uint32_t warp_begin(uint32_t W, uint32_t n_items, uint32_t n_warps) {
-  return (uint32_t)(((unsigned long long)W * n_items) / n_warps);
-}
-__device__ __forceinline__ uint32_t warp_of(uint32_t x, uint32_t n_items, uint32_t n_warps) {
-  return (uint32_t)((((unsigned long long)(x + 1)) * n_warps + n_items - 1) / n_items) - 1;
+// Even split of n items over w parts: first item of part i, and the part that owns item x.
+__device__ __forceinline__ uint32_t part_begin(uint32_t i, uint32_t n, uint32_t w) { return i * n / w; }
+__device__ __forceinline__ uint32_t part_of(uint32_t x, uint32_t n, uint32_t w) { return ((x + 1) * w + n - 1) / n - 1; }
+
+// Runs.  A run is the items of one 16-row group inside one panel (pw consecutive items in memory); runs are
+// numbered panel by panel.  CTA c of a problem owns the runs [c*R/C, (c+1)*R/C); its warps split the items of
+// those runs evenly.
+struct RunGeometry {
+  uint32_t n_rp, n_kt, pw, n_panels, n_runs, n_cta, n_items;
+  __device__ __forceinline__ uint32_t panel_width(uint32_t pn) const {
+    const uint32_t left = n_kt - pn * pw;
+    return left < pw ? left : pw;
+  }
+  // first item (panel-major numbering) of run r; r == n_runs gives the item count
+  __device__ __forceinline__ uint32_t run_start(uint32_t r) const {
+    if (r >= n_runs) return n_items;
+    const uint32_t pn = r / n_rp, rp = r - pn * n_rp;
+    return pn * n_rp * pw + rp * panel_width(pn);
+  }
+  // warps that work on run (pn, rp): how many, and the first one's index inside its CTA
+  __device__ __forceinline__ uint32_t contributors(uint32_t pn, uint32_t rp, uint32_t* first) const {
+    const uint32_t r = pn * n_rp + rp;
+    const uint32_t c = part_of(r, n_runs, n_cta);
+    const uint32_t x0 = run_start(part_begin(c, n_runs, n_cta)), x1 = run_start(part_begin(c + 1, n_runs, n_cta));
+    const uint32_t items = x1 - x0, nw = items < (uint32_t)kWarps ? items : (uint32_t)kWarps;
+    const uint32_t xs = run_start(r) - x0, xe = xs + panel_width(pn) - 1;
+    const uint32_t wf = part_of(xs, items, nw), wl = part_of(xe, items, nw);
+    if (first) *first = wf;
+    return wl - wf + 1;
+  }
+};
+
+// One 16-row x 256-column item: look every weight up in its row's tables and accumulate against the tokens'
+// levels.  item: the item's bytes in shared memory; q[G]: this lane's levels of token group G for the item.
+template <int BITS, int KIND, int MG>
+__device__ __forceinline__ void process_item(const uint8_t* item, const uint8_t* const (&q)[MG],
+                                             const RowTables<BITS, KIND>& Ta, const RowTables<BITS, KIND>& Tb,
+                                             int (&acc)[MG][Planes<BITS, KIND>::value][4], int lane) {
+  constexpr int HALF = 256 * BITS;
+  constexpr int PL = Planes<BITS, KIND>::value;
+  uint32_t raw_a[BITS * 2], raw_b[BITS * 2];
+  if (BITS == 2) {
+    const uint4 wa = *reinterpret_cast<const uint4*>(item + 16 * lane);
+    const uint4 wb = *reinterpret_cast<const uint4*>(item + HALF + 16 * lane);
+    raw_a[0] = wa.x; raw_a[1] = wa.y; raw_a[2] = wa.z; raw_a[3] = wa.w;
+    raw_b[0] = wb.x; raw_b[1] = wb.y; raw_b[2] = wb.z; raw_b[3] = wb.w;
+  } else {
+#pragma unroll
+    for (int b = 0; b < 3; ++b) {
+      const uint2 va = *reinterpret_cast<const uint2*>(item + 256 * b + 8 * lane);
+      const uint2 vb = *reinterpret_cast<const uint2*>(item + HALF + 256 * b + 8 * lane);
+      raw_a[b] = va.x; raw_a[3 + b] = va.y;
+      raw_b[b] = vb.x; raw_b[3 + b] = vb.y;
+    }
+  }
+  uint4 qv[2][2][MG];     // [k-block][staged words 0..3 / 4..7][token group]
+#pragma unroll
+  for (int h = 0; h < 2; ++h)
+#pragma unroll
+    for (int G = 0; G < MG; ++G) {
+      qv[h][0][G] = *reinterpret_cast<const uint4*>(q[G] + h * 128);
+      qv[h][1][G] = *reinterpret_cast<const uint4*>(q[G] + h * 128 + 16);
+    }
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    uint32_t sel_a[8], sel_b[8];    // selector words of rows g and g + 8: lookup l uses the low 16 bits of sel[l]
+    if (BITS == 2) {
+#pragma unroll
+      for (int w = 0; w < 2; ++w) {
+        const uint32_t ua = raw_a[2 * h + w], ub = raw_b[2 * h + w];
+        const uint32_t a0 = ua & 0x33333333u, a1 = (ua >> 2) & 0x33333333u;
+        const uint32_t b0 = ub & 0x33333333u, b1 = (ub >> 2) & 0x33333333u;
+        sel_a[4 * w] = a0; sel_a[4 * w + 1] = a0 >> 16; sel_a[4 * w + 2] = a1; sel_a[4 * w + 3] = a1 >> 16;
+        sel_b[4 * w] = b0; sel_b[4 * w + 1] = b0 >> 16; sel_b[4 * w + 2] = b1; sel_b[4 * w + 3] = b1 >> 16;
+      }
+    } else {
+      const uint32_t* ra = raw_a + 3 * h;
+      const uint32_t* rb = raw_b + 3 * h;
+      // bit b of columns 24..31 sits at bit 3 of the nibbles of word b: gather them into nibbles
+      const uint32_t xa = (((ra[0] >> 3) & 0x11111111u) | ((ra[1] >> 2) & 0x22222222u)) | ((ra[2] >> 1) & 0x44444444u);
+      const uint32_t xb = (((rb[0] >> 3) & 0x11111111u) | ((rb[1] >> 2) & 0x22222222u)) | ((rb[2] >> 1) & 0x44444444u);
+#pragma unroll
+      for (int b = 0; b < 3; ++b) {
+        const uint32_t da = ra[b] & 0x77777777u, db = rb[b] & 0x77777777u;
+        sel_a[2 * b] = da; sel_a[2 * b + 1] = da >> 16;
+        sel_b[2 * b] = db; sel_b[2 * b + 1] = db >> 16;
+      }
+      sel_a[6] = xa; sel_a[7] = xa >> 16;
+      sel_b[6] = xb; sel_b[7] = xb >> 16;
+    }
+    // four MMAs per plane: MMA j takes lookups 2j and 2j + 1 and staged words 2j, 2j + 1
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+#pragma unroll
+      for (int p = 0; p < PL; ++p) {
+        uint32_t a[4];
+        a[0] = pick_lookup<BITS, KIND>(Ta, sel_a[2 * j], p);
+        a[1] = pick_lookup<BITS, KIND>(Tb, sel_b[2 * j], p);
+        a[2] = pick_lookup<BITS, KIND>(Ta, sel_a[2 * j + 1], p);
+        a[3] = pick_lookup<BITS, KIND>(Tb, sel_b[2 * j + 1], p);
+#pragma unroll
+        for (int G = 0; G < MG; ++G) {
+          const uint4& qq = qv[h][j >> 1][G];
+          const uint32_t b0 = (j & 1) ? qq.z : qq.x, b1 = (j & 1) ? qq.w : qq.y;
+          if (KIND == kFixed16 && p == 1) mma_u8(acc[G][p], a, b0, b1);
+          else mma_s8(acc[G][p], a, b0, b1);
+        }
+      }
+    }
+  }
 }
 
 template <int BITS, int KIND, int MG>
@@ -252,9 +356,10 @@ __global__ void __launch_bounds__(kThreads, 1)
 lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ status) {
   extern __shared__ __align__(128) uint8_t smem[];
   constexpr int ITEM = 512 * BITS;
-  constexpr int HALF = ITEM / 2;                 // bytes of one 8-row tile
   constexpr int SLOT = kStageItems * ITEM;
   constexpr int PL = Planes<BITS, KIND>::value;
+  constexpr int ACC_INTS = MG * PL * 128;          // one warp's accumulators, [G][plane][reg][lane]
+  constexpr bool kSmemCombine = KIND == kFixed16;  // partial sums of a CTA meet in shared memory
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
 
@@ -264,15 +369,31 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
   for (int i = 1; i < batch.count; ++i)
     if ((int)blockIdx.x >= batch.p[i].cta0) pi = i;
   const GemvProblem& P = batch.p[pi];
+  RunGeometry geo;
+  geo.n_rp = (uint32_t)P.n_rp; geo.n_kt = (uint32_t)P.n_kt; geo.pw = (uint32_t)P.pw;
+  geo.n_panels = (uint32_t)P.n_panels; geo.n_runs = geo.n_panels * geo.n_rp; geo.n_cta = (uint32_t)P.n_cta;
+  geo.n_items = geo.n_rp * geo.n_kt;
   const uint32_t cta = blockIdx.x - P.cta0;
-  const uint32_t n_items = (uint32_t)P.n_rp * (uint32_t)P.n_kt;
-  const uint32_t n_warps = (uint32_t)P.n_warps;
-  if (cta * kWarps >= n_warps) return;            // whole CTA idle (uniform)
+  // the CTA's items [cx0, cx1) in panel-major numbering and its warps' shares
+  const uint32_t cx0 = geo.run_start(part_begin(cta, geo.n_runs, geo.n_cta));
+  const uint32_t cx1 = geo.run_start(part_begin(cta + 1, geo.n_runs, geo.n_cta));
+  const uint32_t c_items = cx1 - cx0;
+  const uint32_t nw = c_items < (uint32_t)kWarps ? c_items : (uint32_t)kWarps;
+  const bool warp_active = (uint32_t)warp < nw;
+  const uint32_t wx0 = warp_active ? cx0 + part_begin(warp, c_items, nw) : cx0;
+  const uint32_t wx1 = warp_active ? cx0 + part_begin(warp + 1, c_items, nw) : cx0;
+  const uint32_t panel_items = geo.n_rp * geo.pw;
+  const uint32_t pA = cx0 / panel_items, pB = (cx1 - 1) / panel_items;
 
-  uint8_t* ring = smem + kBarBytes + (size_t)warp * kDepth * SLOT;
+  // shared memory: mbarriers | combine tickets | combine slots | rings | activation windows
+  int* s_ticket = reinterpret_cast<int*>(smem + kBarBytes - 64);
+  int* s_acc = reinterpret_cast<int*>(smem + kBarBytes);
+  constexpr int COMBINE_BYTES = kSmemCombine ? kWarps * ACC_INTS * 4 : 0;
+  uint8_t* ring = smem + kBarBytes + COMBINE_BYTES + (size_t)warp * kDepth * SLOT;
   const uint32_t bar0 = smem_u32(smem) + 8u * (uint32_t)(warp * kDepth);
-  uint8_t* act_s = smem + kBarBytes + (size_t)kWarps * kDepth * SLOT;
-  const int win_bytes = (P.M < 8 * MG ? P.M : 8 * MG) * P.tstride;
+  uint8_t* act_s = smem + kBarBytes + COMBINE_BYTES + (size_t)kWarps * kDepth * SLOT;
+  const int n_tok = P.M < 8 * MG ? P.M : 8 * MG;
+  const int win_bytes = n_tok * P.tstride;
 
   if (lane == 0) {
 #pragma unroll
@@ -280,19 +401,11 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
       asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0 + 8u * s));
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    s_ticket[warp] = 0;
   }
+  if (kSmemCombine)
+    for (int i = lane; i < ACC_INTS; i += 32) s_acc[warp * ACC_INTS + i] = 0;
   __syncwarp();
-
-  // this warp's items
-  const uint32_t W = cta * kWarps + warp;
-  const bool warp_active = W < n_warps;
-  const uint32_t wx0 = warp_active ? warp_begin(W, n_items, n_warps) : 0;
-  const uint32_t wx1 = warp_active ? warp_begin(W + 1, n_items, n_warps) : 0;
-  // the CTA's items and the panels they touch
-  const uint32_t last_w = (cta + 1) * kWarps < n_warps ? (cta + 1) * kWarps : n_warps;
-  const uint32_t cx0 = warp_begin(cta * kWarps, n_items, n_warps), cx1 = warp_begin(last_w, n_items, n_warps);
-  const uint32_t panel_items = (uint32_t)P.n_rp * (uint32_t)P.pw;
-  const uint32_t pA = cx0 / panel_items, pB = (cx1 - 1) / panel_items;
 
   uint32_t stage_c = 0, stage_f = 0;    // consumed / fetched stages of this warp (ring position and parity)
   bool aborted = false;
@@ -314,10 +427,10 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
     ++stage_f;
   };
 
-  // The weights do not depend on the kernel that produced the activation indices: start streaming them
-  // before waiting for it.
+  // The weights do not depend on the kernel that produced the activation indices: start streaming them (and
+  // fetch the first rows' codebooks) before waiting for it.
   Cursor fc, cc;
-  uint32_t round_lo = 0, round_hi = 0;
+  uint32_t round_lo, round_hi;
   {
     const uint32_t lo = pA * panel_items, hi = (pA + 2) * panel_items;
     round_lo = wx0 > lo ? wx0 : lo;
@@ -327,11 +440,13 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
     cc = fc;
     while (fc.x < round_hi && stage_f - stage_c < (uint32_t)kDepth) issue(fc, round_hi);
   }
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-
   RowTables<BITS, KIND> Ta, Tb;           // rows 16*rp + g and 16*rp + 8 + g
   RawCodebook<BITS> next_a, next_b;
-  uint32_t tables_rp = 0xffffffffu, next_rp = 0xffffffffu;
+  uint32_t tables_rp = 0xffffffffu, next_rp = cc.rp < geo.n_rp ? cc.rp : 0;
+  next_a = load_codebook<BITS>(P.codebook + ((size_t)next_rp * 16 + g) * (1 << BITS));
+  next_b = load_codebook<BITS>(P.codebook + ((size_t)next_rp * 16 + 8 + g) * (1 << BITS));
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
   int acc[MG][PL][4];
 #pragma unroll
   for (int G = 0; G < MG; ++G)
@@ -341,73 +456,111 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
       for (int r = 0; r < 4; ++r) acc[G][p][r] = 0;
   uint32_t seg_kk0 = 0;
   bool seg_open = false;
+  uint32_t tok_off[MG];
+#pragma unroll
+  for (int G = 0; G < MG; ++G) tok_off[G] = (uint32_t)((8 * G + g < P.M ? 8 * G + g : P.M - 1) * P.tstride + t * 32);
 
-  // Writes the finished sums of 16-row group rp (this warp's share [seg_kk0, kk_end) of panel pn).
-  auto flush = [&](uint32_t rp, uint32_t pn, uint32_t pw_n, uint32_t kk_end) {
-    const bool direct = P.n_panels == 1 && seg_kk0 == 0 && kk_end == pw_n;
-    bool finish = direct;
-    if (!direct) {
-      int* a = P.acc + (size_t)rp * (MG * PL * 128) + lane;
+  // y of the 16-row group rp from complete sums
+  auto write_y = [&](uint32_t rp) {
+#pragma unroll
+    for (int G = 0; G < MG; ++G)
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int m = 8 * G + 2 * t + (r & 1);
+        const int n = 16 * (int)rp + g + ((r & 2) ? 8 : 0);
+        if (m < P.M && n < P.N) {
+          const RowTables<BITS, KIND>& T = (r & 2) ? Tb : Ta;
+          float v;
+          if (KIND == kFixed16) {
+            v = T.scale * ((float)acc[G][0][r] * 256.0f + (float)acc[G][1][r]);
+          } else {
+            // planes 0..C-2 hold the exact bucket sums S_1..S_{C-1}, the last one the token's sum of levels
+            int s0 = acc[G][PL - 1][r];
+#pragma unroll
+            for (int p = 0; p < PL - 1; ++p) s0 -= acc[G][p][r];
+            v = T.c[0] * (float)s0;
+#pragma unroll
+            for (int p = 0; p < PL - 1; ++p) v = fmaf(T.c[p + 1], (float)acc[G][p][r], v);
+          }
+          P.y[(size_t)m * P.ldy + n] = v * __ldg(P.act_scale + m);
+        }
+      }
+  };
+  // Adds this warp's sums to the global scratch of group rp; the warp that brings the count to `expected`
+  // takes the totals back (leaving zeros) and writes y.
+  auto global_combine = [&](uint32_t rp, uint32_t expected) {
+    int* a = P.acc + (size_t)rp * ACC_INTS + lane;
+#pragma unroll
+    for (int G = 0; G < MG; ++G)
+#pragma unroll
+      for (int p = 0; p < PL; ++p)
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+          if (8 * G + 2 * t + (r & 1) < P.M) atomicAdd(a + ((G * PL + p) * 4 + r) * 32, acc[G][p][r]);
+    __threadfence();
+    __syncwarp();
+    int old = 0;
+    if (lane == 0) old = atomicAdd(P.ticket + rp, 1);
+    old = __shfl_sync(0xffffffffu, old, 0);
+    if ((uint32_t)old + 1 == expected) {
+      __threadfence();
 #pragma unroll
       for (int G = 0; G < MG; ++G)
 #pragma unroll
         for (int p = 0; p < PL; ++p)
 #pragma unroll
           for (int r = 0; r < 4; ++r)
-            if (8 * G + 2 * t + (r & 1) < P.M) atomicAdd(a + ((G * PL + p) * 4 + r) * 32, acc[G][p][r]);
-      __threadfence();
-      __syncwarp();
-      // how many warps contribute to this 16-row group: per panel, the warps whose items meet its run
-      uint32_t part = 0;
-      if (lane < P.n_panels) {
-        const int left = P.n_kt - lane * P.pw;
-        const uint32_t w_l = (uint32_t)(left < P.pw ? left : P.pw);
-        const uint32_t r0 = (uint32_t)lane * panel_items + rp * w_l;
-        part = warp_of(r0 + w_l - 1, n_items, n_warps) - warp_of(r0, n_items, n_warps) + 1;
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-      int old = 0;
-      if (lane == 0) old = atomicAdd(P.ticket + rp, 1);
-      old = __shfl_sync(0xffffffffu, old, 0);
-      finish = (uint32_t)old + 1 == part;
-      if (finish) {
-        __threadfence();
+            if (8 * G + 2 * t + (r & 1) < P.M) acc[G][p][r] = atomicExch(a + ((G * PL + p) * 4 + r) * 32, 0);
+      if (lane == 0) atomicExch(P.ticket + rp, 0);
+      write_y(rp);
+    }
+  };
+  // This warp's share [seg_kk0, kk_end) of run (pn, rp) is summed: combine it with the other warps' shares.
+  auto flush = [&](uint32_t rp, uint32_t pn, uint32_t pw_n, uint32_t kk_end) {
+    const bool whole = seg_kk0 == 0 && kk_end == pw_n;
+    if (kSmemCombine) {
+      bool run_done = whole;
+      if (!whole) {
+        uint32_t first = 0;
+        const uint32_t n_contrib = geo.contributors(pn, rp, &first);
+        int* a = s_acc + first * ACC_INTS + lane;
 #pragma unroll
         for (int G = 0; G < MG; ++G)
 #pragma unroll
           for (int p = 0; p < PL; ++p)
 #pragma unroll
-            for (int r = 0; r < 4; ++r)
-              if (8 * G + 2 * t + (r & 1) < P.M) acc[G][p][r] = atomicExch(a + ((G * PL + p) * 4 + r) * 32, 0);
-        if (lane == 0) atomicExch(P.ticket + rp, 0);
-      }
-    }
-    if (finish) {
+            for (int r = 0; r < 4; ++r) atomicAdd(a + ((G * PL + p) * 4 + r) * 32, acc[G][p][r]);
+        __threadfence_block();
+        __syncwarp();
+        int old = 0;
+        if (lane == 0) old = atomicAdd(s_ticket + first, 1);
+        old = __shfl_sync(0xffffffffu, old, 0);
+        run_done = (uint32_t)old + 1 == n_contrib;
+        if (run_done) {
+          __threadfence_block();
 #pragma unroll
-      for (int G = 0; G < MG; ++G)
+          for (int G = 0; G < MG; ++G)
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-          const int m = 8 * G + 2 * t + (r & 1);
-          const int n = 16 * (int)rp + g + ((r & 2) ? 8 : 0);
-          if (m < P.M && n < P.N) {
-            const RowTables<BITS, KIND>& T = (r & 2) ? Tb : Ta;
-            float v;
-            if (KIND == kFixed16) {
-              v = T.scale * ((float)acc[G][0][r] * 256.0f + (float)acc[G][1][r]);
-            } else {
-              // planes 0..C-2 hold the exact bucket sums S_1..S_{C-1}, the last one the token's sum of levels
-              int s0 = acc[G][PL - 1][r];
+            for (int p = 0; p < PL; ++p)
 #pragma unroll
-              for (int p = 0; p < PL - 1; ++p) s0 -= acc[G][p][r];
-              v = T.c[0] * (float)s0;
-#pragma unroll
-              for (int p = 0; p < PL - 1; ++p) v = fmaf(T.c[p + 1], (float)acc[G][p][r], v);
-            }
-            v *= __ldg(P.act_scale + m);
-            P.y[(size_t)m * P.ldy + n] = v;
-          }
+              for (int r = 0; r < 4; ++r)
+                acc[G][p][r] = *reinterpret_cast<volatile int*>(a + ((G * PL + p) * 4 + r) * 32);
         }
+      }
+      if (run_done) {
+        if (P.n_panels == 1) write_y(rp);
+        else global_combine(rp, (uint32_t)P.n_panels);
+      }
+    } else {
+      if (whole && P.n_panels == 1) {
+        write_y(rp);
+      } else {
+        uint32_t part = 0;
+        if (lane < P.n_panels) part = geo.contributors((uint32_t)lane, rp, nullptr);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+        global_combine(rp, part);
+      }
     }
 #pragma unroll
     for (int G = 0; G < MG; ++G)
@@ -434,10 +587,7 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
 #pragma unroll 1
     for (uint32_t wdw = 0; wdw < 2 && pbase + wdw <= pB; ++wdw) {
       const uint32_t pn = pbase + wdw;
-      const int left = P.n_kt - (int)pn * P.pw;
-      const int pw_n = left < P.pw ? left : P.pw;
-      const int n_words = pw_n * 32;
-      const int n_tok = P.M < 8 * MG ? P.M : 8 * MG;
+      const int n_words = (int)geo.panel_width(pn) * 32;
       for (int m = 0; m < n_tok; ++m)
         stage_window<BITS>(reinterpret_cast<uint32_t*>(act_s + wdw * win_bytes + m * P.tstride),
                            reinterpret_cast<const uint32_t*>(P.act_idx + (size_t)m * P.n_kt * 128 +
@@ -451,13 +601,7 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
       while (cc.x < round_hi) {
         const uint32_t n = stage_len(cc, round_hi);
         const uint32_t slot = stage_c % kDepth;
-        const bool ok = __all_sync(0xffffffffu, mbar_wait(bar0 + 8u * slot, (stage_c / kDepth) & 1u));
-        if (!ok) {
-          aborted = true;
-          if (lane == 0 && status) atomicExch(status, (int)LCD_ERR_TIMEOUT);
-          break;
-        }
-        // row tables of this 16-row group
+        // row tables of this 16-row group (its codebook rows were requested one group ahead)
         if (cc.rp != tables_rp) {
           if (next_rp != cc.rp) {
             next_a = load_codebook<BITS>(P.codebook + ((size_t)cc.rp * 16 + g) * (1 << BITS));
@@ -466,109 +610,37 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
           Ta = build_tables<BITS, KIND>(next_a);
           Tb = build_tables<BITS, KIND>(next_b);
           tables_rp = cc.rp;
-          next_rp = cc.rp + 1 < (uint32_t)P.n_rp ? cc.rp + 1 : 0;
+          next_rp = cc.rp + 1 < geo.n_rp ? cc.rp + 1 : 0;
           next_a = load_codebook<BITS>(P.codebook + ((size_t)next_rp * 16 + g) * (1 << BITS));
           next_b = load_codebook<BITS>(P.codebook + ((size_t)next_rp * 16 + 8 + g) * (1 << BITS));
         }
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(bar0 + 8u * slot, (stage_c / kDepth) & 1u));
+        if (!ok) {
+          aborted = true;
+          if (lane == 0 && status) atomicExch(status, (int)LCD_ERR_TIMEOUT);
+          break;
+        }
         if (!seg_open) { seg_kk0 = cc.kk; seg_open = true; }
         const uint8_t* slot_p = ring + slot * SLOT;
-        const uint8_t* win = act_s + (cc.pn - pbase) * win_bytes;
-#pragma unroll 1
-        for (uint32_t i = 0; i < n; ++i) {
-          const uint8_t* item = slot_p + i * ITEM;
-          const uint8_t* qbase = win + (size_t)(cc.kk + i) * 256 + t * 32;
-          // the lane's indices of rows g and g + 8 for both 128-column blocks of the item
-          uint32_t raw_a[BITS * 2], raw_b[BITS * 2];
-          if (BITS == 2) {
-            const uint4 wa = *reinterpret_cast<const uint4*>(item + 16 * lane);
-            const uint4 wb = *reinterpret_cast<const uint4*>(item + HALF + 16 * lane);
-            raw_a[0] = wa.x; raw_a[1] = wa.y; raw_a[2] = wa.z; raw_a[3] = wa.w;
-            raw_b[0] = wb.x; raw_b[1] = wb.y; raw_b[2] = wb.z; raw_b[3] = wb.w;
-          } else {
+        const uint8_t* win = act_s + (cc.pn - pbase) * win_bytes + (size_t)cc.kk * 256;
 #pragma unroll
-            for (int b = 0; b < 3; ++b) {
-              const uint2 va = *reinterpret_cast<const uint2*>(item + 256 * b + 8 * lane);
-              const uint2 vb = *reinterpret_cast<const uint2*>(item + HALF + 256 * b + 8 * lane);
-              raw_a[b] = va.x; raw_a[3 + b] = va.y;
-              raw_b[b] = vb.x; raw_b[3 + b] = vb.y;
-            }
-          }
+        for (uint32_t i = 0; i < (uint32_t)kStageItems; ++i) {
+          if (i < n) {
+            const uint8_t* q[MG];
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            // activation levels of this quarter: words 0..3 and 4..7 of the staged order, per token group
-            uint4 qa[MG], qb[MG];
-#pragma unroll
-            for (int G = 0; G < MG; ++G) {
-              const int tok = 8 * G + g < P.M ? 8 * G + g : P.M - 1;
-              const uint8_t* q = qbase + (size_t)tok * P.tstride + h * 128;
-              qa[G] = *reinterpret_cast<const uint4*>(q);
-              qb[G] = *reinterpret_cast<const uint4*>(q + 16);
-            }
-            uint32_t sel_a[8], sel_b[8];    // selector words of rows g and g + 8: lookup l uses sel[l]
-            if (BITS == 2) {
-              const uint32_t ua[2] = {raw_a[2 * h], raw_a[2 * h + 1]}, ub[2] = {raw_b[2 * h], raw_b[2 * h + 1]};
-#pragma unroll
-              for (int w = 0; w < 2; ++w) {
-                const uint32_t a0 = ua[w] & 0x33333333u, a1 = (ua[w] >> 2) & 0x33333333u;
-                const uint32_t b0 = ub[w] & 0x33333333u, b1 = (ub[w] >> 2) & 0x33333333u;
-                sel_a[4 * w] = a0; sel_a[4 * w + 1] = a0 >> 16; sel_a[4 * w + 2] = a1; sel_a[4 * w + 3] = a1 >> 16;
-                sel_b[4 * w] = b0; sel_b[4 * w + 1] = b0 >> 16; sel_b[4 * w + 2] = b1; sel_b[4 * w + 3] = b1 >> 16;
-              }
-            } else {
-              uint32_t ra[3], rb[3];
-#pragma unroll
-              for (int b = 0; b < 3; ++b) {
-                ra[b] = raw_a[3 * h + b];
-                rb[b] = raw_b[3 * h + b];
-              }
-              const uint32_t xa = ((ra[0] & 0x88888888u) >> 3) | ((ra[1] & 0x88888888u) >> 2) |
-                                  ((ra[2] & 0x88888888u) >> 1);
-              const uint32_t xb = ((rb[0] & 0x88888888u) >> 3) | ((rb[1] & 0x88888888u) >> 2) |
-                                  ((rb[2] & 0x88888888u) >> 1);
-#pragma unroll
-              for (int b = 0; b < 3; ++b) {
-                const uint32_t da = ra[b] & 0x77777777u, db = rb[b] & 0x77777777u;
-                sel_a[2 * b] = da; sel_a[2 * b + 1] = da >> 16;
-                sel_b[2 * b] = db; sel_b[2 * b + 1] = db >> 16;
-              }
-              sel_a[6] = xa; sel_a[7] = xa >> 16;
-              sel_b[6] = xb; sel_b[7] = xb >> 16;
-            }
-            // four MMAs per plane: MMA j takes lookups 2j and 2j + 1 and staged words 2j, 2j + 1
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              uint32_t b0[MG], b1[MG];
-#pragma unroll
-              for (int G = 0; G < MG; ++G) {
-                const uint4& q = j < 2 ? qa[G] : qb[G];
-                b0[G] = (j & 1) ? q.z : q.x;
-                b1[G] = (j & 1) ? q.w : q.y;
-              }
-#pragma unroll
-              for (int p = 0; p < PL; ++p) {
-                uint32_t a[4];
-                a[0] = pick_lookup<BITS, KIND>(Ta, sel_a[2 * j], p);
-                a[1] = pick_lookup<BITS, KIND>(Tb, sel_b[2 * j], p);
-                a[2] = pick_lookup<BITS, KIND>(Ta, sel_a[2 * j + 1], p);
-                a[3] = pick_lookup<BITS, KIND>(Tb, sel_b[2 * j + 1], p);
-#pragma unroll
-                for (int G = 0; G < MG; ++G) {
-                  if (KIND == kFixed16 && p == 1) mma_u8(acc[G][p], a, b0[G], b1[G]);
-                  else mma_s8(acc[G][p], a, b0[G], b1[G]);
-                }
-              }
-            }
+            for (int G = 0; G < MG; ++G) q[G] = win + i * 256 + tok_off[G];
+            process_item<BITS, KIND, MG>(slot_p + i * ITEM, q, Ta, Tb, acc, lane);
           }
         }
         const uint32_t rp_done = cc.rp, pn_done = cc.pn, pw_done = cc.pw, kk_end = cc.kk + n;
         cursor_advance(cc, n, P);
+        __syncwarp();
+        ++stage_c;
+        if (fc.x < round_hi) issue(fc, round_hi);     // the slot just read is free again
         if (kk_end == pw_done || cc.x == round_hi) {
           flush(rp_done, pn_done, pw_done, kk_end);
           seg_open = false;
         }
-        __syncwarp();
-        ++stage_c;
-        if (fc.x < round_hi) issue(fc, round_hi);
       }
     }
     if (aborted) {
@@ -581,6 +653,9 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
   }
 }
 
+}  // namespace
+
+namespace {
 
 int sm_count() {
   static int cached = 0;
@@ -661,7 +736,8 @@ lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void*
 
   const int item_bytes = 512 * bits;
   const size_t ring_bytes = (size_t)kWarps * kDepth * kStageItems * item_bytes;
-  const size_t act_budget = (size_t)kMaxSmem - kBarBytes - ring_bytes;
+  const size_t combine_bytes = kind == kFixed16 ? (size_t)kWarps * MG * planes * 128 * sizeof(int) : 0;
+  const size_t act_budget = (size_t)kMaxSmem - kBarBytes - combine_bytes - ring_bytes;
 
   GemvBatch batch;
   batch.count = count;
@@ -703,25 +779,25 @@ lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void*
     const size_t need = (n_panels == 1 ? 1 : 2) * m_eff * (size_t)g.tstride;
     act_bytes = need > act_bytes ? need : act_bytes;
   }
-  // CTAs per problem: one each, then one more at a time to the problem with the most items per CTA (at most
-  // one CTA per 16 items), until every SM has one
+  // CTAs per problem: one each, then one more at a time to the problem whose most loaded CTA has the most
+  // items (a CTA owns whole runs), until every SM has one
   const int n_sm = sm_count();
   int grid = 0;
   {
-    int given[LCD_MAX_BATCH], cap[LCD_MAX_BATCH];
+    int given[LCD_MAX_BATCH];
+    long long runs[LCD_MAX_BATCH];
     int used = 0;
     for (int i = 0; i < count; ++i) {
-      const long long items = (long long)batch.p[i].n_rp * batch.p[i].n_kt;
-      cap[i] = (int)((items + kWarps - 1) / kWarps);
+      runs[i] = (long long)batch.p[i].n_panels * batch.p[i].n_rp;
       given[i] = 1;
       ++used;
     }
     while (used < n_sm) {
       int best = -1;
-      double best_load = 0.0;
+      long long best_load = 0;
       for (int i = 0; i < count; ++i) {
-        const double load = (double)batch.p[i].n_rp * batch.p[i].n_kt / given[i];
-        if (given[i] < cap[i] && (best < 0 || load > best_load)) { best = i; best_load = load; }
+        const long long load = ((runs[i] + given[i] - 1) / given[i]) * batch.p[i].pw;
+        if (given[i] < runs[i] && (best < 0 || load > best_load)) { best = i; best_load = load; }
       }
       if (best < 0) break;
       ++given[best];
@@ -730,14 +806,11 @@ lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void*
     for (int i = 0; i < count; ++i) {
       batch.p[i].cta0 = grid;
       batch.p[i].n_cta = given[i];
-      const long long items = (long long)batch.p[i].n_rp * batch.p[i].n_kt;
-      const long long w = (long long)given[i] * kWarps;
-      batch.p[i].n_warps = (int)(w < items ? w : items);
       grid += given[i];
     }
   }
   for (int i = count; i < LCD_MAX_BATCH; ++i) batch.p[i] = batch.p[0];
-  const size_t smem = kBarBytes + ring_bytes + act_bytes;
+  const size_t smem = kBarBytes + combine_bytes + ring_bytes + act_bytes;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (bits == 2) {
     if (kind == kFixed16) return MG == 1 ? launch_t<2, kFixed16, 1>(batch, grid, smem, status_word, s)

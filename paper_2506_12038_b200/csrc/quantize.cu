@@ -9,7 +9,8 @@
 
 namespace lcd {
 
-constexpr int kQThreads = 512;
+constexpr int kQThreads = 1024;
+constexpr int kQChunks = 4;    // register-resident path: K <= 8 * kQThreads * kQChunks columns
 
 __device__ __forceinline__ int quant_level(float v) {
   // round half to even, then clip to the 4-bit symmetric range
@@ -129,6 +130,93 @@ __device__ __forceinline__ void smooth_quantize_token(const __half* __restrict__
   }
 }
 
+// Same result as smooth_quantize_token<true>, for rows of at most 8 * kQThreads * kQChunks columns: every thread
+// keeps its products t_k = x_k * inv_smooth_k in registers between the maximum search and the rounding, so x
+// and inv_smooth are read once and all loads are in flight together.
+__device__ __forceinline__ void smooth_quantize_token_cached(const __half* __restrict__ x, int64_t m, int64_t K,
+                                                             int64_t K_pad, int64_t ldx,
+                                                             const float* __restrict__ inv_smooth,
+                                                             const float* __restrict__ static_scale,
+                                                             uint8_t* __restrict__ act_idx,
+                                                             float* __restrict__ act_scale) {
+  __shared__ float s_red[kQThreads / 32];
+  __shared__ float s_mult;
+  const __half* xr = x + m * ldx;
+  uint8_t* out = act_idx + m * (K_pad / 2);
+  const int tid = threadIdx.x;
+  const bool is_static = static_scale != nullptr;
+  float t[kQChunks][8];
+  float amax = 0.0f;
+#pragma unroll
+  for (int c = 0; c < kQChunks; ++c) {
+    const int64_t k = ((int64_t)c * kQThreads + tid) * 8;
+    if (k < K) {
+      const uint4 raw = *reinterpret_cast<const uint4*>(xr + k);
+      const __half2* h = reinterpret_cast<const __half2*>(&raw);
+      float f[8];
+      if (inv_smooth) {
+        const float4 a = *reinterpret_cast<const float4*>(inv_smooth + k);
+        const float4 b = *reinterpret_cast<const float4*>(inv_smooth + k + 4);
+        f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) f[i] = 1.0f;
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 v = __half22float2(h[i]);
+        t[c][2 * i] = __fmul_rn(v.x, f[2 * i]);
+        t[c][2 * i + 1] = __fmul_rn(v.y, f[2 * i + 1]);
+        amax = fmaxf(amax, fmaxf(fabsf(t[c][2 * i]), fabsf(t[c][2 * i + 1])));
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) t[c][i] = 0.0f;
+    }
+  }
+  float r = 1.0f;
+  if (!is_static) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if ((tid & 31) == 0) s_red[tid >> 5] = amax;
+    __syncthreads();
+    if (tid < 32) {
+      float v = tid < kQThreads / 32 ? s_red[tid] : 0.0f;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+      if (tid == 0) {
+        float sq = 1.0f, rr = 0.0f;
+        if (v > 0.0f) {
+          sq = __fdiv_rn(v, 7.0f);
+          rr = __fdiv_rn(7.0f, v);
+        }
+        s_mult = rr;
+        act_scale[m] = sq;
+      }
+    }
+    __syncthreads();
+    r = s_mult;
+  } else if (tid == 0) {
+    act_scale[m] = *static_scale;
+  }
+#pragma unroll
+  for (int c = 0; c < kQChunks; ++c) {
+    const int64_t k = ((int64_t)c * kQThreads + tid) * 8;
+    if (k < K_pad) {
+      uint32_t packed = 0x88888888u;
+      if (k < K) {
+        packed = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float u = is_static ? t[c][i] : __fmul_rn(t[c][i], r);
+          packed |= (uint32_t)(quant_level(u) + 8) << (4 * i);
+        }
+      }
+      *reinterpret_cast<uint32_t*>(out + k / 2) = packed;
+    }
+  }
+}
+
 struct QuantProblem {
   const __half* x;
   const float* inv_smooth;
@@ -146,8 +234,10 @@ struct QuantBatch {
 
 // One CTA per token of every problem of the batch.
 __global__ void __launch_bounds__(kQThreads) smooth_quantize_kernel(const __grid_constant__ QuantBatch batch) {
-  // let a dependent kernel (launched with programmatic stream serialization) start its own prologue now; it
-  // still waits for this grid to finish before it reads the indices
+  // This kernel may itself have been started early (programmatic stream serialization): wait for the kernel
+  // before it, then let the next one start its own prologue; that one still waits for this grid to finish
+  // before it reads the indices.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   int pi = 0;
 #pragma unroll 1
@@ -155,7 +245,9 @@ __global__ void __launch_bounds__(kQThreads) smooth_quantize_kernel(const __grid
     if ((int)blockIdx.x >= batch.p[i].cta0) pi = i;
   const QuantProblem& q = batch.p[pi];
   const int64_t m = (int64_t)blockIdx.x - q.cta0;
-  if (q.vec)
+  if (q.vec && q.K <= (long long)8 * kQThreads * kQChunks)
+    smooth_quantize_token_cached(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx, q.act_scale);
+  else if (q.vec)
     smooth_quantize_token<true>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx, q.act_scale);
   else
     smooth_quantize_token<false>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx, q.act_scale);
@@ -184,8 +276,16 @@ lcd_status launch_smooth_quantize_batch(const lcd_act_problem* probs, int count,
     if (grid > 0x7fffffffLL) return LCD_ERR_INVALID_ARG;
   }
   for (int i = count; i < LCD_MAX_BATCH; ++i) batch.p[i] = batch.p[0];
-  smooth_quantize_kernel<<<(unsigned)grid, kQThreads, 0, static_cast<cudaStream_t>(stream)>>>(batch);
-  const cudaError_t e = cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kQThreads);
+  cfg.stream = static_cast<cudaStream_t>(stream);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, smooth_quantize_kernel, batch);
   if (e != cudaSuccess) {
     set_cuda_error((int)e);
     return LCD_ERR_CUDA;
