@@ -17,7 +17,7 @@ constexpr int kTileRows = 8;    // rows of one tile
 constexpr int kPairRows = 16;   // two adjacent tiles form one 16-row item
 constexpr int kTileK = 256;
 constexpr int kKBlock = 128;
-constexpr bool kHaveDenseTc = false;  // a kernel that is not built yet is skipped by LCD_ALGO_AUTO
+constexpr bool kHaveDenseTc = true;   // a kernel that is not built yet is skipped by LCD_ALGO_AUTO
 
 #pragma pack(push, 1)
 struct Header {

@@ -1,6 +1,496 @@
-// placeholder until the tensor-core kernel lands
+// Batched-prefill path (many tokens): the layer is a dense contraction y[M x N] = diag(s_q) * Q[M x K] * Wd[N x K]^T,
+// where Wd[n][k] = cb[n][idx[n][k]] is what the lookup of Section 4.2 of the LCD paper returns and Q holds the
+// activation levels of Section 4.1.  Both are exact in fp16 (centroids are fp16, levels are integers -8..7), so
+// the tensor cores compute the same sums as the lookup-and-accumulate form, in fp32.
+//
+// Structure (one CTA per SM, persistent over output tiles of 128 weight rows x BN tokens):
+//   warp 0      TMA producer: activation tiles (fp16 levels, expanded once per call into the workspace, in the
+//               column order in which the decoder emits weights) -> shared memory, 128-byte swizzle
+//   warp 1      owns tensor memory; one lane issues tcgen05.mma (kind::f16, A and B from shared memory, fp32
+//               accumulators in tensor memory, two accumulator buffers so that the epilogue overlaps the next tile)
+//   warps 2-5   epilogue: tcgen05.ld, multiply by the token scale, coalesced fp32 stores
+//   warps 6-13  decoder: packed 2/3-bit indices -> PRMT lookups in the row's byte tables (low and high byte of
+//               the fp16 centroids) -> fp16 pairs -> K-major 128-byte-swizzled A tile in shared memory
+// Four pipeline stages of 64 columns; every wait is bounded (status word LCD_ERR_TIMEOUT on expiry, then every
+// role leaves its loop, pending copies and MMAs are drained and tensor memory is released).
+#include <cuda.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
 #include "common.h"
+
 namespace lcd {
-size_t dense_tc_workspace_bytes(int64_t, int64_t) { return 0; }
-lcd_status launch_dense_tc(const Problem&, void*, size_t, int32_t*, void*) { return LCD_ERR_UNSUPPORTED; }
+
+namespace {
+
+constexpr int kBM = 128;                 // weight rows per tile = MMA M
+constexpr int kBK = 64;                  // columns per stage = one 128-byte swizzle row of fp16
+constexpr int kStages = 4;
+constexpr int kDecodeWarps = 8, kEpiWarps = 4;
+constexpr int kFirstEpiWarp = 2, kFirstDecodeWarp = kFirstEpiWarp + kEpiWarps;
+constexpr int kDenseThreads = 32 * (kFirstDecodeWarp + kDecodeWarps);   // 448
+constexpr int kABytes = kBM * kBK * 2;   // 16 KB per stage
+constexpr unsigned long long kWaitNs = 2000000000ull;
+
+__device__ __forceinline__ uint32_t prmt_b(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+  return d;
 }
+__device__ __forceinline__ unsigned long long timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void bar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void bar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool bar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when another role gave up (abort flag) or after kWaitNs, in which case the flag
+// is raised for everybody.
+__device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (bar_try(bar, parity)) return true;
+  const unsigned long long t0 = timer_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (bar_try(bar, parity)) return true;
+    if ((it & 255u) == 0) {
+      if (*abort_flag) return false;
+      if (timer_ns() - t0 > kWaitNs) { *abort_flag = 1; return false; }
+    }
+  }
+}
+// Wait used while draining after an abort: bounded by time only.
+__device__ __forceinline__ void bar_drain(uint32_t bar, uint32_t parity) {
+  const unsigned long long t0 = timer_ns();
+  for (uint32_t it = 1; !bar_try(bar, parity); ++it)
+    if ((it & 255u) == 0 && timer_ns() - t0 > kWaitNs) return;
+}
+
+// 64-bit shared-memory matrix descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  uint64_t d = (uint64_t)((addr & 0x3ffffu) >> 4);       // start address
+  d |= (uint64_t)(1024u >> 4) << 32;                      // stride byte offset
+  d |= (uint64_t)1 << 46;                                 // descriptor version
+  d |= (uint64_t)2 << 61;                                 // 128-byte swizzle
+  return d;
+}
+// kind::f16 instruction descriptor: fp32 accumulate, fp16 A and B, both K-major, M = 128, N = n.
+__host__ __device__ constexpr uint32_t instr_desc(int n) {
+  return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+}
+__device__ __forceinline__ void mma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr) : "memory");
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Activation levels as fp16, in the column order of the decoder.  One thread per (token, 32-column quarter):
+// 16 bytes of packed 4-bit a = q + 8 in, 64 bytes of fp16 out.  Inside a quarter, position p holds column
+//   3 bit: p;      2 bit: 16*(p>>4) + 8*((p>>2)&1) + 2*(p&3) + ((p>>3)&1)
+// (the order in which the selector words of the 2-bit decoder list the weights).
+template <int BITS>
+__global__ void __launch_bounds__(256) expand_levels_kernel(const uint8_t* __restrict__ act_idx, int64_t n_quarters,
+                                                            __half* __restrict__ out) {
+  const int64_t qi = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (qi >= n_quarters) return;
+  const uint4 a = __ldg(reinterpret_cast<const uint4*>(act_idx) + qi);
+  const uint32_t src[4] = {a.x, a.y, a.z, a.w};
+  uint32_t o[16];
+#pragma unroll
+  for (int v = 0; v < 16; ++v) {
+    uint32_t pair = 0;
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int p = 2 * v + e;
+      const int col = BITS == 3 ? p : 16 * (p >> 4) + 8 * ((p >> 2) & 1) + 2 * (p & 3) + ((p >> 3) & 1);
+      const uint32_t nib = (src[col >> 3] >> (4 * (col & 7))) & 15u;
+      pair |= (0x6400u | nib) << (16 * e);        // fp16 bits of 1024 + a
+    }
+    const __half2 h = __hsub2(*reinterpret_cast<const __half2*>(&pair), __floats2half2_rn(1032.0f, 1032.0f));   // a - 8, exact
+    o[v] = *reinterpret_cast<const uint32_t*>(&h);
+  }
+  uint4* dst = reinterpret_cast<uint4*>(out + qi * 32);
+#pragma unroll
+  for (int c = 0; c < 4; ++c) dst[c] = make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+}
+
+// ---------------------------------------------------------------------------------------------------------
+struct DenseParams {
+  const uint8_t* items;
+  const uint16_t* codebook;
+  const float* act_scale;
+  float* y;
+  long long ldy;
+  int N, M, n_rp, n_kt, n_tiles_m, n_tiles;
+  int32_t* status;
+};
+
+template <int BITS, int BN>
+__global__ void __launch_bounds__(kDenseThreads, 1)
+dense_tc_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams P) {
+  extern __shared__ uint8_t smem_raw[];
+  constexpr int ITEM = 512 * BITS, HALF = 256 * BITS;
+  constexpr int kBBytes = BN * kBK * 2;
+  constexpr uint32_t kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  const uint32_t raw_addr = (uint32_t)__cvta_generic_to_shared(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  uint8_t* gen_base = smem_raw + (base - raw_addr);
+  const uint32_t a_base = base, b_base = base + kStages * kABytes, bar_base = b_base + kStages * kBBytes;
+  // barriers: full_a[4] full_b[4] empty[4] tmem_full[2] tmem_empty[2] drain
+  auto full_a = [&](int s) { return bar_base + 8u * s; };
+  auto full_b = [&](int s) { return bar_base + 8u * (kStages + s); };
+  auto empty = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
+  auto tmem_full = [&](int b) { return bar_base + 8u * (3 * kStages + b); };
+  auto tmem_empty = [&](int b) { return bar_base + 8u * (3 * kStages + 2 + b); };
+  const uint32_t drain_bar = bar_base + 8u * (3 * kStages + 4);
+  uint8_t* gen_misc = gen_base + kStages * (kABytes + kBBytes) + 8 * (3 * kStages + 5);
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(gen_misc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_misc + 4);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      bar_init(full_a(s), kDecodeWarps * 32);
+      bar_init(full_b(s), 1);
+      bar_init(empty(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      bar_init(tmem_full(b), 1);
+      bar_init(tmem_empty(b), kEpiWarps * 32);
+    }
+    bar_init(drain_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"((uint32_t)__cvta_generic_to_shared(tmem_holder)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_holder;
+
+  const int n_ks = P.n_kt * 4;     // stages per tile
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile % P.n_tiles_m) * BN;
+        for (int ks = 0; ks < n_ks; ++ks, ++it) {
+          const int slot = it % kStages;
+          if (!bar_wait(empty(slot), ((it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          bar_expect_tx(full_b(slot), kBBytes);
+          asm volatile(
+              "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+              ::"r"(b_base + slot * kBBytes), "l"(&tmap_act), "r"(ks * kBK), "r"(m0), "r"(full_b(slot)) : "memory");
+        }
+      }
+      // nothing this thread issued may still be in flight when the CTA exits
+      const uint32_t n_back = it < (uint32_t)kStages ? it : (uint32_t)kStages;
+      for (uint32_t i = 1; i <= n_back; ++i) {
+        const uint32_t j = it - i;
+        bar_drain(full_b(j % kStages), (j / kStages) & 1u);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc(BN);
+      uint32_t it = 0, tl = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, ++tl) {
+        const uint32_t buf = tl & 1u;
+        if (!bar_wait(tmem_empty(buf), ((tl >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t d_tmem = tmem_base + buf * BN;
+        for (int ks = 0; ks < n_ks; ++ks, ++it) {
+          const int slot = it % kStages;
+          const uint32_t ph = (it / kStages) & 1u;
+          if (!bar_wait(full_a(slot), ph, abort_flag) || !bar_wait(full_b(slot), ph, abort_flag)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k)
+            mma_f16(d_tmem, smem_desc(a_base + slot * kABytes + k * 32), smem_desc(b_base + slot * kBBytes + k * 32),
+                    idesc, (uint32_t)((ks | k) != 0));
+          mma_commit(empty(slot));
+        }
+        if (ok) mma_commit(tmem_full(buf));
+      }
+      // all MMAs issued so far must have finished before tensor memory is released
+      mma_commit(drain_bar);
+      bar_drain(drain_bar, 0);
+    }
+    __syncwarp();
+  } else if (warp < kFirstDecodeWarp) {
+    // ------------------------------------------------------------------ epilogue
+    const int quad = warp & 3;                    // tensor-memory lanes [32*quad, +32) belong to this warp
+    uint32_t tl = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, ++tl) {
+      const uint32_t buf = tl & 1u;
+      const int n = (tile / P.n_tiles_m) * kBM + 32 * quad + lane;
+      const int m0 = (tile % P.n_tiles_m) * BN;
+      ok = __all_sync(0xffffffffu, bar_wait(tmem_full(buf), (tl >> 1) & 1u, abort_flag));
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t v[32];
+        tmem_ld32(tmem_base + ((uint32_t)(32 * quad) << 16) + buf * BN + 32 * c, v);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        const int mc = m0 + 32 * c;
+        const float my_scale = mc + lane < P.M ? __ldg(P.act_scale + mc + lane) : 0.0f;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float s = __shfl_sync(0xffffffffu, my_scale, j);
+          if (mc + j < P.M && n < P.N) P.y[(size_t)(mc + j) * P.ldy + n] = __uint_as_float(v[j]) * s;
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      bar_arrive(tmem_empty(buf));
+    }
+  } else {
+    // ------------------------------------------------------------------ decoder
+    const int dw = warp - kFirstDecodeWarp;       // 16-row group of the tile
+    const int u = lane >> 4, g = (lane >> 1) & 7, tq = lane & 1;
+    const uint32_t row_off = (uint32_t)((2 * dw + u) * 1024 + g * 128);
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x) {
+      int rp = (tile / P.n_tiles_m) * (kBM / 16) + dw;
+      rp = rp < P.n_rp ? rp : P.n_rp - 1;          // rows past the matrix repeat the last group; never stored
+      // byte tables of this thread's row: low and high bytes of the fp16 centroids
+      uint32_t TL[2], TH[2];
+      {
+        const uint16_t* cb = P.codebook + ((size_t)rp * 16 + 8 * u + g) * (1 << BITS);
+        if (BITS == 2) {
+          const uint2 c = __ldg(reinterpret_cast<const uint2*>(cb));
+          TL[0] = TL[1] = prmt_b(c.x, c.y, 0x6420u);
+          TH[0] = TH[1] = prmt_b(c.x, c.y, 0x7531u);
+        } else {
+          const uint4 c = __ldg(reinterpret_cast<const uint4*>(cb));
+          TL[0] = prmt_b(c.x, c.y, 0x6420u); TH[0] = prmt_b(c.x, c.y, 0x7531u);
+          TL[1] = prmt_b(c.z, c.w, 0x6420u); TH[1] = prmt_b(c.z, c.w, 0x7531u);
+        }
+      }
+      const uint8_t* row_items = P.items + (size_t)rp * P.n_kt * ITEM + u * HALF;
+      // packed indices of quarters tq and tq + 2 of this row for one 256-column item: [which][word]
+      uint32_t cur[2][BITS * 2], nxt[2][BITS * 2];
+      auto load_item = [&](uint32_t (&dst)[2][BITS * 2], int kt) {
+        const uint8_t* item = row_items + (size_t)kt * ITEM;
+#pragma unroll
+        for (int w = 0; w < 2; ++w) {
+          const int l = 4 * g + tq + 2 * w;
+          if (BITS == 2) {
+            const uint4 r = __ldg(reinterpret_cast<const uint4*>(item + 16 * l));
+            dst[w][0] = r.x; dst[w][1] = r.y; dst[w][2] = r.z; dst[w][3] = r.w;
+          } else {
+#pragma unroll
+            for (int b = 0; b < 3; ++b) {
+              const uint2 r = __ldg(reinterpret_cast<const uint2*>(item + 256 * b + 8 * l));
+              dst[w][b] = r.x; dst[w][3 + b] = r.y;       // [0..2]: k-block 0, [3..5]: k-block 1
+            }
+          }
+        }
+      };
+      load_item(cur, 0);
+      for (int kt = 0; kt < P.n_kt && ok; ++kt) {
+        if (kt + 1 < P.n_kt) load_item(nxt, kt + 1);
+#pragma unroll
+        for (int j = 0; j < 4; ++j, ++it) {
+          const int slot = it % kStages;
+          if (!bar_wait(empty(slot), ((it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          // stage j of the item: k-block h = j >> 1, quarter tq + 2 * (j & 1)
+          const int w = j & 1, h = j >> 1;
+          uint32_t sel[8];
+          if (BITS == 2) {
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+              const uint32_t wd = cur[w][2 * h + x];
+              const uint32_t s0 = wd & 0x33333333u, s1 = (wd >> 2) & 0x33333333u;
+              sel[4 * x] = s0; sel[4 * x + 1] = s0 >> 16; sel[4 * x + 2] = s1; sel[4 * x + 3] = s1 >> 16;
+            }
+          } else {
+            const uint32_t r0 = cur[w][3 * h], r1 = cur[w][3 * h + 1], r2 = cur[w][3 * h + 2];
+            const uint32_t ex = (((r0 >> 3) & 0x11111111u) | ((r1 >> 2) & 0x22222222u)) | ((r2 >> 1) & 0x44444444u);
+            const uint32_t d0 = r0 & 0x77777777u, d1 = r1 & 0x77777777u, d2 = r2 & 0x77777777u;
+            sel[0] = d0; sel[1] = d0 >> 16; sel[2] = d1; sel[3] = d1 >> 16;
+            sel[4] = d2; sel[5] = d2 >> 16; sel[6] = ex; sel[7] = ex >> 16;
+          }
+          uint8_t* a_row = gen_base + slot * kABytes + row_off;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {            // 16-byte chunk c of this thread's 32 columns
+            uint32_t o[4];
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+              const uint32_t lo = prmt_b(TL[0], TL[1], sel[2 * c + x]), hi = prmt_b(TH[0], TH[1], sel[2 * c + x]);
+              o[2 * x] = prmt_b(lo, hi, 0x5140u);
+              o[2 * x + 1] = prmt_b(lo, hi, 0x7362u);
+            }
+            const int chunk = (4 * tq + c) ^ g;    // 128-byte swizzle: chunk index xor (row mod 8)
+            *reinterpret_cast<uint4*>(a_row + 16 * chunk) = make_uint4(o[0], o[1], o[2], o[3]);
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic stores -> visible to the MMA
+          bar_arrive(full_a(slot));
+        }
+#pragma unroll
+        for (int w = 0; w < 2; ++w)
+#pragma unroll
+          for (int x = 0; x < BITS * 2; ++x) cur[w][x] = nxt[w][x];
+      }
+    }
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+  if (threadIdx.x == 0 && *abort_flag && P.status) atomicExch(P.status, (int)LCD_ERR_TIMEOUT);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+int dense_sm_count() {
+  static int cached = 0;
+  if (cached == 0) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
+      n = 148;
+    cached = n;
+  }
+  return cached;
+}
+
+template <int BITS, int BN>
+lcd_status launch_dense_t(const Problem& p, __half* levels, int32_t* status_word, cudaStream_t stream) {
+  EncodeTiledFn enc = encode_tiled();
+  if (!enc) return LCD_ERR_CUDA;
+  CUtensorMap tmap;
+  const cuuint64_t dims[2] = {(cuuint64_t)p.K_pad, (cuuint64_t)p.M};
+  const cuuint64_t strides[1] = {(cuuint64_t)p.K_pad * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)BN};
+  const cuuint32_t estr[2] = {1, 1};
+  if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, levels, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return LCD_ERR_CUDA;
+  DenseParams dp;
+  dp.items = p.tiles;
+  dp.codebook = p.codebook;
+  dp.act_scale = p.act_scale;
+  dp.y = p.y;
+  dp.ldy = p.ldy;
+  dp.N = (int)p.N;
+  dp.M = (int)p.M;
+  dp.n_rp = (int)(p.N_pad / kPairRows);
+  dp.n_kt = (int)(p.K_pad / kTileK);
+  dp.n_tiles_m = (int)((p.M + BN - 1) / BN);
+  dp.n_tiles = dp.n_tiles_m * (int)((p.N_pad + kBM - 1) / kBM);
+  dp.status = status_word;
+  const size_t smem = 1024 + (size_t)kStages * (kABytes + BN * kBK * 2) + 256;
+  auto kern = dense_tc_kernel<BITS, BN>;
+  static bool attr_set = false;   // per template instance
+  if (!attr_set) {
+    const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
+    attr_set = true;
+  }
+  const int grid = dp.n_tiles < dense_sm_count() ? dp.n_tiles : dense_sm_count();
+  kern<<<grid, kDenseThreads, smem, stream>>>(tmap, dp);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
+  return LCD_OK;
+}
+
+// Tokens per tile: the width whose (waves of tiles) x (tile time) is smallest; the decoder's work per tile does
+// not depend on the width, which is what the constant stands for.
+int pick_bn(int64_t M, int64_t N_pad) {
+  const int n_sm = dense_sm_count();
+  const int64_t tiles_n = (N_pad + kBM - 1) / kBM;
+  int best = 32;
+  int64_t best_cost = -1;
+  for (int bn = 32; bn <= 256; bn *= 2) {
+    const int64_t tiles = tiles_n * ((M + bn - 1) / bn);
+    const int64_t cost = ((tiles + n_sm - 1) / n_sm) * (bn + 48);
+    if (best_cost < 0 || cost < best_cost) { best = bn; best_cost = cost; }
+  }
+  return best;
+}
+
+}  // namespace
+
+size_t dense_tc_workspace_bytes(int64_t M, int64_t K_pad) { return (size_t)round_up_u64((uint64_t)M * K_pad * 2, 256); }
+
+lcd_status launch_dense_tc(const Problem& p, void* workspace, size_t workspace_bytes, int32_t* status_word,
+                           void* stream) {
+  if (!workspace || workspace_bytes < dense_tc_workspace_bytes(p.M, p.K_pad)) return LCD_ERR_BUFFER_TOO_SMALL;
+  if (p.M > 0x7fffffffLL / 2 || p.N > 0x7fffffffLL / 2) return LCD_ERR_UNSUPPORTED;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  __half* levels = static_cast<__half*>(workspace);
+  const int64_t n_quarters = p.M * (p.K_pad / 32);
+  const unsigned blocks = (unsigned)((n_quarters + 255) / 256);
+  if (p.bits == 2) expand_levels_kernel<2><<<blocks, 256, 0, s>>>(p.act_idx, n_quarters, levels);
+  else expand_levels_kernel<3><<<blocks, 256, 0, s>>>(p.act_idx, n_quarters, levels);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
+  const int bn = pick_bn(p.M, p.N_pad);
+#define LCD_DENSE_CASE(B, W) \
+  if (p.bits == B && bn == W) return launch_dense_t<B, W>(p, levels, status_word, s);
+  LCD_DENSE_CASE(2, 32) LCD_DENSE_CASE(2, 64) LCD_DENSE_CASE(2, 128) LCD_DENSE_CASE(2, 256)
+  LCD_DENSE_CASE(3, 32) LCD_DENSE_CASE(3, 64) LCD_DENSE_CASE(3, 128) LCD_DENSE_CASE(3, 256)
+#undef LCD_DENSE_CASE
+  return LCD_ERR_UNSUPPORTED;
+}
+
+}  // namespace lcd
