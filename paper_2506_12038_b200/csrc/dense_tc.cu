@@ -9,7 +9,7 @@
 //   warp 1      owns tensor memory; one lane issues tcgen05.mma (kind::f16, A and B from shared memory, fp32
 //               accumulators in tensor memory, two accumulator buffers so that the epilogue overlaps the next tile)
 //   warps 2-5   epilogue: tcgen05.ld, multiply by the token scale, coalesced fp32 stores
-//   warps 6-13  decoder: packed 2/3-bit indices -> PRMT lookups in the row's byte tables (low and high byte of
+//   warps 6-21  decoder (two groups of 8 warps on alternate stages): packed 2/3-bit indices -> PRMT lookups in the row's byte tables (low and high byte of
 //               the fp16 centroids) -> fp16 pairs -> K-major 128-byte-swizzled A tile in shared memory
 // Four pipeline stages of 64 columns; every wait is bounded (status word LCD_ERR_TIMEOUT on expiry, then every
 // role leaves its loop, pending copies and MMAs are drained and tensor memory is released).
@@ -26,9 +26,9 @@ namespace {
 constexpr int kBM = 128;                 // weight rows per tile = MMA M
 constexpr int kBK = 64;                  // columns per stage = one 128-byte swizzle row of fp16
 constexpr int kStages = 4;
-constexpr int kDecodeWarps = 8, kEpiWarps = 4;
+constexpr int kDecodeWarps = 16, kEpiWarps = 4;   // decoder: two groups of 8 warps
 constexpr int kFirstEpiWarp = 2, kFirstDecodeWarp = kFirstEpiWarp + kEpiWarps;
-constexpr int kDenseThreads = 32 * (kFirstDecodeWarp + kDecodeWarps);   // 448
+constexpr int kDenseThreads = 32 * (kFirstDecodeWarp + kDecodeWarps);   // 704
 constexpr int kABytes = kBM * kBK * 2;   // 16 KB per stage
 constexpr unsigned long long kWaitNs = 2000000000ull;
 
@@ -117,6 +117,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
 template <int BITS>
 __global__ void __launch_bounds__(256) expand_levels_kernel(const uint8_t* __restrict__ act_idx, int64_t n_quarters,
                                                             __half* __restrict__ out) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the tensor-core kernel may set itself up meanwhile
   const int64_t qi = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (qi >= n_quarters) return;
   const uint4 a = __ldg(reinterpret_cast<const uint4*>(act_idx) + qi);
@@ -157,7 +158,7 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
   extern __shared__ uint8_t smem_raw[];
   constexpr int ITEM = 512 * BITS, HALF = 256 * BITS;
   constexpr int kBBytes = BN * kBK * 2;
-  constexpr uint32_t kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;
+  constexpr uint32_t kTmemCols = 2 * BN <= 256 ? 256 : 512;   // a power of two that holds both accumulator buffers
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   const uint32_t raw_addr = (uint32_t)__cvta_generic_to_shared(smem_raw);
@@ -177,7 +178,7 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      bar_init(full_a(s), kDecodeWarps * 32);
+      bar_init(full_a(s), (kDecodeWarps / 2) * 32);   // one decoder group fills a stage
       bar_init(full_b(s), 1);
       bar_init(empty(s), 1);
     }
@@ -207,6 +208,9 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
+      // the fp16 levels are written by the kernel launched just before this one: wait for it here (the other
+      // roles only touch data that was complete before that kernel started)
+      asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x) {
         const int m0 = (tile % P.n_tiles_m) * BN;
         for (int ks = 0; ks < n_ks; ++ks, ++it) {
@@ -285,12 +289,16 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
     }
   } else {
     // ------------------------------------------------------------------ decoder
-    const int dw = warp - kFirstDecodeWarp;       // 16-row group of the tile
+    // Two groups of 8 warps take alternate stages (group = stage parity), so that one group's shared-memory
+    // stores, proxy fence and barrier round trip overlap the other group's lookups.  Inside a group, warp dw
+    // owns the tile's 16-row group dw and a thread owns 32 columns of one row per stage.
+    const int grp = (warp - kFirstDecodeWarp) >> 3, dw = (warp - kFirstDecodeWarp) & 7;
     const int u = lane >> 4, g = (lane >> 1) & 7, tq = lane & 1;
     const uint32_t row_off = (uint32_t)((2 * dw + u) * 1024 + g * 128);
-    uint32_t it = 0;
+    const int rec_lane = 4 * g + tq + 2 * grp;     // the quarter of the row this thread decodes: tq + 2 * grp
+    uint32_t it0 = 0;                              // stage number of the tile's first stage
     bool ok = true;
-    for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x) {
+    for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, it0 += (uint32_t)n_ks) {
       int rp = (tile / P.n_tiles_m) * (kBM / 16) + dw;
       rp = rp < P.n_rp ? rp : P.n_rp - 1;          // rows past the matrix repeat the last group; never stored
       // byte tables of this thread's row: low and high bytes of the fp16 centroids
@@ -308,22 +316,18 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
         }
       }
       const uint8_t* row_items = P.items + (size_t)rp * P.n_kt * ITEM + u * HALF;
-      // packed indices of quarters tq and tq + 2 of this row for one 256-column item: [which][word]
-      uint32_t cur[2][BITS * 2], nxt[2][BITS * 2];
-      auto load_item = [&](uint32_t (&dst)[2][BITS * 2], int kt) {
+      // packed indices of this thread's quarter for one 256-column item: both 128-column k-blocks
+      uint32_t cur[BITS * 2], nxt[BITS * 2];
+      auto load_item = [&](uint32_t (&dst)[BITS * 2], int kt) {
         const uint8_t* item = row_items + (size_t)kt * ITEM;
+        if (BITS == 2) {
+          const uint4 r = __ldg(reinterpret_cast<const uint4*>(item + 16 * rec_lane));
+          dst[0] = r.x; dst[1] = r.y; dst[2] = r.z; dst[3] = r.w;
+        } else {
 #pragma unroll
-        for (int w = 0; w < 2; ++w) {
-          const int l = 4 * g + tq + 2 * w;
-          if (BITS == 2) {
-            const uint4 r = __ldg(reinterpret_cast<const uint4*>(item + 16 * l));
-            dst[w][0] = r.x; dst[w][1] = r.y; dst[w][2] = r.z; dst[w][3] = r.w;
-          } else {
-#pragma unroll
-            for (int b = 0; b < 3; ++b) {
-              const uint2 r = __ldg(reinterpret_cast<const uint2*>(item + 256 * b + 8 * l));
-              dst[w][b] = r.x; dst[w][3 + b] = r.y;       // [0..2]: k-block 0, [3..5]: k-block 1
-            }
+          for (int b = 0; b < 3; ++b) {
+            const uint2 r = __ldg(reinterpret_cast<const uint2*>(item + 256 * b + 8 * rec_lane));
+            dst[b] = r.x; dst[3 + b] = r.y;       // [0..2]: k-block 0, [3..5]: k-block 1
           }
         }
       };
@@ -331,21 +335,21 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
       for (int kt = 0; kt < P.n_kt && ok; ++kt) {
         if (kt + 1 < P.n_kt) load_item(nxt, kt + 1);
 #pragma unroll
-        for (int j = 0; j < 4; ++j, ++it) {
+        for (int h = 0; h < 2; ++h) {
+          // stage 2h + grp of the item: k-block h, quarters 2 * grp and 2 * grp + 1
+          const uint32_t it = it0 + 4u * (uint32_t)kt + 2u * h + grp;
           const int slot = it % kStages;
           if (!bar_wait(empty(slot), ((it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-          // stage j of the item: k-block h = j >> 1, quarter tq + 2 * (j & 1)
-          const int w = j & 1, h = j >> 1;
           uint32_t sel[8];
           if (BITS == 2) {
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
-              const uint32_t wd = cur[w][2 * h + x];
+              const uint32_t wd = cur[2 * h + x];
               const uint32_t s0 = wd & 0x33333333u, s1 = (wd >> 2) & 0x33333333u;
               sel[4 * x] = s0; sel[4 * x + 1] = s0 >> 16; sel[4 * x + 2] = s1; sel[4 * x + 3] = s1 >> 16;
             }
           } else {
-            const uint32_t r0 = cur[w][3 * h], r1 = cur[w][3 * h + 1], r2 = cur[w][3 * h + 2];
+            const uint32_t r0 = cur[3 * h], r1 = cur[3 * h + 1], r2 = cur[3 * h + 2];
             const uint32_t ex = (((r0 >> 3) & 0x11111111u) | ((r1 >> 2) & 0x22222222u)) | ((r2 >> 1) & 0x44444444u);
             const uint32_t d0 = r0 & 0x77777777u, d1 = r1 & 0x77777777u, d2 = r2 & 0x77777777u;
             sel[0] = d0; sel[1] = d0 >> 16; sel[2] = d1; sel[3] = d1 >> 16;
@@ -368,9 +372,7 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
           bar_arrive(full_a(slot));
         }
 #pragma unroll
-        for (int w = 0; w < 2; ++w)
-#pragma unroll
-          for (int x = 0; x < BITS * 2; ++x) cur[w][x] = nxt[w][x];
+        for (int x = 0; x < BITS * 2; ++x) cur[x] = nxt[x];
       }
     }
   }
@@ -447,23 +449,34 @@ lcd_status launch_dense_t(const Problem& p, __half* levels, int32_t* status_word
     attr_set = true;
   }
   const int grid = dp.n_tiles < dense_sm_count() ? dp.n_tiles : dense_sm_count();
-  kern<<<grid, kDenseThreads, smem, stream>>>(tmap, dp);
-  const cudaError_t e = cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kDenseThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see the producer's griddepcontrol.wait
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmap, dp);
   if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
   return LCD_OK;
 }
 
-// Tokens per tile: the width whose (waves of tiles) x (tile time) is smallest; the decoder's work per tile does
-// not depend on the width, which is what the constant stands for.
+// Tokens per tile: the width whose (waves of tiles) x (tile time) is smallest.  A tile's time grows with its
+// width but not below the time the decoder and the shared-memory traffic of the A operand need.
 int pick_bn(int64_t M, int64_t N_pad) {
   const int n_sm = dense_sm_count();
   const int64_t tiles_n = (N_pad + kBM - 1) / kBM;
-  int best = 32;
+  const int widths[3] = {128, 192, 256};
+  int best = 128;
   int64_t best_cost = -1;
-  for (int bn = 32; bn <= 256; bn *= 2) {
+  for (int i = 0; i < 3; ++i) {
+    const int bn = widths[i];
     const int64_t tiles = tiles_n * ((M + bn - 1) / bn);
-    const int64_t cost = ((tiles + n_sm - 1) / n_sm) * (bn + 48);
-    if (best_cost < 0 || cost < best_cost) { best = bn; best_cost = cost; }
+    const int64_t cost = ((tiles + n_sm - 1) / n_sm) * (bn > 150 ? bn : 150);
+    if (best_cost < 0 || cost <= best_cost) { best = bn; best_cost = cost; }
   }
   return best;
 }
@@ -487,8 +500,8 @@ lcd_status launch_dense_tc(const Problem& p, void* workspace, size_t workspace_b
   const int bn = pick_bn(p.M, p.N_pad);
 #define LCD_DENSE_CASE(B, W) \
   if (p.bits == B && bn == W) return launch_dense_t<B, W>(p, levels, status_word, s);
-  LCD_DENSE_CASE(2, 32) LCD_DENSE_CASE(2, 64) LCD_DENSE_CASE(2, 128) LCD_DENSE_CASE(2, 256)
-  LCD_DENSE_CASE(3, 32) LCD_DENSE_CASE(3, 64) LCD_DENSE_CASE(3, 128) LCD_DENSE_CASE(3, 256)
+  LCD_DENSE_CASE(2, 128) LCD_DENSE_CASE(2, 192) LCD_DENSE_CASE(2, 256)
+  LCD_DENSE_CASE(3, 128) LCD_DENSE_CASE(3, 192) LCD_DENSE_CASE(3, 256)
 #undef LCD_DENSE_CASE
   return LCD_ERR_UNSUPPORTED;
 }
