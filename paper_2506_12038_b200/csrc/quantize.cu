@@ -9,7 +9,8 @@
 
 namespace lcd {
 
-constexpr int kQThreads = 1024;
+constexpr int kQThreads = 1024;   // few tokens: one large CTA per token, everything in registers
+constexpr int kQThreadsMany = 256; // many tokens: small CTAs, latency hidden by the number of CTAs
 constexpr int kQChunks = 4;    // register-resident path: K <= 8 * kQThreads * kQChunks columns
 
 __device__ __forceinline__ int quant_level(float v) {
@@ -21,13 +22,13 @@ __device__ __forceinline__ int quant_level(float v) {
 
 // One token per CTA.  VEC: rows are 16-byte aligned and K is a multiple of 8, so each thread handles 8
 // consecutive columns per step (one 16-byte load of x, two of inv_smooth, one 4-byte store).
-template <bool VEC>
+template <bool VEC, int THREADS>
 __device__ __forceinline__ void smooth_quantize_token(const __half* __restrict__ x, int64_t m, int64_t K,
                                                       int64_t K_pad, int64_t ldx,
                                                       const float* __restrict__ inv_smooth,
                                                       const float* __restrict__ static_scale,
                                                       uint8_t* __restrict__ act_idx, float* __restrict__ act_scale) {
-  __shared__ float s_red[kQThreads / 32];
+  __shared__ float s_red[THREADS / 32];
   __shared__ float s_mult;
   const __half* xr = x + m * ldx;
   uint8_t* out = act_idx + m * (K_pad / 2);
@@ -37,7 +38,7 @@ __device__ __forceinline__ void smooth_quantize_token(const __half* __restrict__
   if (!is_static) {
     float amax = 0.0f;
     if (VEC) {
-      for (int64_t k = (int64_t)tid * 8; k < K; k += (int64_t)kQThreads * 8) {
+      for (int64_t k = (int64_t)tid * 8; k < K; k += (int64_t)THREADS * 8) {
         const uint4 raw = *reinterpret_cast<const uint4*>(xr + k);
         const __half2* h = reinterpret_cast<const __half2*>(&raw);
         float f[8];
@@ -57,7 +58,7 @@ __device__ __forceinline__ void smooth_quantize_token(const __half* __restrict__
         }
       }
     } else {
-      for (int64_t k = tid; k < K; k += kQThreads) {
+      for (int64_t k = tid; k < K; k += THREADS) {
         const float f = inv_smooth ? inv_smooth[k] : 1.0f;
         amax = fmaxf(amax, fabsf(__fmul_rn(__half2float(xr[k]), f)));
       }
@@ -67,7 +68,7 @@ __device__ __forceinline__ void smooth_quantize_token(const __half* __restrict__
     if ((tid & 31) == 0) s_red[tid >> 5] = amax;
     __syncthreads();
     if (tid < 32) {
-      float v = tid < kQThreads / 32 ? s_red[tid] : 0.0f;
+      float v = tid < THREADS / 32 ? s_red[tid] : 0.0f;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
       if (tid == 0) {
@@ -87,7 +88,7 @@ __device__ __forceinline__ void smooth_quantize_token(const __half* __restrict__
   const float r = is_static ? 1.0f : s_mult;
 
   if (VEC) {
-    for (int64_t k = (int64_t)tid * 8; k < K_pad; k += (int64_t)kQThreads * 8) {
+    for (int64_t k = (int64_t)tid * 8; k < K_pad; k += (int64_t)THREADS * 8) {
       uint32_t packed = 0x88888888u;
       if (k < K) {
         const uint4 raw = *reinterpret_cast<const uint4*>(xr + k);
@@ -114,7 +115,7 @@ __device__ __forceinline__ void smooth_quantize_token(const __half* __restrict__
       *reinterpret_cast<uint32_t*>(out + k / 2) = packed;
     }
   } else {
-    for (int64_t j = tid; j < K_pad / 2; j += kQThreads) {
+    for (int64_t j = tid; j < K_pad / 2; j += THREADS) {
       uint32_t a[2] = {8u, 8u};
 #pragma unroll
       for (int i = 0; i < 2; ++i) {
@@ -233,7 +234,8 @@ struct QuantBatch {
 };
 
 // One CTA per token of every problem of the batch.
-__global__ void __launch_bounds__(kQThreads) smooth_quantize_kernel(const __grid_constant__ QuantBatch batch) {
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS) smooth_quantize_kernel(const __grid_constant__ QuantBatch batch) {
   // This kernel may itself have been started early (programmatic stream serialization): wait for the kernel
   // before it, then let the next one start its own prologue; that one still waits for this grid to finish
   // before it reads the indices.
@@ -245,12 +247,12 @@ __global__ void __launch_bounds__(kQThreads) smooth_quantize_kernel(const __grid
     if ((int)blockIdx.x >= batch.p[i].cta0) pi = i;
   const QuantProblem& q = batch.p[pi];
   const int64_t m = (int64_t)blockIdx.x - q.cta0;
-  if (q.vec && q.K <= (long long)8 * kQThreads * kQChunks)
+  if (THREADS == kQThreads && q.vec && q.K <= (long long)8 * kQThreads * kQChunks)
     smooth_quantize_token_cached(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx, q.act_scale);
   else if (q.vec)
-    smooth_quantize_token<true>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx, q.act_scale);
+    smooth_quantize_token<true, THREADS>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx, q.act_scale);
   else
-    smooth_quantize_token<false>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx, q.act_scale);
+    smooth_quantize_token<false, THREADS>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx, q.act_scale);
 }
 
 lcd_status launch_smooth_quantize_batch(const lcd_act_problem* probs, int count, void* stream) {
@@ -278,14 +280,16 @@ lcd_status launch_smooth_quantize_batch(const lcd_act_problem* probs, int count,
   for (int i = count; i < LCD_MAX_BATCH; ++i) batch.p[i] = batch.p[0];
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
-  cfg.blockDim = dim3(kQThreads);
+  const bool many = grid > 296;
+  cfg.blockDim = dim3(many ? kQThreadsMany : kQThreads);
   cfg.stream = static_cast<cudaStream_t>(stream);
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  const cudaError_t e = cudaLaunchKernelEx(&cfg, smooth_quantize_kernel, batch);
+  const cudaError_t e = many ? cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany>, batch)
+                             : cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreads>, batch);
   if (e != cudaSuccess) {
     set_cuda_error((int)e);
     return LCD_ERR_CUDA;

@@ -215,3 +215,57 @@ def test_host_buffer_entry_point():
     torch.cuda.synchronize()
     q_ref, s_ref = O.smooth_quantize(L.x, L.inv_s)
     check_y(y_host, O.lut_linear_dequant(L.idx, L.codebook, q_ref, s_ref))
+
+
+# ------------------------------------------------------------------------------- full sizes, bench launch shape
+def _sampled_rows_check(L, y, q_ref, s_ref, n_rows=48, seed=0):
+    rows = np.sort(gen.permutation(seed + L.N, L.N)[:n_rows])
+    y_ref = O.lut_linear_rows(L.idx, L.codebook, q_ref, s_ref, rows)
+    check_y(y[:, torch.from_numpy(rows).cuda()], y_ref)
+
+
+def test_full_size_decode_layer_grouped_launch_sampled_rows():
+    # the LLaMA-7B-shaped layer at M = 1 with 2-bit weights, launched exactly as the benchmark does: one grouped
+    # quantise launch and one grouped lookup launch over the seven projections; activation indices are compared
+    # completely, outputs on sampled rows (the oracle computes those one by one)
+    cfg = gen.CONFIGS[1]
+    acts, items, cases = [], [], []
+    for mi, (name, N, K) in enumerate(cfg["shapes"]):
+        L = gen.make_layer(1, mi, N, K, cfg["bits"], 1, outlier_frac=cfg["frac"], outlier_scale=cfg["scale"])
+        w = lcd.PackedWeights(lcd.pack_weights(L.idx, L.codebook, L.bits))
+        x, inv_s = torch.from_numpy(L.x).cuda(), torch.from_numpy(L.inv_s).cuda()
+        a = torch.empty((1, w.K_pad // 2), dtype=torch.uint8, device="cuda")
+        sc = torch.empty((1,), dtype=torch.float32, device="cuda")
+        y = torch.full((1, N), float("nan"), dtype=torch.float32, device="cuda")
+        acts.append((x, inv_s, a, sc))
+        items.append((w, a, sc, y))
+        cases.append(L)
+    qb, lb = lcd.ActBatch(acts), lcd.LinearBatch(items)
+    qb.run()
+    lb.run()
+    torch.cuda.synchronize()
+    assert not lb.workspace.any()
+    for L, (w, a, sc, y) in zip(cases, items):
+        q_ref, s_ref = O.smooth_quantize(L.x, L.inv_s)
+        assert np.array_equal(a.cpu().numpy(), O.pack_act(q_ref))
+        assert np.array_equal(sc.cpu().numpy(), s_ref)
+        assert torch.isfinite(y).all()
+        _sampled_rows_check(L, y, q_ref, s_ref)
+
+
+@pytest.mark.parametrize("mi", [0, 4])      # q 5120 x 5120 (192-token tiles), gate 13824 x 5120 (256-token tiles)
+def test_full_size_prefill_matrix_sampled_rows(mi):
+    cfg = gen.CONFIGS[3]
+    name, N, K = cfg["shapes"][mi]
+    M = 2048
+    L = gen.make_layer(3, mi, N, K, cfg["bits"], M, outlier_frac=cfg["frac"], outlier_scale=cfg["scale"])
+    w = lcd.PackedWeights(lcd.pack_weights(L.idx, L.codebook, L.bits))
+    a, s = lcd.smooth_quantize_act(torch.from_numpy(L.x).cuda(), torch.from_numpy(L.inv_s).cuda())
+    word = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    y = lcd.lut_linear(w, a, s, status_word=word)
+    torch.cuda.synchronize()
+    assert int(word.item()) == 0
+    q_ref, s_ref = O.smooth_quantize(L.x, L.inv_s)
+    assert np.array_equal(a.cpu().numpy(), O.pack_act(q_ref))
+    assert torch.isfinite(y).all()
+    _sampled_rows_check(L, y, q_ref, s_ref, n_rows=32)
