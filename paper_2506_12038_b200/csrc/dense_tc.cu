@@ -386,6 +386,258 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
   if (threadIdx.x == 0 && *abort_flag && P.status) atomicExch(P.status, (int)LCD_ERR_TIMEOUT);
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Variant for tiles of at most 192 tokens: the decoded A operand never touches shared memory.  The decoder
+// writes fp16 pairs straight from registers into tensor memory (tcgen05.st: a thread owns one row of the tile,
+// a warp the 32 tensor-memory lanes of its quadrant) and the MMA takes A from tensor memory.  Shared memory then
+// carries only the token tiles, which is what bounds the kernel above (see the profile of that kernel).
+// Tensor memory: two accumulators of BN columns, then four A stages of 32 columns (64 fp16 per row).
+// Warps: 0 TMA, 1 MMA, 2-5 epilogue, 6-21 decoder = 4 groups x 4 quadrant warps; group i decodes the stages
+// whose number is i modulo 4.
+__device__ __forceinline__ void mma_f16_ta(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
+        "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
+        "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]) : "memory");
+}
+
+template <int BITS, int BN>
+__global__ void __launch_bounds__(kDenseThreads, 1)
+dense_tc_ta_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams P) {
+  extern __shared__ uint8_t smem_raw[];
+  constexpr int ITEM = 512 * BITS, HALF = 256 * BITS;
+  constexpr int kBBytes = BN * kBK * 2;
+  constexpr uint32_t kTmemCols = 512;
+  constexpr uint32_t kACol0 = 2 * BN;              // first tensor-memory column of the A stages
+  static_assert(2 * BN + kStages * 32 <= 512, "tensor memory holds two accumulators and four A stages");
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  const uint32_t raw_addr = (uint32_t)__cvta_generic_to_shared(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  uint8_t* gen_base = smem_raw + (base - raw_addr);
+  const uint32_t b_base = base, bar_base = b_base + kStages * kBBytes;
+  auto full_a = [&](int s) { return bar_base + 8u * s; };
+  auto full_b = [&](int s) { return bar_base + 8u * (kStages + s); };
+  auto empty = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
+  auto tmem_full = [&](int b) { return bar_base + 8u * (3 * kStages + b); };
+  auto tmem_empty = [&](int b) { return bar_base + 8u * (3 * kStages + 2 + b); };
+  const uint32_t drain_bar = bar_base + 8u * (3 * kStages + 4);
+  uint8_t* gen_misc = gen_base + kStages * kBBytes + 8 * (3 * kStages + 5);
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(gen_misc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_misc + 4);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      bar_init(full_a(s), 4 * 32);                 // the four quadrant warps of one decoder group
+      bar_init(full_b(s), 1);
+      bar_init(empty(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      bar_init(tmem_full(b), 1);
+      bar_init(tmem_empty(b), kEpiWarps * 32);
+    }
+    bar_init(drain_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"((uint32_t)__cvta_generic_to_shared(tmem_holder)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_holder;
+
+  const int n_ks = P.n_kt * 4;     // stages per tile (a multiple of four: stage number mod 4 == stage of the item)
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      asm volatile("griddepcontrol.wait;" ::: "memory");      // the levels come from the kernel launched before
+      for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile % P.n_tiles_m) * BN;
+        for (int ks = 0; ks < n_ks; ++ks, ++it) {
+          const int slot = it % kStages;
+          if (!bar_wait(empty(slot), ((it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          bar_expect_tx(full_b(slot), kBBytes);
+          asm volatile(
+              "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+              ::"r"(b_base + slot * kBBytes), "l"(&tmap_act), "r"(ks * kBK), "r"(m0), "r"(full_b(slot)) : "memory");
+        }
+      }
+      const uint32_t n_back = it < (uint32_t)kStages ? it : (uint32_t)kStages;
+      for (uint32_t i = 1; i <= n_back; ++i) {
+        const uint32_t j = it - i;
+        bar_drain(full_b(j % kStages), (j / kStages) & 1u);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc(BN);
+      uint32_t it = 0, tl = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, ++tl) {
+        const uint32_t buf = tl & 1u;
+        if (!bar_wait(tmem_empty(buf), ((tl >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t d_tmem = tmem_base + buf * BN;
+        for (int ks = 0; ks < n_ks; ++ks, ++it) {
+          const int slot = it % kStages;
+          const uint32_t ph = (it / kStages) & 1u;
+          if (!bar_wait(full_a(slot), ph, abort_flag) || !bar_wait(full_b(slot), ph, abort_flag)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k)
+            mma_f16_ta(d_tmem, tmem_base + kACol0 + slot * 32 + k * 8, smem_desc(b_base + slot * kBBytes + k * 32),
+                       idesc, (uint32_t)((ks | k) != 0));
+          mma_commit(empty(slot));                 // frees the token tile and the A stage
+        }
+        if (ok) mma_commit(tmem_full(buf));
+      }
+      mma_commit(drain_bar);
+      bar_drain(drain_bar, 0);
+    }
+    __syncwarp();
+  } else if (warp < kFirstDecodeWarp) {
+    // ------------------------------------------------------------------ epilogue
+    const int quad = warp & 3;
+    uint32_t tl = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, ++tl) {
+      const uint32_t buf = tl & 1u;
+      const int n = (tile / P.n_tiles_m) * kBM + 32 * quad + lane;
+      const int m0 = (tile % P.n_tiles_m) * BN;
+      ok = __all_sync(0xffffffffu, bar_wait(tmem_full(buf), (tl >> 1) & 1u, abort_flag));
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t v[32];
+        tmem_ld32(tmem_base + ((uint32_t)(32 * quad) << 16) + buf * BN + 32 * c, v);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        const int mc = m0 + 32 * c;
+        const float my_scale = mc + lane < P.M ? __ldg(P.act_scale + mc + lane) : 0.0f;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float s = __shfl_sync(0xffffffffu, my_scale, j);
+          if (mc + j < P.M && n < P.N) P.y[(size_t)(mc + j) * P.ldy + n] = __uint_as_float(v[j]) * s;
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      bar_arrive(tmem_empty(buf));
+    }
+  } else {
+    // ------------------------------------------------------------------ decoder
+    const int grp = (warp - kFirstDecodeWarp) >> 2;     // stage of every item this warp decodes
+    const int quad = warp & 3;                          // tensor-memory lanes [32*quad, +32) = tile rows
+    const int r = 32 * quad + lane;                     // tile row of this thread
+    const int u = (r >> 3) & 1, g = r & 7;
+    const int h = grp >> 1, t0 = 2 * (grp & 1);         // k-block and first quarter of the stage
+    uint32_t it0 = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, it0 += (uint32_t)n_ks) {
+      int rp = (tile / P.n_tiles_m) * (kBM / 16) + (r >> 4);
+      rp = rp < P.n_rp ? rp : P.n_rp - 1;          // rows past the matrix repeat the last group; never stored
+      uint32_t TL[2], TH[2];
+      {
+        const uint16_t* cb = P.codebook + ((size_t)rp * 16 + 8 * u + g) * (1 << BITS);
+        if (BITS == 2) {
+          const uint2 c = __ldg(reinterpret_cast<const uint2*>(cb));
+          TL[0] = TL[1] = prmt_b(c.x, c.y, 0x6420u);
+          TH[0] = TH[1] = prmt_b(c.x, c.y, 0x7531u);
+        } else {
+          const uint4 c = __ldg(reinterpret_cast<const uint4*>(cb));
+          TL[0] = prmt_b(c.x, c.y, 0x6420u); TH[0] = prmt_b(c.x, c.y, 0x7531u);
+          TL[1] = prmt_b(c.z, c.w, 0x6420u); TH[1] = prmt_b(c.z, c.w, 0x7531u);
+        }
+      }
+      // this thread's 64 columns of one item: quarters t0 and t0 + 1 of k-block h -> [quarter][word]
+      const uint8_t* row_items = P.items + (size_t)rp * P.n_kt * ITEM + u * HALF;
+      uint32_t cur[2][BITS == 2 ? 2 : 3], nxt[2][BITS == 2 ? 2 : 3];
+      auto load_stage = [&](uint32_t (&dst)[2][BITS == 2 ? 2 : 3], int kt) {
+        const uint8_t* item = row_items + (size_t)kt * ITEM;
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+          const int l = 4 * g + t0 + x;
+          if (BITS == 2) {
+            const uint2 w = __ldg(reinterpret_cast<const uint2*>(item + 16 * l + 8 * h));
+            dst[x][0] = w.x; dst[x][1] = w.y;
+          } else {
+#pragma unroll
+            for (int b = 0; b < 3; ++b) dst[x][b] = __ldg(reinterpret_cast<const uint32_t*>(item + 256 * b + 8 * l + 4 * h));
+          }
+        }
+      };
+      load_stage(cur, 0);
+      for (int kt = 0; kt < P.n_kt && ok; ++kt) {
+        if (kt + 1 < P.n_kt) load_stage(nxt, kt + 1);
+        const uint32_t it = it0 + 4u * (uint32_t)kt + (uint32_t)grp;
+        const int slot = it % kStages;
+        uint32_t v[32];     // the row's 64 fp16 of this stage, two per tensor-memory column
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+          uint32_t sel[8];
+          if (BITS == 2) {
+#pragma unroll
+            for (int wd = 0; wd < 2; ++wd) {
+              const uint32_t raw = cur[x][wd];
+              const uint32_t s0 = raw & 0x33333333u, s1 = (raw >> 2) & 0x33333333u;
+              sel[4 * wd] = s0; sel[4 * wd + 1] = s0 >> 16; sel[4 * wd + 2] = s1; sel[4 * wd + 3] = s1 >> 16;
+            }
+          } else {
+            const uint32_t r0 = cur[x][0], r1 = cur[x][1], r2 = cur[x][2];
+            const uint32_t ex = (((r0 >> 3) & 0x11111111u) | ((r1 >> 2) & 0x22222222u)) | ((r2 >> 1) & 0x44444444u);
+            const uint32_t d0 = r0 & 0x77777777u, d1 = r1 & 0x77777777u, d2 = r2 & 0x77777777u;
+            sel[0] = d0; sel[1] = d0 >> 16; sel[2] = d1; sel[3] = d1 >> 16;
+            sel[4] = d2; sel[5] = d2 >> 16; sel[6] = ex; sel[7] = ex >> 16;
+          }
+#pragma unroll
+          for (int L = 0; L < 8; ++L) {
+            const uint32_t lo = prmt_b(TL[0], TL[1], sel[L]), hi = prmt_b(TH[0], TH[1], sel[L]);
+            v[16 * x + 2 * L] = prmt_b(lo, hi, 0x5140u);
+            v[16 * x + 2 * L + 1] = prmt_b(lo, hi, 0x7362u);
+          }
+        }
+        if (!bar_wait(empty(slot), ((it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; }
+        ok = __all_sync(0xffffffffu, ok);          // tcgen05.st is a warp-wide instruction
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        tmem_st32(tmem_base + ((uint32_t)(32 * quad) << 16) + kACol0 + slot * 32, v);
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        bar_arrive(full_a(slot));
+#pragma unroll
+        for (int x = 0; x < 2; ++x)
+#pragma unroll
+          for (int b = 0; b < (BITS == 2 ? 2 : 3); ++b) cur[x][b] = nxt[x][b];
+      }
+    }
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+  if (threadIdx.x == 0 && *abort_flag && P.status) atomicExch(P.status, (int)LCD_ERR_TIMEOUT);
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -440,8 +692,9 @@ lcd_status launch_dense_t(const Problem& p, __half* levels, int32_t* status_word
   dp.n_tiles_m = (int)((p.M + BN - 1) / BN);
   dp.n_tiles = dp.n_tiles_m * (int)((p.N_pad + kBM - 1) / kBM);
   dp.status = status_word;
-  const size_t smem = 1024 + (size_t)kStages * (kABytes + BN * kBK * 2) + 256;
-  auto kern = dense_tc_kernel<BITS, BN>;
+  constexpr bool kATmem = BN <= 192;    // A through tensor memory where two accumulators leave room for it
+  const size_t smem = 1024 + (size_t)kStages * ((kATmem ? 0 : kABytes) + BN * kBK * 2) + 256;
+  auto kern = kATmem ? dense_tc_ta_kernel<BITS, (BN <= 192 ? BN : 192)> : dense_tc_kernel<BITS, BN>;
   static bool attr_set = false;   // per template instance
   if (!attr_set) {
     const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
