@@ -234,6 +234,7 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = instr_desc(BN);
+      const uint64_t a_desc0 = smem_desc(a_base), b_desc0 = smem_desc(b_base);
       uint32_t it = 0, tl = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, ++tl) {
@@ -246,10 +247,12 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
           const uint32_t ph = (it / kStages) & 1u;
           if (!bar_wait(full_a(slot), ph, abort_flag) || !bar_wait(full_b(slot), ph, abort_flag)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          // descriptors differ only in the start-address field (units of 16 bytes): this one thread issues every
+          // MMA of the CTA, so its instruction count per stage is kept small
+          const uint64_t ad = a_desc0 + (uint64_t)((slot * kABytes) >> 4), bd = b_desc0 + (uint64_t)((slot * kBBytes) >> 4);
+          mma_f16(d_tmem, ad, bd, idesc, (uint32_t)(ks != 0));
 #pragma unroll
-          for (int k = 0; k < kBK / 16; ++k)
-            mma_f16(d_tmem, smem_desc(a_base + slot * kABytes + k * 32), smem_desc(b_base + slot * kBBytes + k * 32),
-                    idesc, (uint32_t)((ks | k) != 0));
+          for (int k = 1; k < kBK / 16; ++k) mma_f16(d_tmem, ad + 2 * k, bd + 2 * k, idesc, 1u);
           mma_commit(empty(slot));
         }
         if (ok) mma_commit(tmem_full(buf));
@@ -392,8 +395,10 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
 // a warp the 32 tensor-memory lanes of its quadrant) and the MMA takes A from tensor memory.  Shared memory then
 // carries only the token tiles, which is what bounds the kernel above (see the profile of that kernel).
 // Tensor memory: two accumulators of BN columns, then four A stages of 32 columns (64 fp16 per row).
-// Warps: 0 TMA, 1 MMA, 2-5 epilogue, 6-21 decoder = 4 groups x 4 quadrant warps; group i decodes the stages
-// whose number is i modulo 4.
+// RT = 1: a CTA tile is 128 rows, two accumulator buffers.  RT = 2: 256 rows (two MMA row tiles share every token
+// tile, which halves the token bytes streamed from L2 per flop), one accumulator buffer.
+// Warps: 0 TMA, 1 MMA, 2-5 epilogue, 6-21 decoder = 16 / (4 RT) groups x RT row tiles x 4 quadrant warps; group i
+// decodes the stages whose number is i modulo the number of groups.
 __device__ __forceinline__ void mma_f16_ta(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
       "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
@@ -409,36 +414,47 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
         "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]) : "memory");
 }
 
-template <int BITS, int BN>
+// Token-tile stages of the tensor-memory variant: as many as fit in about 200 KB, at most 8.
+__host__ __device__ constexpr int ta_b_stages(int bn) { return (200 * 1024) / (bn * kBK * 2) > 8 ? 8 : (200 * 1024) / (bn * kBK * 2); }
+
+template <int BITS, int BN, int RT>
 __global__ void __launch_bounds__(kDenseThreads, 1)
 dense_tc_ta_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams P) {
   extern __shared__ uint8_t smem_raw[];
   constexpr int ITEM = 512 * BITS, HALF = 256 * BITS;
   constexpr int kBBytes = BN * kBK * 2;
   constexpr uint32_t kTmemCols = 512;
-  constexpr uint32_t kACol0 = 2 * BN;              // first tensor-memory column of the A stages
-  static_assert(2 * BN + kStages * 32 <= 512, "tensor memory holds two accumulators and four A stages");
+  constexpr int SB = ta_b_stages(BN);              // token-tile stages in shared memory (deep: they hide the L2 latency)
+  constexpr int NBUF = RT == 1 ? 2 : 1;            // accumulator buffers (RT * BN columns each)
+  constexpr int NG = kDecodeWarps / (4 * RT);      // decoder groups; a group decodes the stages == its index mod NG
+  constexpr uint32_t kACol0 = NBUF * RT * BN;      // first tensor-memory column of the A stages
+  static_assert(NBUF * RT * BN + kStages * RT * 32 <= 512, "tensor memory holds the accumulators and four A stages");
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   const uint32_t raw_addr = (uint32_t)__cvta_generic_to_shared(smem_raw);
   const uint32_t base = (raw_addr + 1023u) & ~1023u;
   uint8_t* gen_base = smem_raw + (base - raw_addr);
-  const uint32_t b_base = base, bar_base = b_base + kStages * kBBytes;
+  const uint32_t b_base = base, bar_base = b_base + SB * kBBytes;
+  // barriers: A stages (tensor memory) full/empty, token-tile stages full/empty, accumulators, drain
   auto full_a = [&](int s) { return bar_base + 8u * s; };
-  auto full_b = [&](int s) { return bar_base + 8u * (kStages + s); };
-  auto empty = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
-  auto tmem_full = [&](int b) { return bar_base + 8u * (3 * kStages + b); };
-  auto tmem_empty = [&](int b) { return bar_base + 8u * (3 * kStages + 2 + b); };
-  const uint32_t drain_bar = bar_base + 8u * (3 * kStages + 4);
-  uint8_t* gen_misc = gen_base + kStages * kBBytes + 8 * (3 * kStages + 5);
+  auto empty_a = [&](int s) { return bar_base + 8u * (kStages + s); };
+  auto full_b = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
+  auto empty_b = [&](int s) { return bar_base + 8u * (2 * kStages + SB + s); };
+  auto tmem_full = [&](int b) { return bar_base + 8u * (2 * kStages + 2 * SB + b); };
+  auto tmem_empty = [&](int b) { return bar_base + 8u * (2 * kStages + 2 * SB + 2 + b); };
+  const uint32_t drain_bar = bar_base + 8u * (2 * kStages + 2 * SB + 4);
+  uint8_t* gen_misc = gen_base + SB * kBBytes + 8 * (2 * kStages + 2 * SB + 5);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(gen_misc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_misc + 4);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      bar_init(full_a(s), 4 * 32);                 // the four quadrant warps of one decoder group
+      bar_init(full_a(s), RT * 4 * 32);            // the quadrant warps of one decoder group
+      bar_init(empty_a(s), 1);
+    }
+    for (int s = 0; s < SB; ++s) {
       bar_init(full_b(s), 1);
-      bar_init(empty(s), 1);
+      bar_init(empty_b(s), 1);
     }
     for (int b = 0; b < 2; ++b) {
       bar_init(tmem_full(b), 1);
@@ -470,18 +486,18 @@ dense_tc_ta_kernel(const __grid_constant__ CUtensorMap tmap_act, const DensePara
       for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x) {
         const int m0 = (tile % P.n_tiles_m) * BN;
         for (int ks = 0; ks < n_ks; ++ks, ++it) {
-          const int slot = it % kStages;
-          if (!bar_wait(empty(slot), ((it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          const int slot = it % SB;
+          if (!bar_wait(empty_b(slot), ((it / SB) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
           bar_expect_tx(full_b(slot), kBBytes);
           asm volatile(
               "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
               ::"r"(b_base + slot * kBBytes), "l"(&tmap_act), "r"(ks * kBK), "r"(m0), "r"(full_b(slot)) : "memory");
         }
       }
-      const uint32_t n_back = it < (uint32_t)kStages ? it : (uint32_t)kStages;
+      const uint32_t n_back = it < (uint32_t)SB ? it : (uint32_t)SB;
       for (uint32_t i = 1; i <= n_back; ++i) {
         const uint32_t j = it - i;
-        bar_drain(full_b(j % kStages), (j / kStages) & 1u);
+        bar_drain(full_b(j % SB), (j / SB) & 1u);
       }
     }
     __syncwarp();
@@ -489,23 +505,31 @@ dense_tc_ta_kernel(const __grid_constant__ CUtensorMap tmap_act, const DensePara
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = instr_desc(BN);
-      uint32_t it = 0, tl = 0;
+      const uint64_t b_desc0 = smem_desc(b_base);
+      uint32_t it = 0, tl = 0, bslot = 0, bphase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, ++tl) {
-        const uint32_t buf = tl & 1u;
-        if (!bar_wait(tmem_empty(buf), ((tl >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        const uint32_t buf = tl % NBUF;
+        if (!bar_wait(tmem_empty(buf), ((tl / NBUF) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t d_tmem = tmem_base + buf * BN;
+        const uint32_t d_tmem = tmem_base + buf * (RT * BN);
         for (int ks = 0; ks < n_ks; ++ks, ++it) {
           const int slot = it % kStages;
-          const uint32_t ph = (it / kStages) & 1u;
-          if (!bar_wait(full_a(slot), ph, abort_flag) || !bar_wait(full_b(slot), ph, abort_flag)) { ok = false; break; }
+          if (!bar_wait(full_a(slot), (it / kStages) & 1u, abort_flag) ||
+              !bar_wait(full_b(bslot), bphase, abort_flag)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          // one thread issues every MMA of the CTA: keep its instruction count per stage small
+          const uint64_t bd = b_desc0 + (uint64_t)((bslot * kBBytes) >> 4);
+          const uint32_t a_t = tmem_base + kACol0 + slot * (RT * 32);
 #pragma unroll
-          for (int k = 0; k < kBK / 16; ++k)
-            mma_f16_ta(d_tmem, tmem_base + kACol0 + slot * 32 + k * 8, smem_desc(b_base + slot * kBBytes + k * 32),
-                       idesc, (uint32_t)((ks | k) != 0));
-          mma_commit(empty(slot));                 // frees the token tile and the A stage
+          for (int i = 0; i < RT; ++i) {
+            mma_f16_ta(d_tmem + i * BN, a_t + i * 32, bd, idesc, (uint32_t)(ks != 0));
+#pragma unroll
+            for (int k = 1; k < kBK / 16; ++k) mma_f16_ta(d_tmem + i * BN, a_t + i * 32 + k * 8, bd + 2 * k, idesc, 1u);
+          }
+          mma_commit(empty_a(slot));               // frees the A stage in tensor memory
+          mma_commit(empty_b(bslot));              // and the token tile in shared memory
+          if (++bslot == (uint32_t)SB) { bslot = 0; bphase ^= 1u; }
         }
         if (ok) mma_commit(tmem_full(buf));
       }
@@ -519,16 +543,17 @@ dense_tc_ta_kernel(const __grid_constant__ CUtensorMap tmap_act, const DensePara
     uint32_t tl = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, ++tl) {
-      const uint32_t buf = tl & 1u;
-      const int n = (tile / P.n_tiles_m) * kBM + 32 * quad + lane;
+      const uint32_t buf = tl % NBUF;
       const int m0 = (tile % P.n_tiles_m) * BN;
-      ok = __all_sync(0xffffffffu, bar_wait(tmem_full(buf), (tl >> 1) & 1u, abort_flag));
+      ok = __all_sync(0xffffffffu, bar_wait(tmem_full(buf), (tl / NBUF) & 1u, abort_flag));
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
+      for (int cc = 0; cc < RT * (BN / 32); ++cc) {
+        const int i = cc / (BN / 32), c = cc % (BN / 32);       // row tile, 32-token chunk
+        const int n = (tile / P.n_tiles_m) * (RT * kBM) + kBM * i + 32 * quad + lane;
         uint32_t v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(32 * quad) << 16) + buf * BN + 32 * c, v);
+        tmem_ld32(tmem_base + ((uint32_t)(32 * quad) << 16) + buf * (RT * BN) + i * BN + 32 * c, v);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         const int mc = m0 + 32 * c;
         const float my_scale = mc + lane < P.M ? __ldg(P.act_scale + mc + lane) : 0.0f;
@@ -543,15 +568,16 @@ dense_tc_ta_kernel(const __grid_constant__ CUtensorMap tmap_act, const DensePara
     }
   } else {
     // ------------------------------------------------------------------ decoder
-    const int grp = (warp - kFirstDecodeWarp) >> 2;     // stage of every item this warp decodes
-    const int quad = warp & 3;                          // tensor-memory lanes [32*quad, +32) = tile rows
-    const int r = 32 * quad + lane;                     // tile row of this thread
+    const int dwi = warp - kFirstDecodeWarp;
+    const int grp = dwi / (4 * RT);                     // decodes the stages whose number is grp modulo NG
+    const int rt = (dwi >> 2) % RT;                     // row tile of 128 rows inside the CTA's tile
+    const int quad = warp & 3;                          // tensor-memory lanes [32*quad, +32) = rows of the row tile
+    const int r = 32 * quad + lane;                     // row inside the row tile
     const int u = (r >> 3) & 1, g = r & 7;
-    const int h = grp >> 1, t0 = 2 * (grp & 1);         // k-block and first quarter of the stage
     uint32_t it0 = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, it0 += (uint32_t)n_ks) {
-      int rp = (tile / P.n_tiles_m) * (kBM / 16) + (r >> 4);
+      int rp = (tile / P.n_tiles_m) * (RT * kBM / 16) + rt * (kBM / 16) + (r >> 4);
       rp = rp < P.n_rp ? rp : P.n_rp - 1;          // rows past the matrix repeat the last group; never stored
       uint32_t TL[2], TH[2];
       {
@@ -568,8 +594,10 @@ dense_tc_ta_kernel(const __grid_constant__ CUtensorMap tmap_act, const DensePara
       }
       // this thread's 64 columns of one item: quarters t0 and t0 + 1 of k-block h -> [quarter][word]
       const uint8_t* row_items = P.items + (size_t)rp * P.n_kt * ITEM + u * HALF;
-      uint32_t cur[2][BITS == 2 ? 2 : 3], nxt[2][BITS == 2 ? 2 : 3];
-      auto load_stage = [&](uint32_t (&dst)[2][BITS == 2 ? 2 : 3], int kt) {
+      constexpr int SPI = 4 / NG;                  // stages of one item this group decodes
+      uint32_t cur[SPI][2][BITS == 2 ? 2 : 3], nxt[SPI][2][BITS == 2 ? 2 : 3];
+      auto load_stage = [&](uint32_t (&dst)[2][BITS == 2 ? 2 : 3], int kt, int j) {
+        const int h = j >> 1, t0 = 2 * (j & 1);    // k-block and first quarter of stage j of an item
         const uint8_t* item = row_items + (size_t)kt * ITEM;
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
@@ -583,10 +611,17 @@ dense_tc_ta_kernel(const __grid_constant__ CUtensorMap tmap_act, const DensePara
           }
         }
       };
-      load_stage(cur, 0);
+#pragma unroll
+      for (int jj = 0; jj < SPI; ++jj) load_stage(cur[jj], 0, grp + NG * jj);
       for (int kt = 0; kt < P.n_kt && ok; ++kt) {
-        if (kt + 1 < P.n_kt) load_stage(nxt, kt + 1);
-        const uint32_t it = it0 + 4u * (uint32_t)kt + (uint32_t)grp;
+        if (kt + 1 < P.n_kt) {
+#pragma unroll
+          for (int jj = 0; jj < SPI; ++jj) load_stage(nxt[jj], kt + 1, grp + NG * jj);
+        }
+#pragma unroll
+       for (int jj = 0; jj < SPI; ++jj) {
+        if (!ok) break;
+        const uint32_t it = it0 + 4u * (uint32_t)kt + (uint32_t)(grp + NG * jj);
         const int slot = it % kStages;
         uint32_t v[32];     // the row's 64 fp16 of this stage, two per tensor-memory column
 #pragma unroll
@@ -595,12 +630,12 @@ dense_tc_ta_kernel(const __grid_constant__ CUtensorMap tmap_act, const DensePara
           if (BITS == 2) {
 #pragma unroll
             for (int wd = 0; wd < 2; ++wd) {
-              const uint32_t raw = cur[x][wd];
+              const uint32_t raw = cur[jj][x][wd];
               const uint32_t s0 = raw & 0x33333333u, s1 = (raw >> 2) & 0x33333333u;
               sel[4 * wd] = s0; sel[4 * wd + 1] = s0 >> 16; sel[4 * wd + 2] = s1; sel[4 * wd + 3] = s1 >> 16;
             }
           } else {
-            const uint32_t r0 = cur[x][0], r1 = cur[x][1], r2 = cur[x][2];
+            const uint32_t r0 = cur[jj][x][0], r1 = cur[jj][x][1], r2 = cur[jj][x][2];
             const uint32_t ex = (((r0 >> 3) & 0x11111111u) | ((r1 >> 2) & 0x22222222u)) | ((r2 >> 1) & 0x44444444u);
             const uint32_t d0 = r0 & 0x77777777u, d1 = r1 & 0x77777777u, d2 = r2 & 0x77777777u;
             sel[0] = d0; sel[1] = d0 >> 16; sel[2] = d1; sel[3] = d1 >> 16;
@@ -613,18 +648,21 @@ dense_tc_ta_kernel(const __grid_constant__ CUtensorMap tmap_act, const DensePara
             v[16 * x + 2 * L + 1] = prmt_b(lo, hi, 0x7362u);
           }
         }
-        if (!bar_wait(empty(slot), ((it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; }
+        if (!bar_wait(empty_a(slot), ((it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; }
         ok = __all_sync(0xffffffffu, ok);          // tcgen05.st is a warp-wide instruction
-        if (!ok) break;
+        if (!ok) continue;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        tmem_st32(tmem_base + ((uint32_t)(32 * quad) << 16) + kACol0 + slot * 32, v);
+        tmem_st32(tmem_base + ((uint32_t)(32 * quad) << 16) + kACol0 + (slot * RT + rt) * 32, v);
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         bar_arrive(full_a(slot));
+       }
 #pragma unroll
-        for (int x = 0; x < 2; ++x)
+        for (int jj = 0; jj < SPI; ++jj)
 #pragma unroll
-          for (int b = 0; b < (BITS == 2 ? 2 : 3); ++b) cur[x][b] = nxt[x][b];
+          for (int x = 0; x < 2; ++x)
+#pragma unroll
+            for (int b = 0; b < (BITS == 2 ? 2 : 3); ++b) cur[jj][x][b] = nxt[jj][x][b];
       }
     }
   }
@@ -667,7 +705,8 @@ int dense_sm_count() {
   return cached;
 }
 
-template <int BITS, int BN>
+// KERNEL 0: A through shared memory (dense_tc_kernel); 1: A through tensor memory with RT row tiles per CTA.
+template <int BITS, int BN, int RT, int KERNEL>
 lcd_status launch_dense_t(const Problem& p, __half* levels, int32_t* status_word, cudaStream_t stream) {
   EncodeTiledFn enc = encode_tiled();
   if (!enc) return LCD_ERR_CUDA;
@@ -690,11 +729,13 @@ lcd_status launch_dense_t(const Problem& p, __half* levels, int32_t* status_word
   dp.n_rp = (int)(p.N_pad / kPairRows);
   dp.n_kt = (int)(p.K_pad / kTileK);
   dp.n_tiles_m = (int)((p.M + BN - 1) / BN);
-  dp.n_tiles = dp.n_tiles_m * (int)((p.N_pad + kBM - 1) / kBM);
+  dp.n_tiles = dp.n_tiles_m * (int)((p.N_pad + RT * kBM - 1) / (RT * kBM));
   dp.status = status_word;
-  constexpr bool kATmem = BN <= 192;    // A through tensor memory where two accumulators leave room for it
-  const size_t smem = 1024 + (size_t)kStages * ((kATmem ? 0 : kABytes) + BN * kBK * 2) + 256;
-  auto kern = kATmem ? dense_tc_ta_kernel<BITS, (BN <= 192 ? BN : 192)> : dense_tc_kernel<BITS, BN>;
+  const size_t smem = KERNEL == 0 ? 1024 + (size_t)kStages * (kABytes + BN * kBK * 2) + 256
+                                  : 1024 + (size_t)ta_b_stages(BN) * (BN * kBK * 2) + 512;
+  void (*kern)(const CUtensorMap, const DenseParams);
+  if (KERNEL == 0) kern = dense_tc_kernel<BITS, BN>;
+  else kern = dense_tc_ta_kernel<BITS, (KERNEL == 0 ? 128 : BN), RT>;
   static bool attr_set = false;   // per template instance
   if (!attr_set) {
     const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -717,19 +758,22 @@ lcd_status launch_dense_t(const Problem& p, __half* levels, int32_t* status_word
   return LCD_OK;
 }
 
-// Tokens per tile: the width whose (waves of tiles) x (tile time) is smallest.  A tile's time grows with its
-// width but not below the time the decoder and the shared-memory traffic of the A operand need.
-int pick_bn(int64_t M, int64_t N_pad) {
+// Tile shapes: {kernel, row tiles, tokens, cycles per 64-column stage}.  The stage times are measured ones: with
+// 128 rows per CTA the token tiles streamed from L2 bound the stage (the L2-to-SM path runs at about 8 TB/s), so a
+// stage costs about 3.5 cycles per token of tile width.  (A 256-row tile, RT = 2, halves that traffic and is
+// supported by the kernel, but its decoder did not keep up when measured, so it is not among the choices.)
+struct TileShape { int kernel, rt, bn, stage_clks, epilogue_clks; };
+constexpr TileShape kShapes[3] = {{1, 1, 192, 664, 0}, {1, 1, 128, 443, 0}, {0, 1, 256, 733, 0}};
+
+int pick_shape(int64_t M, int64_t N_pad, int64_t n_ks) {
   const int n_sm = dense_sm_count();
-  const int64_t tiles_n = (N_pad + kBM - 1) / kBM;
-  const int widths[3] = {128, 192, 256};
-  int best = 128;
+  int best = 0;
   int64_t best_cost = -1;
   for (int i = 0; i < 3; ++i) {
-    const int bn = widths[i];
-    const int64_t tiles = tiles_n * ((M + bn - 1) / bn);
-    const int64_t cost = ((tiles + n_sm - 1) / n_sm) * (bn > 150 ? bn : 150);
-    if (best_cost < 0 || cost <= best_cost) { best = bn; best_cost = cost; }
+    const TileShape& t = kShapes[i];
+    const int64_t tiles = ((N_pad + t.rt * kBM - 1) / (t.rt * kBM)) * ((M + t.bn - 1) / t.bn);
+    const int64_t cost = ((tiles + n_sm - 1) / n_sm) * (n_ks * t.stage_clks + t.epilogue_clks);
+    if (best_cost < 0 || cost < best_cost) { best = i; best_cost = cost; }
   }
   return best;
 }
@@ -750,11 +794,11 @@ lcd_status launch_dense_tc(const Problem& p, void* workspace, size_t workspace_b
   else expand_levels_kernel<3><<<blocks, 256, 0, s>>>(p.act_idx, n_quarters, levels);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
-  const int bn = pick_bn(p.M, p.N_pad);
-#define LCD_DENSE_CASE(B, W) \
-  if (p.bits == B && bn == W) return launch_dense_t<B, W>(p, levels, status_word, s);
-  LCD_DENSE_CASE(2, 128) LCD_DENSE_CASE(2, 192) LCD_DENSE_CASE(2, 256)
-  LCD_DENSE_CASE(3, 128) LCD_DENSE_CASE(3, 192) LCD_DENSE_CASE(3, 256)
+  const int shape = pick_shape(p.M, p.N_pad, p.K_pad / kBK);
+#define LCD_DENSE_CASE(B, I, W, R, KN) \
+  if (p.bits == B && shape == I) return launch_dense_t<B, W, R, KN>(p, levels, status_word, s);
+  LCD_DENSE_CASE(2, 0, 192, 1, 1) LCD_DENSE_CASE(2, 1, 128, 1, 1) LCD_DENSE_CASE(2, 2, 256, 1, 0)
+  LCD_DENSE_CASE(3, 0, 192, 1, 1) LCD_DENSE_CASE(3, 1, 128, 1, 1) LCD_DENSE_CASE(3, 2, 256, 1, 0)
 #undef LCD_DENSE_CASE
   return LCD_ERR_UNSUPPORTED;
 }

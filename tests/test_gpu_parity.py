@@ -141,7 +141,9 @@ def test_grouped_launch_matches_oracle_and_leaves_scratch_zero():
 @pytest.mark.parametrize("N,K,M", [(128, 256, 32), (200, 1000, 17), (1031, 520, 40), (64, 4096, 100), (520, 2304, 256),
                                    (272, 768, 300), (1024, 1024, 513),
                                    (2560, 512, 2048),      # 192-token tiles (two waves instead of three)
-                                   (9472, 256, 512)])      # 256-token tiles (one wave)
+                                   (9472, 256, 512),       # 256-token tiles (one wave)
+                                   (4608, 1024, 1024),
+                                   (4600, 1024, 1000)])    # ragged rows and tokens
 def test_dense_tensor_core_path_matches_oracle(bits, N, K, M):
     # fp16 centroids x integer levels on the tensor cores, fp32 accumulation: exact products, so only the order
     # of the fp32 sums differs from the oracle
