@@ -407,29 +407,44 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
     for (int i = lane; i < ACC_INTS; i += 32) s_acc[warp * ACC_INTS + i] = 0;
   __syncwarp();
 
-  uint32_t stage_c = 0, stage_f = 0;    // consumed / fetched stages of this warp (ring position and parity)
+  // Ring state.  Fetch side: next slot to fill, stages in flight, the rest of the segment being fetched (a
+  // segment is this warp's share of one run: consecutive items in memory) and the cursor of the segment after
+  // it.  Consumer side: next slot to read and its barrier phase.  Both sides cut every segment into stages of
+  // kStageItems items from its start, so they agree on what each slot holds.
+  uint32_t f_slot = 0, f_inflight = 0, f_left = 0, c_slot = 0, c_phase = 0;
+  const uint8_t* f_src = P.items;
+  const uint32_t ring_u32 = smem_u32(ring);
   bool aborted = false;
+  Cursor fc, cc;
 
-  auto issue = [&](Cursor& fc, uint32_t x_end) {
-    const uint32_t n = stage_len(fc, x_end);
+  auto issue_stage = [&]() {        // f_left > 0
+    const uint32_t n = f_left < (uint32_t)kStageItems ? f_left : (uint32_t)kStageItems;
     if (lane == 0) {
-      const uint32_t slot = stage_f % kDepth;
-      const uint32_t bar = bar0 + 8u * slot;
-      const uint32_t bytes = n * ITEM;
-      const uint8_t* src = P.items + ((size_t)fc.rp * P.n_kt + (size_t)fc.pn * P.pw + fc.kk) * ITEM;
-      const uint32_t dst = smem_u32(ring + slot * SLOT);
+      const uint32_t bar = bar0 + 8u * f_slot, bytes = n * ITEM, dst = ring_u32 + f_slot * SLOT;
       asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
       asm volatile(
           "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-          ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+          ::"r"(dst), "l"(f_src), "r"(bytes), "r"(bar) : "memory");
     }
-    cursor_advance(fc, n, P);
-    ++stage_f;
+    f_src += (size_t)n * ITEM;
+    f_left -= n;
+    f_slot = f_slot + 1 == (uint32_t)kDepth ? 0 : f_slot + 1;
+    ++f_inflight;
+  };
+  // Issues the next stage if there is one before x_end.
+  auto fetch_more = [&](uint32_t x_end) {
+    if (f_left == 0) {
+      if (fc.x >= x_end) return;
+      const uint32_t row_left = fc.pw - fc.kk, range_left = x_end - fc.x;
+      f_left = row_left < range_left ? row_left : range_left;
+      f_src = P.items + ((size_t)fc.rp * P.n_kt + (size_t)fc.pn * P.pw + fc.kk) * ITEM;
+      cursor_advance(fc, f_left, P);
+    }
+    issue_stage();
   };
 
   // The weights do not depend on the kernel that produced the activation indices: start streaming them (and
   // fetch the first rows' codebooks) before waiting for it.
-  Cursor fc, cc;
   uint32_t round_lo, round_hi;
   {
     const uint32_t lo = pA * panel_items, hi = (pA + 2) * panel_items;
@@ -438,7 +453,7 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
     if (round_hi < round_lo) round_hi = round_lo;
     cursor_set(fc, round_lo, P);
     cc = fc;
-    while (fc.x < round_hi && stage_f - stage_c < (uint32_t)kDepth) issue(fc, round_hi);
+    for (int i = 0; i < kDepth; ++i) fetch_more(round_hi);
   }
   RowTables<BITS, KIND> Ta, Tb;           // rows 16*rp + g and 16*rp + 8 + g
   RawCodebook<BITS> next_a, next_b;
@@ -455,7 +470,6 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
 #pragma unroll
       for (int r = 0; r < 4; ++r) acc[G][p][r] = 0;
   uint32_t seg_kk0 = 0;
-  bool seg_open = false;
   uint32_t tok_off[MG];
 #pragma unroll
   for (int G = 0; G < MG; ++G) tok_off[G] = (uint32_t)((8 * G + g < P.M ? 8 * G + g : P.M - 1) * P.tstride + t * 32);
@@ -580,7 +594,7 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
       cursor_set(fc, round_lo, P);
       cc = fc;
       if (!aborted)
-        while (fc.x < round_hi && stage_f - stage_c < (uint32_t)kDepth) issue(fc, round_hi);
+        for (int i = 0; i < kDepth; ++i) fetch_more(round_hi);
       __syncthreads();     // every warp is done with the previous windows
     }
     // stage the activation windows of panels pbase and pbase + 1
@@ -599,56 +613,64 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
     if (warp_active && !aborted) {
 #pragma unroll 1
       while (cc.x < round_hi) {
-        const uint32_t n = stage_len(cc, round_hi);
-        const uint32_t slot = stage_c % kDepth;
+        // one segment: this warp's share of run (cc.pn, cc.rp), seg_len consecutive items from column item cc.kk
+        const uint32_t rp = cc.rp, pn = cc.pn, pw_n = cc.pw, kk0 = cc.kk;
+        const uint32_t row_left = pw_n - kk0, range_left = round_hi - cc.x;
+        const uint32_t seg_len = row_left < range_left ? row_left : range_left;
         // row tables of this 16-row group (its codebook rows were requested one group ahead)
-        if (cc.rp != tables_rp) {
-          if (next_rp != cc.rp) {
-            next_a = load_codebook<BITS>(P.codebook + ((size_t)cc.rp * 16 + g) * (1 << BITS));
-            next_b = load_codebook<BITS>(P.codebook + ((size_t)cc.rp * 16 + 8 + g) * (1 << BITS));
+        if (rp != tables_rp) {
+          if (next_rp != rp) {
+            next_a = load_codebook<BITS>(P.codebook + ((size_t)rp * 16 + g) * (1 << BITS));
+            next_b = load_codebook<BITS>(P.codebook + ((size_t)rp * 16 + 8 + g) * (1 << BITS));
           }
           Ta = build_tables<BITS, KIND>(next_a);
           Tb = build_tables<BITS, KIND>(next_b);
-          tables_rp = cc.rp;
-          next_rp = cc.rp + 1 < geo.n_rp ? cc.rp + 1 : 0;
+          tables_rp = rp;
+          next_rp = rp + 1 < geo.n_rp ? rp + 1 : 0;
           next_a = load_codebook<BITS>(P.codebook + ((size_t)next_rp * 16 + g) * (1 << BITS));
           next_b = load_codebook<BITS>(P.codebook + ((size_t)next_rp * 16 + 8 + g) * (1 << BITS));
         }
-        const bool ok = __all_sync(0xffffffffu, mbar_wait(bar0 + 8u * slot, (stage_c / kDepth) & 1u));
-        if (!ok) {
-          aborted = true;
+        const uint8_t* q[MG];
+#pragma unroll
+        for (int G = 0; G < MG; ++G) q[G] = act_s + (pn - pbase) * win_bytes + (size_t)kk0 * 256 + tok_off[G];
+#pragma unroll 1
+        for (uint32_t left = seg_len; left > 0;) {
+          const uint32_t n = left < (uint32_t)kStageItems ? left : (uint32_t)kStageItems;
+          const bool ok = __all_sync(0xffffffffu, mbar_wait(bar0 + 8u * c_slot, c_phase));
+          if (!ok) { aborted = true; break; }
+          const uint8_t* slot_p = ring + c_slot * SLOT;
+          process_item<BITS, KIND, MG>(slot_p, q, Ta, Tb, acc, lane);
+          if (kStageItems > 1 && n > 1) {
+            const uint8_t* q1[MG];
+#pragma unroll
+            for (int G = 0; G < MG; ++G) q1[G] = q[G] + 256;
+            process_item<BITS, KIND, MG>(slot_p + ITEM, q1, Ta, Tb, acc, lane);
+          }
+#pragma unroll
+          for (int G = 0; G < MG; ++G) q[G] += n * 256;
+          left -= n;
+          __syncwarp();
+          --f_inflight;
+          if (++c_slot == (uint32_t)kDepth) { c_slot = 0; c_phase ^= 1u; }
+          fetch_more(round_hi);                   // the slot just read is free again
+        }
+        if (aborted) {
           if (lane == 0 && status) atomicExch(status, (int)LCD_ERR_TIMEOUT);
           break;
         }
-        if (!seg_open) { seg_kk0 = cc.kk; seg_open = true; }
-        const uint8_t* slot_p = ring + slot * SLOT;
-        const uint8_t* win = act_s + (cc.pn - pbase) * win_bytes + (size_t)cc.kk * 256;
-#pragma unroll
-        for (uint32_t i = 0; i < (uint32_t)kStageItems; ++i) {
-          if (i < n) {
-            const uint8_t* q[MG];
-#pragma unroll
-            for (int G = 0; G < MG; ++G) q[G] = win + i * 256 + tok_off[G];
-            process_item<BITS, KIND, MG>(slot_p + i * ITEM, q, Ta, Tb, acc, lane);
-          }
-        }
-        const uint32_t rp_done = cc.rp, pn_done = cc.pn, pw_done = cc.pw, kk_end = cc.kk + n;
-        cursor_advance(cc, n, P);
-        __syncwarp();
-        ++stage_c;
-        if (fc.x < round_hi) issue(fc, round_hi);     // the slot just read is free again
-        if (kk_end == pw_done || cc.x == round_hi) {
-          flush(rp_done, pn_done, pw_done, kk_end);
-          seg_open = false;
-        }
+        cursor_advance(cc, seg_len, P);
+        seg_kk0 = kk0;
+        flush(rp, pn, pw_n, kk0 + seg_len);
       }
     }
     if (aborted) {
       // copies already issued must land before the CTA may exit
-      while (stage_c < stage_f) {
-        (void)mbar_wait(bar0 + 8u * (stage_c % kDepth), (stage_c / kDepth) & 1u);
-        ++stage_c;
+      while (f_inflight > 0) {
+        (void)mbar_wait(bar0 + 8u * c_slot, c_phase);
+        --f_inflight;
+        if (++c_slot == (uint32_t)kDepth) { c_slot = 0; c_phase ^= 1u; }
       }
+      f_left = 0;
     }
   }
 }
