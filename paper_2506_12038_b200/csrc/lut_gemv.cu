@@ -33,9 +33,11 @@ namespace {
 
 constexpr int kWarps = 16;
 constexpr int kThreads = kWarps * 32;
-constexpr int kDepth = 3;            // ring slots per warp
+// ring slots per warp: three, or two where 16 tokens need the shared memory for their activation levels
+__host__ __device__ constexpr int ring_depth(int mg) { return mg == 2 ? 2 : 3; }
+constexpr int kMaxDepth = 3;
 constexpr int kStageItems = 2;       // items per slot
-constexpr int kBarBytes = 512;       // mbarriers: kWarps * kDepth * 8 = 384 bytes, padded
+constexpr int kBarBytes = 512;       // mbarriers: kWarps * kMaxDepth * 8 = 384 bytes, padded
 constexpr int kMaxSmem = 227 * 1024;
 constexpr unsigned long long kTimeoutNs = 2000000000ull;   // bounded wait on a bulk copy: 2 s
 
@@ -355,6 +357,7 @@ template <int BITS, int KIND, int MG>
 __global__ void __launch_bounds__(kThreads, 1)
 lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ status) {
   extern __shared__ __align__(128) uint8_t smem[];
+  constexpr int kDepth = ring_depth(MG);
   constexpr int ITEM = 512 * BITS;
   constexpr int SLOT = kStageItems * ITEM;
   constexpr int PL = Planes<BITS, KIND>::value;
@@ -390,7 +393,7 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
   int* s_acc = reinterpret_cast<int*>(smem + kBarBytes);
   constexpr int COMBINE_BYTES = kSmemCombine ? kWarps * ACC_INTS * 4 : 0;
   uint8_t* ring = smem + kBarBytes + COMBINE_BYTES + (size_t)warp * kDepth * SLOT;
-  const uint32_t bar0 = smem_u32(smem) + 8u * (uint32_t)(warp * kDepth);
+  const uint32_t bar0 = smem_u32(smem) + 8u * (uint32_t)(warp * kMaxDepth);
   uint8_t* act_s = smem + kBarBytes + COMBINE_BYTES + (size_t)kWarps * kDepth * SLOT;
   const int n_tok = P.M < 8 * MG ? P.M : 8 * MG;
   const int win_bytes = n_tok * P.tstride;
@@ -757,7 +760,7 @@ lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void*
   if (workspace_bytes < lut_gemv_workspace_bytes(probs, count, algo) || !workspace) return LCD_ERR_BUFFER_TOO_SMALL;
 
   const int item_bytes = 512 * bits;
-  const size_t ring_bytes = (size_t)kWarps * kDepth * kStageItems * item_bytes;
+  const size_t ring_bytes = (size_t)kWarps * ring_depth(MG) * kStageItems * item_bytes;
   const size_t combine_bytes = kind == kFixed16 ? (size_t)kWarps * MG * planes * 128 * sizeof(int) : 0;
   const size_t act_budget = (size_t)kMaxSmem - kBarBytes - combine_bytes - ring_bytes;
 
