@@ -34,10 +34,12 @@ from synth import gen  # noqa: E402
 # changed since reports traffic = null.
 NCU_TRAFFIC = {
     # profiles/lut_gemv_kernel_llama7b_2bit_m1.md: one grouped launch of configs[1] at M = 1
-    ("lut_gemv.cu", 1, 1): {"sha256": "f35d381ad0e931346d092f5b8d4a671970b8ab3961186dc2ec80b358f72219bb", "bytes_per_launch": 50985984 + 25856},
-    # profiles/dense_tc_kernel_llama13b_2bit_m2048.md: the q projection of configs[3]; the layer's launches scale
-    # with their packed-weight + level bytes (traffic is those bytes once each)
-    ("dense_tc.cu", 3, 2048): {"sha256": "1ecac43fd227883efb489da9d19396c0898a3b4674232f1f11f4593f10a062e0", "bytes_per_launch": None},
+    ("lut_gemv.cu", 1, 1): {"sha256": "2813124b355499c0d7b9727ec884ce3d565f27dae85537db426cbf394fbf5d03", "bytes_per_launch": 50989056 + 26880},
+    # profiles/dense_tc_kernel_llama13b_2bit_m2048.md: the layer's seven launches of configs[3]: q captured
+    # (27.61 + 2.15 MB, taken four times for q/k/v/o), gate captured (39.22 + 62.68 MB, twice for gate/up), down
+    # scaled from q by its 2.7 times longer rows (same tiles, traffic in proportion to K)
+    ("dense_tc.cu", 3, 2048): {"sha256": "2c9d2410e0eda5b2f6b9dc3d2f6095c2d9a93c9cf3ead495f3685c450933633d",
+                               "bytes_per_launch": int(4 * 29.76e6 + 2 * 101.9e6 + 29.76e6 * 13824 / 5120)},
 }
 L2_BYTES = 126e6
 ROTATE_BYTES = 300e6          # total size of the weight copies the timed loop rotates over
@@ -311,22 +313,34 @@ def run_ours(args):
             kern_name = "lcd_lut_linear launches of one layer (sum of bytes / sum of durations)"
         clocks = sampler.stop()
 
-        # end to end through the host-buffer entry point: pinned host x -> device -> kernels -> pinned host y
+        # end to end through the host-buffer entry points: pinned host x -> device -> kernels -> pinned host y.
+        # Grouped (M <= 16): one copy in, two launches, one copy out per layer; else per matrix.
         e2e_ms, h2d, d2h = None, 0, 0
-        host = []
-        for mt in mats:
-            L = mt["L"]
-            xh = torch.from_numpy(L.x).pin_memory()
-            yh = torch.empty((M, L.N), dtype=torch.float32).pin_memory()
-            sc = torch.empty(lcd.linear_host_scratch_bytes(mt["w"][0], M), dtype=torch.uint8, device=dev)
-            host.append((xh, yh, sc))
-            h2d += xh.numel() * 2
-            d2h += yh.numel() * 4
+        if grouped:
+            hbatch = [lcd.HostBatch([(mt["w"][c], mt["inv_s"], M) for mt in mats], dev) for c in range(copies)]
+            for hb in hbatch:
+                for i, mt in enumerate(mats):
+                    hb.x_view(i).copy_(torch.from_numpy(mt["L"].x))
+            h2d, d2h = hbatch[0].x_host.numel(), hbatch[0].y_host.numel()
 
-        def e2e_step(c):
-            for mt, (xh, yh, sc) in zip(mats, host):
-                lcd.linear_host(mt["w"][c], xh, mt["inv_s"], yh, sc)
-            torch.cuda.current_stream().synchronize()
+            def e2e_step(c):
+                hbatch[c].run()
+                torch.cuda.current_stream().synchronize()
+        else:
+            host = []
+            for mt in mats:
+                L = mt["L"]
+                xh = torch.from_numpy(L.x).pin_memory()
+                yh = torch.empty((M, L.N), dtype=torch.float32).pin_memory()
+                sc = torch.empty(lcd.linear_host_scratch_bytes(mt["w"][0], M), dtype=torch.uint8, device=dev)
+                host.append((xh, yh, sc))
+                h2d += xh.numel() * 2
+                d2h += yh.numel() * 4
+
+            def e2e_step(c):
+                for mt, (xh, yh, sc) in zip(mats, host):
+                    lcd.linear_host(mt["w"][c], xh, mt["inv_s"], yh, sc)
+                torch.cuda.current_stream().synchronize()
 
         n_e2e = max(3, min(args.steps, 50))
         for c in range(min(copies, 3)):

@@ -229,6 +229,26 @@ lcd_status lcd_linear_host(const void* packed_weights_dev, const void* header_ho
                            int64_t M, const float* inv_smooth, float* y_host, void* scratch,
                            size_t scratch_bytes, void* cuda_stream);
 
+/* The same for up to LCD_MAX_BATCH independent problems with M <= 16 and equal index width (the projections of
+ * a decoder layer): ONE host-to-device copy of all inputs, one grouped quantise launch, one grouped lookup
+ * launch, ONE device-to-host copy of all outputs.  The host staging buffers are laid out by the library:
+ * problem i's x (fp16 [M][K], dense) starts at the sum of the earlier problems' M*K*2 bytes rounded up to 16,
+ * its y (fp32 [M][N], dense) at the sum of the earlier problems' M*N*4 bytes rounded up to 16;
+ * lcd_linear_host_batch_sizes returns the total sizes (any of the three outputs may be NULL).  x_host_all and
+ * y_host_all should be pinned; y_host_all is valid once cuda_stream is synchronised. */
+typedef struct {
+  const void* packed_weights_dev; /* device, 256-byte aligned */
+  const void* header_host;        /* host */
+  const float* inv_smooth;        /* device fp32 [K] or NULL */
+  int64_t M;
+} lcd_host_problem;
+
+lcd_status lcd_linear_host_batch_sizes(const lcd_host_problem* problems /* host */, int count, size_t* x_host_bytes,
+                                       size_t* y_host_bytes, size_t* scratch_bytes);
+
+lcd_status lcd_linear_host_batch(const lcd_host_problem* problems /* host */, int count, const void* x_host_all,
+                                 void* y_host_all, void* scratch, size_t scratch_bytes, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -25,7 +25,8 @@ MAX_BATCH = 8
 EXPORTS = ["lcd_status_string", "lcd_last_cuda_error", "lcd_packed_weights_bytes", "lcd_pack_weights",
            "lcd_unpack_weights", "lcd_smooth_quantize_act", "lcd_lut_linear_workspace_bytes", "lcd_lut_linear",
            "lcd_linear_host_scratch_bytes", "lcd_linear_host", "lcd_smooth_quantize_act_batch",
-           "lcd_lut_linear_batch_workspace_bytes", "lcd_lut_linear_batch", "lcd_lut_linear_static"]
+           "lcd_lut_linear_batch_workspace_bytes", "lcd_lut_linear_batch", "lcd_lut_linear_static",
+           "lcd_linear_host_batch_sizes", "lcd_linear_host_batch"]
 STATIC_SCRATCH_BYTES = 4 << 20
 
 
@@ -33,6 +34,11 @@ class ActProblem(Structure):
     """lcd_act_problem"""
     _fields_ = [("x_fp16", c_void_p), ("M", c_int64), ("K", c_int64), ("ldx", c_int64), ("inv_smooth", c_void_p),
                 ("static_scale", c_void_p), ("act_idx", c_void_p), ("act_scale", c_void_p)]
+
+
+class HostProblem(Structure):
+    """lcd_host_problem"""
+    _fields_ = [("packed_weights_dev", c_void_p), ("header_host", c_void_p), ("inv_smooth", c_void_p), ("M", c_int64)]
 
 
 class LinearProblem(Structure):
@@ -73,6 +79,9 @@ def _load() -> ctypes.CDLL:
     lib.lcd_lut_linear_batch.argtypes = [POINTER(LinearProblem), c_int, c_int, c_void_p, c_size_t, c_void_p, c_void_p]
     lib.lcd_lut_linear_static.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_int64, c_int,
                                           c_void_p, c_void_p]
+    lib.lcd_linear_host_batch_sizes.argtypes = [POINTER(HostProblem), c_int, POINTER(c_size_t), POINTER(c_size_t),
+                                                POINTER(c_size_t)]
+    lib.lcd_linear_host_batch.argtypes = [POINTER(HostProblem), c_int, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     for name in EXPORTS:
         if name not in ("lcd_status_string", "lcd_last_cuda_error"):
             getattr(lib, name).restype = c_int
@@ -257,6 +266,50 @@ class LinearBatch:
                                         self.workspace.numel(),
                                         c_void_p(self.status_word.data_ptr()) if self.status_word is not None else None,
                                         _stream_ptr(stream)), "lcd_lut_linear_batch")
+
+
+class HostBatch:
+    """lcd_linear_host_batch: up to MAX_BATCH problems (M <= 16) from pinned host inputs to pinned host outputs with
+    one copy in and one copy out.  items: (PackedWeights, inv_smooth CUDA tensor or None, M).  The pinned staging
+    tensors x_host (uint8) / y_host (uint8) and the device scratch are owned here; x_view(i) / y_view(i) give
+    problem i's fp16 [M, K] input and fp32 [M, N] output inside them."""
+
+    def __init__(self, items, device="cuda"):
+        import torch
+        self._keep = list(items)
+        self.count = len(self._keep)
+        self.arr = (HostProblem * self.count)()
+        for a, (w, inv_s, M) in zip(self.arr, self._keep):
+            a.packed_weights_dev, a.header_host = w.dev.data_ptr(), w.header_ptr
+            a.inv_smooth = inv_s.data_ptr() if inv_s is not None else None
+            a.M = M
+        xb, yb, sb = c_size_t(0), c_size_t(0), c_size_t(0)
+        _check(lib.lcd_linear_host_batch_sizes(self.arr, self.count, byref(xb), byref(yb), byref(sb)),
+               "lcd_linear_host_batch_sizes")
+        self.x_host = torch.zeros(xb.value, dtype=torch.uint8).pin_memory()
+        self.y_host = torch.zeros(yb.value, dtype=torch.uint8).pin_memory()
+        self.scratch = torch.empty(sb.value, dtype=torch.uint8, device=device)
+        self._x_off, self._y_off, xo, yo = [], [], 0, 0
+        for w, _, M in self._keep:
+            self._x_off.append(xo)
+            self._y_off.append(yo)
+            xo += (M * w.K * 2 + 15) // 16 * 16
+            yo += (M * w.N * 4 + 15) // 16 * 16
+
+    def x_view(self, i):
+        import torch
+        w, _, M = self._keep[i]
+        return self.x_host[self._x_off[i]:self._x_off[i] + M * w.K * 2].view(torch.float16).view(M, w.K)
+
+    def y_view(self, i):
+        import torch
+        w, _, M = self._keep[i]
+        return self.y_host[self._y_off[i]:self._y_off[i] + M * w.N * 4].view(torch.float32).view(M, w.N)
+
+    def run(self, stream=None):
+        _check(lib.lcd_linear_host_batch(self.arr, self.count, c_void_p(self.x_host.data_ptr()),
+                                         c_void_p(self.y_host.data_ptr()), c_void_p(self.scratch.data_ptr()),
+                                         self.scratch.numel(), _stream_ptr(stream)), "lcd_linear_host_batch")
 
 
 def linear_host_scratch_bytes(w: PackedWeights, M: int) -> int:

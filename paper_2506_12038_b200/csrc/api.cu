@@ -269,3 +269,95 @@ extern "C" lcd_status lcd_linear_host(const void* packed_weights_dev, const void
   if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
   return LCD_OK;
 }
+
+// ---- host-buffer path, grouped ----------------------------------------------------------------------
+namespace {
+struct HostBatchLayout {
+  size_t x_off[LCD_MAX_BATCH], idx_off[LCD_MAX_BATCH], scale_off[LCD_MAX_BATCH], y_off[LCD_MAX_BATCH];
+  size_t x_bytes, y_bytes;      // staging areas (all inputs / all outputs, contiguous)
+  size_t ws_off, ws_bytes, total;
+};
+// Device scratch: | all x (dense, in problem order) | all y (dense, in problem order) | indices | scales | workspace |
+lcd_status host_batch_layout(const lcd_host_problem* probs, int count, Problem* shapes, HostBatchLayout* L) {
+  if (!probs || count < 1 || count > LCD_MAX_BATCH) return LCD_ERR_INVALID_ARG;
+  size_t o = 0;
+  for (int i = 0; i < count; ++i) {
+    if (!probs[i].header_host || probs[i].M < 1) return LCD_ERR_INVALID_ARG;
+    if (probs[i].M > 16) return LCD_ERR_UNSUPPORTED;
+    if (!shape_problem(probs[i].header_host, probs[i].M, &shapes[i])) return LCD_ERR_BAD_BLOB;
+    if (shapes[i].bits != shapes[0].bits) return LCD_ERR_UNSUPPORTED;
+    L->x_off[i] = o;
+    o += (size_t)round_up_u64((uint64_t)probs[i].M * shapes[i].K * 2, 16);
+  }
+  L->x_bytes = o;
+  o = (size_t)round_up_u64(o, 256);
+  const size_t y0 = o;
+  for (int i = 0; i < count; ++i) {
+    L->y_off[i] = o;
+    o += (size_t)round_up_u64((uint64_t)probs[i].M * shapes[i].N * 4, 16);
+  }
+  L->y_bytes = o - y0;
+  o = (size_t)round_up_u64(o, 256);
+  for (int i = 0; i < count; ++i) {
+    L->idx_off[i] = o;
+    o += (size_t)round_up_u64((uint64_t)probs[i].M * shapes[i].K_pad / 2, 256);
+    L->scale_off[i] = o;
+    o += 256;
+  }
+  L->ws_off = o;
+  L->ws_bytes = lut_gemv_workspace_bytes(shapes, count, LCD_ALGO_REGISTER_LUT);
+  L->total = o + (size_t)round_up_u64(L->ws_bytes, 256);
+  return LCD_OK;
+}
+}  // namespace
+
+extern "C" lcd_status lcd_linear_host_batch_sizes(const lcd_host_problem* problems, int count, size_t* x_host_bytes,
+                                                  size_t* y_host_bytes, size_t* scratch_bytes) {
+  Problem shapes[LCD_MAX_BATCH];
+  HostBatchLayout L;
+  const lcd_status st = host_batch_layout(problems, count, shapes, &L);
+  if (st != LCD_OK) return st;
+  if (x_host_bytes) *x_host_bytes = L.x_bytes;
+  if (y_host_bytes) *y_host_bytes = L.y_bytes;
+  if (scratch_bytes) *scratch_bytes = L.total;
+  return LCD_OK;
+}
+
+extern "C" lcd_status lcd_linear_host_batch(const lcd_host_problem* problems, int count, const void* x_host_all,
+                                            void* y_host_all, void* scratch, size_t scratch_bytes, void* cuda_stream) {
+  if (!x_host_all || !y_host_all || !scratch) return LCD_ERR_INVALID_ARG;
+  Problem shapes[LCD_MAX_BATCH];
+  HostBatchLayout L;
+  lcd_status st = host_batch_layout(problems, count, shapes, &L);
+  if (st != LCD_OK) return st;
+  if (scratch_bytes < L.total) return LCD_ERR_BUFFER_TOO_SMALL;
+  if (!aligned(scratch, 256)) return LCD_ERR_INVALID_ARG;
+  uint8_t* base = static_cast<uint8_t*>(scratch);
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e = cudaMemcpyAsync(base, x_host_all, L.x_bytes, cudaMemcpyHostToDevice, stream);   // one copy in
+  if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
+  lcd_act_problem acts[LCD_MAX_BATCH];
+  Problem p[LCD_MAX_BATCH];
+  for (int i = 0; i < count; ++i) {
+    acts[i].x_fp16 = base + L.x_off[i];
+    acts[i].M = problems[i].M;
+    acts[i].K = shapes[i].K;
+    acts[i].ldx = shapes[i].K;
+    acts[i].inv_smooth = problems[i].inv_smooth;
+    acts[i].static_scale = nullptr;
+    acts[i].act_idx = base + L.idx_off[i];
+    acts[i].act_scale = reinterpret_cast<float*>(base + L.scale_off[i]);
+    st = make_problem(problems[i].packed_weights_dev, problems[i].header_host, acts[i].act_idx, acts[i].act_scale,
+                      problems[i].M, reinterpret_cast<float*>(base + L.y_off[i]), shapes[i].N, &p[i]);
+    if (st != LCD_OK) return st;
+  }
+  st = lcd_smooth_quantize_act_batch(acts, count, LCD_ACT_BITS, cuda_stream);
+  if (st != LCD_OK) return st;
+  e = cudaMemsetAsync(base + L.ws_off, 0, L.ws_bytes, stream);    // the lookup kernel wants its scratch zero-filled
+  if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
+  st = launch_lut_gemv(p, count, LCD_ALGO_REGISTER_LUT, base + L.ws_off, L.ws_bytes, nullptr, cuda_stream);
+  if (st != LCD_OK) return st;
+  e = cudaMemcpyAsync(y_host_all, base + L.y_off[0], L.y_bytes, cudaMemcpyDeviceToHost, stream);   // one copy out
+  if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
+  return LCD_OK;
+}

@@ -219,6 +219,22 @@ def test_host_buffer_entry_point():
     check_y(y_host, O.lut_linear_dequant(L.idx, L.codebook, q_ref, s_ref))
 
 
+def test_grouped_host_buffer_entry_point():
+    shapes = [(200, 1000, 1), (1031, 520, 3), (24, 11008, 5)]
+    cases = [gen.random_case(seed=51 + i, N=N, K=K, bits=3, M=M) for i, (N, K, M) in enumerate(shapes)]
+    ws = [lcd.PackedWeights(lcd.pack_weights(L.idx, L.codebook, 3)) for L in cases]
+    hb = lcd.HostBatch([(w, torch.from_numpy(L.inv_s).cuda(), L.M) for w, L in zip(ws, cases)])
+    for _ in range(2):                      # the second call finds the scratch as the first one left it
+        for i, L in enumerate(cases):
+            hb.x_view(i).copy_(torch.from_numpy(L.x))
+        hb.y_host.fill_(255)
+        hb.run()
+        torch.cuda.synchronize()
+        for i, L in enumerate(cases):
+            q_ref, s_ref = O.smooth_quantize(L.x, L.inv_s)
+            check_y(hb.y_view(i), O.lut_linear_dequant(L.idx, L.codebook, q_ref, s_ref))
+
+
 # ------------------------------------------------------------------------------- full sizes, bench launch shape
 def _sampled_rows_check(L, y, q_ref, s_ref, n_rows=48, seed=0):
     rows = np.sort(gen.permutation(seed + L.N, L.N)[:n_rows])
