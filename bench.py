@@ -185,6 +185,23 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+# ----------------------------------------------------------------------------------------------- ranks
+def max_over_ranks(ms, device):
+    """The slowest rank's time (every rank runs its own replica of the layer; no data-path collective)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def per_layer_us(ms_step, world):
+    """Whole-job metric for replicas: `world` replicas each finish one layer per step."""
+    return ms_step * 1e3 / world
+
+
 # ----------------------------------------------------------------------------------------------- ours
 def run_ours(args):
     import torch
@@ -274,9 +291,7 @@ def run_ours(args):
         torch.cuda.synchronize()
         ms_total = e0.elapsed_time(e1)
         if world > 1:
-            t = torch.tensor([ms_total], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_total = float(t.item())
+            ms_total = max_over_ranks(ms_total, dev)
             dist.barrier()
 
         # dominant kernel: the lookup+accumulate launches alone, back to back inside a graph, every launch on
@@ -355,12 +370,10 @@ def run_ours(args):
         torch.cuda.synchronize()
         e2e_ms = max(g0.elapsed_time(g1), (time.perf_counter() - t0) * 1e3) / n_e2e
         if world > 1:
-            t = torch.tensor([e2e_ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+            e2e_ms = max_over_ranks(e2e_ms, dev)
 
     ms_step = ms_total / args.steps
-    us_per_layer = ms_step * 1e3 / world             # `world` replicas each finish one layer per step
+    us_per_layer = per_layer_us(ms_step, world)
     layer_alg_bytes = sum(mt["bytes"] for mt in mats)
     peaks = {}
     try:
