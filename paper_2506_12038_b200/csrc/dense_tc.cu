@@ -676,6 +676,320 @@ dense_tc_ta_kernel(const __grid_constant__ CUtensorMap tmap_act, const DensePara
   if (threadIdx.x == 0 && *abort_flag && P.status) atomicExch(P.status, (int)LCD_ERR_TIMEOUT);
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Integer variant (the default for many tokens).  The row codebook becomes the same two byte tables as in the
+// M <= 16 kernel (16-bit fixed point: signed high byte, unsigned low byte), the decoder emits two int8 A planes
+// with ONE lookup per plane and four weights (no fp16 interleave), the levels are int8, and every stage of 128
+// columns is multiplied twice with tcgen05.mma kind::i8 (twice the fp16 rate) into two int32 accumulators:
+//     y = s_q * 2^e_n * (256 * D_hi + D_lo).
+// Against the fp16 kernels this halves the token bytes streamed from L2 per flop (what bounds them) and halves
+// the decoder's work; the sums are exact integers, the only error is the 2^-16 table quantisation.
+// Tensor memory: two buffers x (D_hi, D_lo) x 128 columns.  Warps as in dense_tc_kernel; the two decoder groups
+// take the two 128-column k-blocks of every item.
+constexpr int kI8BN = 128;                      // tokens per tile
+constexpr int kI8BK = 128;                      // columns per stage = one 128-byte swizzle row of int8
+constexpr int kI8PlaneBytes = kBM * kI8BK;      // 16 KB per plane and stage
+constexpr int kI8BBytes = kI8BN * kI8BK;        // 16 KB per stage
+
+// kind::i8 instruction descriptor: int32 accumulate, B signed, A signed (high plane) or unsigned (low plane).
+__host__ __device__ constexpr uint32_t instr_desc_i8(int n, bool a_signed) {
+  return (2u << 4) | ((a_signed ? 1u : 0u) << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+}
+__device__ __forceinline__ void mma_i8(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr) : "memory");
+}
+
+// Activation levels as int8 in the decoder's column order (see expand_levels_kernel): one thread per (token,
+// 32-column quarter), 16 bytes in, 32 bytes out.
+template <int BITS>
+__global__ void __launch_bounds__(256) expand_levels_i8_kernel(const uint8_t* __restrict__ act_idx, int64_t n_quarters,
+                                                               int8_t* __restrict__ out) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int64_t qi = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (qi >= n_quarters) return;
+  const uint4 a = __ldg(reinterpret_cast<const uint4*>(act_idx) + qi);
+  const uint32_t src[4] = {a.x, a.y, a.z, a.w};
+  uint32_t o[8];
+#pragma unroll
+  for (int v = 0; v < 8; ++v) {
+    uint32_t word = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int p = 4 * v + e;
+      const int col = BITS == 3 ? p : 16 * (p >> 4) + 8 * ((p >> 2) & 1) + 2 * (p & 3) + ((p >> 3) & 1);
+      const uint32_t nib = (src[col >> 3] >> (4 * (col & 7))) & 15u;
+      word |= ((nib - 8u) & 0xffu) << (8 * e);       // q = a - 8 as a signed byte
+    }
+    o[v] = word;
+  }
+  uint4* dst = reinterpret_cast<uint4*>(out + qi * 32);
+  dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+  dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+}
+
+// 2^(e-15) of a row: e is the exponent with max|centroid| < 2^e (the scale of the row's 16-bit fixed point).
+template <int BITS>
+__device__ __forceinline__ float row_exponent_scale(const uint16_t* cb_row, float* up) {
+  float mx = 0.0f;
+#pragma unroll
+  for (int i = 0; i < (1 << BITS); ++i) mx = fmaxf(mx, fabsf(__half2float(__ushort_as_half(__ldg(cb_row + i)))));
+  int ex = (int)((__float_as_uint(mx) >> 23) & 0xffu) - 126;
+  ex = ex < -30 ? -30 : ex;
+  if (up) *up = __uint_as_float((uint32_t)(15 - ex + 127) << 23);
+  return __uint_as_float((uint32_t)(ex - 15 + 127) << 23);
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(kDenseThreads, 1)
+dense_i8_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams P) {
+  extern __shared__ uint8_t smem_raw[];
+  constexpr int ITEM = 512 * BITS, HALF = 256 * BITS;
+  constexpr int BN = kI8BN;
+  constexpr int kStageBytes = 2 * kI8PlaneBytes + kI8BBytes;      // A high plane | A low plane | tokens
+  constexpr uint32_t kTmemCols = 512;                             // two buffers x (D_hi, D_lo) x 128 columns
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  const uint32_t raw_addr = (uint32_t)__cvta_generic_to_shared(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  uint8_t* gen_base = smem_raw + (base - raw_addr);
+  const uint32_t bar_base = base + kStages * kStageBytes;
+  auto full_a = [&](int s) { return bar_base + 8u * s; };
+  auto full_b = [&](int s) { return bar_base + 8u * (kStages + s); };
+  auto empty = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
+  auto tmem_full = [&](int b) { return bar_base + 8u * (3 * kStages + b); };
+  auto tmem_empty = [&](int b) { return bar_base + 8u * (3 * kStages + 2 + b); };
+  const uint32_t drain_bar = bar_base + 8u * (3 * kStages + 4);
+  uint8_t* gen_misc = gen_base + kStages * kStageBytes + 8 * (3 * kStages + 5);
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(gen_misc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_misc + 4);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      bar_init(full_a(s), (kDecodeWarps / 2) * 32);
+      bar_init(full_b(s), 1);
+      bar_init(empty(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      bar_init(tmem_full(b), 1);
+      bar_init(tmem_empty(b), kEpiWarps * 32);
+    }
+    bar_init(drain_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"((uint32_t)__cvta_generic_to_shared(tmem_holder)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_holder;
+
+  const int n_ks = P.n_kt * 2;     // stages per tile: the two 128-column k-blocks of every item
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (int8 levels)
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile % P.n_tiles_m) * BN;
+        for (int ks = 0; ks < n_ks; ++ks, ++it) {
+          const int slot = it % kStages;
+          if (!bar_wait(empty(slot), ((it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          bar_expect_tx(full_b(slot), kI8BBytes);
+          asm volatile(
+              "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+              ::"r"(base + slot * kStageBytes + 2 * kI8PlaneBytes), "l"(&tmap_act), "r"(ks * kI8BK), "r"(m0),
+                "r"(full_b(slot)) : "memory");
+        }
+      }
+      const uint32_t n_back = it < (uint32_t)kStages ? it : (uint32_t)kStages;
+      for (uint32_t i = 1; i <= n_back; ++i) {
+        const uint32_t j = it - i;
+        bar_drain(full_b(j % kStages), (j / kStages) & 1u);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_hi = instr_desc_i8(BN, true), idesc_lo = instr_desc_i8(BN, false);
+      const uint64_t desc0 = smem_desc(base);
+      uint32_t it = 0, tl = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, ++tl) {
+        const uint32_t buf = tl & 1u;
+        if (!bar_wait(tmem_empty(buf), ((tl >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t d_hi = tmem_base + buf * (2 * BN), d_lo = d_hi + BN;
+        for (int ks = 0; ks < n_ks; ++ks, ++it) {
+          const int slot = it % kStages;
+          const uint32_t ph = (it / kStages) & 1u;
+          if (!bar_wait(full_a(slot), ph, abort_flag) || !bar_wait(full_b(slot), ph, abort_flag)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint64_t ah = desc0 + (uint64_t)((slot * kStageBytes) >> 4);
+          const uint64_t al = ah + (uint64_t)(kI8PlaneBytes >> 4), bd = ah + (uint64_t)((2 * kI8PlaneBytes) >> 4);
+#pragma unroll
+          for (int k = 0; k < kI8BK / 32; ++k) {         // 32 int8 columns = 32 bytes per MMA
+            const uint32_t accumulate = (uint32_t)((ks | k) != 0);
+            mma_i8(d_hi, ah + 2 * k, bd + 2 * k, idesc_hi, accumulate);
+            mma_i8(d_lo, al + 2 * k, bd + 2 * k, idesc_lo, accumulate);
+          }
+          mma_commit(empty(slot));
+        }
+        if (ok) mma_commit(tmem_full(buf));
+      }
+      mma_commit(drain_bar);
+      bar_drain(drain_bar, 0);
+    }
+    __syncwarp();
+  } else if (warp < kFirstDecodeWarp) {
+    // ------------------------------------------------------------------ epilogue
+    const int quad = warp & 3;
+    uint32_t tl = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, ++tl) {
+      const uint32_t buf = tl & 1u;
+      const int n = (tile / P.n_tiles_m) * kBM + 32 * quad + lane;
+      const int m0 = (tile % P.n_tiles_m) * BN;
+      // this thread's row: 2^(e-15) of its fixed-point tables (rows past the matrix are never stored)
+      const int n_cb = n < P.n_rp * 16 ? n : P.n_rp * 16 - 1;
+      const float row_scale = row_exponent_scale<BITS>(P.codebook + (size_t)n_cb * (1 << BITS), nullptr);
+      ok = __all_sync(0xffffffffu, bar_wait(tmem_full(buf), (tl >> 1) & 1u, abort_flag));
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll 1
+      for (int c = 0; c < BN / 16; ++c) {
+        uint32_t hi[16], lo[16];
+        const uint32_t t_hi = tmem_base + ((uint32_t)(32 * quad) << 16) + buf * (2 * BN) + 16 * c;
+        tmem_ld16(t_hi, hi);
+        tmem_ld16(t_hi + BN, lo);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        const int mc = m0 + 16 * c;
+        const float my_scale = (lane < 16 && mc + lane < P.M) ? __ldg(P.act_scale + mc + lane) : 0.0f;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const float s = __shfl_sync(0xffffffffu, my_scale, j) * row_scale;
+          if (mc + j < P.M && n < P.N)
+            P.y[(size_t)(mc + j) * P.ldy + n] = ((float)(int)hi[j] * 256.0f + (float)(int)lo[j]) * s;
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      bar_arrive(tmem_empty(buf));
+    }
+  } else {
+    // ------------------------------------------------------------------ decoder
+    // Group 0 decodes k-block 0 of every item, group 1 k-block 1 (stage number parity).  Warp dw owns the tile's
+    // 16-row group dw; a thread owns 64 columns (quarters 2x and 2x + 1) of one row per stage.
+    const int grp = (warp - kFirstDecodeWarp) >> 3, dw = (warp - kFirstDecodeWarp) & 7;
+    const int u = lane >> 4, g = (lane >> 1) & 7, x = lane & 1;
+    const uint32_t row_off = (uint32_t)((2 * dw + u) * 1024 + g * 128);
+    uint32_t it0 = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, it0 += (uint32_t)n_ks) {
+      int rp = (tile / P.n_tiles_m) * (kBM / 16) + dw;
+      rp = rp < P.n_rp ? rp : P.n_rp - 1;          // rows past the matrix repeat the last group; never stored
+      // byte tables of this thread's row: 16-bit fixed point, high (signed) and low (unsigned) bytes
+      uint32_t TH[2] = {0, 0}, TL[2] = {0, 0};
+      {
+        const uint16_t* cb = P.codebook + ((size_t)rp * 16 + 8 * u + g) * (1 << BITS);
+        float up;
+        (void)row_exponent_scale<BITS>(cb, &up);
+#pragma unroll
+        for (int i = 0; i < (1 << BITS); ++i) {
+          const int f = __float2int_rn(__half2float(__ushort_as_half(__ldg(cb + i))) * up);
+          TH[i >> 2] |= ((uint32_t)(f >> 8) & 0xffu) << (8 * (i & 3));
+          TL[i >> 2] |= ((uint32_t)f & 0xffu) << (8 * (i & 3));
+        }
+        if (BITS == 2) { TH[1] = TH[0]; TL[1] = TL[0]; }
+      }
+      const uint8_t* row_items = P.items + (size_t)rp * P.n_kt * ITEM + u * HALF;
+      uint32_t cur[2][BITS == 2 ? 2 : 3], nxt[2][BITS == 2 ? 2 : 3];      // [quarter][word]
+      auto load_stage = [&](uint32_t (&dst)[2][BITS == 2 ? 2 : 3], int kt) {
+        const uint8_t* item = row_items + (size_t)kt * ITEM;
+#pragma unroll
+        for (int xq = 0; xq < 2; ++xq) {
+          const int l = 4 * g + 2 * x + xq;
+          if (BITS == 2) {
+            const uint2 w = __ldg(reinterpret_cast<const uint2*>(item + 16 * l + 8 * grp));
+            dst[xq][0] = w.x; dst[xq][1] = w.y;
+          } else {
+#pragma unroll
+            for (int b = 0; b < 3; ++b)
+              dst[xq][b] = __ldg(reinterpret_cast<const uint32_t*>(item + 256 * b + 8 * l + 4 * grp));
+          }
+        }
+      };
+      load_stage(cur, 0);
+      for (int kt = 0; kt < P.n_kt && ok; ++kt) {
+        if (kt + 1 < P.n_kt) load_stage(nxt, kt + 1);
+        const uint32_t it = it0 + 2u * (uint32_t)kt + (uint32_t)grp;
+        const int slot = it % kStages;
+        if (!bar_wait(empty(slot), ((it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        uint8_t* a_row = gen_base + slot * kStageBytes + row_off;
+#pragma unroll
+        for (int xq = 0; xq < 2; ++xq) {
+          uint32_t sel[8];
+          if (BITS == 2) {
+#pragma unroll
+            for (int wd = 0; wd < 2; ++wd) {
+              const uint32_t raw = cur[xq][wd];
+              const uint32_t s0 = raw & 0x33333333u, s1 = (raw >> 2) & 0x33333333u;
+              sel[4 * wd] = s0; sel[4 * wd + 1] = s0 >> 16; sel[4 * wd + 2] = s1; sel[4 * wd + 3] = s1 >> 16;
+            }
+          } else {
+            const uint32_t r0 = cur[xq][0], r1 = cur[xq][1], r2 = cur[xq][2];
+            const uint32_t ex = (((r0 >> 3) & 0x11111111u) | ((r1 >> 2) & 0x22222222u)) | ((r2 >> 1) & 0x44444444u);
+            const uint32_t d0 = r0 & 0x77777777u, d1 = r1 & 0x77777777u, d2 = r2 & 0x77777777u;
+            sel[0] = d0; sel[1] = d0 >> 16; sel[2] = d1; sel[3] = d1 >> 16;
+            sel[4] = d2; sel[5] = d2 >> 16; sel[6] = ex; sel[7] = ex >> 16;
+          }
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {            // 16-byte chunk = 16 weights = four lookups, per plane
+            uint32_t h4[4], l4[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              h4[i] = prmt_b(TH[0], TH[1], sel[4 * c + i]);
+              l4[i] = prmt_b(TL[0], TL[1], sel[4 * c + i]);
+            }
+            const int chunk = (4 * x + 2 * xq + c) ^ g;     // 128-byte swizzle
+            *reinterpret_cast<uint4*>(a_row + 16 * chunk) = make_uint4(h4[0], h4[1], h4[2], h4[3]);
+            *reinterpret_cast<uint4*>(a_row + kI8PlaneBytes + 16 * chunk) = make_uint4(l4[0], l4[1], l4[2], l4[3]);
+          }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic stores -> visible to the MMA
+        bar_arrive(full_a(slot));
+#pragma unroll
+        for (int xq = 0; xq < 2; ++xq)
+#pragma unroll
+          for (int b = 0; b < (BITS == 2 ? 2 : 3); ++b) cur[xq][b] = nxt[xq][b];
+      }
+    }
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+  if (threadIdx.x == 0 && *abort_flag && P.status) atomicExch(P.status, (int)LCD_ERR_TIMEOUT);
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -758,18 +1072,67 @@ lcd_status launch_dense_t(const Problem& p, __half* levels, int32_t* status_word
   return LCD_OK;
 }
 
+template <int BITS>
+lcd_status launch_dense_i8(const Problem& p, int8_t* levels, int32_t* status_word, cudaStream_t stream) {
+  EncodeTiledFn enc = encode_tiled();
+  if (!enc) return LCD_ERR_CUDA;
+  CUtensorMap tmap;
+  const cuuint64_t dims[2] = {(cuuint64_t)p.K_pad, (cuuint64_t)p.M};
+  const cuuint64_t strides[1] = {(cuuint64_t)p.K_pad};
+  const cuuint32_t box[2] = {(cuuint32_t)kI8BK, (cuuint32_t)kI8BN};
+  const cuuint32_t estr[2] = {1, 1};
+  if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, levels, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return LCD_ERR_CUDA;
+  DenseParams dp;
+  dp.items = p.tiles;
+  dp.codebook = p.codebook;
+  dp.act_scale = p.act_scale;
+  dp.y = p.y;
+  dp.ldy = p.ldy;
+  dp.N = (int)p.N;
+  dp.M = (int)p.M;
+  dp.n_rp = (int)(p.N_pad / kPairRows);
+  dp.n_kt = (int)(p.K_pad / kTileK);
+  dp.n_tiles_m = (int)((p.M + kI8BN - 1) / kI8BN);
+  dp.n_tiles = dp.n_tiles_m * (int)((p.N_pad + kBM - 1) / kBM);
+  dp.status = status_word;
+  const size_t smem = 1024 + (size_t)kStages * (2 * kI8PlaneBytes + kI8BBytes) + 256;
+  auto kern = dense_i8_kernel<BITS>;
+  static bool attr_set = false;   // per template instance
+  if (!attr_set) {
+    const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
+    attr_set = true;
+  }
+  const int grid = dp.n_tiles < dense_sm_count() ? dp.n_tiles : dense_sm_count();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kDenseThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmap, dp);
+  if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
+  return LCD_OK;
+}
+
 // Tile shapes: {kernel, row tiles, tokens, cycles per 64-column stage}.  The stage times are measured ones: with
 // 128 rows per CTA the token tiles streamed from L2 bound the stage (the L2-to-SM path runs at about 8 TB/s), so a
 // stage costs about 3.5 cycles per token of tile width.  (A 256-row tile, RT = 2, halves that traffic and is
 // supported by the kernel, but its decoder did not keep up when measured, so it is not among the choices.)
 struct TileShape { int kernel, rt, bn, stage_clks, epilogue_clks; };
-constexpr TileShape kShapes[3] = {{1, 1, 192, 664, 0}, {1, 1, 128, 443, 0}, {0, 1, 256, 733, 0}};
+constexpr TileShape kShapes[4] = {{1, 1, 192, 664, 0}, {1, 1, 128, 443, 0}, {0, 1, 256, 733, 0}, {2, 1, 128, 1, 0}};
 
 int pick_shape(int64_t M, int64_t N_pad, int64_t n_ks) {
   const int n_sm = dense_sm_count();
   int best = 0;
   int64_t best_cost = -1;
-  for (int i = 0; i < 3; ++i) {
+  for (int i = 0; i < 4; ++i) {
     const TileShape& t = kShapes[i];
     const int64_t tiles = ((N_pad + t.rt * kBM - 1) / (t.rt * kBM)) * ((M + t.bn - 1) / t.bn);
     const int64_t cost = ((tiles + n_sm - 1) / n_sm) * (n_ks * t.stage_clks + t.epilogue_clks);
@@ -787,14 +1150,22 @@ lcd_status launch_dense_tc(const Problem& p, void* workspace, size_t workspace_b
   if (!workspace || workspace_bytes < dense_tc_workspace_bytes(p.M, p.K_pad)) return LCD_ERR_BUFFER_TOO_SMALL;
   if (p.M > 0x7fffffffLL / 2 || p.N > 0x7fffffffLL / 2) return LCD_ERR_UNSUPPORTED;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  __half* levels = static_cast<__half*>(workspace);
   const int64_t n_quarters = p.M * (p.K_pad / 32);
   const unsigned blocks = (unsigned)((n_quarters + 255) / 256);
+  const int shape = pick_shape(p.M, p.N_pad, p.K_pad / kBK);
+  if (kShapes[shape].kernel == 2) {
+    int8_t* levels = static_cast<int8_t*>(workspace);
+    if (p.bits == 2) expand_levels_i8_kernel<2><<<blocks, 256, 0, s>>>(p.act_idx, n_quarters, levels);
+    else expand_levels_i8_kernel<3><<<blocks, 256, 0, s>>>(p.act_idx, n_quarters, levels);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
+    return p.bits == 2 ? launch_dense_i8<2>(p, levels, status_word, s) : launch_dense_i8<3>(p, levels, status_word, s);
+  }
+  __half* levels = static_cast<__half*>(workspace);
   if (p.bits == 2) expand_levels_kernel<2><<<blocks, 256, 0, s>>>(p.act_idx, n_quarters, levels);
   else expand_levels_kernel<3><<<blocks, 256, 0, s>>>(p.act_idx, n_quarters, levels);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
-  const int shape = pick_shape(p.M, p.N_pad, p.K_pad / kBK);
 #define LCD_DENSE_CASE(B, I, W, R, KN) \
   if (p.bits == B && shape == I) return launch_dense_t<B, W, R, KN>(p, levels, status_word, s);
   LCD_DENSE_CASE(2, 0, 192, 1, 1) LCD_DENSE_CASE(2, 1, 128, 1, 1) LCD_DENSE_CASE(2, 2, 256, 1, 0)
