@@ -684,12 +684,17 @@ dense_tc_ta_kernel(const __grid_constant__ CUtensorMap tmap_act, const DensePara
 //     y = s_q * 2^e_n * (256 * D_hi + D_lo).
 // Against the fp16 kernels this halves the token bytes streamed from L2 per flop (what bounds them) and halves
 // the decoder's work; the sums are exact integers, the only error is the 2^-16 table quantisation.
-// Tensor memory: two buffers x (D_hi, D_lo) x 128 columns.  Warps as in dense_tc_kernel; the two decoder groups
-// take the two 128-column k-blocks of every item.
-constexpr int kI8BN = 128;                      // tokens per tile
+// Tensor memory: (D_hi, D_lo) x BN columns per accumulator buffer.  Warps as in dense_tc_kernel plus a second MMA
+// issuer; the two decoder groups take the two 128-column k-blocks of every item.
 constexpr int kI8BK = 128;                      // columns per stage = one 128-byte swizzle row of int8
 constexpr int kI8PlaneBytes = kBM * kI8BK;      // 16 KB per plane and stage
-constexpr int kI8BBytes = kI8BN * kI8BK;        // 16 KB per stage
+// Tiles of 128 tokens have two accumulator buffers (the epilogue overlaps the next tile); 192 and 256 tokens have
+// one, but their MMAs are long enough (96 / 128 cycles) to hide the issue latency of the two issuing threads.
+__host__ __device__ constexpr int i8_stages(int bn) { return bn <= 192 ? 4 : 3; }   // stages that fit in 227 KB
+// warps: 0 TMA, 1 MMA issuer (high plane), 2-9 epilogue, 10-25 decoder, 26 MMA issuer (low plane)
+constexpr int kI8EpiWarps = 8;
+constexpr int kI8FirstDecodeWarp = kFirstEpiWarp + kI8EpiWarps;
+constexpr int kI8Threads = 32 * (kI8FirstDecodeWarp + kDecodeWarps + 1);   // 864
 
 // kind::i8 instruction descriptor: int32 accumulate, B signed, A signed (high plane) or unsigned (low plane).
 __host__ __device__ constexpr uint32_t instr_desc_i8(int n, bool a_signed) {
@@ -748,22 +753,26 @@ __device__ __forceinline__ float row_exponent_scale(const uint16_t* cb_row, floa
   return __uint_as_float((uint32_t)(ex - 15 + 127) << 23);
 }
 
-template <int BITS>
-__global__ void __launch_bounds__(kDenseThreads, 1)
+template <int BITS, int BN>
+__global__ void __launch_bounds__(kI8Threads, 1)
 dense_i8_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams P) {
   extern __shared__ uint8_t smem_raw[];
   constexpr int ITEM = 512 * BITS, HALF = 256 * BITS;
-  constexpr int BN = kI8BN;
+  constexpr int kI8BBytes = BN * kI8BK;
+  constexpr int kStages = i8_stages(BN);                          // shadows the fp16 kernels' stage count
+  constexpr int NBUF = BN <= 128 ? 2 : 1;                         // accumulator buffers of (D_hi, D_lo) x BN columns
   constexpr int kStageBytes = 2 * kI8PlaneBytes + kI8BBytes;      // A high plane | A low plane | tokens
-  constexpr uint32_t kTmemCols = 512;                             // two buffers x (D_hi, D_lo) x 128 columns
+  constexpr uint32_t kTmemCols = 512;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   const uint32_t raw_addr = (uint32_t)__cvta_generic_to_shared(smem_raw);
   const uint32_t base = (raw_addr + 1023u) & ~1023u;
   uint8_t* gen_base = smem_raw + (base - raw_addr);
   const uint32_t bar_base = base + kStages * kStageBytes;
+  // full(s): the stage's operands are ready = all arrivals of one decoder group + the TMA producer's arrival
+  // with its byte count
   auto full_a = [&](int s) { return bar_base + 8u * s; };
-  auto full_b = [&](int s) { return bar_base + 8u * (kStages + s); };
+  auto full_b = [&](int s) { return bar_base + 8u * s; };
   auto empty = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
   auto tmem_full = [&](int b) { return bar_base + 8u * (3 * kStages + b); };
   auto tmem_empty = [&](int b) { return bar_base + 8u * (3 * kStages + 2 + b); };
@@ -774,15 +783,14 @@ dense_i8_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      bar_init(full_a(s), (kDecodeWarps / 2) * 32);
-      bar_init(full_b(s), 1);
-      bar_init(empty(s), 1);
+      bar_init(full_a(s), (kDecodeWarps / 2) * 32 + 1);
+      bar_init(empty(s), 2);                        // both MMA issuers release a stage
     }
     for (int b = 0; b < 2; ++b) {
-      bar_init(tmem_full(b), 1);
-      bar_init(tmem_empty(b), kEpiWarps * 32);
+      bar_init(tmem_full(b), 2);
+      bar_init(tmem_empty(b), kI8EpiWarps * 32);
     }
-    bar_init(drain_bar, 1);
+    bar_init(drain_bar, 2);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -824,31 +832,30 @@ dense_i8_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
       }
     }
     __syncwarp();
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
+  } else if (warp == 1 || warp == kI8Threads / 32 - 1) {
+    // ------------------------------------------------------------------ MMA issuers
+    // Two threads in two warps, one per byte plane (independent accumulators): a single thread cannot issue the
+    // eight MMAs of a stage as fast as the tensor pipe executes them.
     if (lane == 0) {
-      constexpr uint32_t idesc_hi = instr_desc_i8(BN, true), idesc_lo = instr_desc_i8(BN, false);
-      const uint64_t desc0 = smem_desc(base);
+      const bool is_hi = warp == 1;
+      const uint32_t idesc = is_hi ? instr_desc_i8(BN, true) : instr_desc_i8(BN, false);
+      const uint64_t desc0 = smem_desc(base) + (uint64_t)(is_hi ? 0 : (kI8PlaneBytes >> 4));
       uint32_t it = 0, tl = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, ++tl) {
-        const uint32_t buf = tl & 1u;
-        if (!bar_wait(tmem_empty(buf), ((tl >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        const uint32_t buf = tl % NBUF;
+        if (!bar_wait(tmem_empty(buf), ((tl / NBUF) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t d_hi = tmem_base + buf * (2 * BN), d_lo = d_hi + BN;
+        const uint32_t d = tmem_base + buf * (2 * BN) + (is_hi ? 0 : BN);
         for (int ks = 0; ks < n_ks; ++ks, ++it) {
           const int slot = it % kStages;
-          const uint32_t ph = (it / kStages) & 1u;
-          if (!bar_wait(full_a(slot), ph, abort_flag) || !bar_wait(full_b(slot), ph, abort_flag)) { ok = false; break; }
+          if (!bar_wait(full_a(slot), (it / kStages) & 1u, abort_flag)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint64_t ah = desc0 + (uint64_t)((slot * kStageBytes) >> 4);
-          const uint64_t al = ah + (uint64_t)(kI8PlaneBytes >> 4), bd = ah + (uint64_t)((2 * kI8PlaneBytes) >> 4);
+          const uint64_t ad = desc0 + (uint64_t)((slot * kStageBytes) >> 4);
+          const uint64_t bd = smem_desc(base) + (uint64_t)((slot * kStageBytes + 2 * kI8PlaneBytes) >> 4);
+          mma_i8(d, ad, bd, idesc, (uint32_t)(ks != 0));
 #pragma unroll
-          for (int k = 0; k < kI8BK / 32; ++k) {         // 32 int8 columns = 32 bytes per MMA
-            const uint32_t accumulate = (uint32_t)((ks | k) != 0);
-            mma_i8(d_hi, ah + 2 * k, bd + 2 * k, idesc_hi, accumulate);
-            mma_i8(d_lo, al + 2 * k, bd + 2 * k, idesc_lo, accumulate);
-          }
+          for (int k = 1; k < kI8BK / 32; ++k) mma_i8(d, ad + 2 * k, bd + 2 * k, idesc, 1u);   // 32 bytes per MMA
           mma_commit(empty(slot));
         }
         if (ok) mma_commit(tmem_full(buf));
@@ -857,23 +864,24 @@ dense_i8_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
       bar_drain(drain_bar, 0);
     }
     __syncwarp();
-  } else if (warp < kFirstDecodeWarp) {
+  } else if (warp < kI8FirstDecodeWarp) {
     // ------------------------------------------------------------------ epilogue
-    const int quad = warp & 3;
+    // two warps per tensor-memory quadrant, each drains every other 16-token chunk
+    const int quad = warp & 3, half = (warp - kFirstEpiWarp) >> 2;
     uint32_t tl = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, ++tl) {
-      const uint32_t buf = tl & 1u;
+      const uint32_t buf = tl % NBUF;
       const int n = (tile / P.n_tiles_m) * kBM + 32 * quad + lane;
       const int m0 = (tile % P.n_tiles_m) * BN;
       // this thread's row: 2^(e-15) of its fixed-point tables (rows past the matrix are never stored)
       const int n_cb = n < P.n_rp * 16 ? n : P.n_rp * 16 - 1;
       const float row_scale = row_exponent_scale<BITS>(P.codebook + (size_t)n_cb * (1 << BITS), nullptr);
-      ok = __all_sync(0xffffffffu, bar_wait(tmem_full(buf), (tl >> 1) & 1u, abort_flag));
+      ok = __all_sync(0xffffffffu, bar_wait(tmem_full(buf), (tl / NBUF) & 1u, abort_flag));
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll 1
-      for (int c = 0; c < BN / 16; ++c) {
+      for (int c = half; c < BN / 16; c += kI8EpiWarps / 4) {
         uint32_t hi[16], lo[16];
         const uint32_t t_hi = tmem_base + ((uint32_t)(32 * quad) << 16) + buf * (2 * BN) + 16 * c;
         tmem_ld16(t_hi, hi);
@@ -895,7 +903,7 @@ dense_i8_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
     // ------------------------------------------------------------------ decoder
     // Group 0 decodes k-block 0 of every item, group 1 k-block 1 (stage number parity).  Warp dw owns the tile's
     // 16-row group dw; a thread owns 64 columns (quarters 2x and 2x + 1) of one row per stage.
-    const int grp = (warp - kFirstDecodeWarp) >> 3, dw = (warp - kFirstDecodeWarp) & 7;
+    const int grp = (warp - kI8FirstDecodeWarp) >> 3, dw = (warp - kI8FirstDecodeWarp) & 7;
     const int u = lane >> 4, g = (lane >> 1) & 7, x = lane & 1;
     const uint32_t row_off = (uint32_t)((2 * dw + u) * 1024 + g * 128);
     uint32_t it0 = 0;
@@ -939,8 +947,9 @@ dense_i8_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
         if (kt + 1 < P.n_kt) load_stage(nxt, kt + 1);
         const uint32_t it = it0 + 2u * (uint32_t)kt + (uint32_t)grp;
         const int slot = it % kStages;
-        if (!bar_wait(empty(slot), ((it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-        uint8_t* a_row = gen_base + slot * kStageBytes + row_off;
+        // look everything up first (registers), wait for the stage to be free only then: the wait for the MMAs
+        // that last read this stage overlaps the lookups
+        uint32_t hw[2][2][4], lw[2][2][4];          // [quarter][chunk][word]
 #pragma unroll
         for (int xq = 0; xq < 2; ++xq) {
           uint32_t sel[8];
@@ -959,18 +968,24 @@ dense_i8_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
             sel[4] = d2; sel[5] = d2 >> 16; sel[6] = ex; sel[7] = ex >> 16;
           }
 #pragma unroll
-          for (int c = 0; c < 2; ++c) {            // 16-byte chunk = 16 weights = four lookups, per plane
-            uint32_t h4[4], l4[4];
+          for (int c = 0; c < 2; ++c)
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-              h4[i] = prmt_b(TH[0], TH[1], sel[4 * c + i]);
-              l4[i] = prmt_b(TL[0], TL[1], sel[4 * c + i]);
+              hw[xq][c][i] = prmt_b(TH[0], TH[1], sel[4 * c + i]);
+              lw[xq][c][i] = prmt_b(TL[0], TL[1], sel[4 * c + i]);
             }
-            const int chunk = (4 * x + 2 * xq + c) ^ g;     // 128-byte swizzle
-            *reinterpret_cast<uint4*>(a_row + 16 * chunk) = make_uint4(h4[0], h4[1], h4[2], h4[3]);
-            *reinterpret_cast<uint4*>(a_row + kI8PlaneBytes + 16 * chunk) = make_uint4(l4[0], l4[1], l4[2], l4[3]);
-          }
         }
+        if (!bar_wait(empty(slot), ((it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+        uint8_t* a_row = gen_base + slot * kStageBytes + row_off;
+#pragma unroll
+        for (int xq = 0; xq < 2; ++xq)
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {            // 16-byte chunk = 16 weights = four lookups, per plane
+            const int chunk = (4 * x + 2 * xq + c) ^ g;     // 128-byte swizzle
+            *reinterpret_cast<uint4*>(a_row + 16 * chunk) = make_uint4(hw[xq][c][0], hw[xq][c][1], hw[xq][c][2], hw[xq][c][3]);
+            *reinterpret_cast<uint4*>(a_row + kI8PlaneBytes + 16 * chunk) =
+                make_uint4(lw[xq][c][0], lw[xq][c][1], lw[xq][c][2], lw[xq][c][3]);
+          }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic stores -> visible to the MMA
         bar_arrive(full_a(slot));
 #pragma unroll
@@ -1072,14 +1087,14 @@ lcd_status launch_dense_t(const Problem& p, __half* levels, int32_t* status_word
   return LCD_OK;
 }
 
-template <int BITS>
+template <int BITS, int BN>
 lcd_status launch_dense_i8(const Problem& p, int8_t* levels, int32_t* status_word, cudaStream_t stream) {
   EncodeTiledFn enc = encode_tiled();
   if (!enc) return LCD_ERR_CUDA;
   CUtensorMap tmap;
   const cuuint64_t dims[2] = {(cuuint64_t)p.K_pad, (cuuint64_t)p.M};
   const cuuint64_t strides[1] = {(cuuint64_t)p.K_pad};
-  const cuuint32_t box[2] = {(cuuint32_t)kI8BK, (cuuint32_t)kI8BN};
+  const cuuint32_t box[2] = {(cuuint32_t)kI8BK, (cuuint32_t)BN};
   const cuuint32_t estr[2] = {1, 1};
   if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, levels, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -1094,11 +1109,11 @@ lcd_status launch_dense_i8(const Problem& p, int8_t* levels, int32_t* status_wor
   dp.M = (int)p.M;
   dp.n_rp = (int)(p.N_pad / kPairRows);
   dp.n_kt = (int)(p.K_pad / kTileK);
-  dp.n_tiles_m = (int)((p.M + kI8BN - 1) / kI8BN);
+  dp.n_tiles_m = (int)((p.M + BN - 1) / BN);
   dp.n_tiles = dp.n_tiles_m * (int)((p.N_pad + kBM - 1) / kBM);
   dp.status = status_word;
-  const size_t smem = 1024 + (size_t)kStages * (2 * kI8PlaneBytes + kI8BBytes) + 256;
-  auto kern = dense_i8_kernel<BITS>;
+  const size_t smem = 1024 + (size_t)i8_stages(BN) * (2 * kI8PlaneBytes + BN * kI8BK) + 256;
+  auto kern = dense_i8_kernel<BITS, BN>;
   static bool attr_set = false;   // per template instance
   if (!attr_set) {
     const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -1108,7 +1123,7 @@ lcd_status launch_dense_i8(const Problem& p, int8_t* levels, int32_t* status_wor
   const int grid = dp.n_tiles < dense_sm_count() ? dp.n_tiles : dense_sm_count();
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
-  cfg.blockDim = dim3(kDenseThreads);
+  cfg.blockDim = dim3(kI8Threads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -1121,18 +1136,19 @@ lcd_status launch_dense_i8(const Problem& p, int8_t* levels, int32_t* status_wor
   return LCD_OK;
 }
 
-// Tile shapes: {kernel, row tiles, tokens, cycles per 64-column stage}.  The stage times are measured ones: with
-// 128 rows per CTA the token tiles streamed from L2 bound the stage (the L2-to-SM path runs at about 8 TB/s), so a
-// stage costs about 3.5 cycles per token of tile width.  (A 256-row tile, RT = 2, halves that traffic and is
-// supported by the kernel, but its decoder did not keep up when measured, so it is not among the choices.)
+// Tile shapes: {kernel (0 fp16 / A in shared memory, 1 fp16 / A in tensor memory, 2 int8 planes), row tiles,
+// tokens, cycles per 64 columns of a tile, cycles per tile that do not overlap (epilogue of the shapes with one
+// accumulator buffer)}.  The numbers are measured on the LLaMA-13B shapes (1.7 GHz under load); the launcher takes
+// the shape with the smallest waves x (columns x stage + fixed).
 struct TileShape { int kernel, rt, bn, stage_clks, epilogue_clks; };
-constexpr TileShape kShapes[4] = {{1, 1, 192, 664, 0}, {1, 1, 128, 443, 0}, {0, 1, 256, 733, 0}, {2, 1, 128, 1, 0}};
+constexpr TileShape kShapes[6] = {{1, 1, 192, 664, 0}, {1, 1, 128, 443, 0}, {0, 1, 256, 733, 0},
+                                  {2, 1, 128, 425, 0}, {2, 1, 192, 400, 19900}, {2, 1, 256, 535, 19000}};
 
 int pick_shape(int64_t M, int64_t N_pad, int64_t n_ks) {
   const int n_sm = dense_sm_count();
   int best = 0;
   int64_t best_cost = -1;
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < 6; ++i) {
     const TileShape& t = kShapes[i];
     const int64_t tiles = ((N_pad + t.rt * kBM - 1) / (t.rt * kBM)) * ((M + t.bn - 1) / t.bn);
     const int64_t cost = ((tiles + n_sm - 1) / n_sm) * (n_ks * t.stage_clks + t.epilogue_clks);
@@ -1159,7 +1175,13 @@ lcd_status launch_dense_tc(const Problem& p, void* workspace, size_t workspace_b
     else expand_levels_i8_kernel<3><<<blocks, 256, 0, s>>>(p.act_idx, n_quarters, levels);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
-    return p.bits == 2 ? launch_dense_i8<2>(p, levels, status_word, s) : launch_dense_i8<3>(p, levels, status_word, s);
+    const int bn = kShapes[shape].bn;
+    if (p.bits == 2) return bn == 128 ? launch_dense_i8<2, 128>(p, levels, status_word, s)
+                          : bn == 192 ? launch_dense_i8<2, 192>(p, levels, status_word, s)
+                                      : launch_dense_i8<2, 256>(p, levels, status_word, s);
+    return bn == 128 ? launch_dense_i8<3, 128>(p, levels, status_word, s)
+         : bn == 192 ? launch_dense_i8<3, 192>(p, levels, status_word, s)
+                     : launch_dense_i8<3, 256>(p, levels, status_word, s);
   }
   __half* levels = static_cast<__half*>(workspace);
   if (p.bits == 2) expand_levels_kernel<2><<<blocks, 256, 0, s>>>(p.act_idx, n_quarters, levels);
