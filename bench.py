@@ -407,7 +407,7 @@ def run_ours(args):
         return
     line = {"metric": metric_name(M), "value": us_per_layer, "unit": "us/layer", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
-            "vs_baseline": None, "dtype": "s8 table bytes x s8 levels -> s32 (int8 MMA), f32 epilogue" if not tensor_bound else "f16 x f16 -> f32",
+            "vs_baseline": None, "dtype": "s8 table bytes x s8 levels -> s32 (int8 MMA), f32 epilogue" if not tensor_bound else "s8 table bytes x s8 levels -> s32 (tcgen05 kind::i8), f32 epilogue",
             "data": "synthetic", "config": dict(workload_config(args.config, M, copies),
                                                 launches="1 grouped quantise + 1 grouped lookup per layer" if grouped
                                                 else "per matrix: quantise + lookup"),

@@ -50,8 +50,11 @@ typedef enum {
   LCD_ALGO_REGISTER_LUT = 3,/* Section 4.2 lookup with the row codebook held as byte tables in registers        */
                             /* (16-bit fixed point, high and low byte), four weights looked up per instruction,  */
                             /* accumulated by int8 tensor-core MMAs against the activation levels.  M <= 16.     */
-  LCD_ALGO_DENSE_TC = 4     /* batched prefill: indices decoded through the codebook into fp16 shared-memory   */
-                            /* tiles feeding tcgen05 tensor cores with fp32 accumulators in tensor memory.      */
+  LCD_ALGO_DENSE_TC = 4,    /* batched prefill on tcgen05 tensor cores: the byte tables of REGISTER_LUT decode   */
+                            /* the indices into two int8 planes in shared memory, int8 levels arrive by TMA,     */
+                            /* kind::i8 MMAs accumulate exact int32 sums in tensor memory.                      */
+  LCD_ALGO_DENSE_F16 = 5    /* the same with fp16 operands: indices decoded through the codebook into fp16     */
+                            /* shared-memory tiles, fp32 accumulators (no fixed-point step; slower).            */
 } lcd_algo;
 
 #define LCD_HEADER_BYTES 64

@@ -73,6 +73,7 @@ static lcd_status workspace_for(const Problem& p, lcd_algo algo, size_t* bytes) 
       *bytes = lut_gemv_workspace_bytes(&p, 1, resolve_algo(p.M, algo));
       return LCD_OK;
     case LCD_ALGO_DENSE_TC:
+    case LCD_ALGO_DENSE_F16:
       *bytes = dense_tc_workspace_bytes(p.M, p.K_pad);
       return LCD_OK;
     default:
@@ -153,7 +154,8 @@ extern "C" lcd_status lcd_lut_linear(const void* packed_weights_dev, const void*
     case LCD_ALGO_BUCKET_LUT:
       return launch_lut_gemv(&p, 1, resolved, workspace, workspace_bytes, status_word_dev, cuda_stream);
     case LCD_ALGO_DENSE_TC:
-      return launch_dense_tc(p, workspace, workspace_bytes, status_word_dev, cuda_stream);
+    case LCD_ALGO_DENSE_F16:
+      return launch_dense_tc(p, resolved == LCD_ALGO_DENSE_F16, workspace, workspace_bytes, status_word_dev, cuda_stream);
     default:
       return LCD_ERR_INVALID_ARG;
   }

@@ -59,8 +59,8 @@ size_t lut_gemv_workspace_bytes(const Problem* probs, int count, lcd_algo algo);
 lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void* workspace, size_t workspace_bytes,
                            int32_t* status_word, void* stream);
 size_t dense_tc_workspace_bytes(int64_t M, int64_t K_pad);
-lcd_status launch_dense_tc(const Problem& p, void* workspace, size_t workspace_bytes, int32_t* status_word,
-                           void* stream);
+lcd_status launch_dense_tc(const Problem& p, bool fp16_operands, void* workspace, size_t workspace_bytes,
+                           int32_t* status_word, void* stream);
 
 }  // namespace lcd
 #endif

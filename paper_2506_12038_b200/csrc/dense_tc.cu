@@ -1,18 +1,19 @@
 // Batched-prefill path (many tokens): the layer is a dense contraction y[M x N] = diag(s_q) * Q[M x K] * Wd[N x K]^T,
 // where Wd[n][k] = cb[n][idx[n][k]] is what the lookup of Section 4.2 of the LCD paper returns and Q holds the
-// activation levels of Section 4.1.  Both are exact in fp16 (centroids are fp16, levels are integers -8..7), so
-// the tensor cores compute the same sums as the lookup-and-accumulate form, in fp32.
-//
-// Structure (one CTA per SM, persistent over output tiles of 128 weight rows x BN tokens):
-//   warp 0      TMA producer: activation tiles (fp16 levels, expanded once per call into the workspace, in the
-//               column order in which the decoder emits weights) -> shared memory, 128-byte swizzle
-//   warp 1      owns tensor memory; one lane issues tcgen05.mma (kind::f16, A and B from shared memory, fp32
-//               accumulators in tensor memory, two accumulator buffers so that the epilogue overlaps the next tile)
+// activation levels of Section 4.1.  Two kernels share one structure (one persistent CTA per SM, tiles of 128 weight
+// rows x BN tokens, every role a warp or a group of warps, mbarrier pipelines, accumulators in tensor memory):
+//   dense_i8_kernel  (LCD_ALGO_DENSE_TC, the default)  int8 byte-table planes x int8 levels, kind::i8, int32 sums
+//   dense_tc_kernel  (LCD_ALGO_DENSE_F16)              fp16 centroids x fp16 levels, kind::f16, fp32 sums
+// Roles of dense_tc_kernel:
+//   warp 0      TMA producer: token tiles (levels expanded once per call into the workspace, in the column order in
+//               which the decoder emits weights) -> shared memory, 128-byte swizzle
+//   warp 1      owns tensor memory; one lane issues tcgen05.mma (A and B from shared memory, two accumulator
+//               buffers so that the epilogue overlaps the next tile)
 //   warps 2-5   epilogue: tcgen05.ld, multiply by the token scale, coalesced fp32 stores
-//   warps 6-21  decoder (two groups of 8 warps on alternate stages): packed 2/3-bit indices -> PRMT lookups in the row's byte tables (low and high byte of
-//               the fp16 centroids) -> fp16 pairs -> K-major 128-byte-swizzled A tile in shared memory
-// Four pipeline stages of 64 columns; every wait is bounded (status word LCD_ERR_TIMEOUT on expiry, then every
-// role leaves its loop, pending copies and MMAs are drained and tensor memory is released).
+//   warps 6-21  decoder, two groups of 8 warps on alternate stages: packed 2/3-bit indices -> PRMT lookups in the
+//               row's byte tables -> K-major 128-byte-swizzled A tile in shared memory
+// Every wait is bounded (status word LCD_ERR_TIMEOUT on expiry, then every role leaves its loop, pending copies and
+// MMAs are drained and tensor memory is released).
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -390,293 +391,6 @@ dense_tc_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
 }
 
 // ---------------------------------------------------------------------------------------------------------
-// Variant for tiles of at most 192 tokens: the decoded A operand never touches shared memory.  The decoder
-// writes fp16 pairs straight from registers into tensor memory (tcgen05.st: a thread owns one row of the tile,
-// a warp the 32 tensor-memory lanes of its quadrant) and the MMA takes A from tensor memory.  Shared memory then
-// carries only the token tiles, which is what bounds the kernel above (see the profile of that kernel).
-// Tensor memory: two accumulators of BN columns, then four A stages of 32 columns (64 fp16 per row).
-// RT = 1: a CTA tile is 128 rows, two accumulator buffers.  RT = 2: 256 rows (two MMA row tiles share every token
-// tile, which halves the token bytes streamed from L2 per flop), one accumulator buffer.
-// Warps: 0 TMA, 1 MMA, 2-5 epilogue, 6-21 decoder = 16 / (4 RT) groups x RT row tiles x 4 quadrant warps; group i
-// decodes the stages whose number is i modulo the number of groups.
-__device__ __forceinline__ void mma_f16_ta(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
-      ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
-      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
-        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
-        "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
-        "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]) : "memory");
-}
-
-// Token-tile stages of the tensor-memory variant: as many as fit in about 200 KB, at most 8.
-__host__ __device__ constexpr int ta_b_stages(int bn) { return (200 * 1024) / (bn * kBK * 2) > 8 ? 8 : (200 * 1024) / (bn * kBK * 2); }
-
-template <int BITS, int BN, int RT>
-__global__ void __launch_bounds__(kDenseThreads, 1)
-dense_tc_ta_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams P) {
-  extern __shared__ uint8_t smem_raw[];
-  constexpr int ITEM = 512 * BITS, HALF = 256 * BITS;
-  constexpr int kBBytes = BN * kBK * 2;
-  constexpr uint32_t kTmemCols = 512;
-  constexpr int SB = ta_b_stages(BN);              // token-tile stages in shared memory (deep: they hide the L2 latency)
-  constexpr int NBUF = RT == 1 ? 2 : 1;            // accumulator buffers (RT * BN columns each)
-  constexpr int NG = kDecodeWarps / (4 * RT);      // decoder groups; a group decodes the stages == its index mod NG
-  constexpr uint32_t kACol0 = NBUF * RT * BN;      // first tensor-memory column of the A stages
-  static_assert(NBUF * RT * BN + kStages * RT * 32 <= 512, "tensor memory holds the accumulators and four A stages");
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-  const uint32_t raw_addr = (uint32_t)__cvta_generic_to_shared(smem_raw);
-  const uint32_t base = (raw_addr + 1023u) & ~1023u;
-  uint8_t* gen_base = smem_raw + (base - raw_addr);
-  const uint32_t b_base = base, bar_base = b_base + SB * kBBytes;
-  // barriers: A stages (tensor memory) full/empty, token-tile stages full/empty, accumulators, drain
-  auto full_a = [&](int s) { return bar_base + 8u * s; };
-  auto empty_a = [&](int s) { return bar_base + 8u * (kStages + s); };
-  auto full_b = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
-  auto empty_b = [&](int s) { return bar_base + 8u * (2 * kStages + SB + s); };
-  auto tmem_full = [&](int b) { return bar_base + 8u * (2 * kStages + 2 * SB + b); };
-  auto tmem_empty = [&](int b) { return bar_base + 8u * (2 * kStages + 2 * SB + 2 + b); };
-  const uint32_t drain_bar = bar_base + 8u * (2 * kStages + 2 * SB + 4);
-  uint8_t* gen_misc = gen_base + SB * kBBytes + 8 * (2 * kStages + 2 * SB + 5);
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(gen_misc);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_misc + 4);
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
-      bar_init(full_a(s), RT * 4 * 32);            // the quadrant warps of one decoder group
-      bar_init(empty_a(s), 1);
-    }
-    for (int s = 0; s < SB; ++s) {
-      bar_init(full_b(s), 1);
-      bar_init(empty_b(s), 1);
-    }
-    for (int b = 0; b < 2; ++b) {
-      bar_init(tmem_full(b), 1);
-      bar_init(tmem_empty(b), kEpiWarps * 32);
-    }
-    bar_init(drain_bar, 1);
-    *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"((uint32_t)__cvta_generic_to_shared(tmem_holder)), "r"(kTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tmem_base = *tmem_holder;
-
-  const int n_ks = P.n_kt * 4;     // stages per tile (a multiple of four: stage number mod 4 == stage of the item)
-
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      uint32_t it = 0;
-      bool ok = true;
-      asm volatile("griddepcontrol.wait;" ::: "memory");      // the levels come from the kernel launched before
-      for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x) {
-        const int m0 = (tile % P.n_tiles_m) * BN;
-        for (int ks = 0; ks < n_ks; ++ks, ++it) {
-          const int slot = it % SB;
-          if (!bar_wait(empty_b(slot), ((it / SB) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-          bar_expect_tx(full_b(slot), kBBytes);
-          asm volatile(
-              "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-              ::"r"(b_base + slot * kBBytes), "l"(&tmap_act), "r"(ks * kBK), "r"(m0), "r"(full_b(slot)) : "memory");
-        }
-      }
-      const uint32_t n_back = it < (uint32_t)SB ? it : (uint32_t)SB;
-      for (uint32_t i = 1; i <= n_back; ++i) {
-        const uint32_t j = it - i;
-        bar_drain(full_b(j % SB), (j / SB) & 1u);
-      }
-    }
-    __syncwarp();
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = instr_desc(BN);
-      const uint64_t b_desc0 = smem_desc(b_base);
-      uint32_t it = 0, tl = 0, bslot = 0, bphase = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, ++tl) {
-        const uint32_t buf = tl % NBUF;
-        if (!bar_wait(tmem_empty(buf), ((tl / NBUF) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t d_tmem = tmem_base + buf * (RT * BN);
-        for (int ks = 0; ks < n_ks; ++ks, ++it) {
-          const int slot = it % kStages;
-          if (!bar_wait(full_a(slot), (it / kStages) & 1u, abort_flag) ||
-              !bar_wait(full_b(bslot), bphase, abort_flag)) { ok = false; break; }
-          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          // one thread issues every MMA of the CTA: keep its instruction count per stage small
-          const uint64_t bd = b_desc0 + (uint64_t)((bslot * kBBytes) >> 4);
-          const uint32_t a_t = tmem_base + kACol0 + slot * (RT * 32);
-#pragma unroll
-          for (int i = 0; i < RT; ++i) {
-            mma_f16_ta(d_tmem + i * BN, a_t + i * 32, bd, idesc, (uint32_t)(ks != 0));
-#pragma unroll
-            for (int k = 1; k < kBK / 16; ++k) mma_f16_ta(d_tmem + i * BN, a_t + i * 32 + k * 8, bd + 2 * k, idesc, 1u);
-          }
-          mma_commit(empty_a(slot));               // frees the A stage in tensor memory
-          mma_commit(empty_b(bslot));              // and the token tile in shared memory
-          if (++bslot == (uint32_t)SB) { bslot = 0; bphase ^= 1u; }
-        }
-        if (ok) mma_commit(tmem_full(buf));
-      }
-      mma_commit(drain_bar);
-      bar_drain(drain_bar, 0);
-    }
-    __syncwarp();
-  } else if (warp < kFirstDecodeWarp) {
-    // ------------------------------------------------------------------ epilogue
-    const int quad = warp & 3;
-    uint32_t tl = 0;
-    bool ok = true;
-    for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, ++tl) {
-      const uint32_t buf = tl % NBUF;
-      const int m0 = (tile % P.n_tiles_m) * BN;
-      ok = __all_sync(0xffffffffu, bar_wait(tmem_full(buf), (tl / NBUF) & 1u, abort_flag));
-      if (!ok) break;
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll 1
-      for (int cc = 0; cc < RT * (BN / 32); ++cc) {
-        const int i = cc / (BN / 32), c = cc % (BN / 32);       // row tile, 32-token chunk
-        const int n = (tile / P.n_tiles_m) * (RT * kBM) + kBM * i + 32 * quad + lane;
-        uint32_t v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(32 * quad) << 16) + buf * (RT * BN) + i * BN + 32 * c, v);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        const int mc = m0 + 32 * c;
-        const float my_scale = mc + lane < P.M ? __ldg(P.act_scale + mc + lane) : 0.0f;
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float s = __shfl_sync(0xffffffffu, my_scale, j);
-          if (mc + j < P.M && n < P.N) P.y[(size_t)(mc + j) * P.ldy + n] = __uint_as_float(v[j]) * s;
-        }
-      }
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      bar_arrive(tmem_empty(buf));
-    }
-  } else {
-    // ------------------------------------------------------------------ decoder
-    const int dwi = warp - kFirstDecodeWarp;
-    const int grp = dwi / (4 * RT);                     // decodes the stages whose number is grp modulo NG
-    const int rt = (dwi >> 2) % RT;                     // row tile of 128 rows inside the CTA's tile
-    const int quad = warp & 3;                          // tensor-memory lanes [32*quad, +32) = rows of the row tile
-    const int r = 32 * quad + lane;                     // row inside the row tile
-    const int u = (r >> 3) & 1, g = r & 7;
-    uint32_t it0 = 0;
-    bool ok = true;
-    for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, it0 += (uint32_t)n_ks) {
-      int rp = (tile / P.n_tiles_m) * (RT * kBM / 16) + rt * (kBM / 16) + (r >> 4);
-      rp = rp < P.n_rp ? rp : P.n_rp - 1;          // rows past the matrix repeat the last group; never stored
-      uint32_t TL[2], TH[2];
-      {
-        const uint16_t* cb = P.codebook + ((size_t)rp * 16 + 8 * u + g) * (1 << BITS);
-        if (BITS == 2) {
-          const uint2 c = __ldg(reinterpret_cast<const uint2*>(cb));
-          TL[0] = TL[1] = prmt_b(c.x, c.y, 0x6420u);
-          TH[0] = TH[1] = prmt_b(c.x, c.y, 0x7531u);
-        } else {
-          const uint4 c = __ldg(reinterpret_cast<const uint4*>(cb));
-          TL[0] = prmt_b(c.x, c.y, 0x6420u); TH[0] = prmt_b(c.x, c.y, 0x7531u);
-          TL[1] = prmt_b(c.z, c.w, 0x6420u); TH[1] = prmt_b(c.z, c.w, 0x7531u);
-        }
-      }
-      // this thread's 64 columns of one item: quarters t0 and t0 + 1 of k-block h -> [quarter][word]
-      const uint8_t* row_items = P.items + (size_t)rp * P.n_kt * ITEM + u * HALF;
-      constexpr int SPI = 4 / NG;                  // stages of one item this group decodes
-      uint32_t cur[SPI][2][BITS == 2 ? 2 : 3], nxt[SPI][2][BITS == 2 ? 2 : 3];
-      auto load_stage = [&](uint32_t (&dst)[2][BITS == 2 ? 2 : 3], int kt, int j) {
-        const int h = j >> 1, t0 = 2 * (j & 1);    // k-block and first quarter of stage j of an item
-        const uint8_t* item = row_items + (size_t)kt * ITEM;
-#pragma unroll
-        for (int x = 0; x < 2; ++x) {
-          const int l = 4 * g + t0 + x;
-          if (BITS == 2) {
-            const uint2 w = __ldg(reinterpret_cast<const uint2*>(item + 16 * l + 8 * h));
-            dst[x][0] = w.x; dst[x][1] = w.y;
-          } else {
-#pragma unroll
-            for (int b = 0; b < 3; ++b) dst[x][b] = __ldg(reinterpret_cast<const uint32_t*>(item + 256 * b + 8 * l + 4 * h));
-          }
-        }
-      };
-#pragma unroll
-      for (int jj = 0; jj < SPI; ++jj) load_stage(cur[jj], 0, grp + NG * jj);
-      for (int kt = 0; kt < P.n_kt && ok; ++kt) {
-        if (kt + 1 < P.n_kt) {
-#pragma unroll
-          for (int jj = 0; jj < SPI; ++jj) load_stage(nxt[jj], kt + 1, grp + NG * jj);
-        }
-#pragma unroll
-       for (int jj = 0; jj < SPI; ++jj) {
-        if (!ok) break;
-        const uint32_t it = it0 + 4u * (uint32_t)kt + (uint32_t)(grp + NG * jj);
-        const int slot = it % kStages;
-        uint32_t v[32];     // the row's 64 fp16 of this stage, two per tensor-memory column
-#pragma unroll
-        for (int x = 0; x < 2; ++x) {
-          uint32_t sel[8];
-          if (BITS == 2) {
-#pragma unroll
-            for (int wd = 0; wd < 2; ++wd) {
-              const uint32_t raw = cur[jj][x][wd];
-              const uint32_t s0 = raw & 0x33333333u, s1 = (raw >> 2) & 0x33333333u;
-              sel[4 * wd] = s0; sel[4 * wd + 1] = s0 >> 16; sel[4 * wd + 2] = s1; sel[4 * wd + 3] = s1 >> 16;
-            }
-          } else {
-            const uint32_t r0 = cur[jj][x][0], r1 = cur[jj][x][1], r2 = cur[jj][x][2];
-            const uint32_t ex = (((r0 >> 3) & 0x11111111u) | ((r1 >> 2) & 0x22222222u)) | ((r2 >> 1) & 0x44444444u);
-            const uint32_t d0 = r0 & 0x77777777u, d1 = r1 & 0x77777777u, d2 = r2 & 0x77777777u;
-            sel[0] = d0; sel[1] = d0 >> 16; sel[2] = d1; sel[3] = d1 >> 16;
-            sel[4] = d2; sel[5] = d2 >> 16; sel[6] = ex; sel[7] = ex >> 16;
-          }
-#pragma unroll
-          for (int L = 0; L < 8; ++L) {
-            const uint32_t lo = prmt_b(TL[0], TL[1], sel[L]), hi = prmt_b(TH[0], TH[1], sel[L]);
-            v[16 * x + 2 * L] = prmt_b(lo, hi, 0x5140u);
-            v[16 * x + 2 * L + 1] = prmt_b(lo, hi, 0x7362u);
-          }
-        }
-        if (!bar_wait(empty_a(slot), ((it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; }
-        ok = __all_sync(0xffffffffu, ok);          // tcgen05.st is a warp-wide instruction
-        if (!ok) continue;
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        tmem_st32(tmem_base + ((uint32_t)(32 * quad) << 16) + kACol0 + (slot * RT + rt) * 32, v);
-        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        bar_arrive(full_a(slot));
-       }
-#pragma unroll
-        for (int jj = 0; jj < SPI; ++jj)
-#pragma unroll
-          for (int x = 0; x < 2; ++x)
-#pragma unroll
-            for (int b = 0; b < (BITS == 2 ? 2 : 3); ++b) cur[jj][x][b] = nxt[jj][x][b];
-      }
-    }
-  }
-
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
-  if (warp == 1) {
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
-  }
-  if (threadIdx.x == 0 && *abort_flag && P.status) atomicExch(P.status, (int)LCD_ERR_TIMEOUT);
-}
-
-// ---------------------------------------------------------------------------------------------------------
 // Integer variant (the default for many tokens).  The row codebook becomes the same two byte tables as in the
 // M <= 16 kernel (16-bit fixed point: signed high byte, unsigned low byte), the decoder emits two int8 A planes
 // with ONE lookup per plane and four weights (no fp16 interleave), the levels are int8, and every stage of 128
@@ -1034,8 +748,7 @@ int dense_sm_count() {
   return cached;
 }
 
-// KERNEL 0: A through shared memory (dense_tc_kernel); 1: A through tensor memory with RT row tiles per CTA.
-template <int BITS, int BN, int RT, int KERNEL>
+template <int BITS, int BN>
 lcd_status launch_dense_t(const Problem& p, __half* levels, int32_t* status_word, cudaStream_t stream) {
   EncodeTiledFn enc = encode_tiled();
   if (!enc) return LCD_ERR_CUDA;
@@ -1058,13 +771,10 @@ lcd_status launch_dense_t(const Problem& p, __half* levels, int32_t* status_word
   dp.n_rp = (int)(p.N_pad / kPairRows);
   dp.n_kt = (int)(p.K_pad / kTileK);
   dp.n_tiles_m = (int)((p.M + BN - 1) / BN);
-  dp.n_tiles = dp.n_tiles_m * (int)((p.N_pad + RT * kBM - 1) / (RT * kBM));
+  dp.n_tiles = dp.n_tiles_m * (int)((p.N_pad + kBM - 1) / kBM);
   dp.status = status_word;
-  const size_t smem = KERNEL == 0 ? 1024 + (size_t)kStages * (kABytes + BN * kBK * 2) + 256
-                                  : 1024 + (size_t)ta_b_stages(BN) * (BN * kBK * 2) + 512;
-  void (*kern)(const CUtensorMap, const DenseParams);
-  if (KERNEL == 0) kern = dense_tc_kernel<BITS, BN>;
-  else kern = dense_tc_ta_kernel<BITS, (KERNEL == 0 ? 128 : BN), RT>;
+  const size_t smem = 1024 + (size_t)kStages * (kABytes + BN * kBK * 2) + 256;
+  auto kern = dense_tc_kernel<BITS, BN>;
   static bool attr_set = false;   // per template instance
   if (!attr_set) {
     const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -1136,21 +846,19 @@ lcd_status launch_dense_i8(const Problem& p, int8_t* levels, int32_t* status_wor
   return LCD_OK;
 }
 
-// Tile shapes: {kernel (0 fp16 / A in shared memory, 1 fp16 / A in tensor memory, 2 int8 planes), row tiles,
-// tokens, cycles per 64 columns of a tile, cycles per tile that do not overlap (epilogue of the shapes with one
-// accumulator buffer)}.  The numbers are measured on the LLaMA-13B shapes (1.7 GHz under load); the launcher takes
-// the shape with the smallest waves x (columns x stage + fixed).
-struct TileShape { int kernel, rt, bn, stage_clks, epilogue_clks; };
-constexpr TileShape kShapes[6] = {{1, 1, 192, 664, 0}, {1, 1, 128, 443, 0}, {0, 1, 256, 733, 0},
-                                  {2, 1, 128, 425, 0}, {2, 1, 192, 400, 19900}, {2, 1, 256, 535, 19000}};
+// Tile widths of the int8 kernel: {tokens, cycles per 64 columns of a tile, cycles per tile that do not overlap
+// (the epilogue of the widths with one accumulator buffer)}, measured on the LLaMA-13B shapes at about 1.7 GHz.
+// The launcher takes the width with the smallest waves x (columns x stage + fixed).
+struct TileShape { int bn, stage_clks, epilogue_clks; };
+constexpr TileShape kShapes[3] = {{128, 425, 0}, {192, 400, 13000}, {256, 535, 13000}};
 
 int pick_shape(int64_t M, int64_t N_pad, int64_t n_ks) {
   const int n_sm = dense_sm_count();
   int best = 0;
   int64_t best_cost = -1;
-  for (int i = 0; i < 6; ++i) {
+  for (int i = 0; i < 3; ++i) {
     const TileShape& t = kShapes[i];
-    const int64_t tiles = ((N_pad + t.rt * kBM - 1) / (t.rt * kBM)) * ((M + t.bn - 1) / t.bn);
+    const int64_t tiles = ((N_pad + kBM - 1) / kBM) * ((M + t.bn - 1) / t.bn);
     const int64_t cost = ((tiles + n_sm - 1) / n_sm) * (n_ks * t.stage_clks + t.epilogue_clks);
     if (best_cost < 0 || cost < best_cost) { best = i; best_cost = cost; }
   }
@@ -1161,21 +869,20 @@ int pick_shape(int64_t M, int64_t N_pad, int64_t n_ks) {
 
 size_t dense_tc_workspace_bytes(int64_t M, int64_t K_pad) { return (size_t)round_up_u64((uint64_t)M * K_pad * 2, 256); }
 
-lcd_status launch_dense_tc(const Problem& p, void* workspace, size_t workspace_bytes, int32_t* status_word,
-                           void* stream) {
+lcd_status launch_dense_tc(const Problem& p, bool fp16_operands, void* workspace, size_t workspace_bytes,
+                           int32_t* status_word, void* stream) {
   if (!workspace || workspace_bytes < dense_tc_workspace_bytes(p.M, p.K_pad)) return LCD_ERR_BUFFER_TOO_SMALL;
   if (p.M > 0x7fffffffLL / 2 || p.N > 0x7fffffffLL / 2) return LCD_ERR_UNSUPPORTED;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int64_t n_quarters = p.M * (p.K_pad / 32);
   const unsigned blocks = (unsigned)((n_quarters + 255) / 256);
-  const int shape = pick_shape(p.M, p.N_pad, p.K_pad / kBK);
-  if (kShapes[shape].kernel == 2) {
+  if (!fp16_operands) {
     int8_t* levels = static_cast<int8_t*>(workspace);
     if (p.bits == 2) expand_levels_i8_kernel<2><<<blocks, 256, 0, s>>>(p.act_idx, n_quarters, levels);
     else expand_levels_i8_kernel<3><<<blocks, 256, 0, s>>>(p.act_idx, n_quarters, levels);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
-    const int bn = kShapes[shape].bn;
+    const int bn = kShapes[pick_shape(p.M, p.N_pad, p.K_pad / kBK)].bn;
     if (p.bits == 2) return bn == 128 ? launch_dense_i8<2, 128>(p, levels, status_word, s)
                           : bn == 192 ? launch_dense_i8<2, 192>(p, levels, status_word, s)
                                       : launch_dense_i8<2, 256>(p, levels, status_word, s);
@@ -1186,14 +893,15 @@ lcd_status launch_dense_tc(const Problem& p, void* workspace, size_t workspace_b
   __half* levels = static_cast<__half*>(workspace);
   if (p.bits == 2) expand_levels_kernel<2><<<blocks, 256, 0, s>>>(p.act_idx, n_quarters, levels);
   else expand_levels_kernel<3><<<blocks, 256, 0, s>>>(p.act_idx, n_quarters, levels);
-  cudaError_t e = cudaGetLastError();
+  const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
-#define LCD_DENSE_CASE(B, I, W, R, KN) \
-  if (p.bits == B && shape == I) return launch_dense_t<B, W, R, KN>(p, levels, status_word, s);
-  LCD_DENSE_CASE(2, 0, 192, 1, 1) LCD_DENSE_CASE(2, 1, 128, 1, 1) LCD_DENSE_CASE(2, 2, 256, 1, 0)
-  LCD_DENSE_CASE(3, 0, 192, 1, 1) LCD_DENSE_CASE(3, 1, 128, 1, 1) LCD_DENSE_CASE(3, 2, 256, 1, 0)
-#undef LCD_DENSE_CASE
-  return LCD_ERR_UNSUPPORTED;
+  // 256-token tiles unless 128-token tiles need fewer waves per token
+  const int n_sm = dense_sm_count();
+  const int64_t tiles_n = (p.N_pad + kBM - 1) / kBM;
+  const int64_t w256 = (tiles_n * ((p.M + 255) / 256) + n_sm - 1) / n_sm, w128 = (tiles_n * ((p.M + 127) / 128) + n_sm - 1) / n_sm;
+  const bool wide = 2 * w256 <= w128;
+  if (p.bits == 2) return wide ? launch_dense_t<2, 256>(p, levels, status_word, s) : launch_dense_t<2, 128>(p, levels, status_word, s);
+  return wide ? launch_dense_t<3, 256>(p, levels, status_word, s) : launch_dense_t<3, 128>(p, levels, status_word, s);
 }
 
 }  // namespace lcd

@@ -140,26 +140,26 @@ def test_grouped_launch_matches_oracle_and_leaves_scratch_zero():
 @pytest.mark.parametrize("bits", [2, 3])
 @pytest.mark.parametrize("N,K,M", [(128, 256, 32), (200, 1000, 17), (1031, 520, 40), (64, 4096, 100), (520, 2304, 256),
                                    (272, 768, 300), (1024, 1024, 513),
-                                   (2560, 512, 2048),      # 192-token tiles (two waves instead of three)
-                                   (9472, 256, 512),       # 256-token tiles (one wave)
+                                   (2560, 512, 2048), (9472, 256, 512),
                                    (4608, 1024, 1024),
                                    (4600, 1024, 1000)])    # ragged rows and tokens
-def test_dense_tensor_core_path_matches_oracle(bits, N, K, M):
-    # fp16 centroids x integer levels on the tensor cores, fp32 accumulation: exact products, so only the order
-    # of the fp32 sums differs from the oracle
+@pytest.mark.parametrize("algo", ["int8", "fp16"])
+def test_dense_tensor_core_path_matches_oracle(bits, N, K, M, algo):
+    # int8: 16-bit fixed-point byte tables x integer levels, exact int32 sums (the default above 16 tokens);
+    # fp16: fp16 centroids x integer levels, fp32 accumulation, only the order of the sums differs from the oracle
+    algo = lcd.ALGO_DENSE_TC if algo == "int8" else lcd.ALGO_DENSE_F16
     L = gen.random_case(seed=N + K + M + bits, N=N, K=K, bits=bits, M=M)
     word = torch.zeros((1,), dtype=torch.int32, device="cuda")
     w = lcd.PackedWeights(lcd.pack_weights(L.idx, L.codebook, L.bits, L.C))
     a, s = lcd.smooth_quantize_act(torch.from_numpy(L.x).cuda(), torch.from_numpy(L.inv_s).cuda())
     y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
-    lcd.lut_linear(w, a, s, y=y, algo=lcd.ALGO_DENSE_TC, status_word=word)
+    lcd.lut_linear(w, a, s, y=y, algo=algo, status_word=word)
     torch.cuda.synchronize()
     assert int(word.item()) == 0
     q_ref, s_ref = O.smooth_quantize(L.x, L.inv_s)
     check_y(y, O.lut_linear_dequant(L.idx, L.codebook, q_ref, s_ref))
-    # the default choice above 16 tokens is this path
-    y2 = lcd.lut_linear(w, a, s)
-    assert torch.equal(y2, y)
+    if algo == lcd.ALGO_DENSE_TC:      # the default choice above 16 tokens is this path
+        assert torch.equal(lcd.lut_linear(w, a, s), y)
 
 
 def test_status_word_untouched_on_success():
