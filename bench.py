@@ -36,10 +36,10 @@ NCU_TRAFFIC = {
     # profiles/lut_gemv_kernel_llama7b_2bit_m1.md: one grouped launch of configs[1] at M = 1
     ("lut_gemv.cu", 1, 1): {"sha256": "2813124b355499c0d7b9727ec884ce3d565f27dae85537db426cbf394fbf5d03", "bytes_per_launch": 50989056 + 26880},
     # profiles/dense_tc_kernel_llama13b_2bit_m2048.md: the layer's seven launches of configs[3]: q captured
-    # (27.61 + 2.15 MB, taken four times for q/k/v/o), gate captured (39.22 + 62.68 MB, twice for gate/up), down
+    # (17.11 + 0.23 MB, taken four times for q/k/v/o), gate captured (28.36 + 56.16 MB, twice for gate/up), down
     # scaled from q by its 2.7 times longer rows (same tiles, traffic in proportion to K)
-    ("dense_tc.cu", 3, 2048): {"sha256": "2c9d2410e0eda5b2f6b9dc3d2f6095c2d9a93c9cf3ead495f3685c450933633d",
-                               "bytes_per_launch": int(4 * 29.76e6 + 2 * 101.9e6 + 29.76e6 * 13824 / 5120)},
+    ("dense_tc.cu", 3, 2048): {"sha256": "edefd6132d93e9c889e32fe8be8fc1b7954a843f088f3bc771d89f17959f4a13",
+                               "bytes_per_launch": int(4 * 17.34e6 + 2 * 84.52e6 + 17.34e6 * 13824 / 5120)},
 }
 L2_BYTES = 126e6
 ROTATE_BYTES = 300e6          # total size of the weight copies the timed loop rotates over
