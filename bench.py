@@ -54,6 +54,8 @@ def parse_args():
     ap.add_argument("--M", type=int, default=None, help="token count (default: first M of the config)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--algo", default="auto", choices=["auto", "register", "bucket", "tensor"],
+                    help="lookup kernel for M <= 16 (default: the library's choice)")
     return ap.parse_args()
 
 
@@ -239,12 +241,18 @@ def run_ours(args):
                          bytes=algorithmic_bytes(L.N, L.K, bits, M), flop=2.0 * M * L.N * L.K))
 
     grouped = M <= 16 and len(mats) <= lcd.MAX_BATCH
+    algo = {"auto": lcd.ALGO_AUTO, "register": lcd.ALGO_REGISTER_LUT, "bucket": lcd.ALGO_BUCKET_LUT,
+            "tensor": lcd.ALGO_TC_LUT}[args.algo]
+    # every kernel that can give up on a bounded wait reports it here; a non-zero word voids the run
+    status = torch.zeros((1,), dtype=torch.int32, device=dev)
     if grouped:
         # one launch quantises every matrix's tokens, one launch runs every matrix's lookup: the inputs are
         # independent, so the whole layer is a single grouped problem
         qbatch = lcd.ActBatch([(mt["x"], mt["inv_s"], mt["a"], mt["s"]) for mt in mats])
-        lbatch = [lcd.LinearBatch([(mt["w"][c], mt["a"], mt["s"], mt["y"]) for mt in mats]) for c in range(copies)]
-        single = [[lcd.LinearBatch([(mt["w"][c], mt["a"], mt["s"], mt["y"])]) for c in range(copies)] for mt in mats]
+        lbatch = [lcd.LinearBatch([(mt["w"][c], mt["a"], mt["s"], mt["y"]) for mt in mats], algo=algo, status_word=status)
+                  for c in range(copies)]
+        single = [[lcd.LinearBatch([(mt["w"][c], mt["a"], mt["s"], mt["y"])], algo=algo, status_word=status)
+                   for c in range(copies)] for mt in mats]
 
         def step(c):
             qbatch.run()
@@ -256,11 +264,11 @@ def run_ours(args):
         def step(c):
             for mt in mats:
                 lcd.smooth_quantize_act(mt["x"], mt["inv_s"], act_idx=mt["a"], act_scale=mt["s"])
-                lcd.lut_linear(mt["w"][c], mt["a"], mt["s"], y=mt["y"], workspace=mt["work"])
+                lcd.lut_linear(mt["w"][c], mt["a"], mt["s"], y=mt["y"], workspace=mt["work"], status_word=status)
 
         def lookup_only(mi, c):
             mt = mats[mi]
-            lcd.lut_linear(mt["w"][c], mt["a"], mt["s"], y=mt["y"], workspace=mt["work"])
+            lcd.lut_linear(mt["w"][c], mt["a"], mt["s"], y=mt["y"], workspace=mt["work"], status_word=status)
 
     launches_per_step = 2 if grouped else 2 * len(mats)
     stream = torch.cuda.Stream(device=dev)
@@ -399,6 +407,9 @@ def run_ours(args):
         with open(os.path.join(ROOT, "paper_2506_12038_b200", "csrc", src), "rb") as fh:
             if hashlib.sha256(fh.read()).hexdigest() == rec["sha256"]:
                 roof["traffic"] = rec["bytes_per_launch"]
+    torch.cuda.synchronize()
+    if int(status.item()) != 0:
+        raise RuntimeError(f"a kernel reported status {int(status.item())} (bounded wait expired): timings are void")
     roof["kernel"] = kern_name
     roof["us_per_launch"] = kern_ms * 1e3
     roof["per_matrix"] = per_matrix

@@ -53,8 +53,10 @@ typedef enum {
   LCD_ALGO_DENSE_TC = 4,    /* batched prefill on tcgen05 tensor cores: the byte tables of REGISTER_LUT decode   */
                             /* the indices into two int8 planes in shared memory, int8 levels arrive by TMA,     */
                             /* kind::i8 MMAs accumulate exact int32 sums in tensor memory.                      */
-  LCD_ALGO_DENSE_F16 = 5    /* the same with fp16 operands: indices decoded through the codebook into fp16     */
+  LCD_ALGO_DENSE_F16 = 5,   /* the same with fp16 operands: indices decoded through the codebook into fp16     */
                             /* shared-memory tiles, fp32 accumulators (no fixed-point step; slower).            */
+  LCD_ALGO_TC_LUT = 6       /* REGISTER_LUT's tables and sums, the looked-up bytes written to tensor memory as  */
+                            /* the A operand of tcgen05 kind::i8 MMAs over a 16-token tile.  M <= 16.            */
 } lcd_algo;
 
 #define LCD_HEADER_BYTES 64

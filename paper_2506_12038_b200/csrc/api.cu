@@ -69,6 +69,7 @@ static lcd_status workspace_for(const Problem& p, lcd_algo algo, size_t* bytes) 
       return LCD_OK;
     case LCD_ALGO_REGISTER_LUT:
     case LCD_ALGO_BUCKET_LUT:
+    case LCD_ALGO_TC_LUT:
       if (p.M > 16) return LCD_ERR_UNSUPPORTED;
       *bytes = lut_gemv_workspace_bytes(&p, 1, resolve_algo(p.M, algo));
       return LCD_OK;
@@ -152,6 +153,7 @@ extern "C" lcd_status lcd_lut_linear(const void* packed_weights_dev, const void*
       return launch_reference(p, cuda_stream);
     case LCD_ALGO_REGISTER_LUT:
     case LCD_ALGO_BUCKET_LUT:
+    case LCD_ALGO_TC_LUT:
       return launch_lut_gemv(&p, 1, resolved, workspace, workspace_bytes, status_word_dev, cuda_stream);
     case LCD_ALGO_DENSE_TC:
     case LCD_ALGO_DENSE_F16:
@@ -163,7 +165,8 @@ extern "C" lcd_status lcd_lut_linear(const void* packed_weights_dev, const void*
 
 static lcd_status batch_algo(const lcd_linear_problem* problems, int count, lcd_algo algo, lcd_algo* resolved) {
   if (!problems || count < 1 || count > LCD_MAX_BATCH) return LCD_ERR_INVALID_ARG;
-  if (algo != LCD_ALGO_AUTO && algo != LCD_ALGO_REGISTER_LUT && algo != LCD_ALGO_BUCKET_LUT) return LCD_ERR_UNSUPPORTED;
+  if (algo != LCD_ALGO_AUTO && algo != LCD_ALGO_REGISTER_LUT && algo != LCD_ALGO_BUCKET_LUT && algo != LCD_ALGO_TC_LUT)
+    return LCD_ERR_UNSUPPORTED;
   for (int i = 0; i < count; ++i)
     if (problems[i].M < 1 || problems[i].M > 16) return problems[i].M < 1 ? LCD_ERR_INVALID_ARG : LCD_ERR_UNSUPPORTED;
   *resolved = algo == LCD_ALGO_AUTO ? LCD_ALGO_REGISTER_LUT : algo;

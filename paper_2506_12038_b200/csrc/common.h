@@ -58,6 +58,10 @@ lcd_status launch_smooth_quantize_batch(const lcd_act_problem* probs, int count,
 size_t lut_gemv_workspace_bytes(const Problem* probs, int count, lcd_algo algo);
 lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void* workspace, size_t workspace_bytes,
                            int32_t* status_word, void* stream);
+// LCD_ALGO_TC_LUT: the same arithmetic for up to 16 tokens with the looked-up bytes fed to tcgen05.mma kind::i8
+size_t lut_gemv_tc_workspace_bytes(const Problem* probs, int count);
+lcd_status launch_lut_gemv_tc(const Problem* probs, int count, void* workspace, size_t workspace_bytes,
+                              int32_t* status_word, void* stream);
 size_t dense_tc_workspace_bytes(int64_t M, int64_t K_pad);
 lcd_status launch_dense_tc(const Problem& p, bool fp16_operands, void* workspace, size_t workspace_bytes,
                            int32_t* status_word, void* stream);

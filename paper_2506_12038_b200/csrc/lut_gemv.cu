@@ -735,6 +735,7 @@ lcd_status launch_t(const GemvBatch& batch, int grid, size_t smem, int32_t* stat
 }  // namespace
 
 size_t lut_gemv_workspace_bytes(const Problem* probs, int count, lcd_algo algo) {
+  if (algo == LCD_ALGO_TC_LUT) return lut_gemv_tc_workspace_bytes(probs, count);
   const int kind = algo == LCD_ALGO_BUCKET_LUT ? kBuckets : kFixed16;
   int64_t max_m = 1;
   for (int i = 0; i < count; ++i) max_m = probs[i].M > max_m ? probs[i].M : max_m;
@@ -748,6 +749,7 @@ size_t lut_gemv_workspace_bytes(const Problem* probs, int count, lcd_algo algo) 
 lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void* workspace, size_t workspace_bytes,
                            int32_t* status_word, void* stream) {
   if (count < 1 || count > LCD_MAX_BATCH) return LCD_ERR_INVALID_ARG;
+  if (algo == LCD_ALGO_TC_LUT) return launch_lut_gemv_tc(probs, count, workspace, workspace_bytes, status_word, stream);
   const int kind = algo == LCD_ALGO_BUCKET_LUT ? kBuckets : kFixed16;
   const int bits = probs[0].bits;
   int64_t max_m = 1;

@@ -110,7 +110,30 @@ def test_lookup_with_column_panels(bits, N, K, M):
     run_case(L, lcd.ALGO_REGISTER_LUT)
 
 
-def test_grouped_launch_matches_oracle_and_leaves_scratch_zero():
+@pytest.mark.parametrize("bits", [2, 3])
+@pytest.mark.parametrize("N,K", SHAPES + [(4096, 4096), (300, 28672)])
+@pytest.mark.parametrize("M", [1, 3, 8, 16])
+def test_tensor_core_lut_matches_oracle(bits, N, K, M):
+    # the register-LUT tables and exact integer sums, looked-up bytes fed to tcgen05 kind::i8 through tensor memory;
+    # row tiles whose columns are split over CTAs are finished through the integer scratch, which is left zero
+    L = gen.random_case(seed=N + K + M + bits, N=N, K=K, bits=bits, M=M)
+    w = lcd.PackedWeights(lcd.pack_weights(L.idx, L.codebook, L.bits, L.C))
+    a, s = lcd.smooth_quantize_act(torch.from_numpy(L.x).cuda(), torch.from_numpy(L.inv_s).cuda())
+    word = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    ws = torch.zeros((lcd.lut_linear_workspace_bytes(w, M, lcd.ALGO_TC_LUT),), dtype=torch.uint8, device="cuda")
+    y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    for _ in range(2):
+        lcd.lut_linear(w, a, s, y=y, algo=lcd.ALGO_TC_LUT, workspace=ws, status_word=word)
+    torch.cuda.synchronize()
+    assert int(word.item()) == 0
+    assert not ws.any()
+    q_ref, s_ref = O.smooth_quantize(L.x, L.inv_s)
+    check_y(y, O.lut_linear_dequant(L.idx, L.codebook, q_ref, s_ref))
+
+
+@pytest.mark.parametrize("algo", ["register", "tensor"])
+def test_grouped_launch_matches_oracle_and_leaves_scratch_zero(algo):
+    algo = lcd.ALGO_REGISTER_LUT if algo == "register" else lcd.ALGO_TC_LUT
     shapes = [(2, 200, 1000, 1), (2, 4096, 512, 3), (2, 24, 11008, 5), (2, 1031, 520, 1), (2, 8, 256, 8)]
     for bits in (2, 3):
         cases = [gen.random_case(seed=31 * i + bits, N=N, K=K, bits=bits, M=M) for i, (_, N, K, M) in enumerate(shapes)]
@@ -125,7 +148,7 @@ def test_grouped_launch_matches_oracle_and_leaves_scratch_zero():
             items.append((w, a, sc, y))
             q_ref, s_ref = O.smooth_quantize(L.x, L.inv_s)
             refs.append((q_ref, s_ref, O.lut_linear_dequant(L.idx, L.codebook, q_ref, s_ref)))
-        qb, lb = lcd.ActBatch(acts), lcd.LinearBatch(items)
+        qb, lb = lcd.ActBatch(acts), lcd.LinearBatch(items, algo=algo)
         for _ in range(3):          # repeated calls reuse the scratch the previous call left
             qb.run()
             lb.run()
