@@ -12,10 +12,10 @@
 // zero-filled global scratch, the last arrival (ticket) writes y and leaves zeros.  Integer accumulation is order
 // free, so several threads issue MMAs into one accumulator that the epilogue zero-fills after every use.
 //
-// Warps: 0-1 token producers (4-bit levels -> int8 in lookup order -> swizzled shared-memory tile), 2-7 MMA issuers
-// (one per stage slot), 8-11 epilogue (tensor-memory quadrant each), 12-27 decoders = 4 groups (unit number mod 4) x
-// 4 quadrant warps; a decoder thread owns one row, its warp streams its 32 rows' items through a private
-// shared-memory ring filled by cp.async.bulk.  Every wait is bounded; on expiry the status word is set and all roles
+// Warps: 0-5 MMA issuers (one per stage slot), 6-9 epilogue (tensor-memory quadrant each), 10-25 decoders = 4 groups
+// (unit number mod 4) x 4 quadrant warps; a decoder thread owns one row, its warp streams its 32 rows' items through
+// a private shared-memory ring filled by cp.async.bulk, and the 128 threads of a group also stage the stage's
+// 16 x 128 token levels (4-bit -> int8 in lookup order -> swizzled shared-memory tile, one 16-byte chunk each).  Every wait is bounded; on expiry the status word is set and all roles
 // leave their loops, drain what they issued and release tensor memory.
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -29,12 +29,11 @@ namespace {
 constexpr int kTcTokens = 16;                 // MMA N: tokens per tile (rows past M are zero)
 constexpr int kTcRows = 128;                  // MMA M: weight rows per tile
 constexpr int kTcSlots = 6;                   // pipeline stages (128 columns each): A in tensor memory, B in smem
-constexpr int kTcProducers = 2, kTcIssuers = kTcSlots, kTcEpi = 4, kTcDecoders = 16;
-constexpr int kTcFirstIssuer = kTcProducers, kTcFirstEpi = kTcFirstIssuer + kTcIssuers;
+constexpr int kTcIssuers = kTcSlots, kTcEpi = 4, kTcDecoders = 16;
+constexpr int kTcFirstIssuer = 0, kTcFirstEpi = kTcFirstIssuer + kTcIssuers;
 constexpr int kTcFirstDecoder = kTcFirstEpi + kTcEpi;
-constexpr int kTcThreads = 32 * (kTcFirstDecoder + kTcDecoders);     // 896
+constexpr int kTcThreads = 32 * (kTcFirstDecoder + kTcDecoders);     // 832
 constexpr int kTcRing = 3;                    // ring slots per decoder warp (one 256-column unit of its 32 rows each)
-constexpr int kTcAhead = 4;                   // units whose levels a producer holds in registers ahead of use
 constexpr int kTcBBytes = kTcTokens * 128;    // 2 KB: 16 tokens x 128 int8
 constexpr uint32_t kTcACols = 64;             // tensor-memory columns of one A stage: 32 high plane + 32 low plane
 constexpr uint32_t kTcAccCol0 = kTcSlots * kTcACols;   // accumulators: 2 buffers x (16 high + 16 low) columns
@@ -75,18 +74,18 @@ __device__ __forceinline__ bool tc_try(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait.  After a few immediate retries the thread sleeps between polls, so that the many waiting threads of
-// a CTA (epilogue, issuers, producers) leave the issue slots to the decoders.
+// Bounded wait.  SLEEP: the thread sleeps between polls (roles that wait long and are not on the critical path: the
+// epilogue), so that it leaves the issue slots to the others; otherwise it polls back to back, because the wake-up
+// delay of a sleeping thread would be added to every hand-over of a pipeline stage.
+template <bool SLEEP = false>
 __device__ __forceinline__ bool tc_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-#pragma unroll 1
-  for (int i = 0; i < 4; ++i)
-    if (tc_try(bar, parity)) return true;
+  if (tc_try(bar, parity)) return true;
   const unsigned long long t0 = tc_timer();
 #pragma unroll 1
   for (uint32_t it = 1;; ++it) {
-    __nanosleep(40);
+    if (SLEEP) __nanosleep(200);
     if (tc_try(bar, parity)) return true;
-    if ((it & 63u) == 0) {
+    if ((it & (SLEEP ? 63u : 1023u)) == 0) {
       if (*abort_flag) return false;
       if (tc_timer() - t0 > kTcWaitNs) { *abort_flag = 1; return false; }
     }
@@ -114,6 +113,13 @@ __device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t (&v)[8]) {
                ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
                : "memory");
 }
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "memory");
+}
 __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
@@ -138,23 +144,30 @@ __device__ __forceinline__ uint64_t tc_smem_desc(uint32_t addr) {
 struct Walk {
   uint32_t u;      // global unit number
   int p, rt, kt;
+  int n_kt, n_rt;  // of problem p (kept here: indexing the kernel parameters at every step is slow)
 };
 __device__ __forceinline__ void walk_set(Walk& w, uint32_t u, const TcBatch& B) {
   w.u = u;
   w.p = 0;
   for (int i = 1; i < B.count; ++i)
     if (u >= B.p[i].unit0) w.p = i;
+  w.n_kt = B.p[w.p].n_kt;
+  w.n_rt = B.p[w.p].n_rt;
   const uint32_t local = u - B.p[w.p].unit0;
-  w.rt = (int)(local / (uint32_t)B.p[w.p].n_kt);
-  w.kt = (int)(local - (uint32_t)w.rt * (uint32_t)B.p[w.p].n_kt);
+  w.rt = (int)(local / (uint32_t)w.n_kt);
+  w.kt = (int)(local - (uint32_t)w.rt * (uint32_t)w.n_kt);
 }
 __device__ __forceinline__ void walk_step(Walk& w, const TcBatch& B) {
   ++w.u;
-  if (++w.kt == B.p[w.p].n_kt) {
+  if (++w.kt == w.n_kt) {
     w.kt = 0;
-    if (++w.rt == B.p[w.p].n_rt) {
+    if (++w.rt == w.n_rt) {
       w.rt = 0;
-      if (w.p + 1 < B.count) ++w.p;
+      if (w.p + 1 < B.count) {
+        ++w.p;
+        w.n_kt = B.p[w.p].n_kt;
+        w.n_rt = B.p[w.p].n_rt;
+      }
     }
   }
 }
@@ -206,12 +219,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) lut_gemv_tc_kernel(const TcBatc
     return tc_wait(empty((int)(it % kTcSlots), use - 1), ((use - 1) >> 1) & 1u, abort_flag);
   };
 
+  // token tiles start as zeros: rows of tokens a problem does not have are never written
+  for (int i = threadIdx.x; i < kTcSlots * kTcBBytes / 16; i += kTcThreads)
+    reinterpret_cast<uint4*>(gen_base)[i] = make_uint4(0u, 0u, 0u, 0u);
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   if (threadIdx.x == 0) {
     auto init = [](uint32_t bar, uint32_t count) {
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
     };
     for (int s = 0; s < kTcSlots; ++s) {
-      init(full(s), 4 * 32 + 32);        // one decoder group (4 warps) + one producer warp
+      init(full(s), 4 * 32);             // one decoder group (4 warps)
       init(empty(s, 0), 1);              // the issuer of the stage
       init(empty(s, 1), 1);
     }
@@ -240,69 +257,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) lut_gemv_tc_kernel(const TcBatc
   const uint32_t u0 = unit_begin(blockIdx.x, G, T), u1 = unit_begin(blockIdx.x + 1, G, T);
   const uint32_t n_units = u1 - u0;
 
-  if (warp < kTcProducers) {
-    // ------------------------------------------------------------------ token producers
-    // Warp h stages the levels of k-block h of every unit: lane = (token, 64-column half); 32 bytes of 4-bit levels
-    // become 64 signed bytes in the decoder's lookup order, written as four swizzled 16-byte chunks.  The levels of
-    // the next kTcAhead units are held in registers, so the latency of their loads is off the stage's path.
-    const int h = warp, token = lane >> 1, half = lane & 1;
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    Walk wl;
-    if (n_units) walk_set(wl, u0, B);
-    auto load = [&](uint4& a0, uint4& a1) {       // levels of the unit at wl, then step wl
-      const TcProblem& P = B.p[wl.p];
-      if (token < P.M) {
-        const uint8_t* src = P.act_idx + (size_t)token * ((size_t)P.n_kt * 128) + (size_t)wl.kt * 128 + h * 64 + half * 32;
-        a0 = __ldg(reinterpret_cast<const uint4*>(src));
-        a1 = __ldg(reinterpret_cast<const uint4*>(src) + 1);
-      } else {
-        a0 = a1 = make_uint4(0x88888888u, 0x88888888u, 0x88888888u, 0x88888888u);   // level 0
-      }
-      walk_step(wl, B);
-    };
-    uint4 q0[kTcAhead], q1[kTcAhead];
-#pragma unroll
-    for (int j = 0; j < kTcAhead; ++j)
-      if ((uint32_t)j < n_units) load(q0[j], q1[j]);
-    bool ok = true;
-    for (uint32_t ic0 = 0; ic0 < n_units && ok; ic0 += kTcAhead) {
-#pragma unroll
-      for (int j = 0; j < kTcAhead; ++j) {
-        const uint32_t ic = ic0 + (uint32_t)j;
-        if (ic >= n_units || !ok) break;
-        const uint4 a0 = q0[j], a1 = q1[j];
-        if (ic + kTcAhead < n_units) load(q0[j], q1[j]);
-        const uint32_t s[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-        uint32_t o[16];
-#pragma unroll
-        for (int v = 0; v < 8; ++v) {                 // source word v = 8 columns -> two output words
-          const uint32_t e = s[v] & 0x0f0f0f0fu, od = (s[v] >> 4) & 0x0f0f0f0fu;
-          uint32_t x0, x1;
-          int i0, i1;
-          if (BITS == 2) {   // lookup order of a 16-column pair of words: E(w0) E(w1) O(w0) O(w1)
-            x0 = e; x1 = od;
-            i0 = 4 * (v >> 1) + (v & 1); i1 = i0 + 2;
-          } else {           // natural order
-            x0 = tc_prmt(e, od, 0x5140u); x1 = tc_prmt(e, od, 0x7362u);
-            i0 = 2 * v; i1 = 2 * v + 1;
-          }
-          o[i0] = ((x0 | 0x80808080u) - 0x08080808u) ^ 0x80808080u;    // level - 8 as a signed byte
-          o[i1] = ((x1 | 0x80808080u) - 0x08080808u) ^ 0x80808080u;
-        }
-        const uint32_t it = 2u * ic + (uint32_t)h;
-        const int slot = it % kTcSlots;
-        if (!wait_slot_free(it)) { ok = false; break; }
-        uint8_t* row = gen_base + slot * kTcBBytes + (token >> 3) * 1024 + (token & 7) * 128;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const int chunk = (4 * half + c) ^ (token & 7);
-          *reinterpret_cast<uint4*>(row + 16 * chunk) = make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        tc_arrive(full(slot));
-      }
-    }
-  } else if (warp < kTcFirstEpi) {
+  if (warp < kTcFirstEpi) {
     // ------------------------------------------------------------------ MMA issuers
     // One thread per stage slot: a slot's fill barrier is then always waited on by the same thread, in order.
     if (lane == 0) {
@@ -334,7 +289,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) lut_gemv_tc_kernel(const TcBatc
           for (int k = 0; k < 4; ++k) tc_mma(d_hi + 16, a + 32 + 8 * k, bd + 2 * k, idesc_lo);
           tc_commit(empty(slot, it / kTcSlots));
         }
-        const bool last = (ic + 1 == n_units) || (w.kt + 1 == B.p[w.p].n_kt);
+        const bool last = (ic + 1 == n_units) || (w.kt + 1 == w.n_kt);
         if (last) {
           tc_commit(tmem_full(buf));
           seg_open = false;
@@ -367,7 +322,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) lut_gemv_tc_kernel(const TcBatc
     uint32_t sg = 0;
     int seg_kt0 = n_units ? w.kt : 0;
     for (uint32_t ic = 0; ic < n_units && ok; ++ic) {
-      const bool last = (ic + 1 == n_units) || (w.kt + 1 == B.p[w.p].n_kt);
+      const bool last = (ic + 1 == n_units) || (w.kt + 1 == w.n_kt);
       if (last) {
         const TcProblem& P = B.p[w.p];
         const uint32_t buf = sg & 1u;
@@ -382,7 +337,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) lut_gemv_tc_kernel(const TcBatc
         ex = ex < -30 ? -30 : ex;
         const float row_scale = __uint_as_float((uint32_t)(ex - 15 + 127) << 23);   // 2^(e-15) of the row's tables
         const float my_scale = (lane < 16 && lane < P.M) ? __ldg(P.act_scale + lane) : 0.0f;
-        ok = __all_sync(0xffffffffu, tc_wait(tmem_full(buf), (sg >> 1) & 1u, abort_flag));
+        ok = __all_sync(0xffffffffu, tc_wait<true>(tmem_full(buf), (sg >> 1) & 1u, abort_flag));
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         uint32_t hi[16], lo[16];
@@ -477,6 +432,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) lut_gemv_tc_kernel(const TcBatc
     if (lane == 0)
       for (; fetched < n_own && fetched < (uint32_t)kTcRing; ++fetched) { fetch(fetched); advance4(wf); }
 
+    // Each decoder thread also stages one 16-column piece of one token's levels per stage (128 threads = 16 tokens
+    // x 8 pieces): 8 bytes of 4-bit levels become one 16-byte chunk of signed bytes in the lookup order.
+    const int tk_token = (32 * quad + lane) >> 3, tk_piece = lane & 7;
+    const uint8_t* act_ptr = nullptr;       // this thread's token row (+ piece), null when the problem has no such token
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     uint32_t TH[2] = {0, 0}, TL[2] = {0, 0};
     int tab_p = -1, tab_rt = -1;
     bool ok = true;
@@ -486,6 +446,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) lut_gemv_tc_kernel(const TcBatc
       if (wc.p != tab_p || wc.rt != tab_rt) {
         // byte tables of this thread's row: 16-bit fixed point, high (signed) and low (unsigned) bytes
         tab_p = wc.p; tab_rt = wc.rt;
+        act_ptr = tk_token < P.M ? P.act_idx + (size_t)tk_token * ((size_t)P.n_kt * 128) + tk_piece * 8 : nullptr;
         int n = wc.rt * kTcRows + 32 * quad + lane;
         n = n < P.n_rp * 16 ? n : P.n_rp * 16 - 1;
         const uint16_t* cb = P.codebook + (size_t)n * (1 << BITS);
@@ -503,6 +464,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) lut_gemv_tc_kernel(const TcBatc
           TL[i >> 2] |= ((uint32_t)f & 0xffu) << (8 * (i & 3));
         }
         if (BITS == 2) { TH[1] = TH[0]; TL[1] = TL[0]; }
+      }
+      uint2 lv[2] = {make_uint2(0u, 0u), make_uint2(0u, 0u)};
+      if (act_ptr) {
+        lv[0] = __ldg(reinterpret_cast<const uint2*>(act_ptr + (size_t)wc.kt * 128));
+        lv[1] = __ldg(reinterpret_cast<const uint2*>(act_ptr + (size_t)wc.kt * 128 + 64));
       }
       const uint32_t rslot = oi % kTcRing;
       // tcgen05.st below is warp-collective: the whole warp leaves a wait together
@@ -534,30 +500,52 @@ __global__ void __launch_bounds__(kTcThreads, 1) lut_gemv_tc_kernel(const TcBatc
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t a_col = tmem_base + lane_field + slot * kTcACols;
+        if (act_ptr) {
+          const uint32_t w0 = lv[h].x, w1 = lv[h].y;
+          const uint32_t e0 = w0 & 0x0f0f0f0fu, o0 = (w0 >> 4) & 0x0f0f0f0fu;
+          const uint32_t e1 = w1 & 0x0f0f0f0fu, o1 = (w1 >> 4) & 0x0f0f0f0fu;
+          uint32_t x[4];
+          if (BITS == 2) {      // lookup order of 16 columns: even fields of word 0, of word 1, odd fields of 0, of 1
+            x[0] = e0; x[1] = e1; x[2] = o0; x[3] = o1;
+          } else {              // natural order
+            x[0] = tc_prmt(e0, o0, 0x5140u); x[1] = tc_prmt(e0, o0, 0x7362u);
+            x[2] = tc_prmt(e1, o1, 0x5140u); x[3] = tc_prmt(e1, o1, 0x7362u);
+          }
 #pragma unroll
-        for (int t = 0; t < 4; ++t) {
-          uint32_t sel[8], hw[8], lw[8];
-          if (BITS == 2) {
+          for (int i = 0; i < 4; ++i) x[i] = ((x[i] | 0x80808080u) - 0x08080808u) ^ 0x80808080u;   // level - 8, signed byte
+          uint8_t* row = gen_base + slot * kTcBBytes + (tk_token >> 3) * 1024 + (tk_token & 7) * 128;
+          *reinterpret_cast<uint4*>(row + 16 * (tk_piece ^ (tk_token & 7))) = make_uint4(x[0], x[1], x[2], x[3]);
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+        // two quarters (64 weights) per store: a tcgen05.st costs about as much to issue whatever its width
 #pragma unroll
-            for (int wd = 0; wd < 2; ++wd) {
-              const uint32_t r = raw[t][2 * h + wd];
-              const uint32_t s0 = r & 0x33333333u, s1 = (r >> 2) & 0x33333333u;
-              sel[4 * wd] = s0; sel[4 * wd + 1] = s0 >> 16; sel[4 * wd + 2] = s1; sel[4 * wd + 3] = s1 >> 16;
+        for (int tp = 0; tp < 2; ++tp) {
+          uint32_t sel[16], v[16];
+#pragma unroll
+          for (int tq = 0; tq < 2; ++tq) {
+            const int t = 2 * tp + tq;
+            if (BITS == 2) {
+#pragma unroll
+              for (int wd = 0; wd < 2; ++wd) {
+                const uint32_t r = raw[t][2 * h + wd];
+                const uint32_t s0 = r & 0x33333333u, s1 = (r >> 2) & 0x33333333u;
+                sel[8 * tq + 4 * wd] = s0; sel[8 * tq + 4 * wd + 1] = s0 >> 16;
+                sel[8 * tq + 4 * wd + 2] = s1; sel[8 * tq + 4 * wd + 3] = s1 >> 16;
+              }
+            } else {
+              const uint32_t r0 = raw[t][3 * h], r1 = raw[t][3 * h + 1], r2 = raw[t][3 * h + 2];
+              const uint32_t ex = (((r0 >> 3) & 0x11111111u) | ((r1 >> 2) & 0x22222222u)) | ((r2 >> 1) & 0x44444444u);
+              const uint32_t d0 = r0 & 0x77777777u, d1 = r1 & 0x77777777u, d2 = r2 & 0x77777777u;
+              sel[8 * tq] = d0; sel[8 * tq + 1] = d0 >> 16; sel[8 * tq + 2] = d1; sel[8 * tq + 3] = d1 >> 16;
+              sel[8 * tq + 4] = d2; sel[8 * tq + 5] = d2 >> 16; sel[8 * tq + 6] = ex; sel[8 * tq + 7] = ex >> 16;
             }
-          } else {
-            const uint32_t r0 = raw[t][3 * h], r1 = raw[t][3 * h + 1], r2 = raw[t][3 * h + 2];
-            const uint32_t ex = (((r0 >> 3) & 0x11111111u) | ((r1 >> 2) & 0x22222222u)) | ((r2 >> 1) & 0x44444444u);
-            const uint32_t d0 = r0 & 0x77777777u, d1 = r1 & 0x77777777u, d2 = r2 & 0x77777777u;
-            sel[0] = d0; sel[1] = d0 >> 16; sel[2] = d1; sel[3] = d1 >> 16;
-            sel[4] = d2; sel[5] = d2 >> 16; sel[6] = ex; sel[7] = ex >> 16;
           }
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            hw[i] = tc_prmt(TH[0], TH[1], sel[i]);
-            lw[i] = tc_prmt(TL[0], TL[1], sel[i]);
-          }
-          tc_st8(a_col + 8 * t, hw);
-          tc_st8(a_col + 32 + 8 * t, lw);
+          for (int i = 0; i < 16; ++i) v[i] = tc_prmt(TH[0], TH[1], sel[i]);
+          tc_st16(a_col + 16 * tp, v);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[i] = tc_prmt(TL[0], TL[1], sel[i]);
+          tc_st16(a_col + 32 + 16 * tp, v);
         }
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
