@@ -13,15 +13,19 @@
 // fragments are the tokens' activation levels (int8, staged in shared memory in lookup order): 16 rows x 8
 // tokens per instruction, exact int32 sums, so the result does not depend on the order of summation.
 //
-// Streaming.  The index area is a sequence of 16-row x 256-column items.  The items of one problem are split
-// evenly (stream-K) over the warps of the CTAs that work on it; each warp streams its items through its own
-// shared-memory ring filled by bulk asynchronous copies (cp.async.bulk + mbarrier), so many kilobytes per warp
-// are in flight without holding registers.  A 16-row group whose columns are shared by several warps is summed
-// with integer atomics in global scratch; the warp that arrives last (ticket counter) converts the total to
-// fp32, writes y and leaves the scratch zero again.
+// Streaming.  The index area is a sequence of 16-row x 256-column items.  A run is one 16-row group x one column
+// panel (a single panel when all tokens' levels of a whole row fit in shared memory).  A CTA owns whole runs, its
+// 16 warps split the items of those runs evenly, and each warp streams its share through its own shared-memory
+// ring filled by bulk asynchronous copies (cp.async.bulk + mbarrier), so many kilobytes per warp are in flight
+// without holding registers.
 //
-// Several independent problems (the projections of a decoder layer) can run in one launch: CTAs are divided
-// among the problems in proportion to their index bytes.
+// Combine.  Warps of a CTA that share a run add their integer partial sums in shared-memory slots with an arrival
+// counter; the last one converts to fp32 and writes y.  With several panels (and for the bucket tables) the
+// totals of a 16-row group meet in zero-filled global scratch with integer atomics; the warp that arrives last
+// (ticket counter) writes y and leaves the scratch zero again.
+//
+// Several independent problems (the projections of a decoder layer) can run in one launch: CTAs are handed to the
+// problems one at a time, each to the problem whose most loaded CTA has the most items.
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
