@@ -42,6 +42,13 @@ import numpy as np
 
 QMIN, QMAX = -8, 7            # 4-bit symmetric range [-2^(b-1), 2^(b-1)-1], b = 4
 LEVELS = 16
+
+
+def act_range(act_bits: int):
+    """(qmin, qmax) = (-2^(b-1), 2^(b-1)-1) of Section 4.1's clip for b-bit activations (b = 4 or 8)."""
+    if act_bits not in (4, 8):
+        raise ValueError("act_bits must be 4 or 8")
+    return -(1 << (act_bits - 1)), (1 << (act_bits - 1)) - 1
 MAGIC = 0x5744434C            # "LCDW"
 VERSION = 1
 LAYOUT_PAIR16X256 = 2
@@ -65,7 +72,8 @@ def round_up(v: int, m: int) -> int:
 # --------------------------------------------------------------------------------------
 # Section 4.1 - input transformation
 # --------------------------------------------------------------------------------------
-def smooth_quantize(x_fp16: np.ndarray, inv_s: np.ndarray | None, static_scale: float | None = None):
+def smooth_quantize(x_fp16: np.ndarray, inv_s: np.ndarray | None, static_scale: float | None = None,
+                    act_bits: int = 4):
     """Activation index assignment, Section 4.1.
 
     q = Clip(round(X / (s_m * s_q))): the smoothing divide and the quantisation divide are one
@@ -81,27 +89,32 @@ def smooth_quantize(x_fp16: np.ndarray, inv_s: np.ndarray | None, static_scale: 
     through one binary64 division rounds identically (53 >= 2*24+2), so casting to binary32 after
     each step reproduces IEEE binary32 arithmetic exactly.
 
+    With act_bits = 8 (the paper's b = 8) the same steps run with 127 in place of 7 and the clip range
+    [-128, 127].
+
     Returns (q int8 [M,K], s_q float32 [M]).
     """
+    qmin, qmax = act_range(act_bits)
+    top = float(qmax)
     x = np.asarray(x_fp16, dtype=np.float16).astype(np.float64)
     M, K = x.shape
     f = np.ones(K) if inv_s is None else np.asarray(inv_s, dtype=np.float32).astype(np.float64)
     t = _f32(x * f[None, :])
     if static_scale is not None:
-        q = np.clip(np.rint(t), QMIN, QMAX).astype(np.int8)
+        q = np.clip(np.rint(t), qmin, qmax).astype(np.int8)
         return q, np.full(M, np.float32(static_scale), dtype=np.float32)
     A = np.abs(t).max(axis=1) if K else np.zeros(M)
     s_q = np.ones(M, dtype=np.float64)
     r = np.zeros(M, dtype=np.float64)
     nz = A > 0
-    s_q[nz] = _f32(A[nz] / 7.0)
-    r[nz] = _f32(7.0 / A[nz])
+    s_q[nz] = _f32(A[nz] / top)
+    r[nz] = _f32(top / A[nz])
     u = _f32(t * r[:, None])
-    q = np.clip(np.rint(u), QMIN, QMAX).astype(np.int8)   # np.rint rounds half to even
+    q = np.clip(np.rint(u), qmin, qmax).astype(np.int8)   # np.rint rounds half to even
     return q, s_q.astype(np.float32)
 
 
-def smooth_quantize_ideal(x_fp16, inv_s):
+def smooth_quantize_ideal(x_fp16, inv_s, act_bits: int = 4):
     """The same assignment in unrounded real arithmetic (binary64): x/(s_k*s_q) with s_q = A/7.
     Differs from ``smooth_quantize`` only where the pre-rounding value sits within a few binary32
     ulps of a half-integer; used to count such positions, never as an expected value."""
@@ -109,8 +122,9 @@ def smooth_quantize_ideal(x_fp16, inv_s):
     f = np.ones(x.shape[1]) if inv_s is None else np.asarray(inv_s, dtype=np.float32).astype(np.float64)
     t = x * f[None, :]
     A = np.abs(t).max(axis=1)
-    u = np.where(A[:, None] > 0, t * 7.0 / np.where(A > 0, A, 1.0)[:, None], 0.0)
-    return np.clip(np.rint(u), QMIN, QMAX).astype(np.int8)
+    qmin, qmax = act_range(act_bits)
+    u = np.where(A[:, None] > 0, t * float(qmax) / np.where(A > 0, A, 1.0)[:, None], 0.0)
+    return np.clip(np.rint(u), qmin, qmax).astype(np.int8)
 
 
 def pack_act(q: np.ndarray, K_pad: int | None = None) -> np.ndarray:
@@ -121,6 +135,16 @@ def pack_act(q: np.ndarray, K_pad: int | None = None) -> np.ndarray:
     a = np.full((M, K_pad), 8, dtype=np.uint8)
     a[:, :K] = (q.astype(np.int16) + 8).astype(np.uint8)
     return (a[:, 0::2] | (a[:, 1::2] << 4)).astype(np.uint8)
+
+
+def pad_act8(q: np.ndarray, K_pad: int | None = None) -> np.ndarray:
+    """8-bit activation levels as stored for the lookup: one signed byte per column, row padded to K_pad
+    (multiple of 256) with zeros."""
+    M, K = q.shape
+    K_pad = round_up(K, TILE_K) if K_pad is None else K_pad
+    out = np.zeros((M, K_pad), dtype=np.int8)
+    out[:, :K] = q
+    return out
 
 
 def unpack_act(packed: np.ndarray, K: int) -> np.ndarray:
@@ -162,13 +186,15 @@ def lut_linear_loops(idx, codebook_fp16, q, s_q) -> np.ndarray:
     return y
 
 
-def lut_linear_product(idx, codebook_fp16, q, s_q) -> np.ndarray:
-    """Product table: T_{m,n}[a][w] = ((a-8) * s_q[m]) * cb[n][w];  y[m][n] = sum_k T[a_k][idx_k]."""
+def lut_linear_product(idx, codebook_fp16, q, s_q, act_bits: int = 4) -> np.ndarray:
+    """Product table: T_{m,n}[a][w] = ((a + qmin) * s_q[m]) * cb[n][w];  y[m][n] = sum_k T[a_k][idx_k], with the
+    activation index a = q - qmin in [0, 2^b) (16 rows for b = 4, 256 for b = 8)."""
     cb = np.asarray(codebook_fp16, dtype=np.float16).astype(np.float64)
     M, K = q.shape
     N, C = cb.shape
-    a = q.astype(np.int64) + 8
-    levels = np.arange(LEVELS, dtype=np.float64) - 8.0
+    qmin, _ = act_range(act_bits)
+    a = q.astype(np.int64) - qmin
+    levels = np.arange(1 << act_bits, dtype=np.float64) + float(qmin)
     y = np.zeros((M, N))
     ii = idx.astype(np.int64)
     for m in range(M):
@@ -179,8 +205,9 @@ def lut_linear_product(idx, codebook_fp16, q, s_q) -> np.ndarray:
     return y
 
 
-def lut_linear_signfold(idx, codebook_fp16, q, s_q) -> np.ndarray:
-    """Only |q| in [0,8] is tabulated: T+[|q|][w] = (|q| * s_q) * cb[w]; y = sum_k sgn(q_k) * T+[|q_k|][idx_k]."""
+def lut_linear_signfold(idx, codebook_fp16, q, s_q, act_bits: int = 4) -> np.ndarray:
+    """Only |q| in [0, 2^(b-1)] is tabulated (9 rows for b = 4, 129 for b = 8):
+    T+[|q|][w] = (|q| * s_q) * cb[w]; y = sum_k sgn(q_k) * T+[|q_k|][idx_k]."""
     cb = np.asarray(codebook_fp16, dtype=np.float16).astype(np.float64)
     M, K = q.shape
     N, C = cb.shape
@@ -189,7 +216,7 @@ def lut_linear_signfold(idx, codebook_fp16, q, s_q) -> np.ndarray:
     y = np.zeros((M, N))
     ii = idx.astype(np.int64)
     for m in range(M):
-        lev = np.arange(9, dtype=np.float64) * float(s_q[m])
+        lev = np.arange((1 << (act_bits - 1)) + 1, dtype=np.float64) * float(s_q[m])
         for n in range(N):
             Tp = lev[:, None] * cb[n][None, :]            # 9 x C
             y[m, n] = (sgn[m] * Tp[mag[m], ii[n]]).sum()

@@ -298,3 +298,65 @@ def test_pack_rejects_bad_indices_and_corruption():
     bad = blob.copy(); bad[0] ^= 1
     with pytest.raises(ValueError):
         O.unpack_weights(bad)
+
+
+# ---------------------------------------------------------------- 8-bit activations (the paper's b = 8, Section 4.1)
+def test_quantiser_8bit_hand_example_and_static_levels():
+    # A = 127 with inv_s = 1: s_q = 1 and r = 1 exactly, so q = round-half-even(x)
+    x = np.array([[127, -63.5, 0.5, 1.5, 2.5, -127, 100.25, -0.75]], dtype=np.float16)
+    q, s = O.smooth_quantize(x, None, act_bits=8)
+    assert q.tolist() == [[127, -64, 0, 2, 2, -127, 100, -1]] and s[0] == 1.0
+    # static mode: every level of [-128, 127] is reachable, values beyond are clipped
+    xv = np.arange(-130, 131, dtype=np.float16)[None, :]
+    qs, ss = O.smooth_quantize(xv, np.ones(261, dtype=np.float32), static_scale=0.25, act_bits=8)
+    assert qs[0].tolist() == [max(-128, min(127, v)) for v in range(-130, 131)] and np.all(ss == np.float32(0.25))
+
+
+def test_quantiser_8bit_is_binary32_arithmetic_symmetric_and_bounded():
+    rng = np.random.default_rng(12)
+    x = (rng.standard_normal((4, 512)) * 3).astype(np.float16)
+    inv_s = (rng.random(512) * 3 + 0.01).astype(np.float32)
+    q, s = O.smooth_quantize(x, inv_s, act_bits=8)
+    t = x.astype(np.float32) * inv_s[None, :]
+    A = np.abs(t).max(axis=1)
+    s32 = A / np.float32(127.0)
+    u = t * (np.float32(127.0) / A)[:, None]
+    assert np.array_equal(q, np.clip(np.rint(u), -128, 127).astype(np.int8)) and np.array_equal(s, s32)
+    assert np.all(np.abs(q.astype(int)).max(axis=1) == 127) and q.min() >= -127
+    qn, sn = O.smooth_quantize(-x, inv_s, act_bits=8)
+    assert np.array_equal(qn, -q) and np.array_equal(sn, s)
+    # uniform quantiser of step s_q: |t - s_q q| <= s_q / 2
+    err = np.abs(t.astype(np.float64) - s.astype(np.float64)[:, None] * q)
+    assert np.all(err <= 0.5 * s[:, None] * (1 + 1e-4))
+    assert (O.smooth_quantize_ideal(x, inv_s, act_bits=8) != q).mean() < 2e-3
+    # sixteen times finer than the 4-bit grid of the same row: q4 is q8 rescaled and re-rounded, up to ties
+    q4, s4 = O.smooth_quantize(x, inv_s)
+    assert np.abs(q4.astype(np.float64) - q.astype(np.float64) * 7.0 / 127.0).max() <= 0.5 + 7.0 / 127.0
+
+
+def test_lookup_forms_agree_for_8bit_levels_and_known_values():
+    rng = np.random.default_rng(13)
+    N, K, C, M = 6, 40, 4, 3
+    idx = rng.integers(0, C, size=(N, K), dtype=np.uint8)
+    cb = rng.standard_normal((N, C)).astype(np.float16)
+    q = rng.integers(-128, 128, size=(M, K)).astype(np.int8)
+    q[0, :3] = (-128, 127, 0)
+    s_q = (rng.random(M) + 0.1).astype(np.float32)
+    ref = (q.astype(np.float64) @ cb.astype(np.float64)[np.arange(N)[:, None], idx].T) * s_q.astype(np.float64)[:, None]
+    for f in (O.lut_linear_dequant, O.lut_linear_loops, O.lut_linear_bucket):
+        np.testing.assert_allclose(f(idx, cb, q, s_q), ref, rtol=1e-12, atol=1e-12)
+    for f in (O.lut_linear_product, O.lut_linear_signfold):      # 256 x C and 129 x C tables
+        np.testing.assert_allclose(f(idx, cb, q, s_q, act_bits=8), ref, rtol=1e-12, atol=1e-12)
+    # a 4-bit-sized table cannot hold these levels: the width is part of the definition
+    with pytest.raises(IndexError):
+        O.lut_linear_signfold(idx, cb, q, s_q, act_bits=4)
+    # one weight, one column: y = s_q * q * cb
+    y = O.lut_linear_product(np.array([[1]], dtype=np.uint8), np.array([[0.5, -2.0]], dtype=np.float16),
+                             np.array([[-128]], dtype=np.int8), np.array([0.5], dtype=np.float32), act_bits=8)
+    assert y[0, 0] == 0.5 * -128 * -2.0
+
+
+def test_act8_padding():
+    q = np.arange(-128, 128, dtype=np.int8).reshape(1, 256)[:, :200]
+    p = O.pad_act8(q)
+    assert p.shape == (1, 256) and p.dtype == np.int8 and np.array_equal(p[:, :200], q) and not p[:, 200:].any()
