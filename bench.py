@@ -54,14 +54,16 @@ def parse_args():
     ap.add_argument("--M", type=int, default=None, help="token count (default: first M of the config)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--act-bits", type=int, default=4, choices=[4, 8],
+                    help="activation levels: 4 bit (the benchmark configurations) or 8 bit (the paper's b = 8)")
     ap.add_argument("--algo", default="auto", choices=["auto", "register", "bucket", "tensor"],
                     help="lookup kernel for M <= 16 (default: the library's choice)")
     return ap.parse_args()
 
 
-def algorithmic_bytes(N, K, bits, M):
+def algorithmic_bytes(N, K, bits, M, act_bits=4):
     """index + codebook + activation-index bytes the method must read for one matrix (no padding, no output)."""
-    return N * K * bits / 8 + N * (1 << bits) * 2 + M * (K / 2 + 4)
+    return N * K * bits / 8 + N * (1 << bits) * 2 + M * (K * act_bits / 8 + 4)
 
 
 def build_layers(cfg_id, M):
@@ -137,11 +139,11 @@ def metric_name(M):
     return "lut_linear_us_per_layer_m%d" % M
 
 
-def workload_config(cfg_id, M, copies):
+def workload_config(cfg_id, M, copies, act_bits=4):
     cfg = gen.CONFIGS[cfg_id]
     return {"workload": f"BASELINE configs[{cfg_id}] {cfg['name']}: " +
                         ", ".join(f"{n} {N}x{K}" for n, N, K in cfg["shapes"]),
-            "bits": cfg["bits"], "M": M, "act_bits": 4, "outliers": f"{cfg['frac'] * 100:g}% x{cfg['scale']:g}",
+            "bits": cfg["bits"], "M": M, "act_bits": act_bits, "outliers": f"{cfg['frac'] * 100:g}% x{cfg['scale']:g}",
             "l2": f"weights rotate over {copies} device copies (> {int(L2_BYTES / 1e6)} MB L2)"}
 
 
@@ -232,13 +234,14 @@ def run_ours(args):
         x = torch.from_numpy(L.x).to(dev)
         inv_s = torch.from_numpy(L.inv_s).to(dev)
         K_pad = ws[0].K_pad
-        a = torch.empty((M, K_pad // 2), dtype=torch.uint8, device=dev)
+        a = (torch.empty((M, K_pad // 2), dtype=torch.uint8, device=dev) if args.act_bits == 4 else
+             torch.empty((M, K_pad), dtype=torch.int8, device=dev))
         s = torch.empty((M,), dtype=torch.float32, device=dev)
         y = torch.empty((M, L.N), dtype=torch.float32, device=dev)
         wsb = lcd.lut_linear_workspace_bytes(ws[0], M)
         work = torch.zeros(max(wsb, 256), dtype=torch.uint8, device=dev)
         mats.append(dict(name=name, L=L, w=ws, x=x, inv_s=inv_s, a=a, s=s, y=y, work=work,
-                         bytes=algorithmic_bytes(L.N, L.K, bits, M), flop=2.0 * M * L.N * L.K))
+                         bytes=algorithmic_bytes(L.N, L.K, bits, M, args.act_bits), flop=2.0 * M * L.N * L.K))
 
     grouped = M <= 16 and len(mats) <= lcd.MAX_BATCH
     algo = {"auto": lcd.ALGO_AUTO, "register": lcd.ALGO_REGISTER_LUT, "bucket": lcd.ALGO_BUCKET_LUT,
@@ -263,7 +266,8 @@ def run_ours(args):
     else:
         def step(c):
             for mt in mats:
-                lcd.smooth_quantize_act(mt["x"], mt["inv_s"], act_idx=mt["a"], act_scale=mt["s"])
+                lcd.smooth_quantize_act(mt["x"], mt["inv_s"], act_idx=mt["a"], act_scale=mt["s"],
+                                        act_bits=args.act_bits)
                 lcd.lut_linear(mt["w"][c], mt["a"], mt["s"], y=mt["y"], workspace=mt["work"], status_word=status)
 
         def lookup_only(mi, c):
@@ -339,7 +343,7 @@ def run_ours(args):
         # end to end through the host-buffer entry points: pinned host x -> device -> kernels -> pinned host y.
         # Grouped (M <= 16): one copy in, two launches, one copy out per layer; else per matrix.
         e2e_ms, h2d, d2h = None, 0, 0
-        if grouped:
+        if grouped and args.act_bits == 4:
             hbatch = [lcd.HostBatch([(mt["w"][c], mt["inv_s"], M) for mt in mats], dev) for c in range(copies)]
             for hb in hbatch:
                 for i, mt in enumerate(mats):
@@ -361,8 +365,15 @@ def run_ours(args):
                 d2h += yh.numel() * 4
 
             def e2e_step(c):
-                for mt, (xh, yh, sc) in zip(mats, host):
-                    lcd.linear_host(mt["w"][c], xh, mt["inv_s"], yh, sc)
+                if args.act_bits == 4:
+                    for mt, (xh, yh, sc) in zip(mats, host):
+                        lcd.linear_host(mt["w"][c], xh, mt["inv_s"], yh, sc)
+                else:          # no host-buffer entry point for 8-bit levels: the copies are made here
+                    for mt, (xh, yh, sc) in zip(mats, host):
+                        mt["x"].copy_(xh, non_blocking=True)
+                    step(c)
+                    for mt, (xh, yh, sc) in zip(mats, host):
+                        yh.copy_(mt["y"], non_blocking=True)
                 torch.cuda.current_stream().synchronize()
 
         n_e2e = max(3, min(args.steps, 50))
@@ -419,7 +430,7 @@ def run_ours(args):
     line = {"metric": metric_name(M), "value": us_per_layer, "unit": "us/layer", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
             "vs_baseline": None, "dtype": "s8 table bytes x s8 levels -> s32 (int8 MMA), f32 epilogue" if not tensor_bound else "s8 table bytes x s8 levels -> s32 (tcgen05 kind::i8), f32 epilogue",
-            "data": "synthetic", "config": dict(workload_config(args.config, M, copies),
+            "data": "synthetic", "config": dict(workload_config(args.config, M, copies, args.act_bits),
                                                 launches="1 grouped quantise + 1 grouped lookup per layer" if grouped
                                                 else "per matrix: quantise + lookup"),
             "layer_GBps": layer_alg_bytes * world / (ms_step * 1e-3) / 1e9,

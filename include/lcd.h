@@ -118,9 +118,11 @@ lcd_status lcd_unpack_weights(const void* blob, size_t blob_bytes, uint8_t* idx,
  *   x_fp16:      device, binary16 [M][ldx], ldx >= K;
  *   inv_smooth:  device, fp32 [K], or NULL for all ones;
  *   static_scale device, fp32 scalar, or NULL;
- *   act_bits:    must be 4;
- *   act_idx:     device out, uint8 [M][K_pad/2], K_pad = 256*ceil(K/256): a = q + 8, column k even in the
- *                low nibble; columns K..K_pad-1 are written as a = 8 (q = 0);
+ *   act_bits:    4, or 8 (the paper's own b = 8: the same steps with 127 in place of 7 and the clip range
+ *                [-128, 127]);
+ *   act_idx:     device out.  act_bits = 4: uint8 [M][K_pad/2], K_pad = 256*ceil(K/256): a = q + 8, column k
+ *                even in the low nibble; columns K..K_pad-1 are written as a = 8 (q = 0).
+ *                act_bits = 8: [M][K_pad] signed bytes q, columns K..K_pad-1 written as 0; 16-byte aligned;
  *   act_scale:   device out, fp32 [M] (s_q).
  * -------------------------------------------------------------------------------------------- */
 lcd_status lcd_smooth_quantize_act(const void* x_fp16, int64_t M, int64_t K, int64_t ldx,
@@ -138,6 +140,7 @@ typedef struct {
   float* act_scale;          /* device out */
 } lcd_act_problem;
 
+/* act_bits: 4 or 8, for all problems of the call (8: every act_idx is [M][K_pad] signed bytes). */
 lcd_status lcd_smooth_quantize_act_batch(const lcd_act_problem* problems /* host */, int count, int act_bits,
                                          void* cuda_stream);
 
@@ -168,6 +171,17 @@ lcd_status lcd_lut_linear(const void* packed_weights_dev, const void* header_hos
                           void* workspace, size_t workspace_bytes, int32_t* status_word_dev,
                           void* cuda_stream);
 
+/* The same lookup and accumulation for 8-bit activation levels (Section 4.1 with b = 8; Section 4.2's tables then
+ * have 129 sign-folded rows, here as there never materialised: the weight is looked up, the level multiplies in
+ * the integer MMA).  act_q: device, [M][K_pad] signed bytes as written by lcd_smooth_quantize_act with
+ * act_bits = 8, 16-byte aligned.  Everything else, the workspace size and its zero-fill contract included, as
+ * lcd_lut_linear; algo may be AUTO, REFERENCE, REGISTER_LUT, BUCKET_LUT, TC_LUT or DENSE_TC (DENSE_F16 and
+ * K_pad >= 131072, where the int32 sums could overflow, give LCD_ERR_UNSUPPORTED). */
+lcd_status lcd_lut_linear_act8(const void* packed_weights_dev, const void* header_host, const int8_t* act_q,
+                               const float* act_scale, int64_t M, float* y, int64_t ldy, lcd_algo algo,
+                               void* workspace, size_t workspace_bytes, int32_t* status_word_dev,
+                               void* cuda_stream);
+
 /* Up to LCD_MAX_BATCH independent problems with M <= 16 (e.g. the q/k/v or gate/up projections of a decoder
  * layer, or all projections of a layer when their inputs are independent) in ONE launch: the SMs are divided
  * among the problems in proportion to their index bytes.  All problems must have the same index width.
@@ -186,6 +200,12 @@ lcd_status lcd_lut_linear_batch_workspace_bytes(const lcd_linear_problem* proble
                                                 lcd_algo algo, size_t* bytes);
 
 lcd_status lcd_lut_linear_batch(const lcd_linear_problem* problems /* host */, int count, lcd_algo algo,
+                                void* workspace, size_t workspace_bytes, int32_t* status_word_dev,
+                                void* cuda_stream);
+
+/* lcd_lut_linear_batch for 8-bit levels: every problem's act_idx points at [M][K_pad] signed bytes (see
+ * lcd_lut_linear_act8); workspace size from lcd_lut_linear_batch_workspace_bytes. */
+lcd_status lcd_lut_linear_batch_act8(const lcd_linear_problem* problems /* host */, int count, lcd_algo algo,
                                 void* workspace, size_t workspace_bytes, int32_t* status_word_dev,
                                 void* cuda_stream);
 

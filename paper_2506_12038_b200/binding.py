@@ -26,7 +26,8 @@ EXPORTS = ["lcd_status_string", "lcd_last_cuda_error", "lcd_packed_weights_bytes
            "lcd_unpack_weights", "lcd_smooth_quantize_act", "lcd_lut_linear_workspace_bytes", "lcd_lut_linear",
            "lcd_linear_host_scratch_bytes", "lcd_linear_host", "lcd_smooth_quantize_act_batch",
            "lcd_lut_linear_batch_workspace_bytes", "lcd_lut_linear_batch", "lcd_lut_linear_static",
-           "lcd_linear_host_batch_sizes", "lcd_linear_host_batch"]
+           "lcd_linear_host_batch_sizes", "lcd_linear_host_batch", "lcd_lut_linear_act8",
+           "lcd_lut_linear_batch_act8"]
 STATIC_SCRATCH_BYTES = 4 << 20
 
 
@@ -71,6 +72,8 @@ def _load() -> ctypes.CDLL:
     lib.lcd_lut_linear_workspace_bytes.argtypes = [c_void_p, c_int64, c_int, POINTER(c_size_t)]
     lib.lcd_lut_linear.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_int64, c_int,
                                    c_void_p, c_size_t, c_void_p, c_void_p]
+    lib.lcd_lut_linear_act8.argtypes = lib.lcd_lut_linear.argtypes
+    lib.lcd_lut_linear_batch_act8.argtypes = [POINTER(LinearProblem), c_int, c_int, c_void_p, c_size_t, c_void_p, c_void_p]
     lib.lcd_linear_host_scratch_bytes.argtypes = [c_void_p, c_int64, POINTER(c_size_t)]
     lib.lcd_linear_host.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_size_t,
                                     c_void_p]
@@ -165,20 +168,25 @@ class PackedWeights:
         return ctypes.cast(self._hdr_buf, c_void_p)
 
 
-def smooth_quantize_act(x, inv_smooth=None, static_scale=None, act_idx=None, act_scale=None, stream=None):
-    """x: CUDA fp16 [M,K] (row stride may exceed K) -> (act_idx uint8 [M,K_pad/2], act_scale fp32 [M])."""
+def smooth_quantize_act(x, inv_smooth=None, static_scale=None, act_idx=None, act_scale=None, stream=None,
+                        act_bits: int = 4):
+    """x: CUDA fp16 [M,K] (row stride may exceed K) -> (act_idx uint8 [M,K_pad/2], act_scale fp32 [M]); with
+    act_bits = 8 the levels come back as int8 [M,K_pad]."""
     import torch
     assert x.is_cuda and x.dtype == torch.float16 and x.dim() == 2 and x.stride(1) == 1
     M, K = x.shape
     K_pad = (K + 255) // 256 * 256
+    assert act_bits in (4, 8)
     if act_idx is None:
-        act_idx = torch.empty((M, K_pad // 2), dtype=torch.uint8, device=x.device)
+        act_idx = (torch.empty((M, K_pad // 2), dtype=torch.uint8, device=x.device) if act_bits == 4 else
+                   torch.empty((M, K_pad), dtype=torch.int8, device=x.device))
+    assert act_idx.dtype == (torch.uint8 if act_bits == 4 else torch.int8)
     if act_scale is None:
         act_scale = torch.empty((M,), dtype=torch.float32, device=x.device)
     st = lib.lcd_smooth_quantize_act(c_void_p(x.data_ptr()), M, K, x.stride(0),
                                      c_void_p(inv_smooth.data_ptr()) if inv_smooth is not None else None,
                                      c_void_p(static_scale.data_ptr()) if static_scale is not None else None,
-                                     4, c_void_p(act_idx.data_ptr()), c_void_p(act_scale.data_ptr()),
+                                     act_bits, c_void_p(act_idx.data_ptr()), c_void_p(act_scale.data_ptr()),
                                      _stream_ptr(stream))
     _check(st, "lcd_smooth_quantize_act")
     return act_idx, act_scale
@@ -192,21 +200,24 @@ def lut_linear_workspace_bytes(w: PackedWeights, M: int, algo: int = ALGO_AUTO) 
 
 def lut_linear(w: PackedWeights, act_idx, act_scale, y=None, algo: int = ALGO_AUTO, workspace=None,
                status_word=None, stream=None):
-    """y[m][n] = s_q[m] * sum_k q[m][k] * cb[n][idx[n][k]]  (CUDA fp32 [M,N])."""
+    """y[m][n] = s_q[m] * sum_k q[m][k] * cb[n][idx[n][k]]  (CUDA fp32 [M,N]).  act_idx: uint8 packed 4-bit
+    levels, or int8 8-bit levels (as smooth_quantize_act returns them for act_bits = 8)."""
     import torch
     M = act_idx.shape[0]
+    fn, name = ((lib.lcd_lut_linear_act8, "lcd_lut_linear_act8") if act_idx.dtype == torch.int8 else
+                (lib.lcd_lut_linear, "lcd_lut_linear"))
     if y is None:
         y = torch.empty((M, w.N), dtype=torch.float32, device=act_idx.device)
     need = lut_linear_workspace_bytes(w, M, algo)
     if need and (workspace is None or workspace.numel() * workspace.element_size() < need):
         workspace = torch.zeros(need, dtype=torch.uint8, device=act_idx.device)   # must start zero-filled
-    st = lib.lcd_lut_linear(c_void_p(w.dev.data_ptr()), w.header_ptr, c_void_p(act_idx.data_ptr()),
+    st = fn(c_void_p(w.dev.data_ptr()), w.header_ptr, c_void_p(act_idx.data_ptr()),
                             c_void_p(act_scale.data_ptr()), M, c_void_p(y.data_ptr()), y.stride(0), algo,
                             c_void_p(workspace.data_ptr()) if workspace is not None else None,
                             workspace.numel() * workspace.element_size() if workspace is not None else 0,
                             c_void_p(status_word.data_ptr()) if status_word is not None else None,
                             _stream_ptr(stream))
-    _check(st, "lcd_lut_linear")
+    _check(st, name)
     return y
 
 
@@ -224,10 +235,14 @@ def lut_linear_static(w: PackedWeights, act_idx, act_scale, y, algo: int = ALGO_
 
 class ActBatch:
     """Up to MAX_BATCH activation matrices quantised by one launch.  items: (x, inv_smooth, act_idx, act_scale)
-    CUDA tensors (inv_smooth may be None); the argument array is built once and reused by run()."""
+    CUDA tensors (inv_smooth may be None); the argument array is built once and reused by run().  The level
+    width follows the dtype of the act_idx tensors: uint8 = packed 4-bit, int8 = 8-bit."""
 
     def __init__(self, items):
+        import torch
         self._keep = list(items)
+        self.act_bits = 8 if self._keep[0][2].dtype == torch.int8 else 4
+        assert all((it[2].dtype == torch.int8) == (self.act_bits == 8) for it in self._keep)
         self.count = len(self._keep)
         self.arr = (ActProblem * self.count)()
         for a, (x, inv_s, idx, scale) in zip(self.arr, self._keep):
@@ -237,17 +252,20 @@ class ActBatch:
             a.act_idx, a.act_scale = idx.data_ptr(), scale.data_ptr()
 
     def run(self, stream=None):
-        _check(lib.lcd_smooth_quantize_act_batch(self.arr, self.count, 4, _stream_ptr(stream)),
+        _check(lib.lcd_smooth_quantize_act_batch(self.arr, self.count, self.act_bits, _stream_ptr(stream)),
                "lcd_smooth_quantize_act_batch")
 
 
 class LinearBatch:
     """Up to MAX_BATCH independent lookup problems (M <= 16, same index width) run by one launch.
-    items: (PackedWeights, act_idx, act_scale, y) with CUDA tensors; the zero-filled workspace is owned here."""
+    items: (PackedWeights, act_idx, act_scale, y) with CUDA tensors; the zero-filled workspace is owned here.
+    act_idx tensors of dtype int8 are 8-bit levels (all items alike)."""
 
     def __init__(self, items, algo: int = ALGO_AUTO, status_word=None):
         import torch
         self._keep = list(items)
+        self.act8 = self._keep[0][1].dtype == torch.int8
+        assert all((it[1].dtype == torch.int8) == self.act8 for it in self._keep)
         self.count = len(self._keep)
         self.algo = algo
         self.arr = (LinearProblem * self.count)()
@@ -262,10 +280,10 @@ class LinearBatch:
         self.status_word = status_word
 
     def run(self, stream=None):
-        _check(lib.lcd_lut_linear_batch(self.arr, self.count, self.algo, c_void_p(self.workspace.data_ptr()),
-                                        self.workspace.numel(),
-                                        c_void_p(self.status_word.data_ptr()) if self.status_word is not None else None,
-                                        _stream_ptr(stream)), "lcd_lut_linear_batch")
+        fn = lib.lcd_lut_linear_batch_act8 if self.act8 else lib.lcd_lut_linear_batch
+        _check(fn(self.arr, self.count, self.algo, c_void_p(self.workspace.data_ptr()), self.workspace.numel(),
+                  c_void_p(self.status_word.data_ptr()) if self.status_word is not None else None,
+                  _stream_ptr(stream)), "lcd_lut_linear_batch")
 
 
 class HostBatch:

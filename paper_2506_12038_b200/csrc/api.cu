@@ -107,16 +107,19 @@ extern "C" lcd_status lcd_smooth_quantize_act(const void* x_fp16, int64_t M, int
                                               uint8_t* act_idx, float* act_scale, void* cuda_stream) {
   if (!x_fp16 || !act_idx || !act_scale || M < 1 || K < 1 || ldx < K) return LCD_ERR_INVALID_ARG;
   if (M > 0x7fffffffLL) return LCD_ERR_INVALID_ARG;
-  if (act_bits != LCD_ACT_BITS) return LCD_ERR_UNSUPPORTED;
+  if (act_bits != LCD_ACT_BITS && act_bits != 8) return LCD_ERR_UNSUPPORTED;
   if (!aligned(x_fp16, 2) || !aligned(act_scale, 4) || (inv_smooth && !aligned(inv_smooth, 4)))
     return LCD_ERR_INVALID_ARG;
+  if (act_bits == 8)
+    return launch_smooth_quantize8(x_fp16, M, K, ldx, inv_smooth, static_scale, reinterpret_cast<int8_t*>(act_idx),
+                                   act_scale, cuda_stream);
   return launch_smooth_quantize(x_fp16, M, K, ldx, inv_smooth, static_scale, act_idx, act_scale, cuda_stream);
 }
 
 extern "C" lcd_status lcd_smooth_quantize_act_batch(const lcd_act_problem* problems, int count, int act_bits,
                                                     void* cuda_stream) {
   if (!problems || count < 1 || count > LCD_MAX_BATCH) return LCD_ERR_INVALID_ARG;
-  if (act_bits != LCD_ACT_BITS) return LCD_ERR_UNSUPPORTED;
+  if (act_bits != LCD_ACT_BITS && act_bits != 8) return LCD_ERR_UNSUPPORTED;
   for (int i = 0; i < count; ++i) {
     const lcd_act_problem& q = problems[i];
     if (!q.x_fp16 || !q.act_idx || !q.act_scale || q.M < 1 || q.K < 1 || q.ldx < q.K || q.M > 0x7fffffffLL)
@@ -124,6 +127,7 @@ extern "C" lcd_status lcd_smooth_quantize_act_batch(const lcd_act_problem* probl
     if (!aligned(q.x_fp16, 2) || !aligned(q.act_scale, 4) || (q.inv_smooth && !aligned(q.inv_smooth, 4)))
       return LCD_ERR_INVALID_ARG;
   }
+  if (act_bits == 8) return launch_smooth_quantize8_batch(problems, count, cuda_stream);
   return launch_smooth_quantize_batch(problems, count, cuda_stream);
 }
 
@@ -206,6 +210,60 @@ extern "C" lcd_status lcd_lut_linear_batch(const lcd_linear_problem* problems, i
   if (!workspace || workspace_bytes < need) return LCD_ERR_BUFFER_TOO_SMALL;
   if (!aligned(workspace, 256)) return LCD_ERR_INVALID_ARG;
   return launch_lut_gemv(p, count, resolved, workspace, workspace_bytes, status_word_dev, cuda_stream);
+}
+
+extern "C" lcd_status lcd_lut_linear_batch_act8(const lcd_linear_problem* problems, int count, lcd_algo algo,
+                                           void* workspace, size_t workspace_bytes, int32_t* status_word_dev,
+                                           void* cuda_stream) {
+  lcd_algo resolved;
+  lcd_status st = batch_algo(problems, count, algo, &resolved);
+  if (st != LCD_OK) return st;
+  Problem p[LCD_MAX_BATCH];
+  for (int i = 0; i < count; ++i) {
+    const lcd_linear_problem& q = problems[i];
+    st = make_problem(q.packed_weights_dev, q.header_host, q.act_idx, q.act_scale, q.M, q.y, q.ldy, &p[i]);
+    if (st != LCD_OK) return st;
+    if (p[i].bits != p[0].bits) return LCD_ERR_UNSUPPORTED;
+    p[i].act_bits = 8;
+    if (p[i].K_pad >= (1LL << 17)) return LCD_ERR_UNSUPPORTED;   // int32 sums could overflow
+  }
+  const size_t need = lut_gemv_workspace_bytes(p, count, resolved);
+  if (!workspace || workspace_bytes < need) return LCD_ERR_BUFFER_TOO_SMALL;
+  if (!aligned(workspace, 256)) return LCD_ERR_INVALID_ARG;
+  return launch_lut_gemv(p, count, resolved, workspace, workspace_bytes, status_word_dev, cuda_stream);
+}
+
+extern "C" lcd_status lcd_lut_linear_act8(const void* packed_weights_dev, const void* header_host, const int8_t* act_q,
+                                          const float* act_scale, int64_t M, float* y, int64_t ldy, lcd_algo algo,
+                                          void* workspace, size_t workspace_bytes, int32_t* status_word_dev,
+                                          void* cuda_stream) {
+  Problem p;
+  lcd_status st = make_problem(packed_weights_dev, header_host, reinterpret_cast<const uint8_t*>(act_q), act_scale, M,
+                               y, ldy, &p);
+  if (st != LCD_OK) return st;
+  p.act_bits = 8;
+  // int32 sums of table byte x level: |sum| <= 128 * 128 * K_pad must stay below 2^31
+  if (p.K_pad >= (1LL << 17)) return LCD_ERR_UNSUPPORTED;
+  size_t need = 0;
+  st = workspace_for(p, algo, &need);
+  if (st != LCD_OK) return st;
+  if (need > 0 && (!workspace || workspace_bytes < need)) return LCD_ERR_BUFFER_TOO_SMALL;
+  if (need > 0 && !aligned(workspace, 256)) return LCD_ERR_INVALID_ARG;
+  const lcd_algo resolved = resolve_algo(M, algo);
+  switch (resolved) {
+    case LCD_ALGO_REFERENCE:
+      return launch_reference(p, cuda_stream);
+    case LCD_ALGO_REGISTER_LUT:
+    case LCD_ALGO_BUCKET_LUT:
+    case LCD_ALGO_TC_LUT:
+      return launch_lut_gemv(&p, 1, resolved, workspace, workspace_bytes, status_word_dev, cuda_stream);
+    case LCD_ALGO_DENSE_TC:
+      return launch_dense_tc(p, false, workspace, workspace_bytes, status_word_dev, cuda_stream);
+    case LCD_ALGO_DENSE_F16:
+      return LCD_ERR_UNSUPPORTED;
+    default:
+      return LCD_ERR_INVALID_ARG;
+  }
 }
 
 // ---- host-buffer path -------------------------------------------------------------------------------

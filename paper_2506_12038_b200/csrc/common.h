@@ -40,7 +40,8 @@ struct Problem {
   const uint16_t* codebook; // device: [N_pad][2^bits] fp16 bits
   int64_t N, K, K_pad, N_pad;
   int bits, C;
-  const uint8_t* act_idx;   // device [M][K_pad/2]
+  const uint8_t* act_idx;   // device [M][K_pad/2] (4-bit levels + 8) or [M][K_pad] signed bytes (act_bits == 8)
+  int act_bits = 4;         // 4 or 8
   const float* act_scale;   // device [M]
   int64_t M;
   float* y;
@@ -52,6 +53,9 @@ void set_cuda_error(int err);  // records cudaGetErrorString for lcd_last_cuda_e
 // kernel launchers (each returns LCD_OK or LCD_ERR_CUDA / LCD_ERR_UNSUPPORTED)
 lcd_status launch_smooth_quantize(const void* x, int64_t M, int64_t K, int64_t ldx, const float* inv_smooth,
                                   const float* static_scale, uint8_t* act_idx, float* act_scale, void* stream);
+lcd_status launch_smooth_quantize8(const void* x, int64_t M, int64_t K, int64_t ldx, const float* inv_smooth,
+                                   const float* static_scale, int8_t* act_q, float* act_scale, void* stream);
+lcd_status launch_smooth_quantize8_batch(const lcd_act_problem* probs, int count, void* stream);
 lcd_status launch_reference(const Problem& p, void* stream);
 lcd_status launch_smooth_quantize_batch(const lcd_act_problem* probs, int count, void* stream);
 // LCD_ALGO_REGISTER_LUT / LCD_ALGO_BUCKET_LUT for up to LCD_MAX_BATCH problems of equal index width in one launch

@@ -455,6 +455,32 @@ __global__ void __launch_bounds__(256) expand_levels_i8_kernel(const uint8_t* __
   dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
 }
 
+// 8-bit levels (signed bytes, natural column order) in the 2-bit decoder's column order; one thread per quarter.
+__global__ void __launch_bounds__(256) permute_levels_i8_kernel(const uint8_t* __restrict__ act_q, int64_t n_quarters,
+                                                                int8_t* __restrict__ out) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int64_t qi = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (qi >= n_quarters) return;
+  const uint4 a0 = __ldg(reinterpret_cast<const uint4*>(act_q) + 2 * qi);
+  const uint4 a1 = __ldg(reinterpret_cast<const uint4*>(act_q) + 2 * qi + 1);
+  const uint32_t src[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+  uint32_t o[8];
+#pragma unroll
+  for (int v = 0; v < 8; ++v) {
+    uint32_t word = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int p = 4 * v + e;
+      const int col = 16 * (p >> 4) + 8 * ((p >> 2) & 1) + 2 * (p & 3) + ((p >> 3) & 1);
+      word |= ((src[col >> 2] >> (8 * (col & 3))) & 0xffu) << (8 * e);
+    }
+    o[v] = word;
+  }
+  uint4* dst = reinterpret_cast<uint4*>(out + qi * 32);
+  dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+  dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+}
+
 // 2^(e-15) of a row: e is the exponent with max|centroid| < 2^e (the scale of the row's 16-bit fixed point).
 template <int BITS>
 __device__ __forceinline__ float row_exponent_scale(const uint16_t* cb_row, float* up) {
@@ -876,9 +902,14 @@ lcd_status launch_dense_tc(const Problem& p, bool fp16_operands, void* workspace
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int64_t n_quarters = p.M * (p.K_pad / 32);
   const unsigned blocks = (unsigned)((n_quarters + 255) / 256);
+  if (p.act_bits == 8 && fp16_operands) return LCD_ERR_UNSUPPORTED;
   if (!fp16_operands) {
     int8_t* levels = static_cast<int8_t*>(workspace);
-    if (p.bits == 2) expand_levels_i8_kernel<2><<<blocks, 256, 0, s>>>(p.act_idx, n_quarters, levels);
+    if (p.act_bits == 8) {
+      // signed bytes already: the 3-bit decoder's order is the natural one, the 2-bit one needs the permutation
+      if (p.bits == 2) permute_levels_i8_kernel<<<blocks, 256, 0, s>>>(p.act_idx, n_quarters, levels);
+      else levels = const_cast<int8_t*>(reinterpret_cast<const int8_t*>(p.act_idx));
+    } else if (p.bits == 2) expand_levels_i8_kernel<2><<<blocks, 256, 0, s>>>(p.act_idx, n_quarters, levels);
     else expand_levels_i8_kernel<3><<<blocks, 256, 0, s>>>(p.act_idx, n_quarters, levels);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }

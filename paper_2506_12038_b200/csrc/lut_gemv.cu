@@ -48,7 +48,8 @@ constexpr unsigned long long kTimeoutNs = 2000000000ull;   // bounded wait on a 
 struct GemvProblem {
   const uint8_t* items;       // index area
   const uint16_t* codebook;   // [N_pad][2^bits]
-  const uint8_t* act_idx;     // [M][K_pad/2]
+  const uint8_t* act_idx;     // [M][K_pad/2] packed 4-bit levels + 8, or [M][K_pad] signed bytes
+  int act_bits;               // 4 or 8
   const float* act_scale;     // [M]
   float* y;
   int* acc;                   // scratch: [n_rp][MG][planes][4][32] int32, zero on entry and on exit
@@ -193,17 +194,28 @@ __device__ __forceinline__ uint32_t pick_lookup(const RowTables<BITS, KIND>& T, 
 // nibble) as signed bytes, ordered the way the lookups emit weights.  Per 32-column quarter (4 source words):
 //   2 bit: staged words [E(w0) E(w1) O(w0) O(w1) E(w2) E(w3) O(w2) O(w3)], E/O = even/odd columns of a word;
 //   3 bit: natural column order.
+// With 8-bit levels a group of 8 columns is two source words of signed bytes and only the order changes.
 template <int BITS>
-__device__ __forceinline__ void stage_window(uint32_t* dst, const uint32_t* src, int n_words, int tid) {
+__device__ __forceinline__ void stage_window(uint32_t* dst, const uint32_t* src, int n_words, int tid, bool act8) {
   for (int j = tid; j < n_words; j += kThreads) {
-    const uint32_t a = __ldcg(src + j);
-    uint32_t e = a & 0x0f0f0f0fu, o = (a >> 4) & 0x0f0f0f0fu;
-    e = (e + 0x78787878u) ^ 0x80808080u;   // per byte a - 8, no carry between bytes
-    o = (o + 0x78787878u) ^ 0x80808080u;
+    uint32_t e, o;
+    if (act8) {
+      const uint2 a = __ldcg(reinterpret_cast<const uint2*>(src) + j);
+      if (BITS == 2) { e = prmt(a.x, a.y, 0x6420u); o = prmt(a.x, a.y, 0x7531u); }
+      else { e = a.x; o = a.y; }
+    } else {
+      const uint32_t a = __ldcg(src + j);
+      e = a & 0x0f0f0f0fu; o = (a >> 4) & 0x0f0f0f0fu;
+      e = (e + 0x78787878u) ^ 0x80808080u;   // per byte a - 8, no carry between bytes
+      o = (o + 0x78787878u) ^ 0x80808080u;
+    }
     const int quarter = j >> 2, w = j & 3;
     if (BITS == 2) {
       dst[quarter * 8 + (w & 1) + 4 * (w >> 1)] = e;
       dst[quarter * 8 + 2 + (w & 1) + 4 * (w >> 1)] = o;
+    } else if (act8) {
+      dst[quarter * 8 + 2 * w] = e;
+      dst[quarter * 8 + 2 * w + 1] = o;
     } else {
       dst[quarter * 8 + 2 * w] = prmt(e, o, 0x5140u);
       dst[quarter * 8 + 2 * w + 1] = prmt(e, o, 0x7362u);
@@ -611,9 +623,9 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
       const int n_words = (int)geo.panel_width(pn) * 32;
       for (int m = 0; m < n_tok; ++m)
         stage_window<BITS>(reinterpret_cast<uint32_t*>(act_s + wdw * win_bytes + m * P.tstride),
-                           reinterpret_cast<const uint32_t*>(P.act_idx + (size_t)m * P.n_kt * 128 +
-                                                             (size_t)pn * P.pw * 128),
-                           n_words, tid);
+                           reinterpret_cast<const uint32_t*>(P.act_idx + ((size_t)m * P.n_kt * 128 +
+                                                                          (size_t)pn * P.pw * 128) * (P.act_bits == 8 ? 2 : 1)),
+                           n_words, tid, P.act_bits == 8);
     }
     __syncthreads();
 
@@ -779,6 +791,7 @@ lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void*
     g.items = p.tiles;
     g.codebook = p.codebook;
     g.act_idx = p.act_idx;
+    g.act_bits = p.act_bits;
     g.act_scale = p.act_scale;
     g.y = p.y;
     g.ldy = p.ldy;

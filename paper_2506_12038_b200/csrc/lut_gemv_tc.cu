@@ -49,6 +49,7 @@ struct TcProblem {
   int* ticket;     // scratch [n_rt][4 quadrants] int32, zero on entry and on exit
   long long ldy;
   int N, M, n_rp, n_kt, n_rt;
+  int act_bits;    // 4: act_idx is [M][K_pad/2] packed levels + 8; 8: [M][K_pad] signed bytes
   unsigned unit0;  // number of units of the problems before this one
 };
 struct TcBatch {
@@ -436,6 +437,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) lut_gemv_tc_kernel(const TcBatc
     // x 8 pieces): 8 bytes of 4-bit levels become one 16-byte chunk of signed bytes in the lookup order.
     const int tk_token = (32 * quad + lane) >> 3, tk_piece = lane & 7;
     const uint8_t* act_ptr = nullptr;       // this thread's token row (+ piece), null when the problem has no such token
+    bool act8 = false;                      // 8-bit levels: 16 bytes per piece, only their order changes
     asm volatile("griddepcontrol.wait;" ::: "memory");
     uint32_t TH[2] = {0, 0}, TL[2] = {0, 0};
     int tab_p = -1, tab_rt = -1;
@@ -446,7 +448,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) lut_gemv_tc_kernel(const TcBatc
       if (wc.p != tab_p || wc.rt != tab_rt) {
         // byte tables of this thread's row: 16-bit fixed point, high (signed) and low (unsigned) bytes
         tab_p = wc.p; tab_rt = wc.rt;
-        act_ptr = tk_token < P.M ? P.act_idx + (size_t)tk_token * ((size_t)P.n_kt * 128) + tk_piece * 8 : nullptr;
+        act8 = P.act_bits == 8;
+        act_ptr = tk_token < P.M ? P.act_idx + ((size_t)tk_token * ((size_t)P.n_kt * 128) + tk_piece * 8) * (act8 ? 2 : 1)
+                                 : nullptr;
         int n = wc.rt * kTcRows + 32 * quad + lane;
         n = n < P.n_rp * 16 ? n : P.n_rp * 16 - 1;
         const uint16_t* cb = P.codebook + (size_t)n * (1 << BITS);
@@ -465,10 +469,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) lut_gemv_tc_kernel(const TcBatc
         }
         if (BITS == 2) { TH[1] = TH[0]; TL[1] = TL[0]; }
       }
-      uint2 lv[2] = {make_uint2(0u, 0u), make_uint2(0u, 0u)};
+      uint4 lv[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
       if (act_ptr) {
-        lv[0] = __ldg(reinterpret_cast<const uint2*>(act_ptr + (size_t)wc.kt * 128));
-        lv[1] = __ldg(reinterpret_cast<const uint2*>(act_ptr + (size_t)wc.kt * 128 + 64));
+        if (act8) {
+          lv[0] = __ldg(reinterpret_cast<const uint4*>(act_ptr + (size_t)wc.kt * 256));
+          lv[1] = __ldg(reinterpret_cast<const uint4*>(act_ptr + (size_t)wc.kt * 256 + 128));
+        } else {
+          const uint2 a = __ldg(reinterpret_cast<const uint2*>(act_ptr + (size_t)wc.kt * 128));
+          const uint2 b = __ldg(reinterpret_cast<const uint2*>(act_ptr + (size_t)wc.kt * 128 + 64));
+          lv[0].x = a.x; lv[0].y = a.y; lv[1].x = b.x; lv[1].y = b.y;
+        }
       }
       const uint32_t rslot = oi % kTcRing;
       // tcgen05.st below is warp-collective: the whole warp leaves a wait together
@@ -501,18 +511,27 @@ __global__ void __launch_bounds__(kTcThreads, 1) lut_gemv_tc_kernel(const TcBatc
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t a_col = tmem_base + lane_field + slot * kTcACols;
         if (act_ptr) {
-          const uint32_t w0 = lv[h].x, w1 = lv[h].y;
-          const uint32_t e0 = w0 & 0x0f0f0f0fu, o0 = (w0 >> 4) & 0x0f0f0f0fu;
-          const uint32_t e1 = w1 & 0x0f0f0f0fu, o1 = (w1 >> 4) & 0x0f0f0f0fu;
           uint32_t x[4];
-          if (BITS == 2) {      // lookup order of 16 columns: even fields of word 0, of word 1, odd fields of 0, of 1
-            x[0] = e0; x[1] = e1; x[2] = o0; x[3] = o1;
-          } else {              // natural order
-            x[0] = tc_prmt(e0, o0, 0x5140u); x[1] = tc_prmt(e0, o0, 0x7362u);
-            x[2] = tc_prmt(e1, o1, 0x5140u); x[3] = tc_prmt(e1, o1, 0x7362u);
-          }
+          if (act8) {           // signed bytes already; 2 bit: even columns of 0-7, of 8-15, odd of 0-7, of 8-15
+            if (BITS == 2) {
+              x[0] = tc_prmt(lv[h].x, lv[h].y, 0x6420u); x[1] = tc_prmt(lv[h].z, lv[h].w, 0x6420u);
+              x[2] = tc_prmt(lv[h].x, lv[h].y, 0x7531u); x[3] = tc_prmt(lv[h].z, lv[h].w, 0x7531u);
+            } else {
+              x[0] = lv[h].x; x[1] = lv[h].y; x[2] = lv[h].z; x[3] = lv[h].w;
+            }
+          } else {
+            const uint32_t w0 = lv[h].x, w1 = lv[h].y;
+            const uint32_t e0 = w0 & 0x0f0f0f0fu, o0 = (w0 >> 4) & 0x0f0f0f0fu;
+            const uint32_t e1 = w1 & 0x0f0f0f0fu, o1 = (w1 >> 4) & 0x0f0f0f0fu;
+            if (BITS == 2) {    // lookup order of 16 columns: even fields of word 0, of word 1, odd fields of 0, of 1
+              x[0] = e0; x[1] = e1; x[2] = o0; x[3] = o1;
+            } else {            // natural order
+              x[0] = tc_prmt(e0, o0, 0x5140u); x[1] = tc_prmt(e0, o0, 0x7362u);
+              x[2] = tc_prmt(e1, o1, 0x5140u); x[3] = tc_prmt(e1, o1, 0x7362u);
+            }
 #pragma unroll
-          for (int i = 0; i < 4; ++i) x[i] = ((x[i] | 0x80808080u) - 0x08080808u) ^ 0x80808080u;   // level - 8, signed byte
+            for (int i = 0; i < 4; ++i) x[i] = ((x[i] | 0x80808080u) - 0x08080808u) ^ 0x80808080u;   // level - 8
+          }
           uint8_t* row = gen_base + slot * kTcBBytes + (tk_token >> 3) * 1024 + (tk_token & 7) * 128;
           *reinterpret_cast<uint4*>(row + 16 * (tk_piece ^ (tk_token & 7))) = make_uint4(x[0], x[1], x[2], x[3]);
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -653,6 +672,7 @@ lcd_status launch_lut_gemv_tc(const Problem* probs, int count, void* workspace, 
     g.items = p.tiles;
     g.codebook = p.codebook;
     g.act_idx = p.act_idx;
+    g.act_bits = p.act_bits;
     g.act_scale = p.act_scale;
     g.y = p.y;
     g.ldy = p.ldy;

@@ -13,7 +13,8 @@ namespace lcd {
 // CTA = 8 warps = the 8 rows of one row group; lane = token inside a block of 32 tokens.
 __global__ void __launch_bounds__(256)
 reference_kernel(const uint8_t* __restrict__ tiles, const uint16_t* __restrict__ codebook, int64_t N, int64_t K,
-                 int64_t K_pad, int bits, const uint8_t* __restrict__ act_idx, const float* __restrict__ act_scale,
+                 int64_t K_pad, int bits, int act_bits, const uint8_t* __restrict__ act_idx,
+                 const float* __restrict__ act_scale,
                  int64_t M, float* __restrict__ y, int64_t ldy) {
   __shared__ float s_cb[8][8];
   const int g = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -25,13 +26,18 @@ reference_kernel(const uint8_t* __restrict__ tiles, const uint16_t* __restrict__
   __syncwarp();
   const int64_t n_kt = K_pad / kTileK;
   const size_t tile_bytes = (size_t)kTileRows * kTileK * bits / 8;
-  const uint8_t* act_row = act_idx + (m < M ? m : 0) * (K_pad / 2);
+  const uint8_t* act_row = act_idx + (m < M ? m : 0) * (act_bits == 8 ? K_pad : K_pad / 2);
   float acc = 0.0f;
   for (int64_t k = 0; k < K; ++k) {
     const uint8_t* tile = tiles + (((rg >> 1) * n_kt + k / kTileK) * 2 + (rg & 1)) * tile_bytes;
     const uint32_t w = bits == 2 ? tile_index_2bit(tile, g, (int)(k % kTileK)) : tile_index_3bit(tile, g, (int)(k % kTileK));
-    const uint32_t byte = act_row[k >> 1];
-    const int q = (int)((byte >> (4 * (k & 1))) & 15u) - 8;
+    int q;
+    if (act_bits == 8) {
+      q = (int)(int8_t)act_row[k];
+    } else {
+      const uint32_t byte = act_row[k >> 1];
+      q = (int)((byte >> (4 * (k & 1))) & 15u) - 8;
+    }
     acc = fmaf((float)q, s_cb[g][w], acc);
   }
   if (m < M && n < N) y[m * ldy + n] = act_scale[m] * acc;
@@ -40,7 +46,7 @@ reference_kernel(const uint8_t* __restrict__ tiles, const uint16_t* __restrict__
 lcd_status launch_reference(const Problem& p, void* stream) {
   dim3 grid((unsigned)(p.N_pad / kTileRows), (unsigned)((p.M + 31) / 32));
   reference_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-      p.tiles, p.codebook, p.N, p.K, p.K_pad, p.bits, p.act_idx, p.act_scale, p.M, p.y, p.ldy);
+      p.tiles, p.codebook, p.N, p.K, p.K_pad, p.bits, p.act_bits, p.act_idx, p.act_scale, p.M, p.y, p.ldy);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) {
     set_cuda_error((int)e);

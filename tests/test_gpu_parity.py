@@ -310,3 +310,105 @@ def test_full_size_prefill_matrix_sampled_rows(mi):
     assert np.array_equal(a.cpu().numpy(), O.pack_act(q_ref))
     assert torch.isfinite(y).all()
     _sampled_rows_check(L, y, q_ref, s_ref, n_rows=32)
+
+
+# ------------------------------------------------------------------------------- 8-bit activations (b = 8)
+@pytest.mark.parametrize("M,K,ld_extra,use_inv", [(1, 256, 0, True), (3, 1000, 0, True), (5, 4096, 24, False),
+                                                  (2, 250, 3, False), (1, 1, 0, True), (7, 11008, 0, True),
+                                                  (300, 520, 0, False), (33, 264, 8, True)])
+def test_smooth_quantize_8bit_bit_exact(M, K, ld_extra, use_inv):
+    ch = gen.outlier_channels(11, K, 0.01)
+    x = gen.activations(200 + M + K, M, K, ch, 50.0)
+    inv_s = (1.0 / (np.abs(gen.normal(5, K)) * 3 + 0.05)).astype(np.float32) if use_inv else None
+    xd = torch.zeros((M, K + ld_extra), dtype=torch.float16, device="cuda")
+    xd[:, :K] = torch.from_numpy(x).cuda()
+    a, s = lcd.smooth_quantize_act(xd[:, :K], torch.from_numpy(inv_s).cuda() if use_inv else None, act_bits=8)
+    q_ref, s_ref = O.smooth_quantize(x, inv_s, act_bits=8)
+    assert np.array_equal(a.cpu().numpy(), O.pad_act8(q_ref))
+    assert np.array_equal(s.cpu().numpy().view(np.uint32), s_ref.view(np.uint32))
+
+
+def test_smooth_quantize_8bit_static_mode_reaches_minus_128():
+    K = 512
+    xs = (gen.normal(3, 4 * K).reshape(4, K) * 90).astype(np.float16)
+    f = (1.0 / (np.abs(gen.normal(4, K)) + 0.5)).astype(np.float32)
+    sq = torch.tensor([0.37], dtype=torch.float32, device="cuda")
+    a, s = lcd.smooth_quantize_act(torch.from_numpy(xs).cuda(), torch.from_numpy(f).cuda(), static_scale=sq, act_bits=8)
+    q, sr = O.smooth_quantize(xs, f, static_scale=np.float32(0.37), act_bits=8)
+    assert np.array_equal(a.cpu().numpy(), O.pad_act8(q)) and np.array_equal(s.cpu().numpy(), sr)
+    assert q.min() == -128 and q.max() == 127
+
+
+ALGOS_ACT8 = {"reference": 1, "bucket": 2, "register": 3, "tensor": 6}
+
+
+@pytest.mark.parametrize("bits", [2, 3])
+@pytest.mark.parametrize("N,K,M", [(8, 256, 1), (200, 1000, 2), (1031, 520, 5), (64, 4096, 8), (24, 11008, 16),
+                                   (520, 2304, 11), (4096, 4096, 1), (48, 28672, 8)])
+@pytest.mark.parametrize("algo", sorted(ALGOS_ACT8))
+def test_lookup_with_8bit_levels_matches_oracle(bits, N, K, M, algo):
+    # the same kernels with signed-byte levels: only the staging of the token operand differs
+    L = gen.random_case(seed=N + K + M + bits + 8, N=N, K=K, bits=bits, M=M)
+    w = lcd.PackedWeights(lcd.pack_weights(L.idx, L.codebook, L.bits, L.C))
+    a, s = lcd.smooth_quantize_act(torch.from_numpy(L.x).cuda(), torch.from_numpy(L.inv_s).cuda(), act_bits=8)
+    q_ref, s_ref = O.smooth_quantize(L.x, L.inv_s, act_bits=8)
+    assert np.array_equal(a.cpu().numpy(), O.pad_act8(q_ref))
+    word = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    ws = torch.zeros((max(lcd.lut_linear_workspace_bytes(w, M, ALGOS_ACT8[algo]), 256),), dtype=torch.uint8, device="cuda")
+    for _ in range(2):
+        lcd.lut_linear(w, a, s, y=y, algo=ALGOS_ACT8[algo], workspace=ws, status_word=word)
+    torch.cuda.synchronize()
+    assert int(word.item()) == 0
+    if algo != "reference":
+        assert not ws.any()
+    check_y(y, O.lut_linear_dequant(L.idx, L.codebook, q_ref, s_ref), tight=algo != "reference")
+
+
+@pytest.mark.parametrize("bits", [2, 3])
+@pytest.mark.parametrize("N,K,M", [(128, 256, 32), (200, 1000, 17), (1031, 520, 40), (520, 2304, 256),
+                                   (1024, 1024, 513), (4600, 1024, 1000)])
+def test_dense_path_with_8bit_levels_matches_oracle(bits, N, K, M):
+    L = gen.random_case(seed=N + K + M + bits + 8, N=N, K=K, bits=bits, M=M)
+    w = lcd.PackedWeights(lcd.pack_weights(L.idx, L.codebook, L.bits, L.C))
+    a, s = lcd.smooth_quantize_act(torch.from_numpy(L.x).cuda(), torch.from_numpy(L.inv_s).cuda(), act_bits=8)
+    word = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    lcd.lut_linear(w, a, s, y=y, status_word=word)           # AUTO: the int8 tensor-core kernel above 16 tokens
+    torch.cuda.synchronize()
+    assert int(word.item()) == 0
+    q_ref, s_ref = O.smooth_quantize(L.x, L.inv_s, act_bits=8)
+    assert np.array_equal(a.cpu().numpy(), O.pad_act8(q_ref))
+    check_y(y, O.lut_linear_dequant(L.idx, L.codebook, q_ref, s_ref))
+    with pytest.raises(lcd.LcdError):                          # the fp16-operand kernel takes 4-bit levels only
+        lcd.lut_linear(w, a, s, y=y, algo=lcd.ALGO_DENSE_F16)
+
+
+@pytest.mark.parametrize("algo", ["register", "tensor"])
+def test_grouped_launch_with_8bit_levels(algo):
+    algo = lcd.ALGO_REGISTER_LUT if algo == "register" else lcd.ALGO_TC_LUT
+    shapes = [(200, 1000, 1), (4096, 512, 3), (24, 11008, 5), (1031, 520, 1), (8, 256, 8)]
+    for bits in (2, 3):
+        cases = [gen.random_case(seed=37 * i + bits, N=N, K=K, bits=bits, M=M) for i, (N, K, M) in enumerate(shapes)]
+        acts, items, refs = [], [], []
+        for L in cases:
+            w = lcd.PackedWeights(lcd.pack_weights(L.idx, L.codebook, bits))
+            x, inv_s = torch.from_numpy(L.x).cuda(), torch.from_numpy(L.inv_s).cuda()
+            a = torch.empty((L.M, w.K_pad), dtype=torch.int8, device="cuda")
+            sc = torch.empty((L.M,), dtype=torch.float32, device="cuda")
+            y = torch.full((L.M, L.N), float("nan"), dtype=torch.float32, device="cuda")
+            acts.append((x, inv_s, a, sc))
+            items.append((w, a, sc, y))
+            q_ref, s_ref = O.smooth_quantize(L.x, L.inv_s, act_bits=8)
+            refs.append((q_ref, s_ref, O.lut_linear_dequant(L.idx, L.codebook, q_ref, s_ref)))
+        word = torch.zeros((1,), dtype=torch.int32, device="cuda")
+        qb, lb = lcd.ActBatch(acts), lcd.LinearBatch(items, algo=algo, status_word=word)
+        for _ in range(2):
+            qb.run()
+            lb.run()
+        torch.cuda.synchronize()
+        assert int(word.item()) == 0 and not lb.workspace.any()
+        for (w, a, sc, y), (q_ref, s_ref, y_ref) in zip(items, refs):
+            assert np.array_equal(a.cpu().numpy(), O.pad_act8(q_ref))
+            assert np.array_equal(sc.cpu().numpy(), s_ref)
+            check_y(y, y_ref)

@@ -96,8 +96,17 @@ def test_device_entry_points_reject_bad_arguments_before_any_launch():
     assert lib.lcd_smooth_quantize_act(None, 1, 8, 8, None, None, 4, None, None, None) == 1
     fake = ctypes.c_void_p(4096)
     assert lib.lcd_smooth_quantize_act(fake, 1, 8, 4, None, None, 4, fake, fake, None) == 1      # ldx < K
-    assert lib.lcd_smooth_quantize_act(fake, 1, 8, 8, None, None, 8, fake, fake, None) == 2      # act_bits
+    assert lib.lcd_smooth_quantize_act(fake, 1, 8, 8, None, None, 5, fake, fake, None) == 2      # act_bits: 4 or 8
+    assert lib.lcd_lut_linear_act8(None, hdr, None, None, 1, None, 8, 0, None, 0, None, None) == 1
     assert lib.lcd_lut_linear(fake, hdr, fake, fake, 1, fake, 4, 0, None, 0, None, None) == 1     # ldy < N
     assert lib.lcd_lut_linear(ctypes.c_void_p(4100), hdr, fake, fake, 1, fake, 8, 1, None, 0, None, None) == 1
     assert lib.lcd_lut_linear(fake, hdr, fake, fake, 17, fake, 8, 3, None, 0, None, None) == 2    # M > 16
     assert lib.lcd_linear_host(fake, hdr, fake, 1, None, fake, fake, 16, None) == 3               # scratch small
+
+
+def test_every_export_declares_its_argument_types():
+    # an undeclared prototype makes ctypes pass Python ints as 32-bit values: 64-bit sizes and strides arrive wrong
+    from paper_2506_12038_b200 import binding
+    for name in binding.EXPORTS:
+        if name != "lcd_last_cuda_error":
+            assert getattr(binding.lib, name).argtypes, name
