@@ -56,6 +56,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--act-bits", type=int, default=4, choices=[4, 8],
                     help="activation levels: 4 bit (the benchmark configurations) or 8 bit (the paper's b = 8)")
+    ap.add_argument("--two-call", action="store_true",
+                    help="M <= 16: quantise and look up in two launches per layer instead of the fused one")
     ap.add_argument("--algo", default="auto", choices=["auto", "register", "bucket", "tensor"],
                     help="lookup kernel for M <= 16 (default: the library's choice)")
     return ap.parse_args()
@@ -257,9 +259,21 @@ def run_ours(args):
         single = [[lcd.LinearBatch([(mt["w"][c], mt["a"], mt["s"], mt["y"])], algo=algo, status_word=status)
                    for c in range(copies)] for mt in mats]
 
+        # default: ONE launch per layer, the lookup kernel does the input transformation itself (4-bit levels, the
+        # register or bucket kernel); --two-call, 8-bit levels and the tensor-memory kernel: quantise, then look up
+        # (M = 1 only: with more tokens every CTA would repeat the transformation of all tokens, measured slower)
+        fused = (not args.two_call) and args.act_bits == 4 and args.algo != "tensor" and M == 1
+        if fused:
+            fbatch = [lcd.FusedBatch([(mt["w"][c], mt["x"], mt["inv_s"], mt["y"]) for mt in mats], algo=algo,
+                                     status_word=status) for c in range(copies)]
+            qbatch.run()          # the per-matrix lookup-only timings below use the stored levels
+
         def step(c):
-            qbatch.run()
-            lbatch[c].run()
+            if fused:
+                fbatch[c].run()
+            else:
+                qbatch.run()
+                lbatch[c].run()
 
         def lookup_only(mi, c):
             single[mi][c].run()
@@ -274,7 +288,7 @@ def run_ours(args):
             mt = mats[mi]
             lcd.lut_linear(mt["w"][c], mt["a"], mt["s"], y=mt["y"], workspace=mt["work"], status_word=status)
 
-    launches_per_step = 2 if grouped else 2 * len(mats)
+    launches_per_step = (1 if fused else 2) if grouped else 2 * len(mats)
     stream = torch.cuda.Stream(device=dev)
     with torch.cuda.stream(stream):
         for c in range(copies):
@@ -287,8 +301,15 @@ def run_ours(args):
             with torch.cuda.graph(g, stream=stream):
                 step(c)
             graphs.append(g)
+        # and one graph of `copies` consecutive steps (a model runs its layers back to back): the timed loop replays
+        # it for every full round of copies and finishes the remainder with the single-step graphs
+        round_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(round_graph, stream=stream):
+            for c in range(copies):
+                step(c)
         for i in range(max(args.warmup, 3)):
             graphs[i % copies].replay()
+        round_graph.replay()
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
@@ -297,8 +318,10 @@ def run_ours(args):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         e0.record()
-        for i in range(args.steps):
-            graphs[i % copies].replay()
+        for i in range(args.steps // copies):
+            round_graph.replay()
+        for i in range(args.steps % copies):
+            graphs[i].replay()
         e1.record()
         torch.cuda.synchronize()
         ms_total = e0.elapsed_time(e1)
@@ -332,7 +355,12 @@ def run_ours(args):
                                "GBps": mt["bytes"] / ms / 1e6, "TFLOPs_equiv": mt["flop"] / ms / 1e9})
         kern_bytes = sum(mt["bytes"] for mt in mats)
         kern_flop = sum(mt["flop"] for mt in mats)
-        if grouped:
+        if grouped and fused:
+            kern_ms = time_graph(lambda: [fbatch[c].run() for _ in range(reps) for c in range(copies)], reps * copies)
+            kern_name = "lut_gemv_kernel, one launch per layer: input transformation + lookup of all its matrices"
+            # the launch reads x (fp16) and the smoothing factors instead of stored levels and scales
+            kern_bytes += sum(M * mt["L"].K * 2 + mt["L"].K * 4 - M * (mt["L"].K / 2 + 4) for mt in mats)
+        elif grouped:
             kern_ms = time_graph(lambda: [lbatch[c].run() for _ in range(reps) for c in range(copies)], reps * copies)
             kern_name = "lut_gemv_kernel, one grouped launch over the layer's matrices"
         else:
@@ -431,8 +459,10 @@ def run_ours(args):
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
             "vs_baseline": None, "dtype": "s8 table bytes x s8 levels -> s32 (int8 MMA), f32 epilogue" if not tensor_bound else "s8 table bytes x s8 levels -> s32 (tcgen05 kind::i8), f32 epilogue",
             "data": "synthetic", "config": dict(workload_config(args.config, M, copies, args.act_bits),
-                                                launches="1 grouped quantise + 1 grouped lookup per layer" if grouped
-                                                else "per matrix: quantise + lookup"),
+                                                graphs=f"steps replayed as CUDA graphs of {copies} consecutive steps",
+                                                launches=("1 launch per layer: quantise + lookup fused" if grouped and fused
+                                                          else "1 grouped quantise + 1 grouped lookup per layer" if grouped
+                                                          else "per matrix: quantise + lookup")),
             "layer_GBps": layer_alg_bytes * world / (ms_step * 1e-3) / 1e9,
             "layer_algorithmic_bytes": layer_alg_bytes,
             "TFLOPs_equiv": sum(mt["flop"] for mt in mats) * world / (ms_step * 1e-3) / 1e12,

@@ -210,6 +210,35 @@ lcd_status lcd_lut_linear_batch_act8(const lcd_linear_problem* problems /* host 
                                 void* cuda_stream);
 
 /* ----------------------------------------------------------------------------------------------
+ * Online steps 1+2+3 in one launch for up to LCD_MAX_BATCH independent problems with M <= 16 (the projections
+ * of one decoder layer at decode time): the lookup kernel performs the input transformation of Section 4.1
+ * itself (dynamic per-token scale, 4-bit levels, the operation sequence of lcd_smooth_quantize_act, so the
+ * levels and therefore y are bit-identical to the two-call path) while its first weights are already streaming,
+ * and never writes the levels or scales to memory.
+ *   x_fp16:     device, binary16 [M][ldx], ldx >= K of the blob;
+ *   inv_smooth: device fp32 [K] or NULL;
+ *   algo:       LCD_ALGO_AUTO, REGISTER_LUT or BUCKET_LUT;
+ *   workspace:  as lcd_lut_linear_batch (same size: lcd_linear_fused_batch_workspace_bytes; zero-filled
+ *               before first use, left zero-filled).
+ * -------------------------------------------------------------------------------------------- */
+typedef struct {
+  const void* packed_weights_dev; /* device, 256-byte aligned */
+  const void* header_host;        /* host, the blob's first 64 bytes */
+  const void* x_fp16;             /* device */
+  int64_t M, ldx;
+  const float* inv_smooth;        /* device or NULL */
+  float* y;                       /* device out, fp32 [M][ldy] */
+  int64_t ldy;
+} lcd_fused_problem;
+
+lcd_status lcd_linear_fused_batch_workspace_bytes(const lcd_fused_problem* problems /* host */, int count,
+                                                  lcd_algo algo, size_t* bytes);
+
+lcd_status lcd_linear_fused_batch(const lcd_fused_problem* problems /* host */, int count, lcd_algo algo,
+                                  void* workspace, size_t workspace_bytes, int32_t* status_word_dev,
+                                  void* cuda_stream);
+
+/* ----------------------------------------------------------------------------------------------
  * lcd_lut_linear for M <= 16 without a caller-provided workspace.  (No counterpart in the paper: this is a
  * convenience of the library.)
  *

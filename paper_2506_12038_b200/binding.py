@@ -27,8 +27,14 @@ EXPORTS = ["lcd_status_string", "lcd_last_cuda_error", "lcd_packed_weights_bytes
            "lcd_linear_host_scratch_bytes", "lcd_linear_host", "lcd_smooth_quantize_act_batch",
            "lcd_lut_linear_batch_workspace_bytes", "lcd_lut_linear_batch", "lcd_lut_linear_static",
            "lcd_linear_host_batch_sizes", "lcd_linear_host_batch", "lcd_lut_linear_act8",
-           "lcd_lut_linear_batch_act8"]
+           "lcd_lut_linear_batch_act8", "lcd_linear_fused_batch_workspace_bytes", "lcd_linear_fused_batch"]
 STATIC_SCRATCH_BYTES = 4 << 20
+
+
+class FusedProblem(Structure):
+    """lcd_fused_problem"""
+    _fields_ = [("packed_weights_dev", c_void_p), ("header_host", c_void_p), ("x_fp16", c_void_p), ("M", c_int64),
+                ("ldx", c_int64), ("inv_smooth", c_void_p), ("y", c_void_p), ("ldy", c_int64)]
 
 
 class ActProblem(Structure):
@@ -73,6 +79,8 @@ def _load() -> ctypes.CDLL:
     lib.lcd_lut_linear.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_int64, c_int,
                                    c_void_p, c_size_t, c_void_p, c_void_p]
     lib.lcd_lut_linear_act8.argtypes = lib.lcd_lut_linear.argtypes
+    lib.lcd_linear_fused_batch_workspace_bytes.argtypes = [POINTER(FusedProblem), c_int, c_int, POINTER(c_size_t)]
+    lib.lcd_linear_fused_batch.argtypes = [POINTER(FusedProblem), c_int, c_int, c_void_p, c_size_t, c_void_p, c_void_p]
     lib.lcd_lut_linear_batch_act8.argtypes = [POINTER(LinearProblem), c_int, c_int, c_void_p, c_size_t, c_void_p, c_void_p]
     lib.lcd_linear_host_scratch_bytes.argtypes = [c_void_p, c_int64, POINTER(c_size_t)]
     lib.lcd_linear_host.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_size_t,
@@ -254,6 +262,35 @@ class ActBatch:
     def run(self, stream=None):
         _check(lib.lcd_smooth_quantize_act_batch(self.arr, self.count, self.act_bits, _stream_ptr(stream)),
                "lcd_smooth_quantize_act_batch")
+
+
+class FusedBatch:
+    """Up to MAX_BATCH independent problems (M <= 16) in ONE launch that quantises the activations and runs the
+    lookup: items are (PackedWeights, x fp16 [M,K] CUDA, inv_smooth or None, y fp32 [M,N] CUDA)."""
+
+    def __init__(self, items, algo: int = ALGO_AUTO, status_word=None):
+        import torch
+        self._keep = list(items)
+        self.count = len(self._keep)
+        self.algo = algo
+        self.arr = (FusedProblem * self.count)()
+        for a, (w, x, inv_s, y) in zip(self.arr, self._keep):
+            assert x.dtype == torch.float16 and x.stride(1) == 1 and y.dtype == torch.float32
+            a.packed_weights_dev, a.header_host = w.dev.data_ptr(), w.header_ptr
+            a.x_fp16, a.M, a.ldx = x.data_ptr(), x.shape[0], x.stride(0)
+            a.inv_smooth = inv_s.data_ptr() if inv_s is not None else None
+            a.y, a.ldy = y.data_ptr(), y.stride(0)
+        need = c_size_t(0)
+        _check(lib.lcd_linear_fused_batch_workspace_bytes(self.arr, self.count, algo, byref(need)),
+               "lcd_linear_fused_batch_workspace_bytes")
+        self.workspace = torch.zeros(max(need.value, 256), dtype=torch.uint8, device=self._keep[0][1].device)
+        self.status_word = status_word
+
+    def run(self, stream=None):
+        _check(lib.lcd_linear_fused_batch(self.arr, self.count, self.algo, c_void_p(self.workspace.data_ptr()),
+                                          self.workspace.numel(),
+                                          c_void_p(self.status_word.data_ptr()) if self.status_word is not None else None,
+                                          _stream_ptr(stream)), "lcd_linear_fused_batch")
 
 
 class LinearBatch:

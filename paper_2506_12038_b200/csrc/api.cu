@@ -266,6 +266,61 @@ extern "C" lcd_status lcd_lut_linear_act8(const void* packed_weights_dev, const 
   }
 }
 
+static lcd_status fused_problems(const lcd_fused_problem* problems, int count, lcd_algo algo, bool pointers,
+                                 Problem* p, lcd_algo* resolved) {
+  if (!problems || count < 1 || count > LCD_MAX_BATCH) return LCD_ERR_INVALID_ARG;
+  if (algo != LCD_ALGO_AUTO && algo != LCD_ALGO_REGISTER_LUT && algo != LCD_ALGO_BUCKET_LUT) return LCD_ERR_UNSUPPORTED;
+  *resolved = algo == LCD_ALGO_AUTO ? LCD_ALGO_REGISTER_LUT : algo;
+  for (int i = 0; i < count; ++i) {
+    const lcd_fused_problem& q = problems[i];
+    if (q.M < 1 || !q.header_host) return LCD_ERR_INVALID_ARG;
+    if (q.M > 16) return LCD_ERR_UNSUPPORTED;
+    if (!shape_problem(q.header_host, q.M, &p[i])) return LCD_ERR_BAD_BLOB;
+    if (p[i].bits != p[0].bits) return LCD_ERR_UNSUPPORTED;
+    p[i].act_bits = 16;
+    if (!pointers) continue;
+    if (!q.packed_weights_dev || !q.x_fp16 || !q.y || q.ldx < p[i].K || q.ldy < p[i].N) return LCD_ERR_INVALID_ARG;
+    if (!aligned(q.packed_weights_dev, 256) || !aligned(q.x_fp16, 2) || !aligned(q.y, 4) ||
+        (q.inv_smooth && !aligned(q.inv_smooth, 4)))
+      return LCD_ERR_INVALID_ARG;
+    Header h;
+    parse_header(q.header_host, &h);
+    const uint8_t* blob = static_cast<const uint8_t*>(q.packed_weights_dev);
+    p[i].tiles = blob + h.index_offset;
+    p[i].codebook = reinterpret_cast<const uint16_t*>(blob + h.codebook_offset);
+    p[i].x_fp16 = q.x_fp16;
+    p[i].ldx = q.ldx;
+    p[i].inv_smooth = q.inv_smooth;
+    p[i].y = q.y;
+    p[i].ldy = q.ldy;
+  }
+  return LCD_OK;
+}
+
+extern "C" lcd_status lcd_linear_fused_batch_workspace_bytes(const lcd_fused_problem* problems, int count,
+                                                             lcd_algo algo, size_t* bytes) {
+  Problem p[LCD_MAX_BATCH];
+  lcd_algo resolved;
+  const lcd_status st = fused_problems(problems, count, algo, false, p, &resolved);
+  if (st != LCD_OK) return st;
+  if (!bytes) return LCD_ERR_INVALID_ARG;
+  *bytes = lut_gemv_workspace_bytes(p, count, resolved);
+  return LCD_OK;
+}
+
+extern "C" lcd_status lcd_linear_fused_batch(const lcd_fused_problem* problems, int count, lcd_algo algo,
+                                             void* workspace, size_t workspace_bytes, int32_t* status_word_dev,
+                                             void* cuda_stream) {
+  Problem p[LCD_MAX_BATCH];
+  lcd_algo resolved;
+  const lcd_status st = fused_problems(problems, count, algo, true, p, &resolved);
+  if (st != LCD_OK) return st;
+  const size_t need = lut_gemv_workspace_bytes(p, count, resolved);
+  if (!workspace || workspace_bytes < need) return LCD_ERR_BUFFER_TOO_SMALL;
+  if (!aligned(workspace, 256)) return LCD_ERR_INVALID_ARG;
+  return launch_lut_gemv(p, count, resolved, workspace, workspace_bytes, status_word_dev, cuda_stream);
+}
+
 // ---- host-buffer path -------------------------------------------------------------------------------
 namespace {
 struct HostScratch {
@@ -414,8 +469,22 @@ extern "C" lcd_status lcd_linear_host_batch(const lcd_host_problem* problems, in
                       problems[i].M, reinterpret_cast<float*>(base + L.y_off[i]), shapes[i].N, &p[i]);
     if (st != LCD_OK) return st;
   }
-  st = lcd_smooth_quantize_act_batch(acts, count, LCD_ACT_BITS, cuda_stream);
-  if (st != LCD_OK) return st;
+  // Single tokens: the lookup kernel does the input transformation itself (one launch less, the levels are never
+  // written to memory).  With more tokens every CTA would repeat the transformation of all of them, which costs
+  // more than the separate launch (measured), so that launch stays.
+  bool single_tokens = true;
+  for (int i = 0; i < count; ++i) single_tokens = single_tokens && problems[i].M == 1;
+  if (single_tokens) {
+    for (int i = 0; i < count; ++i) {
+      p[i].act_bits = 16;
+      p[i].x_fp16 = acts[i].x_fp16;
+      p[i].ldx = acts[i].ldx;
+      p[i].inv_smooth = acts[i].inv_smooth;
+    }
+  } else {
+    st = lcd_smooth_quantize_act_batch(acts, count, LCD_ACT_BITS, cuda_stream);
+    if (st != LCD_OK) return st;
+  }
   e = cudaMemsetAsync(base + L.ws_off, 0, L.ws_bytes, stream);    // the lookup kernel wants its scratch zero-filled
   if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
   st = launch_lut_gemv(p, count, LCD_ALGO_REGISTER_LUT, base + L.ws_off, L.ws_bytes, nullptr, cuda_stream);

@@ -41,7 +41,10 @@ struct Problem {
   int64_t N, K, K_pad, N_pad;
   int bits, C;
   const uint8_t* act_idx;   // device [M][K_pad/2] (4-bit levels + 8) or [M][K_pad] signed bytes (act_bits == 8)
-  int act_bits = 4;         // 4 or 8
+  int act_bits = 4;         // 4 or 8; 16 = not quantised yet: the lookup kernel does Section 4.1 itself from x
+  const void* x_fp16 = nullptr;       // act_bits == 16: device fp16 [M][ldx]
+  int64_t ldx = 0;
+  const float* inv_smooth = nullptr;  // act_bits == 16: device fp32 [K] or null
   const float* act_scale;   // device [M]
   int64_t M;
   float* y;

@@ -49,7 +49,12 @@ struct GemvProblem {
   const uint8_t* items;       // index area
   const uint16_t* codebook;   // [N_pad][2^bits]
   const uint8_t* act_idx;     // [M][K_pad/2] packed 4-bit levels + 8, or [M][K_pad] signed bytes
-  int act_bits;               // 4 or 8
+  int act_bits;               // 4 or 8; 16: quantise x here (Section 4.1, dynamic per-token scale)
+  const __half* x;            // act_bits == 16: [M][ldx] fp16
+  const float* inv_smooth;    // act_bits == 16: [K] or null
+  long long ldx;
+  int K;                      // columns of x
+  int x_vec;                  // rows of x and inv_smooth allow 16-byte loads and K % 8 == 0
   const float* act_scale;     // [M]
   float* y;
   int* acc;                   // scratch: [n_rp][MG][planes][4][32] int32, zero on entry and on exit
@@ -219,6 +224,57 @@ __device__ __forceinline__ void stage_window(uint32_t* dst, const uint32_t* src,
     } else {
       dst[quarter * 8 + 2 * w] = prmt(e, o, 0x5140u);
       dst[quarter * 8 + 2 * w + 1] = prmt(e, o, 0x7362u);
+    }
+  }
+}
+
+// The same window straight from the fp16 activations (input transformation of Section 4.1 fused into the lookup
+// kernel): level = clip(rint((x * inv_s) * r)), r = 7 / A with A the token's max |x * inv_s| (found beforehand),
+// every step one binary32 operation as in quantize.cu, so the levels are the ones that kernel would write.
+// k0: first column of the window; columns >= K are level 0.
+template <int BITS>
+__device__ __forceinline__ void stage_window_from_x(uint32_t* dst, const __half* xr, const float* inv_smooth, int k0,
+                                                    int K, bool vec, float r, int n_words, int tid) {
+  for (int j = tid; j < n_words; j += kThreads) {
+    const int k = k0 + 8 * j;
+    float tv[8];
+    if (vec && k < K) {
+      const uint4 raw = *reinterpret_cast<const uint4*>(xr + k);
+      const __half2* h = reinterpret_cast<const __half2*>(&raw);
+      float f[8];
+      if (inv_smooth) {
+        const float4 a = __ldg(reinterpret_cast<const float4*>(inv_smooth + k));
+        const float4 b = __ldg(reinterpret_cast<const float4*>(inv_smooth + k + 4));
+        f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) f[i] = 1.0f;
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 v = __half22float2(h[i]);
+        tv[2 * i] = __fmul_rn(v.x, f[2 * i]);
+        tv[2 * i + 1] = __fmul_rn(v.y, f[2 * i + 1]);
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        tv[i] = k + i < K ? __fmul_rn(__half2float(xr[k + i]), inv_smooth ? __ldg(inv_smooth + k + i) : 1.0f) : 0.0f;
+    }
+    uint32_t b[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      float q = rintf(__fmul_rn(tv[i], r));
+      q = fminf(fmaxf(q, -8.0f), 7.0f);
+      b[i] = (uint32_t)(int)q & 0xffu;
+    }
+    const int quarter = j >> 2, w = j & 3;
+    if (BITS == 2) {
+      dst[quarter * 8 + (w & 1) + 4 * (w >> 1)] = b[0] | (b[2] << 8) | (b[4] << 16) | (b[6] << 24);
+      dst[quarter * 8 + 2 + (w & 1) + 4 * (w >> 1)] = b[1] | (b[3] << 8) | (b[5] << 16) | (b[7] << 24);
+    } else {
+      dst[quarter * 8 + 2 * w] = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
+      dst[quarter * 8 + 2 * w + 1] = b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24);
     }
   }
 }
@@ -481,6 +537,50 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
   next_b = load_codebook<BITS>(P.codebook + ((size_t)next_rp * 16 + 8 + g) * (1 << BITS));
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
+  // act_bits == 16: the tokens' maxima A = max_k |x_k * inv_s_k| first (each CTA for itself; x is a few KB in L2)
+  const bool fused = P.act_bits == 16;
+  float* s_amax = reinterpret_cast<float*>(smem + kWarps * kMaxDepth * 8);   // 16 floats between barriers and tickets
+  if (fused) {
+    float* part = reinterpret_cast<float*>(act_s);                            // [kWarps][16], before the windows exist
+    for (int m = 0; m < n_tok; ++m) {
+      const __half* xr = P.x + (size_t)m * P.ldx;
+      float amax = 0.0f;
+      if (P.x_vec) {
+        for (int k = tid * 8; k < P.K; k += kThreads * 8) {
+          const uint4 raw = *reinterpret_cast<const uint4*>(xr + k);
+          const __half2* h = reinterpret_cast<const __half2*>(&raw);
+          float f[8];
+          if (P.inv_smooth) {
+            const float4 a = __ldg(reinterpret_cast<const float4*>(P.inv_smooth + k));
+            const float4 b = __ldg(reinterpret_cast<const float4*>(P.inv_smooth + k + 4));
+            f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+          } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) f[i] = 1.0f;
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float2 v = __half22float2(h[i]);
+            amax = fmaxf(amax, fmaxf(fabsf(__fmul_rn(v.x, f[2 * i])), fabsf(__fmul_rn(v.y, f[2 * i + 1]))));
+          }
+        }
+      } else {
+        for (int k = tid; k < P.K; k += kThreads)
+          amax = fmaxf(amax, fabsf(__fmul_rn(__half2float(xr[k]), P.inv_smooth ? __ldg(P.inv_smooth + k) : 1.0f)));
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+      if (lane == 0) part[warp * 16 + m] = amax;
+    }
+    __syncthreads();
+    if (tid < n_tok) {
+      float v = 0.0f;
+      for (int w = 0; w < kWarps; ++w) v = fmaxf(v, part[w * 16 + tid]);
+      s_amax[tid] = v;
+    }
+    __syncthreads();
+  }
+
   int acc[MG][PL][4];
 #pragma unroll
   for (int G = 0; G < MG; ++G)
@@ -515,7 +615,14 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
 #pragma unroll
             for (int p = 0; p < PL - 1; ++p) v = fmaf(T.c[p + 1], (float)acc[G][p][r], v);
           }
-          P.y[(size_t)m * P.ldy + n] = v * __ldg(P.act_scale + m);
+          float sq;
+          if (fused) {
+            const float A = s_amax[m];
+            sq = A > 0.0f ? __fdiv_rn(A, 7.0f) : 1.0f;
+          } else {
+            sq = __ldg(P.act_scale + m);
+          }
+          P.y[(size_t)m * P.ldy + n] = v * sq;
         }
       }
   };
@@ -621,11 +728,18 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
     for (uint32_t wdw = 0; wdw < 2 && pbase + wdw <= pB; ++wdw) {
       const uint32_t pn = pbase + wdw;
       const int n_words = (int)geo.panel_width(pn) * 32;
-      for (int m = 0; m < n_tok; ++m)
-        stage_window<BITS>(reinterpret_cast<uint32_t*>(act_s + wdw * win_bytes + m * P.tstride),
-                           reinterpret_cast<const uint32_t*>(P.act_idx + ((size_t)m * P.n_kt * 128 +
-                                                                          (size_t)pn * P.pw * 128) * (P.act_bits == 8 ? 2 : 1)),
-                           n_words, tid, P.act_bits == 8);
+      for (int m = 0; m < n_tok; ++m) {
+        uint32_t* dst = reinterpret_cast<uint32_t*>(act_s + wdw * win_bytes + m * P.tstride);
+        if (fused) {
+          const float A = s_amax[m];
+          stage_window_from_x<BITS>(dst, P.x + (size_t)m * P.ldx, P.inv_smooth, (int)(pn * P.pw) * 256, P.K,
+                                    P.x_vec != 0, A > 0.0f ? __fdiv_rn(7.0f, A) : 0.0f, n_words, tid);
+        } else {
+          stage_window<BITS>(dst, reinterpret_cast<const uint32_t*>(P.act_idx + ((size_t)m * P.n_kt * 128 +
+                                                                                 (size_t)pn * P.pw * 128) * (P.act_bits == 8 ? 2 : 1)),
+                             n_words, tid, P.act_bits == 8);
+        }
+      }
     }
     __syncthreads();
 
@@ -792,6 +906,12 @@ lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void*
     g.codebook = p.codebook;
     g.act_idx = p.act_idx;
     g.act_bits = p.act_bits;
+    g.x = static_cast<const __half*>(p.x_fp16);
+    g.inv_smooth = p.inv_smooth;
+    g.ldx = p.ldx;
+    g.K = (int)p.K;
+    g.x_vec = (p.K % 8 == 0) && (p.ldx % 8 == 0) && ((reinterpret_cast<uintptr_t>(p.x_fp16) & 15) == 0) &&
+              (!p.inv_smooth || (reinterpret_cast<uintptr_t>(p.inv_smooth) & 15) == 0);
     g.act_scale = p.act_scale;
     g.y = p.y;
     g.ldy = p.ldy;
@@ -822,6 +942,8 @@ lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void*
     g.tstride = pw * 256 + 16;
     const size_t need = (n_panels == 1 ? 1 : 2) * m_eff * (size_t)g.tstride;
     act_bytes = need > act_bytes ? need : act_bytes;
+    // act_bits == 16: the window area first holds the warps' partial maxima, kWarps x 16 floats
+    if (p.act_bits == 16 && act_bytes < (size_t)kWarps * 16 * sizeof(float)) act_bytes = (size_t)kWarps * 16 * sizeof(float);
   }
   // CTAs per problem: one each, then one more at a time to the problem whose most loaded CTA has the most
   // items (a CTA owns whole runs), until every SM has one

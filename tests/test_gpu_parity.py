@@ -412,3 +412,40 @@ def test_grouped_launch_with_8bit_levels(algo):
             assert np.array_equal(a.cpu().numpy(), O.pad_act8(q_ref))
             assert np.array_equal(sc.cpu().numpy(), s_ref)
             check_y(y, y_ref)
+
+
+# ------------------------------------------------------------------------------- steps 1+2+3 in one launch
+@pytest.mark.parametrize("bits", [2, 3])
+@pytest.mark.parametrize("algo", ["register", "bucket"])
+def test_fused_launch_equals_two_call_path_and_oracle(bits, algo):
+    # the lookup kernel quantises x itself: same binary32 steps, so y must equal the two-call result bit for bit
+    algo = lcd.ALGO_REGISTER_LUT if algo == "register" else lcd.ALGO_BUCKET_LUT
+    shapes = [(200, 1000, 1), (4096, 512, 3), (24, 11008, 5), (1031, 520, 1), (8, 256, 8), (40, 250, 2),   # 250: unaligned rows
+              (48, 28672, 16)]                                                                           # column panels
+    cases = [gen.random_case(seed=41 * i + bits, N=N, K=K, bits=bits, M=M) for i, (N, K, M) in enumerate(shapes)]
+    cases[0].x[0, :] = 0                                    # an all-zero token: scale 1, levels 0
+    items, two_call, refs = [], [], []
+    for L in cases:
+        w = lcd.PackedWeights(lcd.pack_weights(L.idx, L.codebook, bits))
+        x, inv_s = torch.from_numpy(L.x).cuda(), torch.from_numpy(L.inv_s).cuda()
+        y = torch.full((L.M, L.N), float("nan"), dtype=torch.float32, device="cuda")
+        items.append((w, x, inv_s, y))
+        a, s = lcd.smooth_quantize_act(x, inv_s)
+        two_call.append(lcd.lut_linear(w, a, s, algo=algo))
+        q_ref, s_ref = O.smooth_quantize(L.x, L.inv_s)
+        refs.append(O.lut_linear_dequant(L.idx, L.codebook, q_ref, s_ref))
+    word = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    fb = lcd.FusedBatch(items, algo=algo, status_word=word)
+    for _ in range(2):
+        fb.run()
+    torch.cuda.synchronize()
+    assert int(word.item()) == 0 and not fb.workspace.any()
+    for (w, x, inv_s, y), y2, y_ref in zip(items, two_call, refs):
+        assert torch.equal(y, y2)
+        check_y(y, y_ref)
+    # without smoothing factors
+    w, x, _, y = items[3]
+    fb1 = lcd.FusedBatch([(w, x, None, y)], algo=algo)
+    fb1.run()
+    a, s = lcd.smooth_quantize_act(x, None)
+    assert torch.equal(y, lcd.lut_linear(w, a, s, algo=algo))
