@@ -33,8 +33,8 @@ from synth import gen  # noqa: E402
 # captures summarised under profiles/, with the hash of the kernel source they were taken from: a kernel that has
 # changed since reports traffic = null.
 NCU_TRAFFIC = {
-    # profiles/lut_gemv_kernel_llama7b_2bit_m1.md: one grouped launch of configs[1] at M = 1
-    ("lut_gemv.cu", 1, 1): {"sha256": "de7a82c50470678c2fc5e025fcd3f24651cc60a378eb37fd777b3b5d63b3c890", "bytes_per_launch": 50991104 + 18944},
+    # profiles/lut_gemv_kernel_llama7b_2bit_m1.md: one launch (input transformation + lookup) of configs[1] at M = 1
+    ("lut_gemv.cu", 1, 1): {"sha256": "f70147331c8c03633db381b6d1ea74859aa012a5b041f6b0040f376d05dfe0ce", "bytes_per_launch": 51196416 + 17408},
     # profiles/dense_tc_kernel_llama13b_2bit_m2048.md: the layer's seven launches of configs[3]: q captured
     # (17.11 + 0.23 MB, taken four times for q/k/v/o), gate captured (28.36 + 56.16 MB, twice for gate/up), down
     # scaled from q by its 2.7 times longer rows (same tiles, traffic in proportion to K)
