@@ -397,3 +397,41 @@ def unpack_weights(blob: np.ndarray):
     cbp = blob[h["codebook_offset"]:h["codebook_offset"] + N_pad * (1 << bits) * 2].view(np.float16)
     cbp = cbp.reshape(N_pad, 1 << bits)
     return P[:N, :K].copy(), cbp[:N, :C].copy(), bits, C
+
+
+# --------------------------------------------------------------------------------------
+# Section 3.4 - adaptive smoothing search (offline; needs only a calibration batch)
+# --------------------------------------------------------------------------------------
+def smoothing_factors(xmax, wmax, alpha: float) -> np.ndarray:
+    """Per-input-channel smoothing factors for migration strength alpha:
+    s_k = xmax_k^alpha / wmax_k^(1-alpha), clamped to [1e-5, 1e5]; a channel whose activation or weight maximum
+    is zero keeps s_k = 1.  Computed in binary64 and rounded once to binary32 (what the kernels consume)."""
+    xm = np.asarray(xmax, dtype=np.float64)
+    wm = np.asarray(wmax, dtype=np.float64)
+    ok = (xm > 0) & (wm > 0)
+    s = np.ones_like(xm)
+    s[ok] = np.power(xm[ok], alpha) / np.power(wm[ok], 1.0 - alpha)
+    return np.clip(s, 1e-5, 1e5).astype(np.float32)
+
+
+def smoothing_mse(x_fp16, s) -> float:
+    """The objective of Section 3.4 for one candidate: MSE(X, Q_INT8(X / s) * s) over a calibration batch X [T,K],
+    with Q_INT8 the symmetric per-token 8-bit quantiser of Section 4.1 (scale A/127, round half to even).
+    The level decision is taken in binary32 exactly as ``smooth_quantize`` does (t = x * fl32(1/s)); the
+    reconstruction and the mean are binary64."""
+    x = np.asarray(x_fp16, dtype=np.float16)
+    s32 = np.asarray(s, dtype=np.float32)
+    inv = (np.float32(1.0) / s32).astype(np.float32)
+    q, s_q = smooth_quantize(x, inv, act_bits=8)
+    rec = q.astype(np.float64) * s_q.astype(np.float64)[:, None] * s32.astype(np.float64)[None, :]
+    d = x.astype(np.float64) - rec
+    return float((d * d).mean())
+
+
+def smoothing_search(x_fp16, wmax, alphas):
+    """Grid search of Section 3.4: the activation maxima are taken over the calibration batch itself; returns
+    (index of the best alpha, the MSE of every candidate).  Ties go to the first candidate."""
+    x = np.asarray(x_fp16, dtype=np.float16)
+    xmax = np.abs(x.astype(np.float64)).max(axis=0)
+    mse = np.array([smoothing_mse(x, smoothing_factors(xmax, wmax, float(a))) for a in alphas])
+    return int(np.argmin(mse)), mse

@@ -360,3 +360,60 @@ def test_act8_padding():
     q = np.arange(-128, 128, dtype=np.int8).reshape(1, 256)[:, :200]
     p = O.pad_act8(q)
     assert p.shape == (1, 256) and p.dtype == np.int8 and np.array_equal(p[:, :200], q) and not p[:, 200:].any()
+
+
+# ---------------------------------------------------------------- adaptive smoothing search (Section 3.4)
+def test_smoothing_factors_closed_forms_and_clamps():
+    xmax = np.array([4.0, 9.0, 0.0, 1e12, 1e-12, 2.0])
+    wmax = np.array([1.0, 4.0, 3.0, 1e-12, 1e12, 0.0])
+    s0 = O.smoothing_factors(xmax, wmax, 0.0)       # alpha = 0: 1 / wmax
+    s1 = O.smoothing_factors(xmax, wmax, 1.0)       # alpha = 1: xmax
+    sh = O.smoothing_factors(xmax, wmax, 0.5)       # alpha = 1/2: sqrt(xmax / wmax)
+    assert s0[:2].tolist() == [1.0, 0.25] and s1[:2].tolist() == [4.0, 9.0] and sh[:2].tolist() == [2.0, 1.5]
+    assert sh[2] == 1.0 and sh[5] == 1.0            # a zero maximum leaves the channel alone
+    assert sh[3] == np.float32(1e5) and sh[4] == np.float32(1e-5)
+
+
+def test_smoothing_mse_zero_when_representable_and_matches_loops():
+    # integers up to 127 with a 127 in every row are their own 8-bit levels: no error at s = 1 ...
+    rng = np.random.default_rng(21)
+    x = rng.integers(-127, 128, size=(5, 64)).astype(np.float16)
+    x[:, 0] = 127
+    assert O.smoothing_mse(x, np.ones(64, dtype=np.float32)) == 0.0
+    # ... and at any power-of-two s (division and multiplication are exact)
+    assert O.smoothing_mse(x, np.full(64, 4.0, dtype=np.float32)) == 0.0
+    # brute force on a small case
+    x = (rng.standard_normal((3, 10)) * 5).astype(np.float16)
+    s = (rng.random(10) + 0.5).astype(np.float32)
+    tot = 0.0
+    for t in range(3):
+        tv = [np.float32(x[t, k]) * (np.float32(1.0) / s[k]) for k in range(10)]
+        A = max(abs(v) for v in tv)
+        for k in range(10):
+            lev = float(np.clip(np.rint(np.float32(tv[k] * (np.float32(127.0) / A))), -128, 127))
+            rec = lev * float(np.float32(A / np.float32(127.0))) * float(s[k])
+            tot += (float(x[t, k]) - rec) ** 2
+    assert abs(O.smoothing_mse(x, s) - tot / 30) <= 1e-15 * max(1.0, tot)
+
+
+def test_smoothing_search_prefers_taming_outlier_channels():
+    # a few channels 50x larger than the rest: without smoothing (alpha = 0, equal weights) the 8-bit step is set by
+    # the outliers and the small channels lose their resolution; alpha = 1 equalises the channels completely
+    rng = np.random.default_rng(22)
+    T, K = 64, 256
+    x = rng.standard_normal((T, K))
+    x[:, ::32] *= 50.0
+    x = x.astype(np.float16)
+    wmax = np.ones(K)
+    alphas = [0.0, 0.25, 0.5, 0.75, 1.0]
+    best, mse = O.smoothing_search(x, wmax, alphas)
+    assert best >= 2 and mse[best] < 0.5 * mse[0]
+    # uniform 8-bit quantiser noise of step d is about d^2 / 12: at alpha = 0 (s = 1) the step of a token is A / 127
+    A = np.abs(x.astype(np.float64)).max(axis=1)
+    expect = ((A / 127.0) ** 2 / 12.0).mean()
+    assert 0.8 * expect < mse[0] < 1.2 * expect
+    # scaling X and the factors by a power of two scales the error by its square
+    s = O.smoothing_factors(np.abs(x.astype(np.float64)).max(axis=0), wmax, 0.5)
+    m1 = O.smoothing_mse(x, s)
+    m2 = O.smoothing_mse((x.astype(np.float32) * 4).astype(np.float16), s)
+    assert abs(m2 - 16 * m1) <= 1e-12 * m2
