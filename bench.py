@@ -56,6 +56,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--act-bits", type=int, default=4, choices=[4, 8],
                     help="activation levels: 4 bit (the benchmark configurations) or 8 bit (the paper's b = 8)")
+    ap.add_argument("--aux", default=None, choices=["smoothing"],
+                    help="time an offline piece instead of the hot path: 'smoothing' = the Section 3.4 grid search")
     ap.add_argument("--two-call", action="store_true",
                     help="M <= 16: quantise and look up in two launches per layer instead of the fused one")
     ap.add_argument("--algo", default="auto", choices=["auto", "register", "bucket", "tensor"],
@@ -487,8 +489,42 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_aux_smoothing(args):
+    """Section 3.4 grid search on a 128-token synthetic calibration batch per matrix of the configuration
+    (same outlier recipe as the test tokens): 21 candidates, CUDA events, printed as one JSON line."""
+    import torch
+    import paper_2506_12038_b200 as lcd
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    cfg = gen.CONFIGS[args.config]
+    alphas = [i / 20 for i in range(21)]
+    rows, total_ms = [], 0.0
+    for mi, (name, N, K) in enumerate(cfg["shapes"]):
+        ch = gen.outlier_channels(1000 + mi, K, cfg["frac"])
+        x = torch.from_numpy(gen.activations(2000 + mi, 128, K, ch, cfg["scale"])).to(dev)
+        wmax = torch.from_numpy((np.abs(gen.normal(3000 + mi, K)) * 0.05 + 0.01).astype(np.float32)).to(dev)
+        for _ in range(3):
+            lcd.smoothing_search(x, wmax, alphas)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(10):
+            best, mse, inv = lcd.smoothing_search(x, wmax, alphas)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / 10
+        total_ms += ms
+        rows.append({"matrix": name, "K": K, "us": ms * 1e3, "best_alpha": alphas[int(best.item())]})
+    print(json.dumps({"aux": "smoothing_search", "config": {"workload": f"BASELINE configs[{args.config}] {cfg['name']}",
+                                                            "calibration_tokens": 128, "candidates": len(alphas)},
+                      "us_per_layer": total_ms * 1e3, "per_matrix": rows, "data": "synthetic"}))
+
+
 def main():
     args = parse_args()
+    if args.aux == "smoothing":
+        run_aux_smoothing(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -210,6 +210,27 @@ lcd_status lcd_lut_linear_batch_act8(const lcd_linear_problem* problems /* host 
                                 void* cuda_stream);
 
 /* ----------------------------------------------------------------------------------------------
+ * Offline: adaptive smoothing search (Section 3.4).  For each of n_alphas candidate migration strengths alpha:
+ *     s_k = xmax_k^alpha / wmax_k^(1-alpha), xmax_k = max over the calibration batch of |x_tk|, clamped to
+ *           [1e-5, 1e5], s_k = 1 where either maximum is zero (binary64 powers, rounded once to binary32);
+ *     mse  = mean over the batch of (x - Q_INT8(x / s) * s)^2, Q_INT8 = the per-token 8-bit quantiser of
+ *           lcd_smooth_quantize_act (act_bits = 8, dynamic scale) applied with inv_smooth = 1/s.
+ * The first candidate with the smallest mse is chosen.
+ *   x_fp16:      device, binary16 [T][ldx], the calibration activations of one layer;
+ *   wmax:        device, fp32 [K]: max over output rows of |W[n][k]| of that layer;
+ *   alphas_host: host, fp32 [n_alphas], 1 <= n_alphas <= 64;
+ *   workspace:   device, lcd_smoothing_search_workspace_bytes(...) bytes, 256-byte aligned, contents ignored;
+ *   mse:         device out, fp64 [n_alphas];   best: device out int32 (index) or NULL;
+ *   inv_smooth:  device out fp32 [K] = 1/s_k of the chosen candidate, ready for the online calls, or NULL.
+ * Sums run in a fixed order: results are reproducible from run to run.
+ * -------------------------------------------------------------------------------------------- */
+lcd_status lcd_smoothing_search_workspace_bytes(int64_t T, int64_t K, int n_alphas, size_t* bytes);
+
+lcd_status lcd_smoothing_search(const void* x_fp16, int64_t T, int64_t K, int64_t ldx, const float* wmax,
+                                const float* alphas_host, int n_alphas, void* workspace, size_t workspace_bytes,
+                                double* mse, int32_t* best, float* inv_smooth, void* cuda_stream);
+
+/* ----------------------------------------------------------------------------------------------
  * Online steps 1+2+3 in one launch for up to LCD_MAX_BATCH independent problems with M <= 16 (the projections
  * of one decoder layer at decode time): the lookup kernel performs the input transformation of Section 4.1
  * itself (dynamic per-token scale, 4-bit levels, the operation sequence of lcd_smooth_quantize_act, so the

@@ -27,7 +27,8 @@ EXPORTS = ["lcd_status_string", "lcd_last_cuda_error", "lcd_packed_weights_bytes
            "lcd_linear_host_scratch_bytes", "lcd_linear_host", "lcd_smooth_quantize_act_batch",
            "lcd_lut_linear_batch_workspace_bytes", "lcd_lut_linear_batch", "lcd_lut_linear_static",
            "lcd_linear_host_batch_sizes", "lcd_linear_host_batch", "lcd_lut_linear_act8",
-           "lcd_lut_linear_batch_act8", "lcd_linear_fused_batch_workspace_bytes", "lcd_linear_fused_batch"]
+           "lcd_lut_linear_batch_act8", "lcd_linear_fused_batch_workspace_bytes", "lcd_linear_fused_batch",
+           "lcd_smoothing_search_workspace_bytes", "lcd_smoothing_search"]
 STATIC_SCRATCH_BYTES = 4 << 20
 
 
@@ -79,6 +80,9 @@ def _load() -> ctypes.CDLL:
     lib.lcd_lut_linear.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_int64, c_int,
                                    c_void_p, c_size_t, c_void_p, c_void_p]
     lib.lcd_lut_linear_act8.argtypes = lib.lcd_lut_linear.argtypes
+    lib.lcd_smoothing_search_workspace_bytes.argtypes = [c_int64, c_int64, c_int, POINTER(c_size_t)]
+    lib.lcd_smoothing_search.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_int, c_void_p, c_size_t,
+                                         c_void_p, c_void_p, c_void_p, c_void_p]
     lib.lcd_linear_fused_batch_workspace_bytes.argtypes = [POINTER(FusedProblem), c_int, c_int, POINTER(c_size_t)]
     lib.lcd_linear_fused_batch.argtypes = [POINTER(FusedProblem), c_int, c_int, c_void_p, c_size_t, c_void_p, c_void_p]
     lib.lcd_lut_linear_batch_act8.argtypes = [POINTER(LinearProblem), c_int, c_int, c_void_p, c_size_t, c_void_p, c_void_p]
@@ -262,6 +266,27 @@ class ActBatch:
     def run(self, stream=None):
         _check(lib.lcd_smooth_quantize_act_batch(self.arr, self.count, self.act_bits, _stream_ptr(stream)),
                "lcd_smooth_quantize_act_batch")
+
+
+def smoothing_search(x, wmax, alphas, stream=None):
+    """Section 3.4 grid search on a calibration batch.  x: CUDA fp16 [T,K]; wmax: CUDA fp32 [K]; alphas: list of
+    floats.  Returns (best index tensor int32 [1], mse fp64 [G], inv_smooth fp32 [K]) on the device."""
+    import torch
+    assert x.is_cuda and x.dtype == torch.float16 and x.dim() == 2 and x.stride(1) == 1
+    T, K = x.shape
+    G = len(alphas)
+    need = c_size_t(0)
+    _check(lib.lcd_smoothing_search_workspace_bytes(T, K, G, byref(need)), "lcd_smoothing_search_workspace_bytes")
+    ws = torch.empty(need.value, dtype=torch.uint8, device=x.device)
+    mse = torch.empty((G,), dtype=torch.float64, device=x.device)
+    best = torch.empty((1,), dtype=torch.int32, device=x.device)
+    inv = torch.empty((K,), dtype=torch.float32, device=x.device)
+    al = (ctypes.c_float * G)(*[float(a) for a in alphas])
+    _check(lib.lcd_smoothing_search(c_void_p(x.data_ptr()), T, K, x.stride(0), c_void_p(wmax.data_ptr()), al, G,
+                                    c_void_p(ws.data_ptr()), need.value, c_void_p(mse.data_ptr()),
+                                    c_void_p(best.data_ptr()), c_void_p(inv.data_ptr()), _stream_ptr(stream)),
+           "lcd_smoothing_search")
+    return best, mse, inv
 
 
 class FusedBatch:

@@ -321,6 +321,27 @@ extern "C" lcd_status lcd_linear_fused_batch(const lcd_fused_problem* problems, 
   return launch_lut_gemv(p, count, resolved, workspace, workspace_bytes, status_word_dev, cuda_stream);
 }
 
+extern "C" lcd_status lcd_smoothing_search_workspace_bytes(int64_t T, int64_t K, int n_alphas, size_t* bytes) {
+  if (!bytes || T < 1 || K < 1 || n_alphas < 1 || n_alphas > 64) return LCD_ERR_INVALID_ARG;
+  if (T > 0x7fffffffLL) return LCD_ERR_INVALID_ARG;
+  *bytes = smoothing_search_workspace_bytes(T, K, n_alphas);
+  return LCD_OK;
+}
+
+extern "C" lcd_status lcd_smoothing_search(const void* x_fp16, int64_t T, int64_t K, int64_t ldx, const float* wmax,
+                                           const float* alphas_host, int n_alphas, void* workspace,
+                                           size_t workspace_bytes, double* mse, int32_t* best, float* inv_smooth,
+                                           void* cuda_stream) {
+  if (!x_fp16 || !wmax || !alphas_host || !workspace || !mse || T < 1 || K < 1 || ldx < K) return LCD_ERR_INVALID_ARG;
+  if (n_alphas < 1 || n_alphas > 64 || T > 0x7fffffffLL) return LCD_ERR_INVALID_ARG;
+  if (!aligned(x_fp16, 2) || !aligned(wmax, 4) || !aligned(workspace, 256) || !aligned(mse, 8) ||
+      (best && !aligned(best, 4)) || (inv_smooth && !aligned(inv_smooth, 4)))
+    return LCD_ERR_INVALID_ARG;
+  if (workspace_bytes < smoothing_search_workspace_bytes(T, K, n_alphas)) return LCD_ERR_BUFFER_TOO_SMALL;
+  return launch_smoothing_search(x_fp16, T, K, ldx, wmax, alphas_host, n_alphas, workspace, mse, best, inv_smooth,
+                                 cuda_stream);
+}
+
 // ---- host-buffer path -------------------------------------------------------------------------------
 namespace {
 struct HostScratch {
