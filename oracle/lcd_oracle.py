@@ -435,3 +435,42 @@ def smoothing_search(x_fp16, wmax, alphas):
     xmax = np.abs(x.astype(np.float64)).max(axis=0)
     mse = np.array([smoothing_mse(x, smoothing_factors(xmax, wmax, float(a))) for a in alphas])
     return int(np.argmin(mse)), mse
+
+
+# --------------------------------------------------------------------------------------
+# Section 3.2 - reclassification of weights and centroid update (offline; mechanics only)
+# --------------------------------------------------------------------------------------
+def reclassify(idx, codebook_fp16, delta_w):
+    """One round of Section 3.2's bookkeeping for per-row codebooks sorted in ascending order.
+
+    For a weight in cluster i with update dw:  d_left = (C_i - C_{i-1}) / 2,  d_right = (C_{i+1} - C_i) / 2
+    (binary32: one subtraction, one halving); it moves to cluster i - 1 when dw < -d_left (the update carries it
+    across the half-way point to the left neighbour), to i + 1 when dw > d_right, edge clusters have one side only.
+    Centroid offset, as printed:  dC_i = sum over weights that stay in i of dw
+                                      + sum over weights that arrive from i + 1 of ((C_{i+1} - C_i) + dw)
+                                      + sum over weights that arrive from i - 1 of ((C_{i-1} - C_i) + dw).
+    Returns (new_idx uint8 [N,K], dC float64 [N,C], count int64 [N,C] = members after the move)."""
+    idx = np.asarray(idx, dtype=np.uint8)
+    cb32 = np.asarray(codebook_fp16, dtype=np.float16).astype(np.float32)
+    dw = np.asarray(delta_w, dtype=np.float32)
+    N, K = idx.shape
+    C = cb32.shape[1]
+    if np.any(np.diff(cb32.astype(np.float64), axis=1) < 0):
+        raise ValueError("codebook rows must be sorted in ascending order")
+    half = ((cb32[:, 1:] - cb32[:, :-1]).astype(np.float32) * np.float32(0.5)).astype(np.float32)   # [N, C-1]
+    new_idx = idx.copy()
+    dC = np.zeros((N, C))
+    cnt = np.zeros((N, C), dtype=np.int64)
+    cb = cb32.astype(np.float64)
+    for n in range(N):
+        i = idx[n].astype(np.int64)
+        d_left = np.where(i > 0, half[n][np.maximum(i - 1, 0)], np.float32(np.inf)).astype(np.float32)
+        d_right = np.where(i < C - 1, half[n][np.minimum(i, C - 2)], np.float32(np.inf)).astype(np.float32)
+        go_left = dw[n] < -d_left
+        go_right = (dw[n] > d_right) & ~go_left
+        j = i - go_left.astype(np.int64) + go_right.astype(np.int64)
+        new_idx[n] = j.astype(np.uint8)
+        contrib = dw[n].astype(np.float64) + (cb[n][i] - cb[n][j])
+        dC[n] = np.bincount(j, weights=contrib, minlength=C)
+        cnt[n] = np.bincount(j, minlength=C)
+    return new_idx, dC, cnt

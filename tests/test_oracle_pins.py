@@ -417,3 +417,55 @@ def test_smoothing_search_prefers_taming_outlier_channels():
     m1 = O.smoothing_mse(x, s)
     m2 = O.smoothing_mse((x.astype(np.float32) * 4).astype(np.float16), s)
     assert abs(m2 - 16 * m1) <= 1e-12 * m2
+
+
+# ---------------------------------------------------------------- reclassification + centroid update (Section 3.2)
+def test_reclassify_hand_example():
+    # centroids -1, 0, 2: half-gaps 0.5 and 1
+    cb = np.array([[-1.0, 0.0, 2.0]], dtype=np.float16)
+    idx = np.array([[1, 1, 1, 1, 0, 0, 2, 2]], dtype=np.uint8)
+    dw = np.array([[0.25, -0.5, -0.75, 1.5, -3.0, 0.75, 0.5, -1.25]], dtype=np.float32)
+    new_idx, dC, cnt = O.reclassify(idx, cb, dw)
+    #  0.25 stays in 1; -0.5 is not beyond -0.5: stays; -0.75 crosses to 0; 1.5 > 1 crosses to 2;
+    #  -3 in the leftmost cluster has no left side: stays; 0.75 > 0.5 crosses to 1; 0.5 in the rightmost: stays;
+    #  -1.25 < -1 crosses to 1
+    assert new_idx.tolist() == [[1, 1, 0, 2, 0, 1, 2, 1]]
+    assert cnt.tolist() == [[2, 4, 2]]
+    # cluster 0: stays -3, arrival from 1: (0 - -1) + -0.75 = 0.25             -> -2.75
+    # cluster 1: stays 0.25 - 0.5, from 0: (-1 - 0) + 0.75, from 2: (2 - 0) - 1.25 -> -0.25 - 0.25 + 0.75 = 0.25
+    # cluster 2: stays 0.5, arrival from 1: (0 - 2) + 1.5 = -0.5                -> 0.0
+    assert dC.tolist() == [[-2.75, 0.25, 0.0]]
+
+
+def test_reclassify_invariants_and_brute_force():
+    rng = np.random.default_rng(31)
+    N, K, C = 7, 300, 5
+    cb = np.sort(rng.standard_normal((N, C)), axis=1).astype(np.float16)
+    idx = rng.integers(0, C, size=(N, K), dtype=np.uint8)
+    dw = (rng.standard_normal((N, K)) * 0.4).astype(np.float32)
+    new_idx, dC, cnt = O.reclassify(idx, cb, dw)
+    assert np.all(np.abs(new_idx.astype(int) - idx.astype(int)) <= 1) and new_idx.max() < C
+    assert np.all(cnt.sum(axis=1) == K)
+    # zero updates change nothing
+    z_idx, z_dC, z_cnt = O.reclassify(idx, cb, np.zeros_like(dw))
+    assert np.array_equal(z_idx, idx) and not z_dC.any()
+    # the offsets of a row add up to: sum of updates + sum over moved weights of (old centroid - new centroid)
+    cbd = cb.astype(np.float64)
+    for n in range(N):
+        moved = cbd[n][idx[n]] - cbd[n][new_idx[n]]
+        assert abs(dC[n].sum() - (dw[n].astype(np.float64).sum() + moved.sum())) < 1e-9
+    # triple loop
+    bf = np.zeros((N, C))
+    for n in range(N):
+        for k in range(K):
+            i, j = int(idx[n, k]), int(new_idx[n, k])
+            if i > 0 and dw[n, k] < -np.float32((np.float32(cb[n, i]) - np.float32(cb[n, i - 1])) * np.float32(0.5)):
+                assert j == i - 1
+            elif i < C - 1 and dw[n, k] > np.float32((np.float32(cb[n, i + 1]) - np.float32(cb[n, i])) * np.float32(0.5)):
+                assert j == i + 1
+            else:
+                assert j == i
+            bf[n, j] += float(dw[n, k]) + (float(cb[n, i]) - float(cb[n, j]))
+    np.testing.assert_allclose(dC, bf, rtol=1e-12, atol=1e-12)
+    with pytest.raises(ValueError):
+        O.reclassify(idx, cb[:, ::-1], dw)
