@@ -56,8 +56,9 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--act-bits", type=int, default=4, choices=[4, 8],
                     help="activation levels: 4 bit (the benchmark configurations) or 8 bit (the paper's b = 8)")
-    ap.add_argument("--aux", default=None, choices=["smoothing"],
-                    help="time an offline piece instead of the hot path: 'smoothing' = the Section 3.4 grid search")
+    ap.add_argument("--aux", default=None, choices=["smoothing", "reclassify"],
+                    help="time an offline piece instead of the hot path: 'smoothing' = the Section 3.4 grid search, "
+                         "'reclassify' = the Section 3.2 reclassification and centroid offsets")
     ap.add_argument("--two-call", action="store_true",
                     help="M <= 16: quantise and look up in two launches per layer instead of the fused one")
     ap.add_argument("--algo", default="auto", choices=["auto", "register", "bucket", "tensor"],
@@ -520,10 +521,64 @@ def run_aux_smoothing(args):
                       "us_per_layer": total_ms * 1e3, "per_matrix": rows, "data": "synthetic"}))
 
 
+def run_aux_reclassify(args):
+    """Section 3.2 bookkeeping on every matrix of the configuration: random clusters, sorted random codebooks and
+    N(0, 0.4) updates; 6 bytes per weight (index and update read, index written); CUDA events, one JSON line."""
+    import torch
+    import paper_2506_12038_b200 as lcd
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    cfg = gen.CONFIGS[args.config]
+    C = 1 << cfg["bits"]
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    peak = peaks.get("hbm_gbs", 6650.0)
+    rows, tot_ms, tot_bytes = [], 0.0, 0.0
+    g = torch.Generator(device=dev)
+    g.manual_seed(1234)
+    for name, N, K in cfg["shapes"]:
+        idx = torch.randint(0, C, (N, K), dtype=torch.uint8, device=dev, generator=g)
+        cb = torch.sort(torch.randn((N, C), device=dev, generator=g), dim=1).values.to(torch.float16)
+        dw = torch.randn((N, K), device=dev, generator=g) * 0.4
+        out = lcd.reclassify(idx, cb, dw)
+        stream = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                lcd.reclassify(idx, cb, dw, out=out)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()              # ten launches back to back, no host gaps
+            with torch.cuda.graph(graph, stream=stream):
+                for _ in range(10):
+                    lcd.reclassify(idx, cb, dw, out=out)
+            graph.replay()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / 10
+        b = 6.0 * N * K
+        tot_ms += ms
+        tot_bytes += b
+        rows.append({"matrix": name, "N": N, "K": K, "us": ms * 1e3, "GBps": b / ms / 1e6})
+    print(json.dumps({"aux": "reclassify", "config": {"workload": f"BASELINE configs[{args.config}] {cfg['name']}", "C": C},
+                      "us_per_layer": tot_ms * 1e3, "per_matrix": rows, "data": "synthetic",
+                      "roofline": {"bound": "hbm", "achieved": tot_bytes / tot_ms / 1e6, "peak": peak, "unit": "GB/s",
+                                   "frac": tot_bytes / tot_ms / 1e6 / peak,
+                                   "peak_source": "measured (copy)" if peaks else "fallback"}}))
+
+
 def main():
     args = parse_args()
     if args.aux == "smoothing":
         run_aux_smoothing(args)
+        return
+    if args.aux == "reclassify":
+        run_aux_reclassify(args)
         return
     if args.impl == "reference":
         run_reference(args)

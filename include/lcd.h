@@ -231,6 +231,22 @@ lcd_status lcd_smoothing_search(const void* x_fp16, int64_t T, int64_t K, int64_
                                 double* mse, int32_t* best, float* inv_smooth, void* cuda_stream);
 
 /* ----------------------------------------------------------------------------------------------
+ * Offline: reclassification of weights and centroid offsets after a round of weight updates (Section 3.2, the
+ * half-gap equation and the centroid-update equation), for per-row codebooks sorted in ascending order (the
+ * caller's duty; unsorted rows give meaningless moves).  A weight of cluster i with update dw moves to i - 1 when
+ * dw < -(C_i - C_{i-1})/2 and to i + 1 when dw > (C_{i+1} - C_i)/2 (binary32, one subtraction and one halving;
+ * the paper prints the left test without the sign; edge clusters have one side); never further than one cluster.
+ *     delta_c[n][j] = sum over the weights that end up in j of (dw + (C_old - C_j))      (a sum, as printed)
+ *   idx:           device, uint8 [N][K] cluster of every weight (one byte each, the packer's input form), < C;
+ *   codebook_fp16: device, binary16 [N][C], 1 <= C <= 16;     delta_w: device, fp32 [N][ldw], ldw >= K;
+ *   new_idx:       device out, uint8 [N][K] (may not alias idx);
+ *   delta_c:       device out, fp64 [N][C];     counts: device out, int32 [N][C] members after the move.
+ * Sums run in a fixed order: results are reproducible from run to run.
+ * -------------------------------------------------------------------------------------------- */
+lcd_status lcd_reclassify(const uint8_t* idx, const uint16_t* codebook_fp16, const float* delta_w, int64_t N, int64_t K,
+                          int64_t ldw, int C, uint8_t* new_idx, double* delta_c, int32_t* counts, void* cuda_stream);
+
+/* ----------------------------------------------------------------------------------------------
  * Online steps 1+2+3 in one launch for up to LCD_MAX_BATCH independent problems with M <= 16 (the projections
  * of one decoder layer at decode time): the lookup kernel performs the input transformation of Section 4.1
  * itself (dynamic per-token scale, 4-bit levels, the operation sequence of lcd_smooth_quantize_act, so the

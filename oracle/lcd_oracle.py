@@ -464,8 +464,9 @@ def reclassify(idx, codebook_fp16, delta_w):
     cb = cb32.astype(np.float64)
     for n in range(N):
         i = idx[n].astype(np.int64)
-        d_left = np.where(i > 0, half[n][np.maximum(i - 1, 0)], np.float32(np.inf)).astype(np.float32)
-        d_right = np.where(i < C - 1, half[n][np.minimum(i, C - 2)], np.float32(np.inf)).astype(np.float32)
+        hp = np.concatenate([half[n], np.array([np.inf], dtype=np.float32)])   # a single cluster has no half-gap
+        d_left = np.where(i > 0, hp[np.maximum(i - 1, 0)], np.float32(np.inf)).astype(np.float32)
+        d_right = np.where(i < C - 1, hp[np.minimum(i, max(C - 2, 0))], np.float32(np.inf)).astype(np.float32)
         go_left = dw[n] < -d_left
         go_right = (dw[n] > d_right) & ~go_left
         j = i - go_left.astype(np.int64) + go_right.astype(np.int64)

@@ -28,7 +28,7 @@ EXPORTS = ["lcd_status_string", "lcd_last_cuda_error", "lcd_packed_weights_bytes
            "lcd_lut_linear_batch_workspace_bytes", "lcd_lut_linear_batch", "lcd_lut_linear_static",
            "lcd_linear_host_batch_sizes", "lcd_linear_host_batch", "lcd_lut_linear_act8",
            "lcd_lut_linear_batch_act8", "lcd_linear_fused_batch_workspace_bytes", "lcd_linear_fused_batch",
-           "lcd_smoothing_search_workspace_bytes", "lcd_smoothing_search"]
+           "lcd_smoothing_search_workspace_bytes", "lcd_smoothing_search", "lcd_reclassify"]
 STATIC_SCRATCH_BYTES = 4 << 20
 
 
@@ -80,6 +80,8 @@ def _load() -> ctypes.CDLL:
     lib.lcd_lut_linear.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_int64, c_int,
                                    c_void_p, c_size_t, c_void_p, c_void_p]
     lib.lcd_lut_linear_act8.argtypes = lib.lcd_lut_linear.argtypes
+    lib.lcd_reclassify.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int, c_void_p, c_void_p,
+                                   c_void_p, c_void_p]
     lib.lcd_smoothing_search_workspace_bytes.argtypes = [c_int64, c_int64, c_int, POINTER(c_size_t)]
     lib.lcd_smoothing_search.argtypes = [c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p, c_int, c_void_p, c_size_t,
                                          c_void_p, c_void_p, c_void_p, c_void_p]
@@ -266,6 +268,29 @@ class ActBatch:
     def run(self, stream=None):
         _check(lib.lcd_smooth_quantize_act_batch(self.arr, self.count, self.act_bits, _stream_ptr(stream)),
                "lcd_smooth_quantize_act_batch")
+
+
+def reclassify(idx, codebook, delta_w, stream=None, out=None):
+    """Section 3.2 bookkeeping.  idx: CUDA uint8 [N,K]; codebook: CUDA fp16 [N,C] rows ascending; delta_w: CUDA fp32
+    [N,K].  Returns (new_idx uint8 [N,K], delta_c fp64 [N,C], counts int32 [N,C]); `out` may give those three
+    tensors to write into."""
+    import torch
+    assert idx.dtype == torch.uint8 and codebook.dtype == torch.float16 and delta_w.dtype == torch.float32
+    assert idx.is_contiguous() and codebook.is_contiguous() and delta_w.stride(1) == 1
+    N, K = idx.shape
+    C = codebook.shape[1]
+    if out is None:
+        new_idx = torch.empty_like(idx)
+        delta_c = torch.empty((N, C), dtype=torch.float64, device=idx.device)
+        counts = torch.empty((N, C), dtype=torch.int32, device=idx.device)
+    else:
+        new_idx, delta_c, counts = out
+        assert new_idx.dtype == torch.uint8 and delta_c.dtype == torch.float64 and counts.dtype == torch.int32
+        assert new_idx.shape == idx.shape and delta_c.shape == (N, C) and counts.shape == (N, C)
+    _check(lib.lcd_reclassify(c_void_p(idx.data_ptr()), c_void_p(codebook.data_ptr()), c_void_p(delta_w.data_ptr()), N, K,
+                              delta_w.stride(0), C, c_void_p(new_idx.data_ptr()), c_void_p(delta_c.data_ptr()),
+                              c_void_p(counts.data_ptr()), _stream_ptr(stream)), "lcd_reclassify")
+    return new_idx, delta_c, counts
 
 
 def smoothing_search(x, wmax, alphas, stream=None):

@@ -480,3 +480,20 @@ def test_smoothing_search_matches_oracle(T, K, ld_extra):
     a, sc = lcd.smooth_quantize_act(xd[:, :K], inv, act_bits=8)
     q_ref, s_q_ref = O.smooth_quantize(x, got, act_bits=8)
     assert np.array_equal(a.cpu().numpy(), O.pad_act8(q_ref)) and np.array_equal(sc.cpu().numpy(), s_q_ref)
+
+
+# ------------------------------------------------------------------------------- reclassification (offline)
+@pytest.mark.parametrize("N,K,C,ld_extra", [(64, 4096, 4, 0), (33, 1000, 8, 8), (5, 250, 5, 3), (3, 7, 1, 0), (2, 300, 16, 0)])
+def test_reclassify_matches_oracle(N, K, C, ld_extra):
+    cb = np.sort(gen.normal(50 + N, N * C).reshape(N, C), axis=1).astype(np.float16)
+    idx = (gen.permutation(51 + K, N * K) % C).astype(np.uint8).reshape(N, K)
+    dw = (gen.normal(52 + C, N * K).reshape(N, K) * 0.4).astype(np.float32)
+    dw[0, :min(K, 4)] = 0.0
+    dwd = torch.zeros((N, K + ld_extra), dtype=torch.float32, device="cuda")
+    dwd[:, :K] = torch.from_numpy(dw).cuda()
+    new_idx, dC, cnt = lcd.reclassify(torch.from_numpy(idx).cuda(), torch.from_numpy(cb).cuda(), dwd[:, :K])
+    torch.cuda.synchronize()
+    r_idx, r_dC, r_cnt = O.reclassify(idx, cb, dw)
+    assert np.array_equal(new_idx.cpu().numpy(), r_idx)                    # decisions: bit-exact
+    assert np.array_equal(cnt.cpu().numpy().astype(np.int64), r_cnt)
+    np.testing.assert_allclose(dC.cpu().numpy(), r_dC, rtol=1e-11, atol=1e-11)   # binary64 sums in another order

@@ -469,3 +469,7 @@ def test_reclassify_invariants_and_brute_force():
     np.testing.assert_allclose(dC, bf, rtol=1e-12, atol=1e-12)
     with pytest.raises(ValueError):
         O.reclassify(idx, cb[:, ::-1], dw)
+    # one cluster: no neighbour, nothing moves, the offset is the sum of the updates
+    one_idx, one_dC, one_cnt = O.reclassify(np.zeros((1, 5), dtype=np.uint8), np.array([[0.5]], dtype=np.float16),
+                                            np.array([[1, -2, 3, 0.5, 0.25]], dtype=np.float32))
+    assert not one_idx.any() and one_dC.tolist() == [[2.75]] and one_cnt.tolist() == [[5]]
