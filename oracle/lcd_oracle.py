@@ -475,3 +475,83 @@ def reclassify(idx, codebook_fp16, delta_w):
         dC[n] = np.bincount(j, weights=contrib, minlength=C)
         cnt[n] = np.bincount(j, minlength=C)
     return new_idx, dC, cnt
+
+
+# --------------------------------------------------------------------------------------
+# Section 3.1 - density-based centroid initialisation (DBCI), offline
+# --------------------------------------------------------------------------------------
+DBCI_PERCENTILES = (0.6827, 0.9544, 0.9974)      # the 1, 2 and 3 sigma ranges of a half-normal
+
+
+def _nearest_rank(sorted_vals: np.ndarray, p: float) -> float:
+    """Value at percentile p of an ascending array by the nearest-rank rule, 0 for an empty array."""
+    if sorted_vals.size == 0:
+        return 0.0
+    k = int(np.ceil(p * sorted_vals.size)) - 1
+    return float(sorted_vals[min(max(k, 0), sorted_vals.size - 1)])
+
+
+def dbci(weights):
+    """Density-based centroid initialisation, the six steps of Section 3.1, on a flat array of binary32 weights.
+    All comparisons and the few scalar operations are binary64 on the binary32 data.
+
+    1. sort;  2. sigma = (sum over the 68.27 / 95.44 / 99.74 % nearest-rank percentiles of the positive weights and
+    of the magnitudes of the negative weights) / 12;  3. the smallest and the largest weight seed two clusters that
+    take every point within sigma of them (the right one gives way if they overlap);  4. MinPts = the smaller of the
+    two counts, eps = sigma / MinPts;  5. DBSCAN on the remaining points alone: a point with at least MinPts points
+    (itself included) within eps is a core point, core points closer than eps chain into one cluster, another point
+    within eps of a core point joins the cluster of its nearest core point (the left one on a tie), the rest is
+    noise;  6. the centroid of a cluster is its lower median (an L1 minimiser).
+
+    Returns a dict: sigma, min_pts, eps, left (count), right (count), labels (int64 per sorted point: cluster number
+    in ascending order of position, -1 noise), centroids (float64, ascending), sorted (the sorted weights)."""
+    x = np.sort(np.asarray(weights, dtype=np.float32).ravel())
+    xd = x.astype(np.float64)
+    n = xd.size
+    if n == 0:
+        raise ValueError("no weights")
+    pos = xd[xd > 0]
+    neg = -xd[xd < 0][::-1]
+    sigma = sum(_nearest_rank(pos, p) + _nearest_rank(neg, p) for p in DBCI_PERCENTILES) / 12.0
+    L = int(np.searchsorted(xd, xd[0] + sigma, side="right"))
+    R = int(np.searchsorted(xd, xd[-1] - sigma, side="left"))
+    R = max(R, L)
+    min_pts = min(L, n - R) if n - R > 0 else L
+    eps = sigma / min_pts
+    y = xd[L:R]
+    m = y.size
+    labels = np.full(n, -1, dtype=np.int64)
+    labels[:L] = 0
+    n_mid = 0
+    if m:
+        lo = np.searchsorted(y, y - eps, side="left")
+        hi = np.searchsorted(y, y + eps, side="right")
+        core = (hi - lo) >= min_pts
+        idx = np.arange(m)
+        prev_core = np.maximum.accumulate(np.where(core, idx, -1))                   # nearest core at or before i
+        next_core = np.minimum.accumulate(np.where(core, idx, m)[::-1])[::-1]        # nearest core at or after i
+        prev_before = np.concatenate([[-1], prev_core[:-1]])                         # nearest core strictly before i
+        start = core & ((prev_before < 0) | ((y - y[np.maximum(prev_before, 0)]) > eps))
+        cid = np.cumsum(start) - 1                                                   # cluster of a core point
+        mid = np.full(m, -1, dtype=np.int64)
+        mid[core] = cid[core]
+        nc = np.flatnonzero(~core)
+        if nc.size:
+            pc, nx = prev_core[nc], next_core[nc]
+            dl = np.where(pc >= 0, y[nc] - y[np.maximum(pc, 0)], np.inf)
+            dr = np.where(nx < m, y[np.minimum(nx, m - 1)] - y[nc], np.inf)
+            take_left = (dl <= eps) & (dl <= dr)
+            take_right = (dr <= eps) & ~take_left
+            mid[nc[take_left]] = cid[pc[take_left]]
+            mid[nc[take_right]] = cid[nx[take_right]]
+        n_mid = int(start.sum())
+        labels[L:R] = np.where(mid >= 0, mid + 1, -1)
+    if n - R > 0:
+        labels[R:] = n_mid + 1
+    cents = []
+    for c in range(n_mid + 2):
+        members = np.flatnonzero(labels == c)
+        if members.size:
+            cents.append(xd[members[(members.size - 1) // 2]])
+    return {"sigma": sigma, "min_pts": int(min_pts), "eps": eps, "left": L, "right": n - R, "labels": labels,
+            "centroids": np.array(cents), "sorted": x}

@@ -473,3 +473,79 @@ def test_reclassify_invariants_and_brute_force():
     one_idx, one_dC, one_cnt = O.reclassify(np.zeros((1, 5), dtype=np.uint8), np.array([[0.5]], dtype=np.float16),
                                             np.array([[1, -2, 3, 0.5, 0.25]], dtype=np.float32))
     assert not one_idx.any() and one_dC.tolist() == [[2.75]] and one_cnt.tolist() == [[5]]
+
+
+# ---------------------------------------------------------------- density-based centroid initialisation (Section 3.1)
+def _dbscan_brute(y, eps, min_pts):
+    """Textbook DBSCAN (region queries by full scans, breadth-first expansion) on a small 1-D array."""
+    m = len(y)
+    nbrs = [[j for j in range(m) if abs(y[j] - y[i]) <= eps] for i in range(m)]
+    core = [len(nb) >= min_pts for nb in nbrs]
+    lab = [None] * m
+    c = 0
+    for i in range(m):
+        if lab[i] is not None or not core[i]:
+            continue
+        lab[i] = c
+        queue = list(nbrs[i])
+        while queue:
+            j = queue.pop()
+            if lab[j] is None or lab[j] == -1:
+                lab[j] = c
+                if core[j]:
+                    queue.extend(nbrs[j])
+        c += 1
+    return core, [(-1 if v is None else v) for v in lab]
+
+
+def test_dbci_sigma_of_a_gaussian_and_hand_example():
+    # half-normal percentiles at 68.27 / 95.44 / 99.74 % are 1, 2, 3 sigma: six of them sum to 12 sigma
+    rng = np.random.default_rng(41)
+    w = (rng.standard_normal(200000) * 0.02).astype(np.float32)
+    r = O.dbci(w)
+    assert abs(r["sigma"] / 0.02 - 1.0) < 0.02
+    assert r["min_pts"] == min(r["left"], r["right"]) and r["eps"] == r["sigma"] / r["min_pts"]
+    assert np.all(np.diff(r["centroids"]) > 0) and np.all(np.isin(r["centroids"].astype(np.float32), r["sorted"]))
+    # hand example: two tight groups, two far outliers
+    w = np.array([-10.0, -1.0, -0.9, -1.1, 1.0, 1.1, 0.9, 1.05, 12.0], dtype=np.float32)
+    r = O.dbci(w)
+    # positives 0.9 1 1.05 1.1 12 -> ranks ceil(p * 5) = 4, 5, 5 -> 1.1, 12, 12; negatives (magnitudes) 0.9 1 1.1 10
+    # -> ranks 3, 4, 4 -> 1.1, 10, 10; sigma = 46.2 / 12 = 3.85
+    assert abs(r["sigma"] - 46.2 / 12) < 1e-6
+    assert r["left"] == 1 and r["right"] == 1 and r["min_pts"] == 1     # nothing within 3.85 of -10 or of 12
+    # MinPts 1: every point is a core point, eps = sigma: the seven middle points chain into one cluster
+    assert r["labels"].tolist() == [0, 1, 1, 1, 1, 1, 1, 1, 2]
+    assert r["centroids"].tolist() == [-10.0, float(np.float32(0.9)), 12.0]
+
+
+def test_dbci_middle_matches_textbook_dbscan():
+    rng = np.random.default_rng(42)
+    for trial in range(6):
+        body = rng.standard_normal(300) * 0.02
+        clumps = np.concatenate([0.1 + rng.standard_normal(25) * 0.001, -0.08 + rng.standard_normal(15) * 0.001])
+        outl = np.array([-0.5, -0.49, -0.495, 0.6, 0.61, 0.6050])
+        w = np.concatenate([body, clumps, outl, rng.uniform(-0.3, 0.3, 12)]).astype(np.float32)
+        r = O.dbci(w)
+        x = r["sorted"].astype(np.float64)
+        L, R = r["left"], len(x) - r["right"]
+        core, lab = _dbscan_brute(x[L:R], r["eps"], r["min_pts"])
+        mine = r["labels"][L:R]
+        core_idx = [i for i in range(R - L) if core[i]]
+        # core points: same partition (cluster numbers may be permuted)
+        pairs = {(lab[i], int(mine[i])) for i in core_idx}
+        assert len(pairs) == len({a for a, _ in pairs}) == len({b for _, b in pairs})
+        assert all(mine[i] >= 1 for i in core_idx)
+        # the rest: noise exactly where the textbook says noise; a border point sits within eps of a core of its cluster
+        for i in range(R - L):
+            if core[i]:
+                continue
+            assert (mine[i] == -1) == (lab[i] == -1)
+            if mine[i] != -1:
+                assert any(core[j] and mine[j] == mine[i] and abs(x[L + j] - x[L + i]) <= r["eps"] for j in range(R - L))
+        # clusters are contiguous in sorted order and every centroid is the lower median of its members
+        labs = r["labels"]
+        for c in range(int(labs.max()) + 1):
+            mem = np.flatnonzero(labs == c)
+            if mem.size:
+                assert not np.any((labs[mem[0]:mem[-1] + 1] != c) & (labs[mem[0]:mem[-1] + 1] != -1))
+        assert r["centroids"].size == len({int(v) for v in labs if v >= 0})
