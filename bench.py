@@ -56,9 +56,10 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--act-bits", type=int, default=4, choices=[4, 8],
                     help="activation levels: 4 bit (the benchmark configurations) or 8 bit (the paper's b = 8)")
-    ap.add_argument("--aux", default=None, choices=["smoothing", "reclassify"],
+    ap.add_argument("--aux", default=None, choices=["smoothing", "reclassify", "dbci"],
                     help="time an offline piece instead of the hot path: 'smoothing' = the Section 3.4 grid search, "
-                         "'reclassify' = the Section 3.2 reclassification and centroid offsets")
+                         "'reclassify' = the Section 3.2 reclassification and centroid offsets, 'dbci' = the Section 3.1 "
+                         "centroid initialisation")
     ap.add_argument("--two-call", action="store_true",
                     help="M <= 16: quantise and look up in two launches per layer instead of the fused one")
     ap.add_argument("--algo", default="auto", choices=["auto", "register", "bucket", "tensor"],
@@ -572,10 +573,43 @@ def run_aux_reclassify(args):
                                    "peak_source": "measured (copy)" if peaks else "fallback"}}))
 
 
+def run_aux_dbci(args):
+    """Section 3.1 on every matrix of the configuration taken as one flat array: N(0, 0.02) weights with ten
+    12-sigma outliers; CUDA events around three calls after a warm-up; one JSON line."""
+    import torch
+    import paper_2506_12038_b200 as lcd
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    cfg = gen.CONFIGS[args.config]
+    g = torch.Generator(device=dev)
+    g.manual_seed(4321)
+    rows, tot_ms = [], 0.0
+    for name, N, K in cfg["shapes"]:
+        w = torch.randn((N * K,), device=dev, generator=g) * 0.02
+        w[:: max(N * K // 10, 1)] *= 12
+        r = lcd.dbci(w, want_labels=False)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(3):
+            r = lcd.dbci(w, want_labels=False)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / 3
+        tot_ms += ms
+        rows.append({"matrix": name, "weights": N * K, "ms": ms, "Gweights_per_s": N * K / ms / 1e6,
+                     "centroids": int(r["centroids"].numel()), "sigma": r["sigma"], "min_pts": r["min_pts"]})
+    print(json.dumps({"aux": "dbci", "config": {"workload": f"BASELINE configs[{args.config}] {cfg['name']}"},
+                      "ms_per_layer": tot_ms, "per_matrix": rows, "data": "synthetic"}))
+
+
 def main():
     args = parse_args()
     if args.aux == "smoothing":
         run_aux_smoothing(args)
+        return
+    if args.aux == "dbci":
+        run_aux_dbci(args)
         return
     if args.aux == "reclassify":
         run_aux_reclassify(args)

@@ -231,6 +231,35 @@ lcd_status lcd_smoothing_search(const void* x_fp16, int64_t T, int64_t K, int64_
                                 double* mse, int32_t* best, float* inv_smooth, void* cuda_stream);
 
 /* ----------------------------------------------------------------------------------------------
+ * Offline: density-based centroid initialisation (DBCI, the six steps of Section 3.1) on a flat array of weights.
+ *   1. sort;  2. sigma = (the 68.27 / 95.44 / 99.74 % nearest-rank percentiles of the positive weights and of the
+ *   magnitudes of the negative weights, summed) / 12;  3. the smallest and the largest weight seed two clusters
+ *   that take every weight within sigma of them (the right one gives way where they overlap);  4. MinPts = the
+ *   smaller of the two counts, eps = sigma / MinPts;  5. DBSCAN on the remaining weights alone: a weight with at
+ *   least MinPts weights (itself included) within eps is a core point, core points within eps of each other chain
+ *   into one cluster, another weight within eps of a core point joins the cluster of its nearest core point (the
+ *   left one on a tie), the rest is noise;  6. the centroid of a cluster is its lower median.
+ * Comparisons and scalar operations are binary64 on the binary32 data.
+ *   weights:   device, fp32 [n], 1 <= n < 2^31;     workspace: device, lcd_dbci_workspace_bytes(n, max_centroids)
+ *              bytes, 256-byte aligned, contents ignored;
+ *   centroids: device out, fp32 [max_centroids], ascending; if more clusters exist than fit
+ *              (result->n_clusters_found > max_centroids + 2 or n_centroids > max_centroids) the list is cut;
+ *   labels:    device out int32 [n] or NULL: cluster of every weight IN SORTED ORDER (0 = left seed cluster,
+ *              1.. = DBSCAN clusters from left to right, last = right seed cluster, -1 = noise);
+ *   sorted:    device out fp32 [n] or NULL: the sorted weights;     result: device out.
+ * -------------------------------------------------------------------------------------------- */
+typedef struct {
+  double sigma, eps;
+  int64_t min_pts, left, right;        /* members of the two seed clusters */
+  int32_t n_centroids, n_noise, n_clusters_found;
+} lcd_dbci_result;
+
+lcd_status lcd_dbci_workspace_bytes(int64_t n, int max_centroids, size_t* bytes);
+
+lcd_status lcd_dbci(const float* weights, int64_t n, void* workspace, size_t workspace_bytes, float* centroids,
+                    int max_centroids, int32_t* labels, float* sorted, lcd_dbci_result* result, void* cuda_stream);
+
+/* ----------------------------------------------------------------------------------------------
  * Offline: reclassification of weights and centroid offsets after a round of weight updates (Section 3.2, the
  * half-gap equation and the centroid-update equation), for per-row codebooks sorted in ascending order (the
  * caller's duty; unsorted rows give meaningless moves).  A weight of cluster i with update dw moves to i - 1 when

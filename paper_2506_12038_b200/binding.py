@@ -28,8 +28,16 @@ EXPORTS = ["lcd_status_string", "lcd_last_cuda_error", "lcd_packed_weights_bytes
            "lcd_lut_linear_batch_workspace_bytes", "lcd_lut_linear_batch", "lcd_lut_linear_static",
            "lcd_linear_host_batch_sizes", "lcd_linear_host_batch", "lcd_lut_linear_act8",
            "lcd_lut_linear_batch_act8", "lcd_linear_fused_batch_workspace_bytes", "lcd_linear_fused_batch",
-           "lcd_smoothing_search_workspace_bytes", "lcd_smoothing_search", "lcd_reclassify"]
+           "lcd_smoothing_search_workspace_bytes", "lcd_smoothing_search", "lcd_reclassify",
+           "lcd_dbci_workspace_bytes", "lcd_dbci"]
 STATIC_SCRATCH_BYTES = 4 << 20
+
+
+class DbciResult(Structure):
+    """lcd_dbci_result"""
+    _fields_ = [("sigma", ctypes.c_double), ("eps", ctypes.c_double), ("min_pts", c_int64), ("left", c_int64),
+                ("right", c_int64), ("n_centroids", ctypes.c_int32), ("n_noise", ctypes.c_int32),
+                ("n_clusters_found", ctypes.c_int32)]
 
 
 class FusedProblem(Structure):
@@ -80,6 +88,8 @@ def _load() -> ctypes.CDLL:
     lib.lcd_lut_linear.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_int64, c_int,
                                    c_void_p, c_size_t, c_void_p, c_void_p]
     lib.lcd_lut_linear_act8.argtypes = lib.lcd_lut_linear.argtypes
+    lib.lcd_dbci_workspace_bytes.argtypes = [c_int64, c_int, POINTER(c_size_t)]
+    lib.lcd_dbci.argtypes = [c_void_p, c_int64, c_void_p, c_size_t, c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.lcd_reclassify.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int, c_void_p, c_void_p,
                                    c_void_p, c_void_p]
     lib.lcd_smoothing_search_workspace_bytes.argtypes = [c_int64, c_int64, c_int, POINTER(c_size_t)]
@@ -268,6 +278,29 @@ class ActBatch:
     def run(self, stream=None):
         _check(lib.lcd_smooth_quantize_act_batch(self.arr, self.count, self.act_bits, _stream_ptr(stream)),
                "lcd_smooth_quantize_act_batch")
+
+
+def dbci(weights, max_centroids: int = 4096, want_labels: bool = True, stream=None):
+    """Section 3.1 on a flat CUDA fp32 tensor.  Returns a dict: sigma, eps, min_pts, left, right, n_noise,
+    n_clusters_found, centroids (CUDA fp32, ascending), sorted (CUDA fp32) and labels (CUDA int32, in sorted order)."""
+    import torch
+    w = weights.reshape(-1)
+    assert w.is_cuda and w.dtype == torch.float32 and w.is_contiguous()
+    n = w.numel()
+    need = c_size_t(0)
+    _check(lib.lcd_dbci_workspace_bytes(n, max_centroids, byref(need)), "lcd_dbci_workspace_bytes")
+    ws = torch.empty(need.value, dtype=torch.uint8, device=w.device)
+    cents = torch.empty((max_centroids,), dtype=torch.float32, device=w.device)
+    labels = torch.empty((n,), dtype=torch.int32, device=w.device) if want_labels else None
+    srt = torch.empty((n,), dtype=torch.float32, device=w.device)
+    res = torch.zeros((ctypes.sizeof(DbciResult),), dtype=torch.uint8, device=w.device)
+    _check(lib.lcd_dbci(c_void_p(w.data_ptr()), n, c_void_p(ws.data_ptr()), need.value, c_void_p(cents.data_ptr()),
+                        max_centroids, c_void_p(labels.data_ptr()) if labels is not None else None,
+                        c_void_p(srt.data_ptr()), c_void_p(res.data_ptr()), _stream_ptr(stream)), "lcd_dbci")
+    r = DbciResult.from_buffer_copy(res.cpu().numpy().tobytes())
+    return {"sigma": r.sigma, "eps": r.eps, "min_pts": r.min_pts, "left": r.left, "right": r.right,
+            "n_noise": r.n_noise, "n_clusters_found": r.n_clusters_found,
+            "centroids": cents[:min(r.n_centroids, max_centroids)], "sorted": srt, "labels": labels}
 
 
 def reclassify(idx, codebook, delta_w, stream=None, out=None):

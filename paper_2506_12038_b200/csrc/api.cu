@@ -352,6 +352,24 @@ extern "C" lcd_status lcd_reclassify(const uint8_t* idx, const uint16_t* codeboo
   return launch_reclassify(idx, codebook_fp16, delta_w, N, K, ldw, C, new_idx, delta_c, counts, cuda_stream);
 }
 
+extern "C" lcd_status lcd_dbci_workspace_bytes(int64_t n, int max_centroids, size_t* bytes) {
+  if (!bytes || n < 1 || n >= 0x7fffffffLL || max_centroids < 1 || max_centroids > (1 << 24)) return LCD_ERR_INVALID_ARG;
+  *bytes = dbci_workspace_bytes(n, max_centroids);
+  return LCD_OK;
+}
+
+extern "C" lcd_status lcd_dbci(const float* weights, int64_t n, void* workspace, size_t workspace_bytes, float* centroids,
+                               int max_centroids, int32_t* labels, float* sorted, lcd_dbci_result* result,
+                               void* cuda_stream) {
+  if (!weights || !workspace || !centroids || !result) return LCD_ERR_INVALID_ARG;
+  if (n < 1 || n >= 0x7fffffffLL || max_centroids < 1 || max_centroids > (1 << 24)) return LCD_ERR_INVALID_ARG;
+  if (!aligned(weights, 4) || !aligned(workspace, 256) || !aligned(centroids, 4) || !aligned(result, 8) ||
+      (labels && !aligned(labels, 4)) || (sorted && !aligned(sorted, 4)))
+    return LCD_ERR_INVALID_ARG;
+  if (workspace_bytes < dbci_workspace_bytes(n, max_centroids)) return LCD_ERR_BUFFER_TOO_SMALL;
+  return launch_dbci(weights, n, workspace, centroids, max_centroids, labels, sorted, result, cuda_stream);
+}
+
 // ---- host-buffer path -------------------------------------------------------------------------------
 namespace {
 struct HostScratch {

@@ -64,6 +64,9 @@ lcd_status launch_smoothing_search(const void* x, int64_t T, int64_t K, int64_t 
                                    int G, void* workspace, double* mse, int32_t* best, float* inv_smooth, void* stream);
 lcd_status launch_reclassify(const uint8_t* idx, const uint16_t* codebook, const float* delta_w, int64_t N, int64_t K,
                              int64_t ldw, int C, uint8_t* new_idx, double* delta_c, int32_t* counts, void* stream);
+size_t dbci_workspace_bytes(int64_t n, int max_centroids);
+lcd_status launch_dbci(const float* weights, int64_t n, void* workspace, float* centroids, int max_centroids,
+                       int32_t* labels, float* sorted_out, lcd_dbci_result* result, void* stream);
 lcd_status launch_reference(const Problem& p, void* stream);
 lcd_status launch_smooth_quantize_batch(const lcd_act_problem* probs, int count, void* stream);
 // LCD_ALGO_REGISTER_LUT / LCD_ALGO_BUCKET_LUT for up to LCD_MAX_BATCH problems of equal index width in one launch

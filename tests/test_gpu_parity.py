@@ -497,3 +497,34 @@ def test_reclassify_matches_oracle(N, K, C, ld_extra):
     assert np.array_equal(new_idx.cpu().numpy(), r_idx)                    # decisions: bit-exact
     assert np.array_equal(cnt.cpu().numpy().astype(np.int64), r_cnt)
     np.testing.assert_allclose(dC.cpu().numpy(), r_dC, rtol=1e-11, atol=1e-11)   # binary64 sums in another order
+
+
+# ------------------------------------------------------------------------------- DBCI (offline)
+def _dbci_inputs(case):
+    if case == "gauss":                      # a layer's weights: N(0, 0.02) with a few outliers
+        w = gen.normal(71, 200000) * 0.02
+        w[::20000] *= 12
+    elif case == "clumps":
+        w = np.concatenate([gen.normal(72, 3000) * 0.02, 0.1 + gen.normal(73, 250) * 0.001,
+                            -0.08 + gen.normal(74, 150) * 0.001, [-0.5, -0.49, -0.495, 0.6, 0.61, 0.605]])
+    elif case == "tiny":
+        w = np.array([-10.0, -1.0, -0.9, -1.1, 1.0, 1.1, 0.9, 1.05, 12.0])
+    elif case == "one_sided":                # no negative weights at all
+        w = np.abs(gen.normal(75, 5000)) * 0.02 + 0.001
+    else:                                    # "single"
+        w = np.array([0.25])
+    return w.astype(np.float32)
+
+
+@pytest.mark.parametrize("case", ["gauss", "clumps", "tiny", "one_sided", "single"])
+def test_dbci_matches_oracle(case):
+    w = _dbci_inputs(case)
+    r = lcd.dbci(torch.from_numpy(w).cuda(), max_centroids=4096)
+    torch.cuda.synchronize()
+    ref = O.dbci(w)
+    assert np.array_equal(r["sorted"].cpu().numpy(), ref["sorted"])
+    assert r["sigma"] == ref["sigma"] and r["eps"] == ref["eps"]            # binary64 scalars: identical operations
+    assert (r["min_pts"], r["left"], r["right"]) == (ref["min_pts"], ref["left"], ref["right"])
+    assert np.array_equal(r["labels"].cpu().numpy().astype(np.int64), ref["labels"])
+    assert r["n_noise"] == int((ref["labels"] < 0).sum())
+    assert np.array_equal(r["centroids"].cpu().numpy().astype(np.float64), ref["centroids"])
