@@ -22,42 +22,48 @@ __global__ void __launch_bounds__(kRcThreads) reclassify_kernel(const uint8_t* _
                                                                 uint8_t* __restrict__ new_idx, double* __restrict__ delta_c,
                                                                 int32_t* __restrict__ counts, const bool vec) {
   __shared__ float s_c[CMAX];
-  __shared__ float s_half[CMAX];            // s_half[i] = (C_{i+1} - C_i) / 2
-  __shared__ double s_sum[kRcThreads / 32][CMAX];
-  __shared__ int s_cnt[kRcThreads / 32][CMAX];
+  __shared__ float s_gl[CMAX], s_gr[CMAX];  // half-gaps (C_i - C_{i-1}) / 2 and (C_{i+1} - C_i) / 2, infinite at the edges
+  __shared__ float s_wh[kRcThreads / 32][CMAX], s_wl[kRcThreads / 32][CMAX];
+  __shared__ int s_cnt[kRcThreads / 32][CMAX], s_wfl[kRcThreads / 32][CMAX], s_wfr[kRcThreads / 32][CMAX];
   const int64_t n = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid < C) s_c[tid] = __half2float(__ushort_as_half(codebook[n * C + tid]));
   __syncthreads();
-  if (tid < C - 1) s_half[tid] = __fmul_rn(__fsub_rn(s_c[tid + 1], s_c[tid]), 0.5f);
+  if (tid < CMAX) {
+    const float inf = __int_as_float(0x7f800000);
+    s_gl[tid] = (tid > 0 && tid < C) ? __fmul_rn(__fsub_rn(s_c[tid], s_c[tid - 1]), 0.5f) : inf;
+    s_gr[tid] = (tid < C - 1) ? __fmul_rn(__fsub_rn(s_c[tid + 1], s_c[tid]), 0.5f) : inf;
+  }
   __syncthreads();
-  // Per thread and cluster: the sum of the arriving updates as an unevaluated pair of binary32 numbers (error-free
-  // two-sum: binary64 adds are scarce on this part), and integer counts of members and of arrivals from either side;
-  // the centroid differences of the arrivals are added at the end from the counts.
-  float hi[CMAX], lo[CMAX];
-  int cnt[CMAX], from_left[CMAX], from_right[CMAX];
+  // Per thread and cluster, in the thread's own column of shared memory (indexed by the data-dependent cluster; a
+  // register array would need one predicated copy of every operation per cluster): the sum of the arriving updates
+  // as an unevaluated pair of binary32 numbers (error-free two-sum: binary64 adds are scarce on this part) and
+  // integer counts of members and of arrivals from either side; the centroid differences of the arrivals are
+  // added at the end from the counts.
+  extern __shared__ unsigned long long s_dyn[];
+  float2* s_pair = reinterpret_cast<float2*>(s_dyn);                      // [CMAX][kRcThreads] (hi, lo)
+  unsigned long long* s_cnt3 = s_dyn + CMAX * kRcThreads;                 // members | arrivals from the left << 21
+                                                                          // | arrivals from the right << 42
 #pragma unroll
-  for (int c = 0; c < CMAX; ++c) { hi[c] = 0.0f; lo[c] = 0.0f; cnt[c] = 0; from_left[c] = 0; from_right[c] = 0; }
+  for (int c = 0; c < CMAX; ++c) {
+    s_pair[c * kRcThreads + tid] = make_float2(0.0f, 0.0f);
+    s_cnt3[c * kRcThreads + tid] = 0ull;
+  }
   const uint8_t* ir = idx + n * K;
   const float* dr = delta_w + n * ldw;
   uint8_t* outr = new_idx + n * K;
+  // branch-free: s_gl[i] / s_gr[i] are the half-gaps to the left / right of cluster i, infinite at the edges
   auto one = [&](int i, float dw) {
-    int j = i;
-    if (i > 0 && dw < -s_half[i - 1]) j = i - 1;
-    else if (i < C - 1 && dw > s_half[i]) j = i + 1;
-#pragma unroll
-    for (int c = 0; c < CMAX; ++c) {
-      const bool mine = c == j;
-      const float x = mine ? dw : 0.0f;
-      const float t = __fadd_rn(hi[c], x);                       // two-sum of (hi, x)
-      const float bb = __fsub_rn(t, hi[c]);
-      const float err = __fadd_rn(__fsub_rn(hi[c], __fsub_rn(t, bb)), __fsub_rn(x, bb));
-      hi[c] = t;
-      lo[c] = __fadd_rn(lo[c], err);
-      cnt[c] += mine ? 1 : 0;
-      from_left[c] += (mine && i < j) ? 1 : 0;
-      from_right[c] += (mine && i > j) ? 1 : 0;
-    }
+    const int left = dw < -s_gl[i] ? 1 : 0;
+    const int right = (dw > s_gr[i] ? 1 : 0) & (left ^ 1);
+    const int j = i - left + right;
+    const int slot = j * kRcThreads + tid;
+    const float2 p = s_pair[slot];
+    const float t = __fadd_rn(p.x, dw);                          // two-sum of (hi, dw)
+    const float bb = __fsub_rn(t, p.x);
+    const float err = __fadd_rn(__fsub_rn(p.x, __fsub_rn(t, bb)), __fsub_rn(dw, bb));
+    s_pair[slot] = make_float2(t, __fadd_rn(p.y, err));
+    s_cnt3[slot] += 1ull + ((unsigned long long)right << 21) + ((unsigned long long)left << 42);
     return (uint32_t)j;
   };
   if (vec) {      // 16 weights per thread and step: one 16-byte index load, four 16-byte update loads, one 16-byte store
@@ -79,26 +85,44 @@ __global__ void __launch_bounds__(kRcThreads) reclassify_kernel(const uint8_t* _
   } else {
     for (int64_t k = tid; k < K; k += kRcThreads) outr[k] = (uint8_t)one(ir[k], dr[k]);
   }
+  // Block reduction of the pairs and counts, still in binary32 pairs (binary64 operations only on the C final values
+  // of the row: they are slow enough here that a few dozen per thread dominated the kernel), fixed order.
+  auto two_sum = [](float& h, float& l, float h2, float l2) {
+    const float t = __fadd_rn(h, h2);
+    const float bb = __fsub_rn(t, h);
+    const float err = __fadd_rn(__fsub_rn(h, __fsub_rn(t, bb)), __fsub_rn(h2, bb));
+    h = t;
+    l = __fadd_rn(__fadd_rn(l, l2), err);
+  };
 #pragma unroll
   for (int c = 0; c < CMAX; ++c) {
-    double v = (double)hi[c] + (double)lo[c];
-    if (c < C) {
-      if (c > 0) v += (double)from_left[c] * ((double)s_c[c - 1] - (double)s_c[c]);
-      if (c < C - 1) v += (double)from_right[c] * ((double)s_c[c + 1] - (double)s_c[c]);
-    }
-    int q = cnt[c];
+    const int slot = c * kRcThreads + tid;
+    float h = s_pair[slot].x, l = s_pair[slot].y;
+    const unsigned long long c3 = s_cnt3[slot];
+    int q = (int)(c3 & 0x1fffffull), fl = (int)((c3 >> 21) & 0x1fffffull), fr = (int)((c3 >> 42) & 0x1fffffull);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
-      v += __shfl_xor_sync(0xffffffffu, v, o);
+      const float h2 = __shfl_xor_sync(0xffffffffu, h, o), l2 = __shfl_xor_sync(0xffffffffu, l, o);
+      two_sum(h, l, h2, l2);
       q += __shfl_xor_sync(0xffffffffu, q, o);
+      fl += __shfl_xor_sync(0xffffffffu, fl, o);
+      fr += __shfl_xor_sync(0xffffffffu, fr, o);
     }
-    if (lane == 0) { s_sum[warp][c] = v; s_cnt[warp][c] = q; }
+    if (lane == 0) {
+      s_wh[warp][c] = h; s_wl[warp][c] = l; s_cnt[warp][c] = q; s_wfl[warp][c] = fl; s_wfr[warp][c] = fr;
+    }
   }
   __syncthreads();
   if (tid < C) {
-    double v = 0.0;
-    int q = 0;
-    for (int w = 0; w < kRcThreads / 32; ++w) { v += s_sum[w][tid]; q += s_cnt[w][tid]; }
+    float h = 0.0f, l = 0.0f;
+    int q = 0, fl = 0, fr = 0;
+    for (int w = 0; w < kRcThreads / 32; ++w) {
+      two_sum(h, l, s_wh[w][tid], s_wl[w][tid]);
+      q += s_cnt[w][tid]; fl += s_wfl[w][tid]; fr += s_wfr[w][tid];
+    }
+    double v = (double)h + (double)l;
+    if (tid > 0) v += (double)fl * ((double)s_c[tid - 1] - (double)s_c[tid]);
+    if (tid < C - 1) v += (double)fr * ((double)s_c[tid + 1] - (double)s_c[tid]);
     delta_c[n * C + tid] = v;
     counts[n * C + tid] = q;
   }
@@ -111,9 +135,18 @@ lcd_status launch_reclassify(const uint8_t* idx, const uint16_t* codebook, const
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   auto al16 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; };
   const bool vec = K % 16 == 0 && ldw % 4 == 0 && al16(idx) && al16(delta_w) && al16(new_idx);
-  if (C <= 4) reclassify_kernel<4><<<(unsigned)N, kRcThreads, 0, s>>>(idx, codebook, delta_w, K, ldw, C, new_idx, delta_c, counts, vec);
-  else if (C <= 8) reclassify_kernel<8><<<(unsigned)N, kRcThreads, 0, s>>>(idx, codebook, delta_w, K, ldw, C, new_idx, delta_c, counts, vec);
-  else reclassify_kernel<kRcMaxC><<<(unsigned)N, kRcThreads, 0, s>>>(idx, codebook, delta_w, K, ldw, C, new_idx, delta_c, counts, vec);
+  if (C <= 4) reclassify_kernel<4><<<(unsigned)N, kRcThreads, 4 * kRcThreads * 16, s>>>(idx, codebook, delta_w, K, ldw, C, new_idx, delta_c, counts, vec);
+  else if (C <= 8) reclassify_kernel<8><<<(unsigned)N, kRcThreads, 8 * kRcThreads * 16, s>>>(idx, codebook, delta_w, K, ldw, C, new_idx, delta_c, counts, vec);
+  else {
+    static bool attr_set = false;     // 80 KB of dynamic shared memory needs the opt-in
+    if (!attr_set) {
+      const cudaError_t ea = cudaFuncSetAttribute(reclassify_kernel<kRcMaxC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                  kRcMaxC * kRcThreads * 16);
+      if (ea != cudaSuccess) { set_cuda_error((int)ea); return LCD_ERR_CUDA; }
+      attr_set = true;
+    }
+    reclassify_kernel<kRcMaxC><<<(unsigned)N, kRcThreads, kRcMaxC * kRcThreads * 16, s>>>(idx, codebook, delta_w, K, ldw, C, new_idx, delta_c, counts, vec);
+  }
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
   return LCD_OK;
