@@ -228,6 +228,27 @@ __device__ __forceinline__ void stage_window(uint32_t* dst, const uint32_t* src,
   }
 }
 
+// Levels of the 8 columns of group j (t = x * inv_s given) into a staged window: clip(rint(t * r)) as signed bytes in
+// the lookup order.
+template <int BITS>
+__device__ __forceinline__ void store_levels(uint32_t* dst, int j, const float (&tv)[8], float r) {
+  uint32_t b[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    float q = rintf(__fmul_rn(tv[i], r));
+    q = fminf(fmaxf(q, -8.0f), 7.0f);
+    b[i] = (uint32_t)(int)q & 0xffu;
+  }
+  const int quarter = j >> 2, w = j & 3;
+  if (BITS == 2) {
+    dst[quarter * 8 + (w & 1) + 4 * (w >> 1)] = b[0] | (b[2] << 8) | (b[4] << 16) | (b[6] << 24);
+    dst[quarter * 8 + 2 + (w & 1) + 4 * (w >> 1)] = b[1] | (b[3] << 8) | (b[5] << 16) | (b[7] << 24);
+  } else {
+    dst[quarter * 8 + 2 * w] = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
+    dst[quarter * 8 + 2 * w + 1] = b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24);
+  }
+}
+
 // The same window straight from the fp16 activations (input transformation of Section 4.1 fused into the lookup
 // kernel): level = clip(rint((x * inv_s) * r)), r = 7 / A with A the token's max |x * inv_s| (found beforehand),
 // every step one binary32 operation as in quantize.cu, so the levels are the ones that kernel would write.
@@ -261,21 +282,7 @@ __device__ __forceinline__ void stage_window_from_x(uint32_t* dst, const __half*
       for (int i = 0; i < 8; ++i)
         tv[i] = k + i < K ? __fmul_rn(__half2float(xr[k + i]), inv_smooth ? __ldg(inv_smooth + k + i) : 1.0f) : 0.0f;
     }
-    uint32_t b[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      float q = rintf(__fmul_rn(tv[i], r));
-      q = fminf(fmaxf(q, -8.0f), 7.0f);
-      b[i] = (uint32_t)(int)q & 0xffu;
-    }
-    const int quarter = j >> 2, w = j & 3;
-    if (BITS == 2) {
-      dst[quarter * 8 + (w & 1) + 4 * (w >> 1)] = b[0] | (b[2] << 8) | (b[4] << 16) | (b[6] << 24);
-      dst[quarter * 8 + 2 + (w & 1) + 4 * (w >> 1)] = b[1] | (b[3] << 8) | (b[5] << 16) | (b[7] << 24);
-    } else {
-      dst[quarter * 8 + 2 * w] = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
-      dst[quarter * 8 + 2 * w + 1] = b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24);
-    }
+    store_levels<BITS>(dst, j, tv, r);
   }
 }
 
@@ -492,14 +499,18 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
   bool aborted = false;
   Cursor fc, cc;
 
+  uint64_t stream_policy;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_policy));
   auto issue_stage = [&]() {        // f_left > 0
     const uint32_t n = f_left < (uint32_t)kStageItems ? f_left : (uint32_t)kStageItems;
     if (lane == 0) {
       const uint32_t bar = bar0 + 8u * f_slot, bytes = n * ITEM, dst = ring_u32 + f_slot * SLOT;
       asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+      // weights are read once: evict-first keeps them from displacing what every CTA and every launch re-reads
+      // (activations, smoothing factors, codebooks) from L2
       asm volatile(
-          "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-          ::"r"(dst), "l"(f_src), "r"(bytes), "r"(bar) : "memory");
+          "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+          ::"r"(dst), "l"(f_src), "r"(bytes), "r"(bar), "l"(stream_policy) : "memory");
     }
     f_src += (size_t)n * ITEM;
     f_left -= n;
@@ -535,12 +546,75 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
   uint32_t tables_rp = 0xffffffffu, next_rp = cc.rp < geo.n_rp ? cc.rp : 0;
   next_a = load_codebook<BITS>(P.codebook + ((size_t)next_rp * 16 + g) * (1 << BITS));
   next_b = load_codebook<BITS>(P.codebook + ((size_t)next_rp * 16 + 8 + g) * (1 << BITS));
+  // act_bits == 16, one token, one panel, at most kFastChunks * 4096 columns: the products x * inv_s stay in
+  // registers between the maximum and the rounding, and the lines are asked into L2 before the dependency wait
+  // (the weight stream evicts them between launches; a prefetch cannot read stale data, L2 is the coherence point)
+  constexpr int kFastChunks = 3;
+  const bool fused = P.act_bits == 16;
+  const bool fast_stage = fused && P.x_vec && n_tok == 1 && P.n_panels == 1 && P.K <= kFastChunks * kThreads * 8;
+  if (fast_stage) {
+#pragma unroll
+    for (int c = 0; c < kFastChunks; ++c) {
+      const int k = (c * kThreads + tid) * 8;
+      if (k < P.K) {
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(P.x + k));
+        if (P.inv_smooth) {
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(P.inv_smooth + k));
+        }
+      }
+    }
+  }
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
   // act_bits == 16: the tokens' maxima A = max_k |x_k * inv_s_k| first (each CTA for itself; x is a few KB in L2)
-  const bool fused = P.act_bits == 16;
   float* s_amax = reinterpret_cast<float*>(smem + kWarps * kMaxDepth * 8);   // 16 floats between barriers and tickets
-  if (fused) {
+  if (fast_stage) {
+    float* part = reinterpret_cast<float*>(act_s);
+    float tv[kFastChunks][8];
+    float amax = 0.0f;
+#pragma unroll
+    for (int c = 0; c < kFastChunks; ++c) {
+      const int k = (c * kThreads + tid) * 8;
+      if (k < P.K) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(P.x + k);
+        const __half2* h = reinterpret_cast<const __half2*>(&raw);
+        float f[8];
+        if (P.inv_smooth) {
+          const float4 a = __ldg(reinterpret_cast<const float4*>(P.inv_smooth + k));
+          const float4 b = __ldg(reinterpret_cast<const float4*>(P.inv_smooth + k + 4));
+          f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+        } else {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) f[i] = 1.0f;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 v = __half22float2(h[i]);
+          tv[c][2 * i] = __fmul_rn(v.x, f[2 * i]);
+          tv[c][2 * i + 1] = __fmul_rn(v.y, f[2 * i + 1]);
+          amax = fmaxf(amax, fmaxf(fabsf(tv[c][2 * i]), fabsf(tv[c][2 * i + 1])));
+        }
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if (lane == 0) part[warp] = amax;
+    __syncthreads();
+    float A = 0.0f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) A = fmaxf(A, part[w]);
+    if (tid == 0) s_amax[0] = A;
+    __syncthreads();                                   // every thread has read the partial maxima: the window may be written
+    const float r = A > 0.0f ? __fdiv_rn(7.0f, A) : 0.0f;
+    uint32_t* dst = reinterpret_cast<uint32_t*>(act_s);
+#pragma unroll
+    for (int c = 0; c < kFastChunks; ++c) {
+      const int k = (c * kThreads + tid) * 8;
+      if (k < P.K) store_levels<BITS>(dst, k >> 3, tv[c], r);
+    }
+    const float zero[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
+    for (int j = (P.K >> 3) + tid; j < P.n_kt * 32; j += kThreads) store_levels<BITS>(dst, j, zero, 0.0f);   // padding columns
+  } else if (fused) {
     float* part = reinterpret_cast<float*>(act_s);                            // [kWarps][16], before the windows exist
     for (int m = 0; m < n_tok; ++m) {
       const __half* xr = P.x + (size_t)m * P.ldx;
@@ -728,7 +802,7 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
     for (uint32_t wdw = 0; wdw < 2 && pbase + wdw <= pB; ++wdw) {
       const uint32_t pn = pbase + wdw;
       const int n_words = (int)geo.panel_width(pn) * 32;
-      for (int m = 0; m < n_tok; ++m) {
+      for (int m = 0; m < n_tok && !fast_stage; ++m) {
         uint32_t* dst = reinterpret_cast<uint32_t*>(act_s + wdw * win_bytes + m * P.tstride);
         if (fused) {
           const float A = s_amax[m];
@@ -946,7 +1020,9 @@ lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void*
     if (p.act_bits == 16 && act_bytes < (size_t)kWarps * 16 * sizeof(float)) act_bytes = (size_t)kWarps * 16 * sizeof(float);
   }
   // CTAs per problem: one each, then one more at a time to the problem whose most loaded CTA has the most
-  // items (a CTA owns whole runs), until every SM has one
+  // work (a CTA owns whole runs), until every SM has one.  Work = items + the CTA's fixed cost of staging the
+  // tokens' levels, in items (measured: about 1 item per token and 1024 columns from stored levels, 3 when the
+  // kernel quantises x itself), so that CTAs of long-row problems get fewer items and all finish together
   const int n_sm = sm_count();
   int grid = 0;
   {
@@ -962,7 +1038,10 @@ lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void*
       int best = -1;
       long long best_load = 0;
       for (int i = 0; i < count; ++i) {
-        const long long load = ((runs[i] + given[i] - 1) / given[i]) * batch.p[i].pw;
+        const GemvProblem& gp = batch.p[i];
+        const long long tokens = gp.M < 8 * MG ? gp.M : 8 * MG;
+        const long long stage = (gp.act_bits == 16 ? 3 : 1) * tokens * ((long long)gp.n_kt * 256 / 1024);
+        const long long load = ((runs[i] + given[i] - 1) / given[i]) * gp.pw + stage;
         if (given[i] < runs[i] && (best < 0 || load > best_load)) { best = i; best_load = load; }
       }
       if (best < 0) break;
