@@ -552,14 +552,20 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
   constexpr int kFastChunks = 3;
   const bool fused = P.act_bits == 16;
   const bool fast_stage = fused && P.x_vec && n_tok == 1 && P.n_panels == 1 && P.K <= kFastChunks * kThreads * 8;
+  float fsm[kFastChunks][8];          // the smoothing factors do not depend on the previous kernel: read them now
   if (fast_stage) {
 #pragma unroll
     for (int c = 0; c < kFastChunks; ++c) {
       const int k = (c * kThreads + tid) * 8;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) fsm[c][i] = 1.0f;
       if (k < P.K) {
         asm volatile("prefetch.global.L2 [%0];" ::"l"(P.x + k));
         if (P.inv_smooth) {
-          asm volatile("prefetch.global.L2 [%0];" ::"l"(P.inv_smooth + k));
+          const float4 a = __ldg(reinterpret_cast<const float4*>(P.inv_smooth + k));
+          const float4 b = __ldg(reinterpret_cast<const float4*>(P.inv_smooth + k + 4));
+          fsm[c][0] = a.x; fsm[c][1] = a.y; fsm[c][2] = a.z; fsm[c][3] = a.w;
+          fsm[c][4] = b.x; fsm[c][5] = b.y; fsm[c][6] = b.z; fsm[c][7] = b.w;
         }
       }
     }
@@ -578,20 +584,11 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
       if (k < P.K) {
         const uint4 raw = *reinterpret_cast<const uint4*>(P.x + k);
         const __half2* h = reinterpret_cast<const __half2*>(&raw);
-        float f[8];
-        if (P.inv_smooth) {
-          const float4 a = __ldg(reinterpret_cast<const float4*>(P.inv_smooth + k));
-          const float4 b = __ldg(reinterpret_cast<const float4*>(P.inv_smooth + k + 4));
-          f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
-        } else {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) f[i] = 1.0f;
-        }
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float2 v = __half22float2(h[i]);
-          tv[c][2 * i] = __fmul_rn(v.x, f[2 * i]);
-          tv[c][2 * i + 1] = __fmul_rn(v.y, f[2 * i + 1]);
+          tv[c][2 * i] = __fmul_rn(v.x, fsm[c][2 * i]);
+          tv[c][2 * i + 1] = __fmul_rn(v.y, fsm[c][2 * i + 1]);
           amax = fmaxf(amax, fmaxf(fabsf(tv[c][2 * i]), fabsf(tv[c][2 * i + 1])));
         }
       }
