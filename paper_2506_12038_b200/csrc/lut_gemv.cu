@@ -539,8 +539,9 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
     if (round_hi < round_lo) round_hi = round_lo;
     cursor_set(fc, round_lo, P);
     cc = fc;
-    for (int i = 0; i < kDepth; ++i) fetch_more(round_hi);
   }
+  // Small loads first, bulk copies after them: an SM's loads return in the order they were queued, and a load
+  // issued behind the ring's first fill waits for all of it (two microseconds for three stages of sixteen warps).
   RowTables<BITS, KIND> Ta, Tb;           // rows 16*rp + g and 16*rp + 8 + g
   RawCodebook<BITS> next_a, next_b;
   uint32_t tables_rp = 0xffffffffu, next_rp = cc.rp < geo.n_rp ? cc.rp : 0;
@@ -570,20 +571,30 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
       }
     }
   }
+  // With the fast staging only one stage per warp is queued before the activations are asked for; the others follow
+  // right behind that request.
+  for (int i = 0; i < (fast_stage ? 1 : kDepth); ++i) fetch_more(round_hi);
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
   // act_bits == 16: the tokens' maxima A = max_k |x_k * inv_s_k| first (each CTA for itself; x is a few KB in L2)
   float* s_amax = reinterpret_cast<float*>(smem + kWarps * kMaxDepth * 8);   // 16 floats between barriers and tickets
   if (fast_stage) {
     float* part = reinterpret_cast<float*>(act_s);
+    uint4 xraw[kFastChunks];
+#pragma unroll
+    for (int c = 0; c < kFastChunks; ++c) {
+      const int k = (c * kThreads + tid) * 8;
+      xraw[c] = make_uint4(0u, 0u, 0u, 0u);
+      if (k < P.K) xraw[c] = *reinterpret_cast<const uint4*>(P.x + k);
+    }
+    for (int i = 1; i < kDepth; ++i) fetch_more(round_hi);
     float tv[kFastChunks][8];
     float amax = 0.0f;
 #pragma unroll
     for (int c = 0; c < kFastChunks; ++c) {
       const int k = (c * kThreads + tid) * 8;
       if (k < P.K) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(P.x + k);
-        const __half2* h = reinterpret_cast<const __half2*>(&raw);
+        const __half2* h = reinterpret_cast<const __half2*>(&xraw[c]);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const float2 v = __half22float2(h[i]);
