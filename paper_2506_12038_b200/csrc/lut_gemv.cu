@@ -571,9 +571,10 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
       }
     }
   }
-  // With the fast staging only one stage per warp is queued before the activations are asked for; the others follow
-  // right behind that request.
-  for (int i = 0; i < (fast_stage ? 1 : kDepth); ++i) fetch_more(round_hi);
+  // Only one stage per warp is queued before the activations (or their stored levels) are asked for; the others
+  // follow right behind that request.
+  fetch_more(round_hi);
+  bool ring_primed = false;
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
   // act_bits == 16: the tokens' maxima A = max_k |x_k * inv_s_k| first (each CTA for itself; x is a few KB in L2)
@@ -588,6 +589,7 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
       if (k < P.K) xraw[c] = *reinterpret_cast<const uint4*>(P.x + k);
     }
     for (int i = 1; i < kDepth; ++i) fetch_more(round_hi);
+    ring_primed = true;
     float tv[kFastChunks][8];
     float amax = 0.0f;
 #pragma unroll
@@ -822,6 +824,10 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
                              n_words, tid, P.act_bits == 8);
         }
       }
+    }
+    if (!ring_primed) {            // first round: the staging loads above are queued, now the rest of the ring
+      for (int i = 1; i < kDepth; ++i) fetch_more(round_hi);
+      ring_primed = true;
     }
     __syncthreads();
 
