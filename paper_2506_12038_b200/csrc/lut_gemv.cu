@@ -485,8 +485,6 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     s_ticket[warp] = 0;
   }
-  if (kSmemCombine)
-    for (int i = lane; i < ACC_INTS; i += 32) s_acc[warp * ACC_INTS + i] = 0;
   __syncwarp();
 
   // Ring state.  Fetch side: next slot to fill, stages in flight, the rest of the segment being fetched (a
@@ -576,6 +574,10 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
   fetch_more(round_hi);
   bool ring_primed = false;
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  // the warp's combine slot is cleared here, with the first loads already under way (every use of it comes after
+  // the block-wide barrier that ends the staging)
+  if (kSmemCombine && !fast_stage)
+    for (int i = lane; i < ACC_INTS; i += 32) s_acc[warp * ACC_INTS + i] = 0;
 
   // act_bits == 16: the tokens' maxima A = max_k |x_k * inv_s_k| first (each CTA for itself; x is a few KB in L2)
   float* s_amax = reinterpret_cast<float*>(smem + kWarps * kMaxDepth * 8);   // 16 floats between barriers and tickets
@@ -590,6 +592,8 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
     }
     for (int i = 1; i < kDepth; ++i) fetch_more(round_hi);
     ring_primed = true;
+    if (kSmemCombine)                        // cleared while the activations are on their way
+      for (int i = lane; i < ACC_INTS; i += 32) s_acc[warp * ACC_INTS + i] = 0;
     float tv[kFastChunks][8];
     float amax = 0.0f;
 #pragma unroll
