@@ -294,7 +294,7 @@ struct Cursor {
 __device__ __forceinline__ void cursor_set(Cursor& c, uint32_t x, const GemvProblem& P) {
   const uint32_t panel_items = (uint32_t)P.n_rp * (uint32_t)P.pw;
   c.x = x;
-  c.pn = x / panel_items;
+  c.pn = P.n_panels == 1 ? 0u : x / panel_items;
   const uint32_t r = x - c.pn * panel_items;
   const int left = P.n_kt - (int)c.pn * P.pw;
   c.pw = (uint32_t)(left < P.pw ? (left > 0 ? left : 1) : P.pw);
@@ -321,7 +321,10 @@ __device__ __forceinline__ void cursor_advance(Cursor& c, uint32_t n, const Gemv
   }
 }
 // Even split of n items over w parts: first item of part i, and the part that owns item x.
-__device__ __forceinline__ uint32_t part_begin(uint32_t i, uint32_t n, uint32_t w) { return i * n / w; }
+__device__ __forceinline__ uint32_t part_begin(uint32_t i, uint32_t n, uint32_t w) {
+  return w == (uint32_t)kWarps ? (i * n) >> 4 : i * n / w;      // the split over a CTA's 16 warps needs no division
+}
+static_assert(kWarps == 16, "part_begin shifts by log2(kWarps)");
 __device__ __forceinline__ uint32_t part_of(uint32_t x, uint32_t n, uint32_t w) { return ((x + 1) * w + n - 1) / n - 1; }
 
 // Runs.  A run is the items of one 16-row group inside one panel (pw consecutive items in memory); runs are
@@ -336,6 +339,7 @@ struct RunGeometry {
   // first item (panel-major numbering) of run r; r == n_runs gives the item count
   __device__ __forceinline__ uint32_t run_start(uint32_t r) const {
     if (r >= n_runs) return n_items;
+    if (n_panels == 1) return r * pw;          // the common case without a division (they are on the launch's critical path)
     const uint32_t pn = r / n_rp, rp = r - pn * n_rp;
     return pn * n_rp * pw + rp * panel_width(pn);
   }
@@ -465,7 +469,7 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
   const uint32_t wx0 = warp_active ? cx0 + part_begin(warp, c_items, nw) : cx0;
   const uint32_t wx1 = warp_active ? cx0 + part_begin(warp + 1, c_items, nw) : cx0;
   const uint32_t panel_items = geo.n_rp * geo.pw;
-  const uint32_t pA = cx0 / panel_items, pB = (cx1 - 1) / panel_items;
+  const uint32_t pA = geo.n_panels == 1 ? 0u : cx0 / panel_items, pB = geo.n_panels == 1 ? 0u : (cx1 - 1) / panel_items;
 
   // shared memory: mbarriers | combine tickets | combine slots | rings | activation windows
   int* s_ticket = reinterpret_cast<int*>(smem + kBarBytes - 64);
