@@ -36,10 +36,10 @@ NCU_TRAFFIC = {
     # profiles/lut_gemv_kernel_llama7b_2bit_m1.md: one launch (input transformation + lookup) of configs[1] at M = 1
     ("lut_gemv.cu", 1, 1): {"sha256": "3c7655a830ae52fd5cdce4571d79daebc70f9cc9f85e8357843aa4d5cb1b6e8a", "bytes_per_launch": 51208704 + 20224},
     # profiles/dense_tc_kernel_llama13b_2bit_m2048.md: the layer's seven launches of configs[3]: q captured
-    # (17.11 + 0.23 MB, taken four times for q/k/v/o), gate captured (28.36 + 56.16 MB, twice for gate/up), down
+    # (17.11 + 0.44 MB, taken four times for q/k/v/o), gate captured (28.37 + 56.32 MB, twice for gate/up), down
     # scaled from q by its 2.7 times longer rows (same tiles, traffic in proportion to K)
-    ("dense_tc.cu", 3, 2048): {"sha256": "edefd6132d93e9c889e32fe8be8fc1b7954a843f088f3bc771d89f17959f4a13",
-                               "bytes_per_launch": int(4 * 17.34e6 + 2 * 84.52e6 + 17.34e6 * 13824 / 5120)},
+    ("dense_tc.cu", 3, 2048): {"sha256": "c29890f9ab90dad858f8486d69f2bb16e902631e75ef856b650a66523b6d474b",
+                               "bytes_per_launch": int(4 * 17.55e6 + 2 * 84.70e6 + 17.55e6 * 13824 / 5120)},
 }
 L2_BYTES = 126e6
 ROTATE_BYTES = 300e6          # total size of the weight copies the timed loop rotates over
