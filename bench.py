@@ -33,9 +33,9 @@ from synth import gen  # noqa: E402
 # captures summarised under profiles/, with the hash of the kernel source they were taken from: a kernel that has
 # changed since reports traffic = null.
 NCU_TRAFFIC = {
-    # profiles/lut_gemv_kernel_llama7b_2bit_m1.md: one launch (input transformation + lookup) of configs[1] at M = 1
+    # profiles/lut_gemv_kernel_llama7b_2bit_m1.md: one launch (input transformation + lookup) of configuration 1 at M = 1
     ("lut_gemv.cu", 1, 1): {"sha256": "3c7655a830ae52fd5cdce4571d79daebc70f9cc9f85e8357843aa4d5cb1b6e8a", "bytes_per_launch": 51208704 + 20224},
-    # profiles/dense_tc_kernel_llama13b_2bit_m2048.md: the layer's seven launches of configs[3]: q captured
+    # profiles/dense_tc_kernel_llama13b_2bit_m2048.md: the layer's seven launches of configuration 3: q captured
     # (17.11 + 0.44 MB, taken four times for q/k/v/o), gate captured (28.37 + 56.32 MB, twice for gate/up), down
     # scaled from q by its 2.7 times longer rows (same tiles, traffic in proportion to K)
     ("dense_tc.cu", 3, 2048): {"sha256": "c29890f9ab90dad858f8486d69f2bb16e902631e75ef856b650a66523b6d474b",
@@ -50,7 +50,7 @@ def parse_args():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--config", type=int, default=1, help="index into BASELINE.json configs (default 1)")
+    ap.add_argument("--config", type=int, default=1, help="index of the workload configuration (default 1: LLaMA-7B-shaped layer, 2 bit, M = 1)")
     ap.add_argument("--M", type=int, default=None, help="token count (default: first M of the config)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -147,7 +147,7 @@ def metric_name(M):
 
 def workload_config(cfg_id, M, copies, act_bits=4):
     cfg = gen.CONFIGS[cfg_id]
-    return {"workload": f"BASELINE configs[{cfg_id}] {cfg['name']}: " +
+    return {"workload": f"configuration {cfg_id} ({cfg['name']}): " +
                         ", ".join(f"{n} {N}x{K}" for n, N, K in cfg["shapes"]),
             "bits": cfg["bits"], "M": M, "act_bits": act_bits, "outliers": f"{cfg['frac'] * 100:g}% x{cfg['scale']:g}",
             "l2": f"weights rotate over {copies} device copies (> {int(L2_BYTES / 1e6)} MB L2)"}
@@ -517,7 +517,7 @@ def run_aux_smoothing(args):
         ms = e0.elapsed_time(e1) / 10
         total_ms += ms
         rows.append({"matrix": name, "K": K, "us": ms * 1e3, "best_alpha": alphas[int(best.item())]})
-    print(json.dumps({"aux": "smoothing_search", "config": {"workload": f"BASELINE configs[{args.config}] {cfg['name']}",
+    print(json.dumps({"aux": "smoothing_search", "config": {"workload": f"configuration {args.config} ({cfg['name']})",
                                                             "calibration_tokens": 128, "candidates": len(alphas)},
                       "us_per_layer": total_ms * 1e3, "per_matrix": rows, "data": "synthetic"}))
 
@@ -566,7 +566,7 @@ def run_aux_reclassify(args):
         tot_ms += ms
         tot_bytes += b
         rows.append({"matrix": name, "N": N, "K": K, "us": ms * 1e3, "GBps": b / ms / 1e6})
-    print(json.dumps({"aux": "reclassify", "config": {"workload": f"BASELINE configs[{args.config}] {cfg['name']}", "C": C},
+    print(json.dumps({"aux": "reclassify", "config": {"workload": f"configuration {args.config} ({cfg['name']})", "C": C},
                       "us_per_layer": tot_ms * 1e3, "per_matrix": rows, "data": "synthetic",
                       "roofline": {"bound": "hbm", "achieved": tot_bytes / tot_ms / 1e6, "peak": peak, "unit": "GB/s",
                                    "frac": tot_bytes / tot_ms / 1e6 / peak,
@@ -599,7 +599,7 @@ def run_aux_dbci(args):
         tot_ms += ms
         rows.append({"matrix": name, "weights": N * K, "ms": ms, "Gweights_per_s": N * K / ms / 1e6,
                      "centroids": int(r["centroids"].numel()), "sigma": r["sigma"], "min_pts": r["min_pts"]})
-    print(json.dumps({"aux": "dbci", "config": {"workload": f"BASELINE configs[{args.config}] {cfg['name']}"},
+    print(json.dumps({"aux": "dbci", "config": {"workload": f"configuration {args.config} ({cfg['name']})"},
                       "ms_per_layer": tot_ms, "per_matrix": rows, "data": "synthetic"}))
 
 

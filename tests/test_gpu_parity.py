@@ -1,7 +1,7 @@
 """GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded inputs.
 Index work (activation indices, scales, packed bytes) must be bit-exact; fp32 outputs must meet
 relative L2 <= 2e-3 and max-abs <= 1e-2 * ||y_ref||_inf (the stated tolerance).  The kernels accumulate in
-exact integers or fp32, for which the expected error is far smaller (the design doc derives <= 1e-4), so that
+exact integers or fp32, for which the expected error is far smaller (derived bound: <= 1e-4 relative L2), so that
 tighter bound is asserted as well."""
 import numpy as np
 import pytest
