@@ -34,7 +34,7 @@ from synth import gen  # noqa: E402
 # changed since reports traffic = null.
 NCU_TRAFFIC = {
     # profiles/lut_gemv_kernel_llama7b_2bit_m1.md: one launch (input transformation + lookup) of configuration 1 at M = 1
-    ("lut_gemv.cu", 1, 1): {"sha256": "3c7655a830ae52fd5cdce4571d79daebc70f9cc9f85e8357843aa4d5cb1b6e8a", "bytes_per_launch": 51208704 + 20224},
+    ("lut_gemv.cu", 1, 1): {"sha256": "ad1eec2679f61945c235cc9c15ca7aa1a36efaf65692539c1eca2916de51bfba", "bytes_per_launch": 51208704 + 20224},
     # profiles/dense_tc_kernel_llama13b_2bit_m2048.md: the layer's seven launches of configuration 3: q captured
     # (17.11 + 0.44 MB, taken four times for q/k/v/o), gate captured (28.37 + 56.32 MB, twice for gate/up), down
     # scaled from q by its 2.7 times longer rows (same tiles, traffic in proportion to K)

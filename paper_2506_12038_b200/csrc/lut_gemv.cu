@@ -833,7 +833,7 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
         }
       }
     }
-    if (!ring_primed) {            // first round: the staging loads above are queued, now the rest of the ring
+    if (!ring_primed) {            // first pass: the staging loads above are queued, now the rest of the ring
       for (int i = 1; i < kDepth; ++i) fetch_more(round_hi);
       ring_primed = true;
     }
