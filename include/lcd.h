@@ -267,6 +267,7 @@ lcd_status lcd_dbci(const float* weights, int64_t n, void* workspace, size_t wor
  * the paper prints the left test without the sign; edge clusters have one side); never further than one cluster.
  *     delta_c[n][j] = sum over the weights that end up in j of (dw + (C_old - C_j))      (a sum, as printed)
  *   idx:           device, uint8 [N][K] cluster of every weight (one byte each, the packer's input form), < C;
+ *                  K <= 2^25;
  *   codebook_fp16: device, binary16 [N][C], 1 <= C <= 16;     delta_w: device, fp32 [N][ldw], ldw >= K;
  *   new_idx:       device out, uint8 [N][K] (may not alias idx);
  *   delta_c:       device out, fp64 [N][C];     counts: device out, int32 [N][C] members after the move.

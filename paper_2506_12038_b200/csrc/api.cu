@@ -346,7 +346,7 @@ extern "C" lcd_status lcd_reclassify(const uint8_t* idx, const uint16_t* codeboo
                                      int64_t K, int64_t ldw, int C, uint8_t* new_idx, double* delta_c, int32_t* counts,
                                      void* cuda_stream) {
   if (!idx || !codebook_fp16 || !delta_w || !new_idx || !delta_c || !counts) return LCD_ERR_INVALID_ARG;
-  if (N < 1 || K < 1 || ldw < K || C < 1 || C > 16 || N > 0x7fffffffLL || K > (1LL << 28)) return LCD_ERR_INVALID_ARG;
+  if (N < 1 || K < 1 || ldw < K || C < 1 || C > 16 || N > 0x7fffffffLL || K > (1LL << 25)) return LCD_ERR_INVALID_ARG;
   if (!aligned(codebook_fp16, 2) || !aligned(delta_w, 4) || !aligned(delta_c, 8) || !aligned(counts, 4))
     return LCD_ERR_INVALID_ARG;
   return launch_reclassify(idx, codebook_fp16, delta_w, N, K, ldw, C, new_idx, delta_c, counts, cuda_stream);

@@ -22,17 +22,15 @@ __global__ void __launch_bounds__(kRcThreads) reclassify_kernel(const uint8_t* _
                                                                 uint8_t* __restrict__ new_idx, double* __restrict__ delta_c,
                                                                 int32_t* __restrict__ counts, const bool vec) {
   __shared__ float s_c[CMAX];
-  __shared__ float s_gl[CMAX], s_gr[CMAX];  // half-gaps (C_i - C_{i-1}) / 2 and (C_{i+1} - C_i) / 2, infinite at the edges
-  __shared__ float s_wh[kRcThreads / 32][CMAX], s_wl[kRcThreads / 32][CMAX];
-  __shared__ int s_cnt[kRcThreads / 32][CMAX], s_wfl[kRcThreads / 32][CMAX], s_wfr[kRcThreads / 32][CMAX];
+  __shared__ float2 s_gap[CMAX];            // half-gaps (C_i - C_{i-1}) / 2 and (C_{i+1} - C_i) / 2, infinite at the edges
   const int64_t n = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid < C) s_c[tid] = __half2float(__ushort_as_half(codebook[n * C + tid]));
   __syncthreads();
   if (tid < CMAX) {
     const float inf = __int_as_float(0x7f800000);
-    s_gl[tid] = (tid > 0 && tid < C) ? __fmul_rn(__fsub_rn(s_c[tid], s_c[tid - 1]), 0.5f) : inf;
-    s_gr[tid] = (tid < C - 1) ? __fmul_rn(__fsub_rn(s_c[tid + 1], s_c[tid]), 0.5f) : inf;
+    s_gap[tid] = make_float2((tid > 0 && tid < C) ? __fmul_rn(__fsub_rn(s_c[tid], s_c[tid - 1]), 0.5f) : inf,
+                             (tid < C - 1) ? __fmul_rn(__fsub_rn(s_c[tid + 1], s_c[tid]), 0.5f) : inf);
   }
   __syncthreads();
   // Per thread and cluster, in the thread's own column of shared memory (indexed by the data-dependent cluster; a
@@ -40,30 +38,35 @@ __global__ void __launch_bounds__(kRcThreads) reclassify_kernel(const uint8_t* _
   // as an unevaluated pair of binary32 numbers (error-free two-sum: binary64 adds are scarce on this part) and
   // integer counts of members and of arrivals from either side; the centroid differences of the arrivals are
   // added at the end from the counts.
-  extern __shared__ unsigned long long s_dyn[];
-  float2* s_pair = reinterpret_cast<float2*>(s_dyn);                      // [CMAX][kRcThreads] (hi, lo)
-  unsigned long long* s_cnt3 = s_dyn + CMAX * kRcThreads;                 // members | arrivals from the left << 21
-                                                                          // | arrivals from the right << 42
+  extern __shared__ uint4 s_dyn[];
+  // one 16-byte slot per thread and cluster: (hi, lo, counts low word, counts high word); the 64-bit count word is
+  // members | arrivals from the left << 21 | arrivals from the right << 42.  One load and one store per weight: the
+  // load/store unit's queue is what bounds this kernel.
+  uint4* s_slot = s_dyn;                                                  // [CMAX][kRcThreads]
 #pragma unroll
-  for (int c = 0; c < CMAX; ++c) {
-    s_pair[c * kRcThreads + tid] = make_float2(0.0f, 0.0f);
-    s_cnt3[c * kRcThreads + tid] = 0ull;
-  }
+  for (int c = 0; c < CMAX; ++c) s_slot[c * kRcThreads + tid] = make_uint4(0u, 0u, 0u, 0u);
   const uint8_t* ir = idx + n * K;
   const float* dr = delta_w + n * ldw;
   uint8_t* outr = new_idx + n * K;
-  // branch-free: s_gl[i] / s_gr[i] are the half-gaps to the left / right of cluster i, infinite at the edges
+  // branch-free: s_gap[i] = (half-gap to the left, half-gap to the right) of cluster i, infinite at the edges
   auto one = [&](int i, float dw) {
-    const int left = dw < -s_gl[i] ? 1 : 0;
-    const int right = (dw > s_gr[i] ? 1 : 0) & (left ^ 1);
+    const float2 gap = s_gap[i];
+    const int left = dw < -gap.x ? 1 : 0;
+    const int right = (dw > gap.y ? 1 : 0) & (left ^ 1);
     const int j = i - left + right;
     const int slot = j * kRcThreads + tid;
-    const float2 p = s_pair[slot];
-    const float t = __fadd_rn(p.x, dw);                          // two-sum of (hi, dw)
-    const float bb = __fsub_rn(t, p.x);
-    const float err = __fadd_rn(__fsub_rn(p.x, __fsub_rn(t, bb)), __fsub_rn(dw, bb));
-    s_pair[slot] = make_float2(t, __fadd_rn(p.y, err));
-    s_cnt3[slot] += 1ull + ((unsigned long long)right << 21) + ((unsigned long long)left << 42);
+    uint4 v = s_slot[slot];
+    const float h = __uint_as_float(v.x), l = __uint_as_float(v.y);
+    const float t = __fadd_rn(h, dw);                            // two-sum of (hi, dw)
+    const float bb = __fsub_rn(t, h);
+    const float err = __fadd_rn(__fsub_rn(h, __fsub_rn(t, bb)), __fsub_rn(dw, bb));
+    unsigned long long cnt = ((unsigned long long)v.w << 32) | v.z;
+    cnt += 1ull + ((unsigned long long)right << 21) + ((unsigned long long)left << 42);
+    v.x = __float_as_uint(t);
+    v.y = __float_as_uint(__fadd_rn(l, err));
+    v.z = (uint32_t)cnt;
+    v.w = (uint32_t)(cnt >> 32);
+    s_slot[slot] = v;
     return (uint32_t)j;
   };
   if (vec) {      // 16 weights per thread and step: one 16-byte index load, four 16-byte update loads, one 16-byte store
@@ -94,37 +97,38 @@ __global__ void __launch_bounds__(kRcThreads) reclassify_kernel(const uint8_t* _
     h = t;
     l = __fadd_rn(__fadd_rn(l, l2), err);
   };
-#pragma unroll
-  for (int c = 0; c < CMAX; ++c) {
-    const int slot = c * kRcThreads + tid;
-    float h = s_pair[slot].x, l = s_pair[slot].y;
-    const unsigned long long c3 = s_cnt3[slot];
-    int q = (int)(c3 & 0x1fffffull), fl = (int)((c3 >> 21) & 0x1fffffull), fr = (int)((c3 >> 42) & 0x1fffffull);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float h2 = __shfl_xor_sync(0xffffffffu, h, o), l2 = __shfl_xor_sync(0xffffffffu, l, o);
-      two_sum(h, l, h2, l2);
-      q += __shfl_xor_sync(0xffffffffu, q, o);
-      fl += __shfl_xor_sync(0xffffffffu, fl, o);
-      fr += __shfl_xor_sync(0xffffffffu, fr, o);
-    }
-    if (lane == 0) {
-      s_wh[warp][c] = h; s_wl[warp][c] = l; s_cnt[warp][c] = q; s_wfl[warp][c] = fl; s_wfr[warp][c] = fr;
-    }
-  }
+  // One warp folds the 256 columns of slots: every lane adds its eight columns, then a butterfly over the lanes.
+  // (A butterfly in every warp made this reduction as expensive as the 16 weights a thread handles per 4096 columns.)
   __syncthreads();
-  if (tid < C) {
-    float h = 0.0f, l = 0.0f;
-    int q = 0, fl = 0, fr = 0;
-    for (int w = 0; w < kRcThreads / 32; ++w) {
-      two_sum(h, l, s_wh[w][tid], s_wl[w][tid]);
-      q += s_cnt[w][tid]; fl += s_wfl[w][tid]; fr += s_wfr[w][tid];
+  if (warp == 0) {
+#pragma unroll
+    for (int c = 0; c < CMAX; ++c) {
+      float h = 0.0f, l = 0.0f;
+      unsigned long long c3 = 0ull;
+#pragma unroll
+      for (int w = 0; w < kRcThreads / 32; ++w) {
+        const uint4 sv = s_slot[c * kRcThreads + w * 32 + lane];
+        two_sum(h, l, __uint_as_float(sv.x), __uint_as_float(sv.y));
+        c3 += ((unsigned long long)sv.w << 32) | sv.z;          // K <= 2^25: a thread counts at most 2^17, eight of them 2^20 < 2^21
+      }
+      // fields of the packed count word may carry into each other once summed over threads: unpack before the lanes meet
+      int q = (int)(c3 & 0x1fffffull), fl = (int)((c3 >> 21) & 0x1fffffull), fr = (int)((c3 >> 42) & 0x1fffffull);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float h2 = __shfl_xor_sync(0xffffffffu, h, o), l2 = __shfl_xor_sync(0xffffffffu, l, o);
+        two_sum(h, l, h2, l2);
+        q += __shfl_xor_sync(0xffffffffu, q, o);
+        fl += __shfl_xor_sync(0xffffffffu, fl, o);
+        fr += __shfl_xor_sync(0xffffffffu, fr, o);
+      }
+      if (lane == 0 && c < C) {
+        double v = (double)h + (double)l;
+        if (c > 0) v += (double)fl * ((double)s_c[c - 1] - (double)s_c[c]);
+        if (c < C - 1) v += (double)fr * ((double)s_c[c + 1] - (double)s_c[c]);
+        delta_c[n * C + c] = v;
+        counts[n * C + c] = q;
+      }
     }
-    double v = (double)h + (double)l;
-    if (tid > 0) v += (double)fl * ((double)s_c[tid - 1] - (double)s_c[tid]);
-    if (tid < C - 1) v += (double)fr * ((double)s_c[tid + 1] - (double)s_c[tid]);
-    delta_c[n * C + tid] = v;
-    counts[n * C + tid] = q;
   }
 }
 
