@@ -491,38 +491,104 @@ def _nearest_rank(sorted_vals: np.ndarray, p: float) -> float:
     return float(sorted_vals[min(max(k, 0), sorted_vals.size - 1)])
 
 
+def _dbci_seeds(xd: np.ndarray):
+    """Steps 2-4 on the sorted binary64 copy of the weights: sigma, the two seed clusters as index ranges
+    [0, L) and [R, n), MinPts and eps."""
+    n = xd.size
+    pos = xd[xd > 0]
+    neg = -xd[xd < 0][::-1]
+    sigma = sum(_nearest_rank(pos, p) + _nearest_rank(neg, p) for p in DBCI_PERCENTILES) / 12.0
+    L = int(np.count_nonzero(xd <= xd[0] + sigma))            # sorted: these are the first L points
+    R = n - int(np.count_nonzero(xd >= xd[-1] - sigma))       # and these the points from R on
+    R = max(R, L)                          # a weight both seeds reach stays with the left one
+    n_right = n - R
+    min_pts = min(L, n_right) if n_right > 0 else L      # an empty right cluster cannot set MinPts to zero
+    return sigma, L, R, int(min_pts), sigma / min_pts
+
+
+def _dbci_finish(x, xd, sigma, L, R, min_pts, eps, mid):
+    """Labels of all points from the labels `mid` of the middle points (0.. = DBSCAN clusters from left to
+    right, -1 noise) and step 6: the centroid of a cluster is its lower median (an L1 minimiser)."""
+    n = xd.size
+    labels = np.full(n, -1, dtype=np.int64)
+    labels[:L] = 0
+    n_mid = int(mid.max()) + 1 if mid.size and mid.max() >= 0 else 0
+    labels[L:R] = np.where(mid >= 0, mid + 1, -1)
+    if n - R > 0:
+        labels[R:] = n_mid + 1
+    cents = []
+    for c in range(n_mid + 2):
+        members = np.flatnonzero(labels == c)
+        if members.size:
+            cents.append(xd[members[(members.size - 1) // 2]])
+    return {"sigma": sigma, "min_pts": int(min_pts), "eps": eps, "left": L, "right": n - R, "labels": labels,
+            "centroids": np.array(cents), "sorted": x}
+
+
 def dbci(weights):
-    """Density-based centroid initialisation, the six steps of Section 3.1, on a flat array of binary32 weights.
-    All comparisons and the few scalar operations are binary64 on the binary32 data.
+    """Density-based centroid initialisation, the six steps of Section 3.1, on a flat array of binary32 weights,
+    written out plainly (quadratic in the number of weights: for small inputs).  All comparisons and the few
+    scalar operations are binary64 on the binary32 data.
 
     1. sort;  2. sigma = (sum over the 68.27 / 95.44 / 99.74 % nearest-rank percentiles of the positive weights and
     of the magnitudes of the negative weights) / 12;  3. the smallest and the largest weight seed two clusters that
     take every point within sigma of them (the right one gives way if they overlap);  4. MinPts = the smaller of the
-    two counts, eps = sigma / MinPts;  5. DBSCAN on the remaining points alone: a point with at least MinPts points
-    (itself included) within eps is a core point, core points closer than eps chain into one cluster, another point
-    within eps of a core point joins the cluster of its nearest core point (the left one on a tie), the rest is
-    noise;  6. the centroid of a cluster is its lower median (an L1 minimiser).
+    two counts, eps = sigma / MinPts;  5. DBSCAN on the remaining points alone: the eps-neighbourhood of a point is
+    found by a scan over all of them (the point itself counts); a point with at least MinPts neighbours is a core
+    point; clusters grow breadth-first from core point to core point; another point within eps of a core point
+    joins the cluster of its nearest core point, found by explicit search (the left one on a tie: textbook DBSCAN
+    leaves this to the visiting order), the rest is noise;  6. the centroid of a cluster is its lower median.
 
     Returns a dict: sigma, min_pts, eps, left (count), right (count), labels (int64 per sorted point: cluster number
     in ascending order of position, -1 noise), centroids (float64, ascending), sorted (the sorted weights)."""
     x = np.sort(np.asarray(weights, dtype=np.float32).ravel())
     xd = x.astype(np.float64)
+    if xd.size == 0:
+        raise ValueError("no weights")
+    sigma, L, R, min_pts, eps = _dbci_seeds(xd)
+    y = xd[L:R]
+    m = y.size
+    neighbours = [np.flatnonzero(np.abs(y - y[i]) <= eps) for i in range(m)]         # region query: full scan
+    core = np.array([nb.size >= min_pts for nb in neighbours], dtype=bool)
+    mid = np.full(m, -1, dtype=np.int64)
+    n_clusters = 0
+    for i in range(m):                     # ascending position, so clusters are numbered from left to right
+        if not core[i] or mid[i] >= 0:
+            continue
+        mid[i] = n_clusters
+        queue = [i]
+        while queue:                       # breadth-first over core points
+            a = queue.pop(0)
+            for b in neighbours[a]:
+                if core[b] and mid[b] < 0:
+                    mid[b] = n_clusters
+                    queue.append(int(b))
+        n_clusters += 1
+    cores = np.flatnonzero(core)
+    for i in np.flatnonzero(~core):        # border points and noise
+        best, best_d = -1, np.inf
+        for c in cores:                    # ascending position: a strict comparison keeps the left one on a tie
+            d = abs(y[c] - y[i])
+            if d <= eps and d < best_d:
+                best, best_d = int(c), d
+        if best >= 0:
+            mid[i] = mid[best]
+    return _dbci_finish(x, xd, sigma, L, R, min_pts, eps, mid)
+
+
+def dbci_scan(weights):
+    """The result of ``dbci`` for large inputs, computed on the sorted array with searches and running
+    extrema instead of scans over all pairs (n log n).  tests/test_oracle_pins.py checks it against ``dbci``
+    on small inputs with many ties; it is used where the plain form would take hours."""
+    x = np.sort(np.asarray(weights, dtype=np.float32).ravel())
+    xd = x.astype(np.float64)
     n = xd.size
     if n == 0:
         raise ValueError("no weights")
-    pos = xd[xd > 0]
-    neg = -xd[xd < 0][::-1]
-    sigma = sum(_nearest_rank(pos, p) + _nearest_rank(neg, p) for p in DBCI_PERCENTILES) / 12.0
-    L = int(np.searchsorted(xd, xd[0] + sigma, side="right"))
-    R = int(np.searchsorted(xd, xd[-1] - sigma, side="left"))
-    R = max(R, L)
-    min_pts = min(L, n - R) if n - R > 0 else L
-    eps = sigma / min_pts
+    sigma, L, R, min_pts, eps = _dbci_seeds(xd)
     y = xd[L:R]
     m = y.size
-    labels = np.full(n, -1, dtype=np.int64)
-    labels[:L] = 0
-    n_mid = 0
+    mid = np.full(m, -1, dtype=np.int64)
     if m:
         lo = np.searchsorted(y, y - eps, side="left")
         hi = np.searchsorted(y, y + eps, side="right")
@@ -533,7 +599,6 @@ def dbci(weights):
         prev_before = np.concatenate([[-1], prev_core[:-1]])                         # nearest core strictly before i
         start = core & ((prev_before < 0) | ((y - y[np.maximum(prev_before, 0)]) > eps))
         cid = np.cumsum(start) - 1                                                   # cluster of a core point
-        mid = np.full(m, -1, dtype=np.int64)
         mid[core] = cid[core]
         nc = np.flatnonzero(~core)
         if nc.size:
@@ -544,14 +609,4 @@ def dbci(weights):
             take_right = (dr <= eps) & ~take_left
             mid[nc[take_left]] = cid[pc[take_left]]
             mid[nc[take_right]] = cid[nx[take_right]]
-        n_mid = int(start.sum())
-        labels[L:R] = np.where(mid >= 0, mid + 1, -1)
-    if n - R > 0:
-        labels[R:] = n_mid + 1
-    cents = []
-    for c in range(n_mid + 2):
-        members = np.flatnonzero(labels == c)
-        if members.size:
-            cents.append(xd[members[(members.size - 1) // 2]])
-    return {"sigma": sigma, "min_pts": int(min_pts), "eps": eps, "left": L, "right": n - R, "labels": labels,
-            "centroids": np.array(cents), "sorted": x}
+    return _dbci_finish(x, xd, sigma, L, R, min_pts, eps, mid)

@@ -502,7 +502,7 @@ def test_dbci_sigma_of_a_gaussian_and_hand_example():
     # half-normal percentiles at 68.27 / 95.44 / 99.74 % are 1, 2, 3 sigma: six of them sum to 12 sigma
     rng = np.random.default_rng(41)
     w = (rng.standard_normal(200000) * 0.02).astype(np.float32)
-    r = O.dbci(w)
+    r = O.dbci_scan(w)         # 200000 weights: the n log n form (checked against the plain one below)
     assert abs(r["sigma"] / 0.02 - 1.0) < 0.02
     assert r["min_pts"] == min(r["left"], r["right"]) and r["eps"] == r["sigma"] / r["min_pts"]
     assert np.all(np.diff(r["centroids"]) > 0) and np.all(np.isin(r["centroids"].astype(np.float32), r["sorted"]))
@@ -549,3 +549,75 @@ def test_dbci_middle_matches_textbook_dbscan():
             if mem.size:
                 assert not np.any((labs[mem[0]:mem[-1] + 1] != c) & (labs[mem[0]:mem[-1] + 1] != -1))
         assert r["centroids"].size == len({int(v) for v in labs if v >= 0})
+
+
+def test_dbci_border_point_rule_by_hand():
+    # Four outliers on either side seed the two outer clusters; positives 0.95 1.05 1.15 1.25 7.97 7.98 7.99 8 ->
+    # nearest ranks ceil(p * 8) = 6, 8, 8 -> 7.98 + 8 + 8, the same for the negative magnitudes:
+    # sigma = 47.96 / 12 = 3.99667; each seed takes its four outliers (nothing else within sigma of -8 or 8), so
+    # MinPts = 4 and eps = sigma / 4 = 0.99917.  Both groups of four are core points (four points within 0.3);
+    # the point 0 sees only -0.95, itself and 0.95 (three points), so it is not a core point, and it lies
+    # exactly 0.95 from the rightmost core of the left group and from the leftmost core of the right group:
+    # the left cluster takes it.
+    w = np.array([-8, -7.99, -7.98, -7.97, -1.25, -1.15, -1.05, -0.95, 0, 0.95, 1.05, 1.15, 1.25, 7.97, 7.98, 7.99, 8],
+                 dtype=np.float32)
+    for f in (O.dbci, O.dbci_scan):
+        r = f(w)
+        assert abs(r["sigma"] - 47.96 / 12) < 1e-6 and r["min_pts"] == 4 and abs(r["eps"] - 47.96 / 48) < 1e-6
+        assert (r["left"], r["right"]) == (4, 4)
+        assert r["labels"].tolist() == [0] * 4 + [1] * 5 + [2] * 4 + [3] * 4
+        # lower medians: member 1 of four, member 2 of five
+        assert r["centroids"].astype(np.float32).tolist() == [np.float32(v) for v in (-7.99, -1.05, 1.05, 7.98)]
+    # the same with the lonely point at 0.02: nine positives, ranks ceil(p * 9) = 7, 9, 9 -> the same three values,
+    # so sigma and eps are unchanged; 0.02 is 0.97 from -0.95 and 0.93 from 0.95, both within eps: the nearer,
+    # right cluster takes it
+    w2 = np.sort(np.where(w == 0, np.float32(0.02), w))
+    for f in (O.dbci, O.dbci_scan):
+        r = f(w2)
+        assert r["labels"].tolist() == [0] * 4 + [1] * 4 + [2] * 5 + [3] * 4
+        assert r["centroids"].astype(np.float32).tolist() == [np.float32(v) for v in (-7.99, -1.15, 1.05, 7.98)]
+    # ... and a point no core point reaches is noise: 0 moved out to 3.0 (more than eps from 1.25 and from 7.97)
+    w3 = np.sort(np.where(w == 0, np.float32(3.0), w))
+    r = O.dbci(w3)        # nine positives again: ranks 7, 9, 9 -> 7.98 + 8 + 8, sigma and eps as before
+    assert abs(r["sigma"] - 47.96 / 12) < 1e-6
+    assert r["labels"].tolist() == [0] * 4 + [1] * 4 + [2] * 4 + [-1] + [3] * 4
+
+
+def test_dbci_seed_clusters_by_hand():
+    # every weight within sigma of the smallest one: positives 1.0 1.1 1.2, ranks ceil(p * 3) = 3, 3, 3 ->
+    # sigma = 3.6 / 12 = 0.3; the left seed takes all three, the right one gives way completely, so MinPts is
+    # the left count and nothing is left for DBSCAN
+    for f in (O.dbci, O.dbci_scan):
+        r = f(np.array([1.0, 1.1, 1.2], dtype=np.float32))
+        assert abs(r["sigma"] - 0.3) < 1e-6 and (r["left"], r["right"], r["min_pts"]) == (3, 0, 3)
+        assert abs(r["eps"] - 0.1) < 1e-6 and r["labels"].tolist() == [0, 0, 0]
+        assert r["centroids"].astype(np.float32).tolist() == [np.float32(1.1)]
+        # partial overlap: 10 12.5 13.5 16 -> ranks 3, 4, 4 -> sigma = (13.5 + 16 + 16) / 12 = 3.79167; the left seed
+        # reaches 13.79 (three weights), the right one 12.21 (three weights): 12.5 and 13.5 stay with the left
+        r = f(np.array([10, 12.5, 13.5, 16], dtype=np.float32))
+        assert abs(r["sigma"] - 45.5 / 12) < 1e-9 and (r["left"], r["right"], r["min_pts"]) == (3, 1, 1)
+        assert r["labels"].tolist() == [0, 0, 0, 1] and r["centroids"].tolist() == [12.5, 16.0]
+        # a single weight
+        r = f(np.array([0.25], dtype=np.float32))
+        assert (r["left"], r["right"], r["min_pts"]) == (1, 0, 1) and r["labels"].tolist() == [0]
+
+
+def test_dbci_scan_form_equals_plain_form():
+    # the n log n form used for large inputs against the plain one, on inputs with many exact ties (values on a
+    # grid), clumps, one-sided data and uniform noise
+    rng = np.random.default_rng(7)
+    for trial in range(40):
+        kind = trial % 4
+        if kind == 0:
+            w = np.round(rng.standard_normal(400) * 0.02, 3)
+            w = np.concatenate([w, [-0.5, -0.499, 0.6, 0.601, 0.602]])
+        elif kind == 1:
+            w = np.concatenate([rng.standard_normal(300) * 0.02, 0.1 + rng.standard_normal(25) * 0.001,
+                                rng.uniform(-0.3, 0.3, 20), [-0.5, -0.49, -0.495, 0.6, 0.61, 0.605]])
+        elif kind == 2:
+            w = np.abs(np.round(rng.standard_normal(300) * 0.02, 3)) + 0.001
+        else:
+            w = np.round(rng.uniform(-1, 1, 200), 2)
+        a, b = O.dbci(w.astype(np.float32)), O.dbci_scan(w.astype(np.float32))
+        assert (a["sigma"], a["eps"], a["min_pts"], a["left"], a["right"]) == (b["sigma"], b["eps"], b["min_pts"], b["left"], b["right"])
+        assert np.array_equal(a["labels"], b["labels"]) and np.array_equal(a["centroids"], b["centroids"])
