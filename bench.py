@@ -62,7 +62,7 @@ def parse_args():
                          "centroid initialisation")
     ap.add_argument("--two-call", action="store_true",
                     help="M <= 16: quantise and look up in two launches per layer instead of the fused one")
-    ap.add_argument("--algo", default="auto", choices=["auto", "register", "bucket", "tensor"],
+    ap.add_argument("--algo", default="auto", choices=["auto", "register", "bucket", "tensor", "shared"],
                     help="lookup kernel for M <= 16 (default: the library's choice)")
     return ap.parse_args()
 
@@ -251,7 +251,7 @@ def run_ours(args):
 
     grouped = M <= 16 and len(mats) <= lcd.MAX_BATCH
     algo = {"auto": lcd.ALGO_AUTO, "register": lcd.ALGO_REGISTER_LUT, "bucket": lcd.ALGO_BUCKET_LUT,
-            "tensor": lcd.ALGO_TC_LUT}[args.algo]
+            "tensor": lcd.ALGO_TC_LUT, "shared": lcd.ALGO_SHARED_BUCKET}[args.algo]
     # every kernel that can give up on a bounded wait reports it here; a non-zero word voids the run
     status = torch.zeros((1,), dtype=torch.int32, device=dev)
     if grouped:

@@ -41,7 +41,8 @@ typedef enum {
 
 /* Which kernel family lcd_lut_linear uses.  Every family computes the same y. */
 typedef enum {
-  LCD_ALGO_AUTO = 0,        /* REGISTER_LUT for M <= 16, DENSE_TC above                                        */
+  LCD_ALGO_AUTO = 0,        /* M <= 16: SHARED_BUCKET where it applies and the layer is large enough to pay    */
+                            /* for its tables, else REGISTER_LUT; DENSE_TC above                                */
   LCD_ALGO_REFERENCE = 1,   /* plain per-weight lookup cb[n][idx] and multiply-accumulate; any M, slow        */
   LCD_ALGO_BUCKET_LUT = 2,  /* Section 4.2 centroid-stationary buckets: per output and per centroid w the exact */
                             /* integer sum S_w of the activation levels whose weight index is w (one-hot byte   */
@@ -55,8 +56,13 @@ typedef enum {
                             /* kind::i8 MMAs accumulate exact int32 sums in tensor memory.                      */
   LCD_ALGO_DENSE_F16 = 5,   /* the same with fp16 operands: indices decoded through the codebook into fp16     */
                             /* shared-memory tiles, fp32 accumulators (no fixed-point step; slower).            */
-  LCD_ALGO_TC_LUT = 6       /* REGISTER_LUT's tables and sums, the looked-up bytes written to tensor memory as  */
+  LCD_ALGO_TC_LUT = 6,      /* REGISTER_LUT's tables and sums, the looked-up bytes written to tensor memory as  */
                             /* the A operand of tcgen05 kind::i8 MMAs over a 16-token tile.  M <= 16.            */
+  LCD_ALGO_SHARED_BUCKET = 7/* Section 4.2 centroid-stationary buckets with the tables in shared memory: for    */
+                            /* every four columns a table indexed by the byte of their four weight indices      */
+                            /* holds the four partial bucket sums of the token's levels, so one load looks four */
+                            /* weights up for all centroids; exact integer S_w, y = s_q * sum_w cb[w] * S_w.     */
+                            /* One token (M = 1), 2-bit indices, 4-bit levels.                                   */
 } lcd_algo;
 
 #define LCD_HEADER_BYTES 64
@@ -266,8 +272,9 @@ lcd_status lcd_dbci(const float* weights, int64_t n, void* workspace, size_t wor
  * dw < -(C_i - C_{i-1})/2 and to i + 1 when dw > (C_{i+1} - C_i)/2 (binary32, one subtraction and one halving;
  * the paper prints the left test without the sign; edge clusters have one side); never further than one cluster.
  *     delta_c[n][j] = sum over the weights that end up in j of (dw + (C_old - C_j))      (a sum, as printed)
- *   idx:           device, uint8 [N][K] cluster of every weight (one byte each, the packer's input form), < C;
- *                  K <= 2^25;
+ *   idx:           device, uint8 [N][K] cluster of every weight (one byte each, the packer's input form), < C
+ *                  (not checked on the device: a byte >= C is reduced modulo 4, 8 or 16, whichever holds C, kept as
+ *                  that value in new_idx and counted in no cluster; nothing faults);  K <= 2^25;
  *   codebook_fp16: device, binary16 [N][C], 1 <= C <= 16;     delta_w: device, fp32 [N][ldw], ldw >= K;
  *   new_idx:       device out, uint8 [N][K] (may not alias idx);
  *   delta_c:       device out, fp64 [N][C];     counts: device out, int32 [N][C] members after the move.

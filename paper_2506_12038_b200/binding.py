@@ -19,6 +19,7 @@ LCD_OK = 0
 STATUS_NAMES = {0: "LCD_OK", 1: "LCD_ERR_INVALID_ARG", 2: "LCD_ERR_UNSUPPORTED", 3: "LCD_ERR_BUFFER_TOO_SMALL",
                 4: "LCD_ERR_INDEX_RANGE", 5: "LCD_ERR_BAD_BLOB", 6: "LCD_ERR_CUDA", 7: "LCD_ERR_TIMEOUT"}
 ALGO_AUTO, ALGO_REFERENCE, ALGO_BUCKET_LUT, ALGO_REGISTER_LUT, ALGO_DENSE_TC, ALGO_DENSE_F16, ALGO_TC_LUT = 0, 1, 2, 3, 4, 5, 6
+ALGO_SHARED_BUCKET = 7
 HEADER_BYTES = 64
 MAX_BATCH = 8
 

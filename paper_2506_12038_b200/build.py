@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liblcd_b200.so")
-SOURCES = ["api.cu", "pack.cpp", "quantize.cu", "quantize8.cu", "smoothing.cu", "reclassify.cu", "dbci.cu", "reference.cu", "lut_gemv.cu", "lut_gemv_tc.cu", "dense_tc.cu", "static_scratch.cu"]
+SOURCES = ["api.cu", "pack.cpp", "quantize.cu", "quantize8.cu", "smoothing.cu", "reclassify.cu", "dbci.cu", "reference.cu", "lut_gemv.cu", "lut_smem.cu", "lut_gemv_tc.cu", "dense_tc.cu", "static_scratch.cu"]
 
 
 def nvcc_path() -> str:

@@ -15,10 +15,14 @@ void set_cuda_error(int err) { g_cuda_error = cudaGetErrorString(static_cast<cud
 
 static bool aligned(const void* p, size_t a) { return reinterpret_cast<uintptr_t>(p) % a == 0; }
 
-static lcd_algo resolve_algo(int64_t M, lcd_algo algo) {
+static lcd_algo resolve_algo(const Problem& p, lcd_algo algo) {
   if (algo != LCD_ALGO_AUTO) return algo;
-  if (M <= 16) return LCD_ALGO_REGISTER_LUT;
+  if (p.M <= 16) return resolve_small_m(&p, 1, algo);
   return kHaveDenseTc ? LCD_ALGO_DENSE_TC : LCD_ALGO_REFERENCE;
+}
+
+static bool small_m_family(lcd_algo a) {
+  return a == LCD_ALGO_REGISTER_LUT || a == LCD_ALGO_BUCKET_LUT || a == LCD_ALGO_TC_LUT || a == LCD_ALGO_SHARED_BUCKET;
 }
 
 // Fills everything of a Problem that follows from the blob header and the call's pointers.
@@ -63,15 +67,18 @@ static bool shape_problem(const void* header_host, int64_t M, Problem* p) {
 }
 
 static lcd_status workspace_for(const Problem& p, lcd_algo algo, size_t* bytes) {
-  switch (resolve_algo(p.M, algo)) {
+  const lcd_algo resolved = resolve_algo(p, algo);
+  switch (resolved) {
     case LCD_ALGO_REFERENCE:
       *bytes = 0;
       return LCD_OK;
     case LCD_ALGO_REGISTER_LUT:
     case LCD_ALGO_BUCKET_LUT:
     case LCD_ALGO_TC_LUT:
+    case LCD_ALGO_SHARED_BUCKET:
       if (p.M > 16) return LCD_ERR_UNSUPPORTED;
-      *bytes = lut_gemv_workspace_bytes(&p, 1, resolve_algo(p.M, algo));
+      if (resolved == LCD_ALGO_SHARED_BUCKET && !lut_smem_supported(&p, 1)) return LCD_ERR_UNSUPPORTED;
+      *bytes = lut_gemv_workspace_bytes(&p, 1, resolved);
       return LCD_OK;
     case LCD_ALGO_DENSE_TC:
     case LCD_ALGO_DENSE_F16:
@@ -151,13 +158,14 @@ extern "C" lcd_status lcd_lut_linear(const void* packed_weights_dev, const void*
   if (st != LCD_OK) return st;
   if (need > 0 && (!workspace || workspace_bytes < need)) return LCD_ERR_BUFFER_TOO_SMALL;
   if (need > 0 && !aligned(workspace, 256)) return LCD_ERR_INVALID_ARG;
-  const lcd_algo resolved = resolve_algo(M, algo);
+  const lcd_algo resolved = resolve_algo(p, algo);
   switch (resolved) {
     case LCD_ALGO_REFERENCE:
       return launch_reference(p, cuda_stream);
     case LCD_ALGO_REGISTER_LUT:
     case LCD_ALGO_BUCKET_LUT:
     case LCD_ALGO_TC_LUT:
+    case LCD_ALGO_SHARED_BUCKET:
       return launch_lut_gemv(&p, 1, resolved, workspace, workspace_bytes, status_word_dev, cuda_stream);
     case LCD_ALGO_DENSE_TC:
     case LCD_ALGO_DENSE_F16:
@@ -167,20 +175,24 @@ extern "C" lcd_status lcd_lut_linear(const void* packed_weights_dev, const void*
   }
 }
 
-static lcd_status batch_algo(const lcd_linear_problem* problems, int count, lcd_algo algo, lcd_algo* resolved) {
+static lcd_status batch_algo(const lcd_linear_problem* problems, int count, lcd_algo algo) {
   if (!problems || count < 1 || count > LCD_MAX_BATCH) return LCD_ERR_INVALID_ARG;
-  if (algo != LCD_ALGO_AUTO && algo != LCD_ALGO_REGISTER_LUT && algo != LCD_ALGO_BUCKET_LUT && algo != LCD_ALGO_TC_LUT)
-    return LCD_ERR_UNSUPPORTED;
+  if (algo != LCD_ALGO_AUTO && !small_m_family(algo)) return LCD_ERR_UNSUPPORTED;
   for (int i = 0; i < count; ++i)
     if (problems[i].M < 1 || problems[i].M > 16) return problems[i].M < 1 ? LCD_ERR_INVALID_ARG : LCD_ERR_UNSUPPORTED;
-  *resolved = algo == LCD_ALGO_AUTO ? LCD_ALGO_REGISTER_LUT : algo;
+  return LCD_OK;
+}
+// The family a grouped call runs: the caller's, or the library's choice for these shapes.
+static lcd_status batch_family(const Problem* p, int count, lcd_algo algo, lcd_algo* resolved) {
+  *resolved = resolve_small_m(p, count, algo);
+  if (*resolved == LCD_ALGO_SHARED_BUCKET && !lut_smem_supported(p, count)) return LCD_ERR_UNSUPPORTED;
   return LCD_OK;
 }
 
 extern "C" lcd_status lcd_lut_linear_batch_workspace_bytes(const lcd_linear_problem* problems, int count,
                                                            lcd_algo algo, size_t* bytes) {
   lcd_algo resolved;
-  lcd_status st = batch_algo(problems, count, algo, &resolved);
+  lcd_status st = batch_algo(problems, count, algo);
   if (st != LCD_OK) return st;
   if (!bytes) return LCD_ERR_INVALID_ARG;
   Problem p[LCD_MAX_BATCH];
@@ -189,6 +201,8 @@ extern "C" lcd_status lcd_lut_linear_batch_workspace_bytes(const lcd_linear_prob
     if (!shape_problem(problems[i].header_host, problems[i].M, &p[i])) return LCD_ERR_BAD_BLOB;
     if (p[i].bits != p[0].bits) return LCD_ERR_UNSUPPORTED;
   }
+  st = batch_family(p, count, algo, &resolved);
+  if (st != LCD_OK) return st;
   *bytes = lut_gemv_workspace_bytes(p, count, resolved);
   return LCD_OK;
 }
@@ -197,7 +211,7 @@ extern "C" lcd_status lcd_lut_linear_batch(const lcd_linear_problem* problems, i
                                            void* workspace, size_t workspace_bytes, int32_t* status_word_dev,
                                            void* cuda_stream) {
   lcd_algo resolved;
-  lcd_status st = batch_algo(problems, count, algo, &resolved);
+  lcd_status st = batch_algo(problems, count, algo);
   if (st != LCD_OK) return st;
   Problem p[LCD_MAX_BATCH];
   for (int i = 0; i < count; ++i) {
@@ -206,6 +220,8 @@ extern "C" lcd_status lcd_lut_linear_batch(const lcd_linear_problem* problems, i
     if (st != LCD_OK) return st;
     if (p[i].bits != p[0].bits) return LCD_ERR_UNSUPPORTED;
   }
+  st = batch_family(p, count, algo, &resolved);
+  if (st != LCD_OK) return st;
   const size_t need = lut_gemv_workspace_bytes(p, count, resolved);
   if (!workspace || workspace_bytes < need) return LCD_ERR_BUFFER_TOO_SMALL;
   if (!aligned(workspace, 256)) return LCD_ERR_INVALID_ARG;
@@ -216,7 +232,7 @@ extern "C" lcd_status lcd_lut_linear_batch_act8(const lcd_linear_problem* proble
                                            void* workspace, size_t workspace_bytes, int32_t* status_word_dev,
                                            void* cuda_stream) {
   lcd_algo resolved;
-  lcd_status st = batch_algo(problems, count, algo, &resolved);
+  lcd_status st = batch_algo(problems, count, algo);
   if (st != LCD_OK) return st;
   Problem p[LCD_MAX_BATCH];
   for (int i = 0; i < count; ++i) {
@@ -227,6 +243,8 @@ extern "C" lcd_status lcd_lut_linear_batch_act8(const lcd_linear_problem* proble
     p[i].act_bits = 8;
     if (p[i].K_pad >= (1LL << 17)) return LCD_ERR_UNSUPPORTED;   // int32 sums could overflow
   }
+  st = batch_family(p, count, algo, &resolved);
+  if (st != LCD_OK) return st;
   const size_t need = lut_gemv_workspace_bytes(p, count, resolved);
   if (!workspace || workspace_bytes < need) return LCD_ERR_BUFFER_TOO_SMALL;
   if (!aligned(workspace, 256)) return LCD_ERR_INVALID_ARG;
@@ -249,7 +267,7 @@ extern "C" lcd_status lcd_lut_linear_act8(const void* packed_weights_dev, const 
   if (st != LCD_OK) return st;
   if (need > 0 && (!workspace || workspace_bytes < need)) return LCD_ERR_BUFFER_TOO_SMALL;
   if (need > 0 && !aligned(workspace, 256)) return LCD_ERR_INVALID_ARG;
-  const lcd_algo resolved = resolve_algo(M, algo);
+  const lcd_algo resolved = resolve_algo(p, algo);
   switch (resolved) {
     case LCD_ALGO_REFERENCE:
       return launch_reference(p, cuda_stream);
@@ -260,6 +278,7 @@ extern "C" lcd_status lcd_lut_linear_act8(const void* packed_weights_dev, const 
     case LCD_ALGO_DENSE_TC:
       return launch_dense_tc(p, false, workspace, workspace_bytes, status_word_dev, cuda_stream);
     case LCD_ALGO_DENSE_F16:
+    case LCD_ALGO_SHARED_BUCKET:      // the shared-memory tables hold sums of four 4-bit levels per byte
       return LCD_ERR_UNSUPPORTED;
     default:
       return LCD_ERR_INVALID_ARG;
@@ -269,8 +288,9 @@ extern "C" lcd_status lcd_lut_linear_act8(const void* packed_weights_dev, const 
 static lcd_status fused_problems(const lcd_fused_problem* problems, int count, lcd_algo algo, bool pointers,
                                  Problem* p, lcd_algo* resolved) {
   if (!problems || count < 1 || count > LCD_MAX_BATCH) return LCD_ERR_INVALID_ARG;
-  if (algo != LCD_ALGO_AUTO && algo != LCD_ALGO_REGISTER_LUT && algo != LCD_ALGO_BUCKET_LUT) return LCD_ERR_UNSUPPORTED;
-  *resolved = algo == LCD_ALGO_AUTO ? LCD_ALGO_REGISTER_LUT : algo;
+  if (algo != LCD_ALGO_AUTO && algo != LCD_ALGO_REGISTER_LUT && algo != LCD_ALGO_BUCKET_LUT &&
+      algo != LCD_ALGO_SHARED_BUCKET)
+    return LCD_ERR_UNSUPPORTED;
   for (int i = 0; i < count; ++i) {
     const lcd_fused_problem& q = problems[i];
     if (q.M < 1 || !q.header_host) return LCD_ERR_INVALID_ARG;
@@ -294,7 +314,7 @@ static lcd_status fused_problems(const lcd_fused_problem* problems, int count, l
     p[i].y = q.y;
     p[i].ldy = q.ldy;
   }
-  return LCD_OK;
+  return batch_family(p, count, algo, resolved);
 }
 
 extern "C" lcd_status lcd_linear_fused_batch_workspace_bytes(const lcd_fused_problem* problems, int count,
@@ -472,7 +492,7 @@ lcd_status host_batch_layout(const lcd_host_problem* probs, int count, Problem* 
     o += 256;
   }
   L->ws_off = o;
-  L->ws_bytes = lut_gemv_workspace_bytes(shapes, count, LCD_ALGO_REGISTER_LUT);
+  L->ws_bytes = lut_gemv_workspace_bytes(shapes, count, resolve_small_m(shapes, count, LCD_ALGO_AUTO));
   L->total = o + (size_t)round_up_u64(L->ws_bytes, 256);
   return LCD_OK;
 }
@@ -536,7 +556,7 @@ extern "C" lcd_status lcd_linear_host_batch(const lcd_host_problem* problems, in
   }
   e = cudaMemsetAsync(base + L.ws_off, 0, L.ws_bytes, stream);    // the lookup kernel wants its scratch zero-filled
   if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
-  st = launch_lut_gemv(p, count, LCD_ALGO_REGISTER_LUT, base + L.ws_off, L.ws_bytes, nullptr, cuda_stream);
+  st = launch_lut_gemv(p, count, resolve_small_m(shapes, count, LCD_ALGO_AUTO), base + L.ws_off, L.ws_bytes, nullptr, cuda_stream);
   if (st != LCD_OK) return st;
   e = cudaMemcpyAsync(y_host_all, base + L.y_off[0], L.y_bytes, cudaMemcpyDeviceToHost, stream);   // one copy out
   if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }

@@ -73,6 +73,13 @@ lcd_status launch_smooth_quantize_batch(const lcd_act_problem* probs, int count,
 size_t lut_gemv_workspace_bytes(const Problem* probs, int count, lcd_algo algo);
 lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void* workspace, size_t workspace_bytes,
                            int32_t* status_word, void* stream);
+// LCD_ALGO_SHARED_BUCKET: one token, 2-bit indices, bucket tables in shared memory (4-bit levels or fp16 x)
+bool lut_smem_supported(const Problem* probs, int count);
+size_t lut_smem_workspace_bytes(const Problem* probs, int count);
+lcd_status launch_lut_smem(const Problem* probs, int count, void* workspace, size_t workspace_bytes,
+                           int32_t* status_word, void* stream);
+// The family LCD_ALGO_AUTO stands for when every problem has at most 16 tokens.
+lcd_algo resolve_small_m(const Problem* probs, int count, lcd_algo algo);
 // LCD_ALGO_TC_LUT: the same arithmetic for up to 16 tokens with the looked-up bytes fed to tcgen05.mma kind::i8
 size_t lut_gemv_tc_workspace_bytes(const Problem* probs, int count);
 lcd_status launch_lut_gemv_tc(const Problem* probs, int count, void* workspace, size_t workspace_bytes,

@@ -19,6 +19,7 @@
 #include <cuda_runtime.h>
 
 #include "common.h"
+#include "device_util.h"
 
 namespace lcd {
 
@@ -762,17 +763,7 @@ EncodeTiledFn encode_tiled() {
   return fn;
 }
 
-int dense_sm_count() {
-  static int cached = 0;
-  if (cached == 0) {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
-      n = 148;
-    cached = n;
-  }
-  return cached;
-}
+int dense_sm_count() { return current_sm_count(); }
 
 template <int BITS, int BN>
 lcd_status launch_dense_t(const Problem& p, __half* levels, int32_t* status_word, cudaStream_t stream) {
@@ -801,11 +792,12 @@ lcd_status launch_dense_t(const Problem& p, __half* levels, int32_t* status_word
   dp.status = status_word;
   const size_t smem = 1024 + (size_t)kStages * (kABytes + BN * kBK * 2) + 256;
   auto kern = dense_tc_kernel<BITS, BN>;
-  static bool attr_set = false;   // per template instance
-  if (!attr_set) {
+  static PerDeviceFlag attr_set;   // per template instance and device
+  int dev;
+  if (attr_set.first(&dev)) {
     const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
-    attr_set = true;
+    attr_set.done(dev);
   }
   const int grid = dp.n_tiles < dense_sm_count() ? dp.n_tiles : dense_sm_count();
   cudaLaunchConfig_t cfg = {};
@@ -850,11 +842,12 @@ lcd_status launch_dense_i8(const Problem& p, int8_t* levels, int32_t* status_wor
   dp.status = status_word;
   const size_t smem = 1024 + (size_t)i8_stages(BN) * (2 * kI8PlaneBytes + BN * kI8BK) + 256;
   auto kern = dense_i8_kernel<BITS, BN>;
-  static bool attr_set = false;   // per template instance
-  if (!attr_set) {
+  static PerDeviceFlag attr_set;   // per template instance and device
+  int dev;
+  if (attr_set.first(&dev)) {
     const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
-    attr_set = true;
+    attr_set.done(dev);
   }
   const int grid = dp.n_tiles < dense_sm_count() ? dp.n_tiles : dense_sm_count();
   cudaLaunchConfig_t cfg = {};

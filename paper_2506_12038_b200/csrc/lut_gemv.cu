@@ -30,6 +30,7 @@
 #include <cuda_runtime.h>
 
 #include "common.h"
+#include "device_util.h"
 
 namespace lcd {
 
@@ -908,16 +909,10 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
 
 namespace {
 
-int sm_count() {
-  static int cached = 0;
-  if (cached == 0) {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
-      n = 148;
-    cached = n;
-  }
-  return cached;
-}
+int sm_count() { return current_sm_count(); }
+
+// items (16 rows x 256 columns) of a launch from which LCD_ALGO_AUTO takes the shared-memory bucket tables
+constexpr long long kSharedBucketMinItems = 1;
 
 int planes_of(int bits, int kind) { return kind == kFixed16 ? 2 : (1 << bits); }
 
@@ -935,11 +930,12 @@ ScratchLayout scratch_layout(size_t begin, int64_t n_rp, int MG, int planes) {
 template <int BITS, int KIND, int MG>
 lcd_status launch_t(const GemvBatch& batch, int grid, size_t smem, int32_t* status, cudaStream_t stream) {
   auto kern = lut_gemv_kernel<BITS, KIND, MG>;
-  static bool attr_set = false;   // per template instance
-  if (!attr_set) {
+  static PerDeviceFlag attr_set;   // per template instance and device
+  int dev;
+  if (attr_set.first(&dev)) {
     const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
     if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
-    attr_set = true;
+    attr_set.done(dev);
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
@@ -960,8 +956,19 @@ lcd_status launch_t(const GemvBatch& batch, int grid, size_t smem, int32_t* stat
 
 }  // namespace
 
+// LCD_ALGO_AUTO for at most 16 tokens: the shared-memory bucket tables where they apply (one token, 2-bit indices)
+// and the launch has enough rows per CTA to pay for building them, else the register tables.
+lcd_algo resolve_small_m(const Problem* probs, int count, lcd_algo algo) {
+  if (algo != LCD_ALGO_AUTO) return algo;
+  if (!lut_smem_supported(probs, count)) return LCD_ALGO_REGISTER_LUT;
+  long long items = 0;
+  for (int i = 0; i < count; ++i) items += (probs[i].N_pad / kPairRows) * (probs[i].K_pad / kTileK);
+  return items >= kSharedBucketMinItems ? LCD_ALGO_SHARED_BUCKET : LCD_ALGO_REGISTER_LUT;
+}
+
 size_t lut_gemv_workspace_bytes(const Problem* probs, int count, lcd_algo algo) {
   if (algo == LCD_ALGO_TC_LUT) return lut_gemv_tc_workspace_bytes(probs, count);
+  if (algo == LCD_ALGO_SHARED_BUCKET) return lut_smem_workspace_bytes(probs, count);
   const int kind = algo == LCD_ALGO_BUCKET_LUT ? kBuckets : kFixed16;
   int64_t max_m = 1;
   for (int i = 0; i < count; ++i) max_m = probs[i].M > max_m ? probs[i].M : max_m;
@@ -976,6 +983,7 @@ lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void*
                            int32_t* status_word, void* stream) {
   if (count < 1 || count > LCD_MAX_BATCH) return LCD_ERR_INVALID_ARG;
   if (algo == LCD_ALGO_TC_LUT) return launch_lut_gemv_tc(probs, count, workspace, workspace_bytes, status_word, stream);
+  if (algo == LCD_ALGO_SHARED_BUCKET) return launch_lut_smem(probs, count, workspace, workspace_bytes, status_word, stream);
   const int kind = algo == LCD_ALGO_BUCKET_LUT ? kBuckets : kFixed16;
   const int bits = probs[0].bits;
   int64_t max_m = 1;

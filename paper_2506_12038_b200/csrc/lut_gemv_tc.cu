@@ -21,6 +21,7 @@
 #include <cuda_runtime.h>
 
 #include "common.h"
+#include "device_util.h"
 
 namespace lcd {
 
@@ -597,16 +598,7 @@ size_t tc_smem_bytes() {
 
 inline size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
-int tc_sm_count() {
-  static int cached = 0;
-  if (cached == 0) {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
-      n = 148;
-    cached = n;
-  }
-  return cached;
-}
+int tc_sm_count() { return current_sm_count(); }
 
 // scratch of one problem: integer sums [n_rt][2][16][128], then tickets [n_rt][4]
 struct TcScratch {
@@ -624,11 +616,12 @@ template <int BITS>
 lcd_status tc_launch_t(const TcBatch& batch, int grid, int32_t* status, cudaStream_t stream) {
   auto kern = lut_gemv_tc_kernel<BITS>;
   const size_t smem = tc_smem_bytes<BITS>();
-  static bool attr_set = false;
-  if (!attr_set) {
+  static PerDeviceFlag attr_set;   // per template instance and device
+  int dev;
+  if (attr_set.first(&dev)) {
     const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
-    attr_set = true;
+    attr_set.done(dev);
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);

@@ -8,6 +8,7 @@
 #include <cuda_runtime.h>
 
 #include "common.h"
+#include "device_util.h"
 
 namespace lcd {
 
@@ -48,7 +49,9 @@ __global__ void __launch_bounds__(kRcThreads) reclassify_kernel(const uint8_t* _
   const uint8_t* ir = idx + n * K;
   const float* dr = delta_w + n * ldw;
   uint8_t* outr = new_idx + n * K;
-  // branch-free: s_gap[i] = (half-gap to the left, half-gap to the right) of cluster i, infinite at the edges
+  // branch-free: s_gap[i] = (half-gap to the left, half-gap to the right) of cluster i, infinite at the edges.
+  // An index is reduced to the table size CMAX before it addresses shared memory, so a byte >= C (the caller's
+  // error) cannot reach outside the slots: such a weight keeps its reduced index and is counted in no cluster.
   auto one = [&](int i, float dw) {
     const float2 gap = s_gap[i];
     const int left = dw < -gap.x ? 1 : 0;
@@ -80,13 +83,13 @@ __global__ void __launch_bounds__(kRcThreads) reclassify_kernel(const uint8_t* _
         const float dv[4] = {d.x, d.y, d.z, d.w};
         uint32_t o = 0;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) o |= one((int)((iw[q] >> (8 * e)) & 0xffu), dv[e]) << (8 * e);
+        for (int e = 0; e < 4; ++e) o |= one((int)((iw[q] >> (8 * e)) & (uint32_t)(CMAX - 1)), dv[e]) << (8 * e);
         ow[q] = o;
       }
       *reinterpret_cast<uint4*>(outr + k) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
     }
   } else {
-    for (int64_t k = tid; k < K; k += kRcThreads) outr[k] = (uint8_t)one(ir[k], dr[k]);
+    for (int64_t k = tid; k < K; k += kRcThreads) outr[k] = (uint8_t)one(ir[k] & (CMAX - 1), dr[k]);
   }
   // Block reduction of the pairs and counts, still in binary32 pairs (binary64 operations only on the C final values
   // of the row: they are slow enough here that a few dozen per thread dominated the kernel), fixed order.
@@ -142,12 +145,13 @@ lcd_status launch_reclassify(const uint8_t* idx, const uint16_t* codebook, const
   if (C <= 4) reclassify_kernel<4><<<(unsigned)N, kRcThreads, 4 * kRcThreads * 16, s>>>(idx, codebook, delta_w, K, ldw, C, new_idx, delta_c, counts, vec);
   else if (C <= 8) reclassify_kernel<8><<<(unsigned)N, kRcThreads, 8 * kRcThreads * 16, s>>>(idx, codebook, delta_w, K, ldw, C, new_idx, delta_c, counts, vec);
   else {
-    static bool attr_set = false;     // 80 KB of dynamic shared memory needs the opt-in
-    if (!attr_set) {
+    static PerDeviceFlag attr_set;    // 80 KB of dynamic shared memory needs the opt-in, on every device
+    int dev;
+    if (attr_set.first(&dev)) {
       const cudaError_t ea = cudaFuncSetAttribute(reclassify_kernel<kRcMaxC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                   kRcMaxC * kRcThreads * 16);
       if (ea != cudaSuccess) { set_cuda_error((int)ea); return LCD_ERR_CUDA; }
-      attr_set = true;
+      attr_set.done(dev);
     }
     reclassify_kernel<kRcMaxC><<<(unsigned)N, kRcThreads, kRcMaxC * kRcThreads * 16, s>>>(idx, codebook, delta_w, K, ldw, C, new_idx, delta_c, counts, vec);
   }
