@@ -23,9 +23,7 @@
 //
 // Decomposition.  The work of a launch is the sequence (problem, column slice, 16-row group); it is cut into one
 // contiguous piece per CTA (the cut counts the table build of every slice a piece touches).  Each of a CTA's 16
-// lookup warps takes every 16th row group of a piece; a seventeenth warp streams their index bytes into per-warp
-// rings of bulk copies (lane w feeds warp w: full/empty mbarriers per slot), so the lookup warps never issue or
-// track a copy.
+// warps takes every 16th row group of a piece and streams its index bytes through its own ring of bulk copies.
 // Per slice a row's four bucket sums are added to zero-filled scratch [row][4] as fp32 (integers below 2^24, so
 // the additions are exact and their order does not matter: one vector reduction per row).  When every CTA of the
 // launch has added its last sum (a counter in the scratch that all CTAs wait for, bounded; the launch is
@@ -45,7 +43,7 @@ namespace {
 constexpr int kMaxSmem = 227 * 1024;
 constexpr uint32_t kBlockBytes = 0x10000u;  // tables of one 256-column block: 64 groups x 256 entries x 4 bytes
 constexpr int kItemBytes = 1024;            // one 16-row x 256-column item at 2 bit
-constexpr int kMiscBytes = 1024;            // full and empty mbarriers, partial maxima, flags
+constexpr int kMiscBytes = 512;             // mbarriers, partial maxima
 constexpr int kMaxCta = 304;
 constexpr unsigned long long kTimeoutNs = 2000000000ull;
 
@@ -55,8 +53,7 @@ constexpr unsigned long long kTimeoutNs = 2000000000ull;
 // the shared window on this architecture; the kernel checks what it finds and gives up cleanly otherwise.
 template <int W, int DEPTH, int WARPS>
 struct Shape {
-  static constexpr int kThreads = WARPS * 32;          // lookup warps
-  static constexpr int kBlock = kThreads + 32;         // + the warp that feeds the rings
+  static constexpr int kThreads = WARPS * 32;
   static constexpr uint32_t kSlot = W * kItemBytes;
   static constexpr uint32_t kRingBytes = WARPS * DEPTH * kSlot;
   static constexpr uint32_t kTableAddr = (0x400u + kMiscBytes + kRingBytes + 0x3ffu) & ~0x3ffu;
@@ -174,13 +171,12 @@ __device__ __forceinline__ void half_item(uint32_t x0, uint32_t y0, uint32_t x1,
 }
 
 template <int W, int DEPTH, int WARPS>
-__global__ void __launch_bounds__(WARPS * 32 + 32, 1)
+__global__ void __launch_bounds__(WARPS * 32, 1)
 lut_smem_kernel(const __grid_constant__ SbBatch batch, int32_t* __restrict__ status) {
   extern __shared__ __align__(1024) uint8_t smem[];
   using S = Shape<W, DEPTH, WARPS>;
   constexpr uint32_t SLOT = S::kSlot, kTableAddr = S::kTableAddr;
   constexpr int kThreads = S::kThreads;
-  static_assert(WARPS <= 32, "one lane of the feeding warp per lookup warp");
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3, hl = g >> 2, rot = g & 3;
   const uint32_t dyn = smem_u32(smem);
@@ -188,97 +184,23 @@ lut_smem_kernel(const __grid_constant__ SbBatch batch, int32_t* __restrict__ sta
     if (tid == 0 && status) atomicExch(status, (int)LCD_ERR_UNSUPPORTED);   // the window is not laid out as assumed
     return;
   }
-  // misc area: full barriers [WARPS][DEPTH] | empty barriers [WARPS][DEPTH] | partial maxima [WARPS] | go | abort
-  constexpr int kBarBytes = WARPS * DEPTH * 8;
-  static_assert(2 * kBarBytes + WARPS * 4 + 8 <= kMiscBytes, "barriers, maxima and flags");
-  float* s_part = reinterpret_cast<float*>(smem + 2 * kBarBytes);
-  int& s_go = *reinterpret_cast<int*>(smem + 2 * kBarBytes + WARPS * 4);
-  volatile int& s_abort = *reinterpret_cast<volatile int*>(smem + 2 * kBarBytes + WARPS * 4 + 4);
-  if (tid == 0) {
-    for (int i = 0; i < 2 * WARPS * DEPTH; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(dyn + 8u * i));
+  const uint32_t ring0 = dyn + kMiscBytes + (uint32_t)(warp * DEPTH) * SLOT;
+  const uint32_t bar0 = dyn + 8u * (uint32_t)(warp * DEPTH);
+  float* s_part = reinterpret_cast<float*>(smem + WARPS * DEPTH * 8);          // [WARPS]
+  static_assert(WARPS * DEPTH * 8 + WARPS * 4 + 4 <= kMiscBytes, "barriers, maxima and the go flag");
+  if (lane == 0) {
+#pragma unroll
+    for (int i = 0; i < DEPTH; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0 + 8u * i));
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    s_abort = 0;
   }
-  __syncthreads();
+  __syncwarp();
 
   // the CTA's piece of the work sequence
   const uint2 st0 = batch.start[blockIdx.x], st1 = batch.start[blockIdx.x + 1];
   Piece geo{batch, (int)(st1.x >> 16), (int)(st1.x & 0xffffu), (int)st1.y};
   const int p0 = (int)(st0.x >> 16), s0 = (int)(st0.x & 0xffffu), rp0 = (int)st0.y;
   const bool has_work = !geo.at_end(p0, s0, rp0);
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-
-  if (warp == WARPS) {
-    // ---- the feeding warp: lane w walks lookup warp w's row groups (every WARPS-th group of every segment of the
-    // piece, a fixed stride apart inside a segment) and keeps that warp's ring full ----------------------------
-    uint64_t stream_policy;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_policy));
-    const int w = lane;
-    const uint32_t full0 = dyn + 8u * (uint32_t)(w * DEPTH), empty0 = full0 + kBarBytes;
-    const uint32_t slot0 = dyn + kMiscBytes + (uint32_t)(w * DEPTH) * SLOT;
-    int f_p = p0, f_s = s0, f_rp = rp0 + w, f_rp_end = 0;
-    bool f_live = has_work && w < WARPS;
-    uint32_t f_bytes = 0, n_issued = 0;
-    const uint8_t* f_src = nullptr;
-    size_t f_stride = 0;
-    auto f_enter = [&]() {      // settles on the first segment from (f_p, f_s) in which warp w has a row group
-      while (f_live) {
-        const int rp_end = geo.seg_end(f_p, f_s);
-        if (f_rp < rp_end) {
-          const SbProblem& P = batch.p[f_p];
-          int kt0, width;
-          slice_range(P, f_s, &kt0, &width);
-          f_rp_end = rp_end;
-          f_bytes = (uint32_t)width * kItemBytes;
-          f_src = P.items + ((size_t)f_rp * P.n_kt + kt0) * kItemBytes;
-          f_stride = (size_t)WARPS * P.n_kt * kItemBytes;
-          return;
-        }
-        f_live = geo.next_segment(f_p, f_s);
-        f_rp = w;
-      }
-    };
-    f_enter();
-    bool gave_up = false;
-    // Use j of a slot (j = n_issued / DEPTH) may start when the lookup warp has released use j - 1.  Weights do not
-    // depend on the previous kernel of the stream, so the stream starts before the dependency wait of the others.
-    while (__any_sync(0xffffffffu, f_live) && !gave_up) {
-      if (f_live) {
-        const uint32_t d = n_issued % DEPTH, use = n_issued / DEPTH;
-        bool free_now = use == 0 || mbar_try(empty0 + 8u * d, (use - 1) & 1u);
-        if (!free_now) {
-          const unsigned long long t0 = globaltimer();
-          for (uint32_t it = 1; !free_now; ++it) {
-            free_now = mbar_try(empty0 + 8u * d, (use - 1) & 1u);
-            if (!free_now && (it & 255u) == 0 && (s_abort || globaltimer() - t0 > kTimeoutNs)) break;
-          }
-        }
-        if (free_now) {
-          const uint32_t bar = full0 + 8u * d;
-          asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(f_bytes) : "memory");
-          // weights are read once: evict-first keeps them from displacing what every CTA and every launch re-reads
-          asm volatile(
-              "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-              ::"r"(slot0 + d * SLOT), "l"(f_src), "r"(f_bytes), "r"(bar), "l"(stream_policy) : "memory");
-          ++n_issued;
-          f_src += f_stride;
-          f_rp += WARPS;
-          if (f_rp >= f_rp_end) {
-            f_live = geo.next_segment(f_p, f_s);
-            f_rp = w;
-            f_enter();
-          }
-        } else {
-          f_live = false;         // the lookup warp gave up (or never came): stop feeding it
-          if (!s_abort) { s_abort = 1; if (status) atomicExch(status, (int)LCD_ERR_TIMEOUT); }
-        }
-      }
-    }
-    // copies already issued must land before the CTA may exit
-    for (uint32_t k = n_issued > (uint32_t)DEPTH ? n_issued - DEPTH : 0; k < n_issued; ++k)
-      (void)mbar_wait(full0 + 8u * (k % DEPTH), (k / DEPTH) & 1u);
-  }
 
   // per-lane constants of the lookups
   uint32_t sel[4], c_first = 0, c_second = 0;
@@ -290,12 +212,61 @@ lut_smem_kernel(const __grid_constant__ SbBatch batch, int32_t* __restrict__ sta
     c_second |= (4u * (uint32_t)(16 * (1 - hl) + 4 * t) + 4u * r) << (8 * s);
   }
   const uint32_t bsel = g < 4 ? 1u << (8 * g) : 0u;     // B fragment: k-row 4t + i feeds column i
-  const bool looker = warp < WARPS;
-  const uint32_t full0 = dyn + 8u * (uint32_t)((looker ? warp : 0) * DEPTH), empty0 = full0 + kBarBytes;
-  const uint32_t ring0 = dyn + kMiscBytes + (uint32_t)((looker ? warp : 0) * DEPTH) * SLOT;
-  auto sync_lookers = [&]() { asm volatile("bar.sync 1, %0;" ::"n"(WARPS * 32) : "memory"); };
 
-  if (looker && has_work && batch.p[p0].act_bits == 16) {
+  // ---- fetch side of the ring: runs ahead of the consumer over the same walk -------------------------
+  // A warp takes every WARPS-th row group of every segment (problem, slice) of the piece.  Inside a segment the next
+  // row group is a fixed stride further in memory; the slice's geometry is worked out once per segment.
+  uint64_t stream_policy;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_policy));
+  int f_p = p0, f_s = s0, f_rp = rp0 + warp, f_rp_end = 0;
+  bool f_live = has_work;
+  uint32_t f_slot = 0, f_inflight = 0, f_bytes = 0;
+  const uint8_t* f_src = nullptr;
+  size_t f_stride = 0;
+  auto f_enter = [&]() {      // settles on the first segment from (f_p, f_s) in which this warp has a row group
+    while (f_live) {
+      const int rp_end = geo.seg_end(f_p, f_s);
+      if (f_rp < rp_end) {
+        const SbProblem& P = batch.p[f_p];
+        int kt0, width;
+        slice_range(P, f_s, &kt0, &width);
+        f_rp_end = rp_end;
+        f_bytes = (uint32_t)width * kItemBytes;
+        f_src = P.items + ((size_t)f_rp * P.n_kt + kt0) * kItemBytes;
+        f_stride = (size_t)WARPS * P.n_kt * kItemBytes;
+        return;
+      }
+      f_live = geo.next_segment(f_p, f_s);
+      f_rp = warp;
+    }
+  };
+  f_enter();
+  auto fetch_one = [&]() {
+    if (!f_live) return;
+    if (lane == 0) {
+      const uint32_t bar = bar0 + 8u * f_slot;
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(f_bytes) : "memory");
+      // weights are read once: evict-first keeps them from displacing what every CTA and every launch re-reads
+      asm volatile(
+          "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+          ::"r"(ring0 + f_slot * SLOT), "l"(f_src), "r"(f_bytes), "r"(bar), "l"(stream_policy) : "memory");
+    }
+    f_slot = f_slot + 1 == (uint32_t)DEPTH ? 0u : f_slot + 1;
+    ++f_inflight;
+    f_src += f_stride;
+    f_rp += WARPS;
+    if (f_rp >= f_rp_end) {
+      f_live = geo.next_segment(f_p, f_s);
+      f_rp = warp;
+      f_enter();
+    }
+  };
+
+  // Weights do not depend on the previous kernel of the stream: one stage per warp is queued before the dependency
+  // wait, the others right behind the first requests for the activations (an SM's loads return in the order they
+  // were queued, and the small ones must not wait behind the whole ring).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (has_work && batch.p[p0].act_bits == 16) {
     // ask the token and its smoothing factors into L2 (the weight stream evicts them between launches); a prefetch
     // cannot read stale data, L2 is the point of coherence
     const SbProblem& P = batch.p[p0];
@@ -307,14 +278,16 @@ lut_smem_kernel(const __grid_constant__ SbBatch batch, int32_t* __restrict__ sta
       }
     }
   }
-  if (looker) asm volatile("griddepcontrol.wait;" ::: "memory");
+  fetch_one();
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  bool ring_primed = false;
 
   uint32_t c_slot = 0, c_phase = 0;
   bool aborted = false;
   int cur_p = -1;
   float amax = 0.0f;          // fused: the token's max |x * inv_s| of problem cur_p
   int seg_p = p0, seg_s = s0, seg_rp = rp0;
-  bool seg_live = has_work && looker;
+  bool seg_live = has_work;
 
 #pragma unroll 1
   while (seg_live) {
@@ -385,11 +358,15 @@ lut_smem_kernel(const __grid_constant__ SbBatch batch, int32_t* __restrict__ sta
           for (int k = tid; k < P.K; k += kThreads)
             m = fmaxf(m, fabsf(__fmul_rn(__half2float(P.x[k]), P.inv_smooth ? __ldg(P.inv_smooth + k) : 1.0f)));
         }
+        if (!ring_primed) {
+          for (int i = 1; i < DEPTH; ++i) fetch_one();
+          ring_primed = true;
+        }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-        sync_lookers();                         // the previous problem's maxima have been read
+        __syncthreads();                        // the previous problem's maxima have been read
         if (lane == 0) s_part[warp] = m;
-        sync_lookers();
+        __syncthreads();
         amax = 0.0f;
 #pragma unroll
         for (int w = 0; w < WARPS; ++w) amax = fmaxf(amax, s_part[w]);
@@ -437,76 +414,67 @@ lut_smem_kernel(const __grid_constant__ SbBatch batch, int32_t* __restrict__ sta
         }
       }
     }
-    sync_lookers();
+    if (!ring_primed) {
+      for (int i = 1; i < DEPTH; ++i) fetch_one();
+      ring_primed = true;
+    }
+    __syncthreads();
 
     // ---- this warp's row groups of the segment: seg_rp + warp, + WARPS, ... ------------------------------
-    // wv[b][0..3]: this lane's index words of the tile of rows g in block b, k-block hl first ([0], [1]) and the other
-    // one second ([2], [3]); wv[b][4..7]: the same of the tile of rows g + 8.  The words of the next row group are
-    // taken out of the ring, and its slot handed back, while the MMAs of the current one are still in flight.
     const int bias = 32 * 64 * width;           // every table byte carries + 32, a row takes 64 lookups per block
     const int rp_first = seg_rp + warp;
-    uint32_t wv[W][8];
-    auto grab = [&]() -> bool {
-      if (!__all_sync(0xffffffffu, mbar_wait(full0 + 8u * c_slot, c_phase))) return false;
-      const uint32_t item0 = ring0 + c_slot * SLOT + 16u * (uint32_t)lane;
-      uint32_t seen = 0;
-#pragma unroll
-      for (int b = 0; b < W; ++b) {
-        if (b < width) {
-          const uint4 r0 = lds128(item0 + (uint32_t)b * kItemBytes), r1 = lds128(item0 + (uint32_t)b * kItemBytes + 512u);
-          wv[b][0] = hl ? r0.z : r0.x; wv[b][1] = hl ? r0.w : r0.y; wv[b][2] = hl ? r0.x : r0.z; wv[b][3] = hl ? r0.y : r0.w;
-          wv[b][4] = hl ? r1.z : r1.x; wv[b][5] = hl ? r1.w : r1.y; wv[b][6] = hl ? r1.x : r1.z; wv[b][7] = hl ? r1.y : r1.w;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) seen ^= wv[b][i];
-        }
-      }
-      // the slot may be refilled once every lane holds its words: the release is made to depend on them
-      asm volatile("" ::"r"(seen) : "memory");
-      __syncwarp();
-      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty0 + 8u * c_slot) : "memory");
-      if (++c_slot == (uint32_t)DEPTH) { c_slot = 0; c_phase ^= 1u; }
-      return true;
-    };
-    if (!aborted && rp_first < rp_end) {
+    if (!aborted) {
       float* dst = P.sums + ((size_t)rp_first * 16 + g) * 4 + (t == 1 ? 32 : 0);
-      aborted = !grab();
 #pragma unroll 1
-      for (int rp = rp_first; rp < rp_end && !aborted; rp += WARPS) {
-        int acc[4] = {-bias, -bias, -bias, -bias}, acc2[4] = {0, 0, 0, 0};    // two chains of dependent MMAs
+      for (int rp = rp_first; rp < rp_end; rp += WARPS) {
+        if (!__all_sync(0xffffffffu, mbar_wait(bar0 + 8u * c_slot, c_phase))) { aborted = true; break; }
+        const uint32_t item0 = ring0 + c_slot * SLOT + 16u * (uint32_t)lane;
+        int acc[4] = {0, 0, 0, 0}, acc2[4] = {0, 0, 0, 0};    // two chains of dependent MMAs
 #pragma unroll
         for (int b = 0; b < W; ++b) {
           if (b < width) {
+            const uint32_t it = item0 + (uint32_t)b * kItemBytes;
+            const uint4 r0 = lds128(it), r1 = lds128(it + 512u);        // this lane's 16 bytes of both tiles
+            // k-block hl first, the other one second
+            const uint32_t f0x = hl ? r0.z : r0.x, f0y = hl ? r0.w : r0.y, g0x = hl ? r0.x : r0.z, g0y = hl ? r0.y : r0.w;
+            const uint32_t f1x = hl ? r1.z : r1.x, f1y = hl ? r1.w : r1.y, g1x = hl ? r1.x : r1.z, g1y = hl ? r1.y : r1.w;
             if (b == 0) {
-              half_item<kTableAddr>(wv[b][0], wv[b][1], wv[b][4], wv[b][5], c_first, sel, bsel, acc, acc2);
-              half_item<kTableAddr>(wv[b][2], wv[b][3], wv[b][6], wv[b][7], c_second, sel, bsel, acc, acc2);
+              half_item<kTableAddr>(f0x, f0y, f1x, f1y, c_first, sel, bsel, acc, acc2);
+              half_item<kTableAddr>(g0x, g0y, g1x, g1y, c_second, sel, bsel, acc, acc2);
             } else if (b == 1) {
-              half_item<kTableAddr + kBlockBytes>(wv[b][0], wv[b][1], wv[b][4], wv[b][5], c_first, sel, bsel, acc, acc2);
-              half_item<kTableAddr + kBlockBytes>(wv[b][2], wv[b][3], wv[b][6], wv[b][7], c_second, sel, bsel, acc, acc2);
+              half_item<kTableAddr + kBlockBytes>(f0x, f0y, f1x, f1y, c_first, sel, bsel, acc, acc2);
+              half_item<kTableAddr + kBlockBytes>(g0x, g0y, g1x, g1y, c_second, sel, bsel, acc, acc2);
             } else {
-              half_item<kTableAddr + 2u * kBlockBytes>(wv[b][0], wv[b][1], wv[b][4], wv[b][5], c_first, sel, bsel, acc, acc2);
-              half_item<kTableAddr + 2u * kBlockBytes>(wv[b][2], wv[b][3], wv[b][6], wv[b][7], c_second, sel, bsel, acc, acc2);
+              half_item<kTableAddr + 2u * kBlockBytes>(f0x, f0y, f1x, f1y, c_first, sel, bsel, acc, acc2);
+              half_item<kTableAddr + 2u * kBlockBytes>(g0x, g0y, g1x, g1y, c_second, sel, bsel, acc, acc2);
             }
           }
         }
-        if (rp + WARPS < rp_end) aborted = !grab();
+        --f_inflight;
+        if (++c_slot == (uint32_t)DEPTH) { c_slot = 0; c_phase ^= 1u; }
         // lanes t = 0, 1 hold buckets 2t, 2t + 1 of rows g and g + 8
-        const float f0 = (float)(acc[0] + acc2[0]), f1 = (float)(acc[1] + acc2[1]);
-        const float f2 = (float)(acc[2] + acc2[2]), f3 = (float)(acc[3] + acc2[3]);
+        const float f0 = (float)(acc[0] + acc2[0] - bias), f1 = (float)(acc[1] + acc2[1] - bias);
+        const float f2 = (float)(acc[2] + acc2[2] - bias), f3 = (float)(acc[3] + acc2[3] - bias);
         // lane t = 0 collects the four buckets of row g, lane t = 1 those of row g + 8
         const float x0 = __shfl_xor_sync(0xffffffffu, t == 0 ? f2 : f0, 1);
         const float x1 = __shfl_xor_sync(0xffffffffu, t == 0 ? f3 : f1, 1);
+        fetch_one();       // the sums are formed, so every read of the slot has completed: it may be refilled
         if (t == 0) red_add_v4(dst, f0, f1, x0, x1);
         if (t == 1) red_add_v4(dst, x0, x1, f2, f3);
         dst += (size_t)WARPS * 64;
       }
-      if (aborted) {
-        s_abort = 1;
-        if (lane == 0 && status) atomicExch(status, (int)LCD_ERR_TIMEOUT);
-      }
+      if (aborted && lane == 0 && status) atomicExch(status, (int)LCD_ERR_TIMEOUT);
     }
     seg_live = geo.next_segment(seg_p, seg_s);
     seg_rp = 0;
-    if (seg_live) sync_lookers();      // every warp is done with the tables before they are rebuilt
+    if (seg_live) __syncthreads();     // every warp is done with the tables before they are rebuilt
+  }
+  if (aborted) {      // copies already issued must land before the CTA may exit
+    while (f_inflight > 0) {
+      (void)mbar_wait(bar0 + 8u * c_slot, c_phase);
+      --f_inflight;
+      if (++c_slot == (uint32_t)DEPTH) { c_slot = 0; c_phase ^= 1u; }
+    }
   }
 
   // ---- every CTA's sums must be in the scratch before a row can be finished ---------------------------------
@@ -520,13 +488,14 @@ lut_smem_kernel(const __grid_constant__ SbBatch batch, int32_t* __restrict__ sta
     *n = r - batch.row0[p];
     return p;
   };
-  int r = (int)blockIdx.x * S::kBlock + tid;
+  int r = (int)blockIdx.x * kThreads + tid;
   int n_cur = 0, p_cur = 0;
   uint2 c_cur = make_uint2(0u, 0u);
   if (r < total_rows) {
     p_cur = locate(r, &n_cur);
     c_cur = __ldg(reinterpret_cast<const uint2*>(batch.p[p_cur].codebook + (size_t)n_cur * 4));
   }
+  int& s_go = *reinterpret_cast<int*>(smem + WARPS * DEPTH * 8 + WARPS * 4);   // in the misc area: no static shared memory
   __threadfence();                       // this thread's reductions are performed
   __syncthreads();
   if (tid == 0) {
@@ -547,7 +516,7 @@ lut_smem_kernel(const __grid_constant__ SbBatch batch, int32_t* __restrict__ sta
     if (tid == 0 && status) atomicExch(status, (int)LCD_ERR_TIMEOUT);
     return;
   }
-  for (; r < total_rows; r += (int)gridDim.x * S::kBlock) {
+  for (; r < total_rows; r += (int)gridDim.x * kThreads) {
     const SbProblem& P = batch.p[p_cur];
     float4* src = reinterpret_cast<float4*>(P.sums) + n_cur;
     const float4 Sw = __ldcg(src);
@@ -557,7 +526,7 @@ lut_smem_kernel(const __grid_constant__ SbBatch batch, int32_t* __restrict__ sta
     const float2 c23 = __half22float2(*reinterpret_cast<const __half2*>(&c_cur.y));
     const float v = (c01.x * Sw.x + c01.y * Sw.y) + (c23.x * Sw.z + c23.y * Sw.w);
     if (n_cur < P.N) P.y[n_cur] = v * sq;
-    const int r_next = r + (int)gridDim.x * S::kBlock;
+    const int r_next = r + (int)gridDim.x * kThreads;
     if (r_next < total_rows) {
       p_cur = locate(r_next, &n_cur);
       c_cur = __ldg(reinterpret_cast<const uint2*>(batch.p[p_cur].codebook + (size_t)n_cur * 4));
@@ -643,10 +612,12 @@ lcd_status launch_lut_smem(const Problem* probs, int count, void* workspace, siz
   // for every slice it touches, the table build (in items, measured); the smallest cost limit that fits into the
   // CTAs is found by bisection over a greedy sweep.
   const int n_cta = sm_count_now() < kMaxCta ? sm_count_now() : kMaxCta;
-  // fixed cost of a segment in items (measured at about 30 ns per item): its tables take 1.2 us, the token's maximum
-  // of another problem 1.3 us, the barriers around a rebuild 0.5 us
-  auto build_cost = [](int width, bool first, bool new_problem) {
-    return 10 + 15 * width + (first ? 0 : 15) + (new_problem ? 45 : 0);
+  // Costs in units of 9 ns (measured): a row group takes 27 ns plus 18 ns per item (3 + 2 * width), a segment's
+  // tables 1.2 us, the token's maximum of another problem 0.9 us plus 0.1 us per 1024 columns, the barriers around a
+  // rebuild and the warps' uneven ends 1.5 us.
+  auto group_cost = [](int width) { return 3 + 2 * width; };
+  auto build_cost = [](int width, bool first, int new_problem_K) {
+    return 30 + 50 * width + (first ? 0 : 165) + (new_problem_K > 0 ? 100 + new_problem_K / 90 : 0);
   };
   auto sweep = [&](long long limit, uint2* start) -> int {
     int cta = 0, last_p = -1;   // last_p: problem of the current CTA's latest segment
@@ -658,8 +629,8 @@ lcd_status launch_lut_smem(const Problem* probs, int count, void* workspace, siz
         const int width = (int)((long long)(s + 1) * g.n_kt / g.n_slices - (long long)s * g.n_kt / g.n_slices);
         int rp = 0;
         while (rp < g.n_rp) {
-          const int fixed = build_cost(width, !open, !open || last_p != p);
-          long long room = (limit - used - fixed) / width;
+          const int fixed = build_cost(width, !open, (!open || last_p != p) ? g.K : 0);
+          long long room = (limit - used - fixed) / group_cost(width);
           if (room < 1 && open) {      // no room for even one row group of this slice: next CTA
             ++cta;
             used = 0;
@@ -672,7 +643,7 @@ lcd_status launch_lut_smem(const Problem* probs, int count, void* workspace, siz
             open = true;
           }
           const int take = (int)(room < g.n_rp - rp ? room : g.n_rp - rp);
-          used += fixed + (long long)take * width;
+          used += fixed + (long long)take * group_cost(width);
           last_p = p;
           rp += take;
           if (rp < g.n_rp) {           // the slice continues in the next CTA
@@ -687,8 +658,9 @@ lcd_status launch_lut_smem(const Problem* probs, int count, void* workspace, siz
   };
   long long total = 0, lo = 1, hi;
   for (int p = 0; p < count; ++p)
-    total += (long long)batch.p[p].n_rp * batch.p[p].n_kt + (long long)batch.p[p].n_slices * build_cost(kSliceBlocks, false, true);
-  hi = total + build_cost(kSliceBlocks, false, true) + kSliceBlocks;
+    total += (long long)batch.p[p].n_rp * batch.p[p].n_slices * group_cost(kSliceBlocks) +
+             (long long)batch.p[p].n_slices * build_cost(kSliceBlocks, false, batch.p[p].K);
+  hi = total + build_cost(kSliceBlocks, false, 1 << 20) + group_cost(kSliceBlocks);
   while (lo < hi) {
     const long long mid = (lo + hi) / 2;
     if (sweep(mid, nullptr) <= n_cta) hi = mid; else lo = mid + 1;
@@ -707,7 +679,7 @@ lcd_status launch_lut_smem(const Problem* probs, int count, void* workspace, siz
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)used);
-  cfg.blockDim = dim3(LaunchShape::kBlock);
+  cfg.blockDim = dim3(LaunchShape::kThreads);
   cfg.dynamicSmemBytes = LaunchShape::kSmemBytes;
   cfg.stream = static_cast<cudaStream_t>(stream);
   // cooperative: all CTAs wait for one another before the rows are finished, so all of them must be resident
