@@ -29,15 +29,15 @@ import numpy as np  # noqa: E402
 
 from synth import gen  # noqa: E402
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, bytes per launch) of the dominant kernel from the ncu
-# captures summarised under profiles/, with the hash of the kernel source they were taken from: a kernel that has
-# changed since reports traffic = null.
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, bytes per launch) of the dominant kernel of a workload,
+# from one ncu capture each, with the hash of the kernel source the capture was taken from: a kernel that has changed
+# since reports traffic = null.  Keys: (kernel source, configuration, M).
 NCU_TRAFFIC = {
-    # profiles/lut_gemv_kernel_llama7b_2bit_m1.md: one launch (input transformation + lookup) of configuration 1 at M = 1
-    ("lut_gemv.cu", 1, 1): {"sha256": "ad1eec2679f61945c235cc9c15ca7aa1a36efaf65692539c1eca2916de51bfba", "bytes_per_launch": 51208704 + 20224},
-    # profiles/dense_tc_kernel_llama13b_2bit_m2048.md: the layer's seven launches of configuration 3: q captured
-    # (17.11 + 0.44 MB, taken four times for q/k/v/o), gate captured (28.37 + 56.32 MB, twice for gate/up), down
-    # scaled from q by its 2.7 times longer rows (same tiles, traffic in proportion to K)
+    # one launch (input transformation + lookup) of the LLaMA-7B-shaped 2-bit layer at M = 1
+    ("lut_smem.cu", 1, 1): {"sha256": "", "bytes_per_launch": 51875584 + 48640},
+    # the seven launches of the LLaMA-13B-shaped layer at M = 2048: q captured (17.11 + 0.44 MB, taken four times for
+    # q/k/v/o), gate captured (28.37 + 56.32 MB, twice for gate/up), down scaled from q by its 2.7 times longer rows
+    # (same tiles, traffic in proportion to K)
     ("dense_tc.cu", 3, 2048): {"sha256": "c29890f9ab90dad858f8486d69f2bb16e902631e75ef856b650a66523b6d474b",
                                "bytes_per_launch": int(4 * 17.55e6 + 2 * 84.70e6 + 17.55e6 * 13824 / 5120)},
 }
@@ -54,6 +54,7 @@ def parse_args():
     ap.add_argument("--M", type=int, default=None, help="token count (default: first M of the config)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true", help="default workload only: skip the M = 2048 and other workloads of the line")
     ap.add_argument("--act-bits", type=int, default=4, choices=[4, 8],
                     help="activation levels: 4 bit (the benchmark configurations) or 8 bit (the paper's b = 8)")
     ap.add_argument("--aux", default=None, choices=["smoothing", "reclassify", "dbci"],
@@ -216,7 +217,6 @@ def per_layer_us(ms_step, world):
 def run_ours(args):
     import torch
     import torch.distributed as dist
-    import paper_2506_12038_b200 as lcd
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -225,13 +225,41 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
-
     cfg = gen.CONFIGS[args.config]
     M = args.M or cfg["Ms"][0]
+    line = measure_config(args, args.config, M, dev, world, local, primary=True)
+    if rank == 0 and line is not None:
+        if world == 1 and not args.no_secondary and args.config == 1 and args.M is None and args.act_bits == 4 \
+                and args.algo == "auto" and not args.two_call:
+            # the rest of the metric in the same line: the prefill half (M = 2048) and the other single-token workloads
+            line["secondary"] = []
+            for cid, m in ((3, 2048), (4, 1), (0, 1)):
+                sec = measure_config(args, cid, m, dev, 1, local, primary=False)
+                line["secondary"].append({k: sec[k] for k in ("metric", "value", "unit", "ms_per_step", "timing", "config",
+                                                              "TFLOPs_equiv", "layer_GBps", "roofline", "parity",
+                                                              "gpu_launches") if k in sec})
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def measure_config(args, cfg_id, M, dev, world, local, primary):
+    """One workload: builds its layer, times the step (median over repeats of exactly --steps steps, at least 0.2 s in
+    all), the dominant kernel and (primary only) the end-to-end path, compares the timed path's outputs with the
+    oracle and returns the JSON line as a dict (None on ranks other than 0)."""
+    import torch
+    import torch.distributed as dist
+    import paper_2506_12038_b200 as lcd
+
+    rank = int(os.environ.get("RANK", "0"))
+    cfg = gen.CONFIGS[cfg_id]
     bits = cfg["bits"]
-    _, layers = build_layers(args.config, M)       # every rank: its own replica of the layer (weak scaling)
+    steps = args.steps if primary else max(10, min(args.steps, 40))
+    _, layers = build_layers(cfg_id, M)            # every rank: its own replica of the layer (weak scaling)
     layer_bytes = sum(lcd.packed_weights_bytes(L.N, L.K, bits) for _, L in layers)
     copies = max(2, int(np.ceil(ROTATE_BYTES / layer_bytes)))
+    if not primary:
+        steps = max(steps, 2 * copies)       # whole rounds of the back-to-back graph, as in a long run
 
     mats = []
     for name, L in layers:
@@ -252,6 +280,10 @@ def run_ours(args):
     grouped = M <= 16 and len(mats) <= lcd.MAX_BATCH
     algo = {"auto": lcd.ALGO_AUTO, "register": lcd.ALGO_REGISTER_LUT, "bucket": lcd.ALGO_BUCKET_LUT,
             "tensor": lcd.ALGO_TC_LUT, "shared": lcd.ALGO_SHARED_BUCKET}[args.algo]
+    # which lookup kernel the library runs for this launch shape (its own answer, not a guess made here)
+    shared_bucket = grouped and lcd.resolve_batch_algo([(mt["w"][0], M) for mt in mats], algo) == lcd.ALGO_SHARED_BUCKET \
+        and args.act_bits == 4
+    lookup_kernel = "lut_smem_kernel" if shared_bucket else "lut_gemv_kernel"
     # every kernel that can give up on a bounded wait reports it here; a non-zero word voids the run
     status = torch.zeros((1,), dtype=torch.int32, device=dev)
     if grouped:
@@ -311,7 +343,7 @@ def run_ours(args):
         with torch.cuda.graph(round_graph, stream=stream):
             for c in range(copies):
                 step(c)
-        for i in range(max(args.warmup, 3)):
+        for i in range(max(args.warmup, 3) if primary else 3):
             graphs[i % copies].replay()
         round_graph.replay()
         torch.cuda.synchronize()
@@ -319,18 +351,26 @@ def run_ours(args):
             dist.barrier()
         sampler = ClockSampler(local)
         sampler.start()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        # Every repeat times exactly `steps` steps between two events; repeats go on until at least 5 were taken and
+        # 0.2 s were timed in all (a short --steps run would otherwise be a fraction of a millisecond and one clock
+        # sample).  The reported step time is the median over the repeats, the minimum is given beside it.
+        rep_ms = []
         torch.cuda.synchronize()
-        e0.record()
-        for i in range(args.steps // copies):
-            round_graph.replay()
-        for i in range(args.steps % copies):
-            graphs[i].replay()
-        e1.record()
-        torch.cuda.synchronize()
-        ms_total = e0.elapsed_time(e1)
+        while len(rep_ms) < 5 or (sum(rep_ms) < 200.0 and len(rep_ms) < 2000):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(steps // copies):
+                round_graph.replay()
+            for i in range(steps % copies):
+                graphs[i].replay()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+            if world > 1:
+                ms = max_over_ranks(ms, dev)          # the same number of repeats on every rank: the maxima decide
+            rep_ms.append(ms)
+        ms_total = statistics.median(rep_ms)
         if world > 1:
-            ms_total = max_over_ranks(ms_total, dev)
             dist.barrier()
 
         # dominant kernel: the lookup+accumulate launches alone, back to back inside a graph, every launch on
@@ -342,7 +382,7 @@ def run_ours(args):
             g.replay()
             torch.cuda.synchronize()
             k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            n_rep = max(3, min(args.steps, 20))
+            n_rep = max(3, min(steps, 20))
             k0.record()
             for _ in range(n_rep):
                 g.replay()
@@ -361,12 +401,12 @@ def run_ours(args):
         kern_flop = sum(mt["flop"] for mt in mats)
         if grouped and fused:
             kern_ms = time_graph(lambda: [fbatch[c].run() for _ in range(reps) for c in range(copies)], reps * copies)
-            kern_name = "lut_gemv_kernel, one launch per layer: input transformation + lookup of all its matrices"
+            kern_name = lookup_kernel + ", one launch per layer: input transformation + lookup of all its matrices"
             # the launch reads x (fp16) and the smoothing factors instead of stored levels and scales
             kern_bytes += sum(M * mt["L"].K * 2 + mt["L"].K * 4 - M * (mt["L"].K / 2 + 4) for mt in mats)
         elif grouped:
             kern_ms = time_graph(lambda: [lbatch[c].run() for _ in range(reps) for c in range(copies)], reps * copies)
-            kern_name = "lut_gemv_kernel, one grouped launch over the layer's matrices"
+            kern_name = lookup_kernel + ", one grouped launch over the layer's matrices"
         else:
             kern_ms = sum_ms
             kern_name = "lcd_lut_linear launches of one layer (sum of bytes / sum of durations)"
@@ -375,7 +415,9 @@ def run_ours(args):
         # end to end through the host-buffer entry points: pinned host x -> device -> kernels -> pinned host y.
         # Grouped (M <= 16): one copy in, two launches, one copy out per layer; else per matrix.
         e2e_ms, h2d, d2h = None, 0, 0
-        if grouped and args.act_bits == 4:
+        if not primary:
+            pass
+        elif grouped and args.act_bits == 4:
             hbatch = [lcd.HostBatch([(mt["w"][c], mt["inv_s"], M) for mt in mats], dev) for c in range(copies)]
             for hb in hbatch:
                 for i, mt in enumerate(mats):
@@ -408,22 +450,26 @@ def run_ours(args):
                         yh.copy_(mt["y"], non_blocking=True)
                 torch.cuda.current_stream().synchronize()
 
-        n_e2e = max(3, min(args.steps, 50))
-        for c in range(min(copies, 3)):
-            e2e_step(c)
+        if primary:
+            n_e2e = max(3, min(steps, 50))
+            for c in range(min(copies, 3)):
+                e2e_step(c)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            g0.record()
+            for i in range(n_e2e):
+                e2e_step(i % copies)
+            g1.record()
+            torch.cuda.synchronize()
+            e2e_ms = max(g0.elapsed_time(g1), (time.perf_counter() - t0) * 1e3) / n_e2e
+            if world > 1:
+                e2e_ms = max_over_ranks(e2e_ms, dev)
+        # the outputs and stored levels of the timed path, for the comparison with the oracle below
+        step(0)
         torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        g0.record()
-        for i in range(n_e2e):
-            e2e_step(i % copies)
-        g1.record()
-        torch.cuda.synchronize()
-        e2e_ms = max(g0.elapsed_time(g1), (time.perf_counter() - t0) * 1e3) / n_e2e
-        if world > 1:
-            e2e_ms = max_over_ranks(e2e_ms, dev)
 
-    ms_step = ms_total / args.steps
+    ms_step = ms_total / steps
     us_per_layer = per_layer_us(ms_step, world)
     layer_alg_bytes = sum(mt["bytes"] for mt in mats)
     peaks = {}
@@ -436,15 +482,17 @@ def run_ours(args):
         peak = peaks.get("bf16_tflops", 1590.0)
         achieved = kern_flop / kern_ms / 1e9
         roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                "traffic": None, "peak_source": "measured (cuBLAS bf16 burst)" if peaks else "fallback"}
+                "traffic": None, "peak_source": "measured (cuBLAS bf16 burst)" if peaks else "fallback",
+                "frac_of_sustained": achieved / peaks.get("bf16_tflops_sustained", 1400.0),
+                "frac_of_2250_nominal": achieved / 2250.0}
     else:
         peak = peaks.get("hbm_gbs", 6650.0)
         achieved = kern_bytes / kern_ms / 1e6
         roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": None, "peak_source": "measured (copy)" if peaks else "fallback",
                 "frac_of_8TBps_nominal": achieved / 8000.0}
-    src = "dense_tc.cu" if tensor_bound else "lut_gemv.cu"
-    rec = NCU_TRAFFIC.get((src, args.config, M))
+    src = "dense_tc.cu" if tensor_bound else ("lut_smem.cu" if shared_bucket else "lut_gemv.cu")
+    rec = NCU_TRAFFIC.get((src, cfg_id, M))
     if rec and rec["bytes_per_launch"] is not None:
         import hashlib
         with open(os.path.join(ROOT, "paper_2506_12038_b200", "csrc", src), "rb") as fh:
@@ -458,37 +506,74 @@ def run_ours(args):
     roof["per_matrix"] = per_matrix
 
     if rank != 0:
-        return
-    line = {"metric": metric_name(M), "value": us_per_layer, "unit": "us/layer", "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
-            "vs_baseline": None, "dtype": "s8 table bytes x s8 levels -> s32 (int8 MMA), f32 epilogue" if not tensor_bound else "s8 table bytes x s8 levels -> s32 (tcgen05 kind::i8), f32 epilogue",
-            "data": "synthetic", "config": dict(workload_config(args.config, M, copies, args.act_bits),
+        return None
+    line = {"metric": metric_name(M), "value": us_per_layer, "unit": "us/layer", "n_gpus": world, "steps": steps,
+            "warmup": max(args.warmup, 3) if primary else 3, "ms_per_step": ms_step, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": ("s8 table bytes x s8 levels -> s32 (tcgen05 kind::i8), f32 epilogue" if tensor_bound else
+                      "u8 bucket-table bytes -> s32 (int8 MMA), f32 sums and epilogue" if shared_bucket else
+                      "s8 table bytes x s8 levels -> s32 (int8 MMA), f32 epilogue"),
+            "data": "synthetic", "config": dict(workload_config(cfg_id, M, copies, args.act_bits),
                                                 graphs=f"steps replayed as CUDA graphs of {copies} consecutive steps",
                                                 launches=("1 launch per layer: quantise + lookup fused" if grouped and fused
                                                           else "1 grouped quantise + 1 grouped lookup per layer" if grouped
                                                           else "per matrix: quantise + lookup")),
+            "timing": {"repeats": len(rep_ms), "steps_per_repeat": steps, "timed_ms_total": sum(rep_ms),
+                       "us_per_step_median": statistics.median(rep_ms) / steps * 1e3 / world,
+                       "us_per_step_min": min(rep_ms) / steps * 1e3 / world},
             "layer_GBps": layer_alg_bytes * world / (ms_step * 1e-3) / 1e9,
             "layer_algorithmic_bytes": layer_alg_bytes,
             "TFLOPs_equiv": sum(mt["flop"] for mt in mats) * world / (ms_step * 1e-3) / 1e12,
-            "clocks": clocks, "gpu_launches": launches_per_step * args.steps,
-            "e2e": {"value": e2e_ms * 1e3 / world, "unit": "us/layer", "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h},
+            "clocks": clocks, "gpu_launches": launches_per_step * steps * len(rep_ms),
             "roofline": roof}
-    if not args.no_cpu_baseline and world == 1:
-        sample, scale, desc = oracle_sample(args.config, layers, M)
+    if e2e_ms is not None:
+        line["e2e"] = {"value": e2e_ms * 1e3 / world, "unit": "us/layer", "h2d_bytes_per_step": h2d,
+                       "d2h_bytes_per_step": d2h}
+    if world == 1 and not args.no_cpu_baseline:
+        # The oracle on the same inputs: its outputs judge the timed path (every output at small M, the sample at
+        # M = 2048), its running time is the CPU baseline (primary workload only).
+        sample, scale, desc = oracle_sample(cfg_id, layers, M)
         t0 = time.perf_counter()
         n = 0
         while True:
-            oracle_layer_pass(sample)
+            outs = oracle_layer_pass(sample)
             n += 1
-            if time.perf_counter() - t0 > 10.0 or n >= 5:
+            if not primary or time.perf_counter() - t0 > 10.0 or n >= 5:
                 break
         us = (time.perf_counter() - t0) / n * scale * 1e6
-        line["cpu_baseline"] = {"value": us, "unit": "us/layer", "cores": oracle_threads(), "kind": "oracle",
-                                "sample": desc + f", mean of {n} passes"}
-    print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+        if primary:
+            line["cpu_baseline"] = {"value": us, "unit": "us/layer", "cores": oracle_threads(), "kind": "oracle",
+                                    "sample": desc + f", mean of {n} passes"}
+        line["parity"] = parity_verdict(sample, outs, mats, args.act_bits)
+        if not line["parity"]["ok"]:
+            print(json.dumps(line))
+            raise SystemExit("parity with the oracle lost: " + json.dumps(line["parity"]))
+    return line
+
+
+def parity_verdict(sample, oracle_outs, mats, act_bits):
+    """The timed path's outputs against the oracle's on the same inputs: per matrix relative L2 error and
+    max-abs error over the largest reference magnitude (stated tolerance 2e-3 and 1e-2), and the stored activation
+    levels and scales bit for bit.  `sample` is the whole layer, or (large M) the leading rows and tokens of its first
+    matrix: the corresponding corner of the device output is compared."""
+    from oracle import lcd_oracle as O
+    rel_max, abs_max, exact = 0.0, 0.0, True
+    by_name = {mt["name"]: mt for mt in mats}
+    for (name, S), y_ref in zip(sample, oracle_outs):
+        mt = by_name[name]
+        y = mt["y"][:S.M, :S.N].detach().cpu().numpy().astype(np.float64)
+        if not np.all(np.isfinite(y)):
+            return {"ok": False, "reason": f"{name}: non-finite output"}
+        d = np.linalg.norm(y_ref)
+        rel_max = max(rel_max, float(np.linalg.norm(y - y_ref) / (d if d > 0 else 1.0)))
+        ninf = np.abs(y_ref).max()
+        abs_max = max(abs_max, float(np.abs(y - y_ref).max() / (ninf if ninf > 0 else 1.0)))
+        q, sq = O.smooth_quantize(S.x, S.inv_s, act_bits=act_bits)
+        packed = O.pack_act(q) if act_bits == 4 else O.pad_act8(q)
+        exact = exact and np.array_equal(mt["a"][:S.M].cpu().numpy(), packed) and np.array_equal(mt["s"][:S.M].cpu().numpy(), sq)
+    return {"ok": bool(rel_max <= 2e-3 and abs_max <= 1e-2 and exact), "rel_l2_max": rel_max,
+            "max_abs_over_inf": abs_max, "indices_bit_exact": bool(exact),
+            "compared": f"{len(sample)} matrices, " + ("every output" if len(sample) == len(mats) else "the sampled corner (see cpu_baseline.sample)")}
 
 
 def run_aux_smoothing(args):

@@ -209,6 +209,11 @@ lcd_status lcd_lut_linear_batch(const lcd_linear_problem* problems /* host */, i
                                 void* workspace, size_t workspace_bytes, int32_t* status_word_dev,
                                 void* cuda_stream);
 
+/* Which family a grouped call with these shapes and this `algo` runs (what LCD_ALGO_AUTO stands for): only the
+ * header_host and M fields of the problems are read.  The fused call (lcd_linear_fused_batch) chooses the same way. */
+lcd_status lcd_lut_linear_batch_resolve(const lcd_linear_problem* problems /* host */, int count, lcd_algo algo,
+                                        lcd_algo* resolved);
+
 /* lcd_lut_linear_batch for 8-bit levels: every problem's act_idx points at [M][K_pad] signed bytes (see
  * lcd_lut_linear_act8); workspace size from lcd_lut_linear_batch_workspace_bytes. */
 lcd_status lcd_lut_linear_batch_act8(const lcd_linear_problem* problems /* host */, int count, lcd_algo algo,

@@ -26,7 +26,7 @@ MAX_BATCH = 8
 EXPORTS = ["lcd_status_string", "lcd_last_cuda_error", "lcd_packed_weights_bytes", "lcd_pack_weights",
            "lcd_unpack_weights", "lcd_smooth_quantize_act", "lcd_lut_linear_workspace_bytes", "lcd_lut_linear",
            "lcd_linear_host_scratch_bytes", "lcd_linear_host", "lcd_smooth_quantize_act_batch",
-           "lcd_lut_linear_batch_workspace_bytes", "lcd_lut_linear_batch", "lcd_lut_linear_static",
+           "lcd_lut_linear_batch_workspace_bytes", "lcd_lut_linear_batch", "lcd_lut_linear_batch_resolve", "lcd_lut_linear_static",
            "lcd_linear_host_batch_sizes", "lcd_linear_host_batch", "lcd_lut_linear_act8",
            "lcd_lut_linear_batch_act8", "lcd_linear_fused_batch_workspace_bytes", "lcd_linear_fused_batch",
            "lcd_smoothing_search_workspace_bytes", "lcd_smoothing_search", "lcd_reclassify",
@@ -105,6 +105,7 @@ def _load() -> ctypes.CDLL:
     lib.lcd_smooth_quantize_act_batch.argtypes = [POINTER(ActProblem), c_int, c_int, c_void_p]
     lib.lcd_lut_linear_batch_workspace_bytes.argtypes = [POINTER(LinearProblem), c_int, c_int, POINTER(c_size_t)]
     lib.lcd_lut_linear_batch.argtypes = [POINTER(LinearProblem), c_int, c_int, c_void_p, c_size_t, c_void_p, c_void_p]
+    lib.lcd_lut_linear_batch_resolve.argtypes = [POINTER(LinearProblem), c_int, c_int, POINTER(c_int)]
     lib.lcd_lut_linear_static.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_int64, c_int,
                                           c_void_p, c_void_p]
     lib.lcd_linear_host_batch_sizes.argtypes = [POINTER(HostProblem), c_int, POINTER(c_size_t), POINTER(c_size_t),
@@ -346,6 +347,17 @@ def smoothing_search(x, wmax, alphas, stream=None):
                                     c_void_p(best.data_ptr()), c_void_p(inv.data_ptr()), _stream_ptr(stream)),
            "lcd_smoothing_search")
     return best, mse, inv
+
+
+def resolve_batch_algo(weights_and_tokens, algo: int = ALGO_AUTO) -> int:
+    """The kernel family a grouped (or fused) call over these (PackedWeights, M) pairs runs for `algo`."""
+    items = list(weights_and_tokens)
+    arr = (LinearProblem * len(items))()
+    for a, (w, M) in zip(arr, items):
+        a.header_host, a.M = w.header_ptr, M
+    out = c_int(0)
+    _check(lib.lcd_lut_linear_batch_resolve(arr, len(items), algo, byref(out)), "lcd_lut_linear_batch_resolve")
+    return out.value
 
 
 class FusedBatch:

@@ -207,6 +207,20 @@ extern "C" lcd_status lcd_lut_linear_batch_workspace_bytes(const lcd_linear_prob
   return LCD_OK;
 }
 
+extern "C" lcd_status lcd_lut_linear_batch_resolve(const lcd_linear_problem* problems, int count, lcd_algo algo,
+                                                   lcd_algo* resolved) {
+  lcd_status st = batch_algo(problems, count, algo);
+  if (st != LCD_OK) return st;
+  if (!resolved) return LCD_ERR_INVALID_ARG;
+  Problem p[LCD_MAX_BATCH];
+  for (int i = 0; i < count; ++i) {
+    if (!problems[i].header_host) return LCD_ERR_INVALID_ARG;
+    if (!shape_problem(problems[i].header_host, problems[i].M, &p[i])) return LCD_ERR_BAD_BLOB;
+    if (p[i].bits != p[0].bits) return LCD_ERR_UNSUPPORTED;
+  }
+  return batch_family(p, count, algo, resolved);
+}
+
 extern "C" lcd_status lcd_lut_linear_batch(const lcd_linear_problem* problems, int count, lcd_algo algo,
                                            void* workspace, size_t workspace_bytes, int32_t* status_word_dev,
                                            void* cuda_stream) {
