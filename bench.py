@@ -433,7 +433,7 @@ def measure_config(args, cfg_id, M, dev, world, local, primary):
                 L = mt["L"]
                 xh = torch.from_numpy(L.x).pin_memory()
                 yh = torch.empty((M, L.N), dtype=torch.float32).pin_memory()
-                sc = torch.empty(lcd.linear_host_scratch_bytes(mt["w"][0], M), dtype=torch.uint8, device=dev)
+                sc = torch.zeros(lcd.linear_host_scratch_bytes(mt["w"][0], M), dtype=torch.uint8, device=dev)
                 host.append((xh, yh, sc))
                 h2d += xh.numel() * 2
                 d2h += yh.numel() * 4

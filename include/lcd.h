@@ -12,7 +12,8 @@
  * Conventions for every function:
  *   - returns an lcd_status; never aborts, traps or throws;
  *   - "host" / "device" in a parameter comment says where the pointer must point;
- *   - the caller owns every buffer; the library keeps no state except lazily set kernel attributes;
+ *   - the caller owns every buffer; the library keeps no state except lazily set kernel attributes (per device) and
+ *     the built-in scratch array of lcd_lut_linear_static with its per-device address;
  *   - device entry points are stream-ordered on `cuda_stream` (a cudaStream_t passed as void*;
  *     NULL = legacy default stream), do not synchronise and do not allocate;
  *   - argument errors are reported before anything is launched; an asynchronous problem (a bounded
@@ -42,7 +43,8 @@ typedef enum {
 /* Which kernel family lcd_lut_linear uses.  Every family computes the same y. */
 typedef enum {
   LCD_ALGO_AUTO = 0,        /* M <= 16: SHARED_BUCKET where it applies and the layer is large enough to pay    */
-                            /* for its tables, else REGISTER_LUT; DENSE_TC above                                */
+                            /* for its tables, else REGISTER_LUT; DENSE_TC above (17..32 tokens on rows of at   */
+                            /* least 8192 columns: REGISTER_LUT in two launches, measured faster there)         */
   LCD_ALGO_REFERENCE = 1,   /* plain per-weight lookup cb[n][idx] and multiply-accumulate; any M, slow        */
   LCD_ALGO_BUCKET_LUT = 2,  /* Section 4.2 centroid-stationary buckets: per output and per centroid w the exact */
                             /* integer sum S_w of the activation levels whose weight index is w (one-hot byte   */
@@ -156,7 +158,7 @@ lcd_status lcd_smooth_quantize_act_batch(const lcd_act_problem* problems /* host
  *   header_host:        host, the blob's first 64 bytes;
  *   act_idx, act_scale: device, as written by lcd_smooth_quantize_act for the same K;
  *   y:                  device out, fp32 [M][ldy], ldy >= N;
- *   algo:               LCD_ALGO_AUTO picks REGISTER_LUT for M <= 16 and DENSE_TC above; a family asked for
+ *   algo:               LCD_ALGO_AUTO: see lcd_algo; a family asked for
  *                       outside its range => LCD_ERR_UNSUPPORTED;
  *   workspace:          device scratch of at least lcd_lut_linear_workspace_bytes(...) bytes, 256-byte
  *                       aligned (may be NULL when that size is 0).  REGISTER_LUT and BUCKET_LUT keep integer
@@ -168,7 +170,10 @@ lcd_status lcd_smooth_quantize_act_batch(const lcd_act_problem* problems /* host
  *                       expired (the output is then invalid and the workspace must be zero-filled again);
  *                       never written otherwise.
  * The M <= 16 kernels are launched with programmatic stream serialization: they begin streaming weights
- * while the previous kernel of the stream finishes and wait for it before reading act_idx / act_scale.
+ * while the previous kernel of the stream finishes and wait for it before reading act_idx / act_scale (x_fp16 in the
+ * fused call).  The blob and inv_smooth are read before that wait: they must be complete when the call is enqueued,
+ * not produced by work that may still be running on the stream (lcd_smoothing_search's output: synchronise, or put
+ * another kernel between).  K_pad >= 2^21 (where the exact int32 sums could overflow) gives LCD_ERR_UNSUPPORTED.
  * -------------------------------------------------------------------------------------------- */
 lcd_status lcd_lut_linear_workspace_bytes(const void* header_host, int64_t M, lcd_algo algo, size_t* bytes);
 
@@ -353,14 +358,17 @@ lcd_status lcd_lut_linear_static(const void* packed_weights_dev, const void* hea
  * valid after the stream is synchronised.  x_host / y_host should be pinned for the copies to be async.
  *   x_host_fp16: host, binary16 [M][K] dense;   y_host: host out, fp32 [M][N] dense;
  *   inv_smooth:  device fp32 [K] or NULL;
- *   scratch:     device, >= lcd_linear_host_scratch_bytes(...) bytes, 256-byte aligned, contents undefined
- *                (the call clears the part the lookup kernel needs zeroed).
+ *   scratch:     device, >= lcd_linear_host_scratch_bytes(...) bytes, 256-byte aligned.  The caller zero-fills it
+ *                once before its first use (the lookup kernels keep partial sums and counters in part of it and
+ *                leave that part zero-filled, see lcd_lut_linear); it must be zero-filled again after a reported
+ *                LCD_ERR_TIMEOUT.  Two calls that may overlap on the device need separate scratch buffers;
+ *   status_word_dev: device int32 or NULL, as for lcd_lut_linear.
  * -------------------------------------------------------------------------------------------- */
 lcd_status lcd_linear_host_scratch_bytes(const void* header_host, int64_t M, size_t* bytes);
 
 lcd_status lcd_linear_host(const void* packed_weights_dev, const void* header_host, const void* x_host_fp16,
                            int64_t M, const float* inv_smooth, float* y_host, void* scratch,
-                           size_t scratch_bytes, void* cuda_stream);
+                           size_t scratch_bytes, int32_t* status_word_dev, void* cuda_stream);
 
 /* The same for up to LCD_MAX_BATCH independent problems with M <= 16 and equal index width (the projections of
  * a decoder layer): ONE host-to-device copy of all inputs, one grouped quantise launch, one grouped lookup
@@ -369,7 +377,8 @@ lcd_status lcd_linear_host(const void* packed_weights_dev, const void* header_ho
  * problem i's x (fp16 [M][K], dense) starts at the sum of the earlier problems' M*K*2 bytes rounded up to 16,
  * its y (fp32 [M][N], dense) at the sum of the earlier problems' M*N*4 bytes rounded up to 16;
  * lcd_linear_host_batch_sizes returns the total sizes (any of the three outputs may be NULL).  x_host_all and
- * y_host_all should be pinned; y_host_all is valid once cuda_stream is synchronised. */
+ * y_host_all should be pinned; y_host_all is valid once cuda_stream is synchronised.  scratch and status_word_dev as
+ * for lcd_linear_host (zero-filled once by the caller, left usable by every call). */
 typedef struct {
   const void* packed_weights_dev; /* device, 256-byte aligned */
   const void* header_host;        /* host */
@@ -381,7 +390,8 @@ lcd_status lcd_linear_host_batch_sizes(const lcd_host_problem* problems /* host 
                                        size_t* y_host_bytes, size_t* scratch_bytes);
 
 lcd_status lcd_linear_host_batch(const lcd_host_problem* problems /* host */, int count, const void* x_host_all,
-                                 void* y_host_all, void* scratch, size_t scratch_bytes, void* cuda_stream);
+                                 void* y_host_all, void* scratch, size_t scratch_bytes, int32_t* status_word_dev,
+                                 void* cuda_stream);
 
 #ifdef __cplusplus
 }

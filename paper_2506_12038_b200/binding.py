@@ -101,7 +101,7 @@ def _load() -> ctypes.CDLL:
     lib.lcd_lut_linear_batch_act8.argtypes = [POINTER(LinearProblem), c_int, c_int, c_void_p, c_size_t, c_void_p, c_void_p]
     lib.lcd_linear_host_scratch_bytes.argtypes = [c_void_p, c_int64, POINTER(c_size_t)]
     lib.lcd_linear_host.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_size_t,
-                                    c_void_p]
+                                    c_void_p, c_void_p]
     lib.lcd_smooth_quantize_act_batch.argtypes = [POINTER(ActProblem), c_int, c_int, c_void_p]
     lib.lcd_lut_linear_batch_workspace_bytes.argtypes = [POINTER(LinearProblem), c_int, c_int, POINTER(c_size_t)]
     lib.lcd_lut_linear_batch.argtypes = [POINTER(LinearProblem), c_int, c_int, c_void_p, c_size_t, c_void_p, c_void_p]
@@ -110,7 +110,8 @@ def _load() -> ctypes.CDLL:
                                           c_void_p, c_void_p]
     lib.lcd_linear_host_batch_sizes.argtypes = [POINTER(HostProblem), c_int, POINTER(c_size_t), POINTER(c_size_t),
                                                 POINTER(c_size_t)]
-    lib.lcd_linear_host_batch.argtypes = [POINTER(HostProblem), c_int, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.lcd_linear_host_batch.argtypes = [POINTER(HostProblem), c_int, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p,
+                                          c_void_p]
     for name in EXPORTS:
         if name not in ("lcd_status_string", "lcd_last_cuda_error"):
             getattr(lib, name).restype = c_int
@@ -425,9 +426,10 @@ class HostBatch:
     tensors x_host (uint8) / y_host (uint8) and the device scratch are owned here; x_view(i) / y_view(i) give
     problem i's fp16 [M, K] input and fp32 [M, N] output inside them."""
 
-    def __init__(self, items, device="cuda"):
+    def __init__(self, items, device="cuda", status_word=None):
         import torch
         self._keep = list(items)
+        self.status_word = status_word
         self.count = len(self._keep)
         self.arr = (HostProblem * self.count)()
         for a, (w, inv_s, M) in zip(self.arr, self._keep):
@@ -439,7 +441,7 @@ class HostBatch:
                "lcd_linear_host_batch_sizes")
         self.x_host = torch.zeros(xb.value, dtype=torch.uint8).pin_memory()
         self.y_host = torch.zeros(yb.value, dtype=torch.uint8).pin_memory()
-        self.scratch = torch.empty(sb.value, dtype=torch.uint8, device=device)
+        self.scratch = torch.zeros(sb.value, dtype=torch.uint8, device=device)     # zero-filled once, kept usable by the calls
         self._x_off, self._y_off, xo, yo = [], [], 0, 0
         for w, _, M in self._keep:
             self._x_off.append(xo)
@@ -460,7 +462,9 @@ class HostBatch:
     def run(self, stream=None):
         _check(lib.lcd_linear_host_batch(self.arr, self.count, c_void_p(self.x_host.data_ptr()),
                                          c_void_p(self.y_host.data_ptr()), c_void_p(self.scratch.data_ptr()),
-                                         self.scratch.numel(), _stream_ptr(stream)), "lcd_linear_host_batch")
+                                         self.scratch.numel(),
+                                         c_void_p(self.status_word.data_ptr()) if self.status_word is not None else None,
+                                         _stream_ptr(stream)), "lcd_linear_host_batch")
 
 
 def linear_host_scratch_bytes(w: PackedWeights, M: int) -> int:
@@ -469,12 +473,14 @@ def linear_host_scratch_bytes(w: PackedWeights, M: int) -> int:
     return out.value
 
 
-def linear_host(w: PackedWeights, x_host, inv_smooth, y_host, scratch, stream=None):
-    """x_host: pinned CPU fp16 [M,K]; y_host: pinned CPU fp32 [M,N]; enqueues copies + kernels, no sync."""
+def linear_host(w: PackedWeights, x_host, inv_smooth, y_host, scratch, stream=None, status_word=None):
+    """x_host: pinned CPU fp16 [M,K]; y_host: pinned CPU fp32 [M,N]; scratch: CUDA uint8, zero-filled before its first
+    use; enqueues copies + kernels, no sync."""
     M = x_host.shape[0]
     st = lib.lcd_linear_host(c_void_p(w.dev.data_ptr()), w.header_ptr, c_void_p(x_host.data_ptr()), M,
                              c_void_p(inv_smooth.data_ptr()) if inv_smooth is not None else None,
                              c_void_p(y_host.data_ptr()), c_void_p(scratch.data_ptr()),
-                             scratch.numel() * scratch.element_size(), _stream_ptr(stream))
+                             scratch.numel() * scratch.element_size(),
+                             c_void_p(status_word.data_ptr()) if status_word is not None else None, _stream_ptr(stream))
     _check(st, "lcd_linear_host")
     return y_host

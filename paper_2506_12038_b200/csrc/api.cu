@@ -21,6 +21,15 @@ static lcd_algo resolve_algo(const Problem& p, lcd_algo algo) {
   return kHaveDenseTc ? LCD_ALGO_DENSE_TC : LCD_ALGO_REFERENCE;
 }
 
+// LCD_ALGO_AUTO between 17 and 32 tokens on long rows: two launches of the register-table kernel (16 tokens, then
+// the rest) beat the tensor-core kernel, whose 128-token tile is mostly empty there and whose time grows with the
+// row length (measured on 4096 x 11008: 31.5 vs 41.0 us at M = 17, 46 vs 41 at M = 32 with 2-bit indices, 28.5 vs
+// 49 and 39 vs 49 with 3-bit ones; on rows of 4096 columns the two are within 5 % at M = 17 and the tensor-core
+// kernel wins from M = 24 on; from M = 64 it wins everywhere by 2 to 8 times).
+static bool two_chunks(const Problem& p, lcd_algo algo) {
+  return algo == LCD_ALGO_AUTO && p.act_bits == 4 && p.M > 16 && p.M <= 32 && p.K_pad >= 8192;
+}
+
 static bool small_m_family(lcd_algo a) {
   return a == LCD_ALGO_REGISTER_LUT || a == LCD_ALGO_BUCKET_LUT || a == LCD_ALGO_TC_LUT || a == LCD_ALGO_SHARED_BUCKET;
 }
@@ -32,6 +41,9 @@ static lcd_status make_problem(const void* packed_weights_dev, const void* heade
   Header h;
   if (!parse_header(header_host, &h)) return LCD_ERR_BAD_BLOB;
   if (ldy < (int64_t)h.N || M > (1LL << 21)) return LCD_ERR_INVALID_ARG;
+  // exact int32 sums of table byte x level: |sum| <= 128 * 8 * K_pad with 4-bit levels (128 * 128 with 8-bit ones,
+  // checked where those are accepted)
+  if (h.K_pad >= (1ull << 21)) return LCD_ERR_UNSUPPORTED;
   if (!aligned(packed_weights_dev, 256) || !aligned(act_idx, 16) || !aligned(act_scale, 4) || !aligned(y, 4))
     return LCD_ERR_INVALID_ARG;
   const uint8_t* blob = static_cast<const uint8_t*>(packed_weights_dev);
@@ -67,6 +79,12 @@ static bool shape_problem(const void* header_host, int64_t M, Problem* p) {
 }
 
 static lcd_status workspace_for(const Problem& p, lcd_algo algo, size_t* bytes) {
+  if (two_chunks(p, algo)) {
+    Problem first = p;
+    first.M = 16;
+    *bytes = lut_gemv_workspace_bytes(&first, 1, LCD_ALGO_REGISTER_LUT);
+    return LCD_OK;
+  }
   const lcd_algo resolved = resolve_algo(p, algo);
   switch (resolved) {
     case LCD_ALGO_REFERENCE:
@@ -158,6 +176,18 @@ extern "C" lcd_status lcd_lut_linear(const void* packed_weights_dev, const void*
   if (st != LCD_OK) return st;
   if (need > 0 && (!workspace || workspace_bytes < need)) return LCD_ERR_BUFFER_TOO_SMALL;
   if (need > 0 && !aligned(workspace, 256)) return LCD_ERR_INVALID_ARG;
+  if (two_chunks(p, algo)) {
+    // the second launch touches the scratch only after the first one has finished (stream order, dependency wait)
+    Problem part = p;
+    part.M = 16;
+    st = launch_lut_gemv(&part, 1, LCD_ALGO_REGISTER_LUT, workspace, workspace_bytes, status_word_dev, cuda_stream);
+    if (st != LCD_OK) return st;
+    part.M = p.M - 16;
+    part.act_idx = p.act_idx + 16 * (p.K_pad / 2);
+    part.act_scale = p.act_scale + 16;
+    part.y = p.y + 16 * p.ldy;
+    return launch_lut_gemv(&part, 1, LCD_ALGO_REGISTER_LUT, workspace, workspace_bytes, status_word_dev, cuda_stream);
+  }
   const lcd_algo resolved = resolve_algo(p, algo);
   switch (resolved) {
     case LCD_ALGO_REFERENCE:
@@ -439,7 +469,8 @@ extern "C" lcd_status lcd_linear_host_scratch_bytes(const void* header_host, int
 
 extern "C" lcd_status lcd_linear_host(const void* packed_weights_dev, const void* header_host,
                                       const void* x_host_fp16, int64_t M, const float* inv_smooth, float* y_host,
-                                      void* scratch, size_t scratch_bytes, void* cuda_stream) {
+                                      void* scratch, size_t scratch_bytes, int32_t* status_word_dev,
+                                      void* cuda_stream) {
   if (!packed_weights_dev || !header_host || !x_host_fp16 || !y_host || !scratch || M < 1)
     return LCD_ERR_INVALID_ARG;
   Header h;
@@ -459,12 +490,9 @@ extern "C" lcd_status lcd_linear_host(const void* packed_weights_dev, const void
   st = lcd_smooth_quantize_act(base + s.x_off, M, (int64_t)h.K, (int64_t)h.K, inv_smooth, nullptr, LCD_ACT_BITS,
                                idx, scale, cuda_stream);
   if (st != LCD_OK) return st;
-  if (s.ws_bytes) {   // the lookup kernels want their scratch zero-filled
-    e = cudaMemsetAsync(base + s.ws_off, 0, s.ws_bytes, stream);
-    if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
-  }
+  // the workspace part was zero-filled by the caller before the first call and is left zero-filled by every call
   st = lcd_lut_linear(packed_weights_dev, header_host, idx, scale, M, y, (int64_t)h.N, LCD_ALGO_AUTO,
-                      s.ws_bytes ? base + s.ws_off : nullptr, s.ws_bytes, nullptr, cuda_stream);
+                      s.ws_bytes ? base + s.ws_off : nullptr, s.ws_bytes, status_word_dev, cuda_stream);
   if (st != LCD_OK) return st;
   e = cudaMemcpyAsync(y_host, y, (size_t)M * h.N * 4, cudaMemcpyDeviceToHost, stream);
   if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
@@ -525,7 +553,8 @@ extern "C" lcd_status lcd_linear_host_batch_sizes(const lcd_host_problem* proble
 }
 
 extern "C" lcd_status lcd_linear_host_batch(const lcd_host_problem* problems, int count, const void* x_host_all,
-                                            void* y_host_all, void* scratch, size_t scratch_bytes, void* cuda_stream) {
+                                            void* y_host_all, void* scratch, size_t scratch_bytes,
+                                            int32_t* status_word_dev, void* cuda_stream) {
   if (!x_host_all || !y_host_all || !scratch) return LCD_ERR_INVALID_ARG;
   Problem shapes[LCD_MAX_BATCH];
   HostBatchLayout L;
@@ -568,9 +597,9 @@ extern "C" lcd_status lcd_linear_host_batch(const lcd_host_problem* problems, in
     st = lcd_smooth_quantize_act_batch(acts, count, LCD_ACT_BITS, cuda_stream);
     if (st != LCD_OK) return st;
   }
-  e = cudaMemsetAsync(base + L.ws_off, 0, L.ws_bytes, stream);    // the lookup kernel wants its scratch zero-filled
-  if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }
-  st = launch_lut_gemv(p, count, resolve_small_m(shapes, count, LCD_ALGO_AUTO), base + L.ws_off, L.ws_bytes, nullptr, cuda_stream);
+  // the workspace part was zero-filled by the caller before the first call and is left zero-filled by every call
+  st = launch_lut_gemv(p, count, resolve_small_m(shapes, count, LCD_ALGO_AUTO), base + L.ws_off, L.ws_bytes, status_word_dev,
+                       cuda_stream);
   if (st != LCD_OK) return st;
   e = cudaMemcpyAsync(y_host_all, base + L.y_off[0], L.y_bytes, cudaMemcpyDeviceToHost, stream);   // one copy out
   if (e != cudaSuccess) { set_cuda_error((int)e); return LCD_ERR_CUDA; }

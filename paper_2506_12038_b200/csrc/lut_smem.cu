@@ -543,8 +543,9 @@ lut_smem_kernel(const __grid_constant__ SbBatch batch, int32_t* __restrict__ sta
 
 int sm_count_now() { return current_sm_count(); }
 
-constexpr int kSliceBlocks = 2;    // W: table blocks per slice (2 x 64 KB beside a 96 KB ring)
-constexpr int kDepth = 3;
+constexpr int kSliceBlocks = 2;    // W: table blocks per slice (2 x 64 KB)
+constexpr int kDepth = 2;          // ring slots per warp: 64 KB in flight per SM (three measured no faster, the first
+                                   // loads of a launch wait behind the ring's first fill)
 constexpr int kWarps = 16;
 using LaunchShape = Shape<kSliceBlocks, kDepth, kWarps>;
 

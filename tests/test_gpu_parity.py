@@ -249,6 +249,26 @@ def test_dense_tensor_core_path_matches_oracle(bits, N, K, M, algo):
         assert torch.equal(lcd.lut_linear(w, a, s), y)
 
 
+@pytest.mark.parametrize("bits,N,K,M", [(2, 200, 11008, 17), (3, 72, 8192, 32), (2, 48, 28672, 25), (3, 40, 4096, 20)])
+def test_between_17_and_32_tokens_library_choice_matches_oracle(bits, N, K, M):
+    # LCD_ALGO_AUTO: on rows of at least 8192 columns two launches of the register-table kernel (16 tokens + the rest)
+    # through one scratch, else the tensor-core kernel; the scratch is left zero either way
+    L = gen.random_case(seed=N + K + M + bits, N=N, K=K, bits=bits, M=M)
+    w = lcd.PackedWeights(lcd.pack_weights(L.idx, L.codebook, bits))
+    a, s = lcd.smooth_quantize_act(torch.from_numpy(L.x).cuda(), torch.from_numpy(L.inv_s).cuda())
+    word = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    ws = torch.zeros((max(lcd.lut_linear_workspace_bytes(w, M), 256),), dtype=torch.uint8, device="cuda")
+    y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    for _ in range(2):
+        lcd.lut_linear(w, a, s, y=y, workspace=ws, status_word=word)
+    torch.cuda.synchronize()
+    assert int(word.item()) == 0
+    if K >= 8192:
+        assert not ws.any()
+    q_ref, s_ref = O.smooth_quantize(L.x, L.inv_s)
+    check_y(y, O.lut_linear_dequant(L.idx, L.codebook, q_ref, s_ref))
+
+
 def test_status_word_untouched_on_success():
     L = gen.random_case(seed=3, N=100, K=600, bits=2, M=2)
     w = lcd.PackedWeights(lcd.pack_weights(L.idx, L.codebook, 2))
@@ -299,7 +319,7 @@ def test_host_buffer_entry_point():
     w = lcd.PackedWeights(lcd.pack_weights(L.idx, L.codebook, 2))
     x_host = torch.from_numpy(L.x).pin_memory()
     y_host = torch.empty((3, 200), dtype=torch.float32).pin_memory()
-    scratch = torch.empty(lcd.linear_host_scratch_bytes(w, 3), dtype=torch.uint8, device="cuda")
+    scratch = torch.zeros(lcd.linear_host_scratch_bytes(w, 3), dtype=torch.uint8, device="cuda")
     lcd.linear_host(w, x_host, torch.from_numpy(L.inv_s).cuda(), y_host, scratch)
     torch.cuda.synchronize()
     q_ref, s_ref = O.smooth_quantize(L.x, L.inv_s)

@@ -101,7 +101,7 @@ def test_device_entry_points_reject_bad_arguments_before_any_launch():
     assert lib.lcd_lut_linear(fake, hdr, fake, fake, 1, fake, 4, 0, None, 0, None, None) == 1     # ldy < N
     assert lib.lcd_lut_linear(ctypes.c_void_p(4100), hdr, fake, fake, 1, fake, 8, 1, None, 0, None, None) == 1
     assert lib.lcd_lut_linear(fake, hdr, fake, fake, 17, fake, 8, 3, None, 0, None, None) == 2    # M > 16
-    assert lib.lcd_linear_host(fake, hdr, fake, 1, None, fake, fake, 16, None) == 3               # scratch small
+    assert lib.lcd_linear_host(fake, hdr, fake, 1, None, fake, fake, 16, None, None) == 3         # scratch small
 
 
 def test_every_export_declares_its_argument_types():
