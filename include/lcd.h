@@ -2,7 +2,7 @@
  * lcd.h - C ABI of the B200 (sm_100a) LUT-based inference matmul of the LCD paper
  *         ("Inference with Table Lookup", Section 4).
  *
- * A linear layer y = x W^T (W is N x K) whose clustered weights are stored as packed 2- or 3-bit
+ * A linear layer y = x W^T (W is N x K) whose clustered weights are stored as packed 2-, 3- or 4-bit
  * centroid indices idx[n][k] plus a per-output-row fp16 codebook cb[n][w].  Activations are
  * smoothed per input channel, mapped to 4-bit indices a = q + 8 (q in [-8,7]) with one fp32 scale
  * per token, and every output is formed by table lookup and accumulation:
@@ -86,7 +86,7 @@ const char* lcd_last_cuda_error(void);
  *     u64 codebook_offset.
  *   index area: rows padded to N_pad = 16*ceil(N/16), columns to K_pad = 256*ceil(K/256) with index 0,
  *     cut into items of 16 rows x 256 columns stored row-group major: item (rp, kt) starts at
- *     index_offset + (rp*(K_pad/256) + kt)*2T and is two tiles of T = 512 (2 bit) or 768 (3 bit) bytes, rows
+ *     index_offset + (rp*(K_pad/256) + kt)*2T and is two tiles of T = 512 (2 bit), 768 (3 bit) or 1024 (4 bit) bytes, rows
  *     16rp..16rp+7 then rows 16rp+8..16rp+15.  Inside a tile, lane l = 4*g + t (g = row 0..7, t = quarter
  *     0..3) owns columns 128*h + 32*t .. +31 of row g for both 128-column k-blocks h = 0,1 of the tile:
  *       2 bit: 16 bytes at tile + 16*l; bytes [8h, 8h+8) belong to k-block h; byte p of those holds the
@@ -94,10 +94,12 @@ const char* lcd_last_cuda_error(void);
  *       3 bit: three 256-byte planes; plane b has, at plane + 8*l + 4*h, word b of the lane's 12-byte
  *              record of k-block h.  A record packs columns 128h + 32t + m: m = 8i+j (i < 3) at bits
  *              [4j, 4j+3) of word i; m = 24+j has bit b of its index at bit 4j+3 of word b.
+ *       4 bit: two 512-byte planes, one per k-block h; plane h has the lane's 16 bytes at plane + 16*l, byte p of
+ *              which holds the two columns 128h + 32t + 2p + i (i = 0, 1, at bits [4i, 4i+4)).
  *   codebook area: N_pad rows of 2^bits fp16 values; entries >= C and padding rows are zero.
  * -------------------------------------------------------------------------------------------- */
 
-/* Size in bytes of the blob for an N x K layer.  bits in {2,3}.  *bytes is written on LCD_OK. */
+/* Size in bytes of the blob for an N x K layer.  bits in {2,3,4}.  *bytes is written on LCD_OK. */
 lcd_status lcd_packed_weights_bytes(int64_t N, int64_t K, int bits, size_t* bytes);
 
 /* idx: host, uint8 [N][K] row-major (ld = K), every value < C else LCD_ERR_INDEX_RANGE

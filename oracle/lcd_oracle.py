@@ -293,7 +293,7 @@ def pack_weights(idx: np.ndarray, codebook_fp16: np.ndarray, bits: int, C: int |
     u64 index_offset (=256), u64 codebook_offset.  Bytes 64..255 are zero.
 
     Index area: rows padded to N_pad = 16*ceil(N/16), columns to K_pad = 256*ceil(K/256), padding
-    index 0.  Tiles of 8 rows x 256 columns of T = 512 bytes (2 bit) or 768 bytes (3 bit); the two
+    index 0.  Tiles of 8 rows x 256 columns of T = 512 (2 bit), 768 (3 bit) or 1024 bytes (4 bit); the two
     tiles of a 16-row group rp (rows 16rp..16rp+7, then 16rp+8..16rp+15) are adjacent and form one
     item: tile (rg, kt), rg = 2*rp + u, is at index_offset + (rp*(K_pad/256) + kt)*2T + u*T.
     Lane l = 4*g + t (g = 0..7 row inside the tile, t = 0..3 quarter) owns, for each of the tile's
@@ -304,12 +304,14 @@ def pack_weights(idx: np.ndarray, codebook_fp16: np.ndarray, bits: int, C: int |
              record for k-block 0 then word b of its record for k-block 1.  A record packs the 32
              columns 128h + 32t + m: m = 8i+j (i<3) in bits [4j,4j+3) of word i; m = 24+j has its bit b
              at bit 4j+3 of word b.
+      4 bit: the tile is two 512-byte planes, one per k-block h; plane h holds, at plane + 16*l, the lane's
+             16 bytes, byte p of which packs the columns 128h + 32t + 2p (low nibble) and 128h + 32t + 2p + 1.
     Codebook area: N_pad rows of 2^bits fp16 values (entries >= C and padded rows are zero).
     """
     idx = np.asarray(idx, dtype=np.uint8)
     N, K = idx.shape
     C = (1 << bits) if C is None else C
-    if bits not in (2, 3) or not (1 <= C <= (1 << bits)):
+    if bits not in (2, 3, 4) or not (1 <= C <= (1 << bits)):
         raise ValueError("bits/C")
     if idx.size and int(idx.max()) >= C:
         raise ValueError("index out of range")
@@ -331,6 +333,11 @@ def pack_weights(idx: np.ndarray, codebook_fp16: np.ndarray, bits: int, C: int |
                     lane = 4 * g + t
                     if bits == 2:
                         blob[base + 16 * lane: base + 16 * lane + 16] = _tile_lane_bytes_2bit(sub, g, t)
+                    elif bits == 4:
+                        for h in range(2):
+                            for p in range(16):
+                                k = KBLOCK * h + 32 * t + 2 * p
+                                blob[base + 512 * h + 16 * lane + p] = int(sub[g, k]) | (int(sub[g, k + 1]) << 4)
                     else:
                         for h in range(2):
                             rec = _record_3bit(sub[g, KBLOCK * h + 32 * t: KBLOCK * h + 32 * t + 32])
@@ -382,6 +389,11 @@ def unpack_weights(blob: np.ndarray):
                                 b = int(blob[base + 16 * lane + 8 * hb + p])
                                 for i in range(4):
                                     P[rg * 8 + g, k0 + 4 * G + i] = (b >> (2 * i)) & 3
+                        elif bits == 4:
+                            for p in range(16):
+                                b = int(blob[base + 512 * hb + 16 * lane + p])
+                                P[rg * 8 + g, k0 + 32 * t + 2 * p] = b & 15
+                                P[rg * 8 + g, k0 + 32 * t + 2 * p + 1] = b >> 4
                         else:
                             words = []
                             for b in range(3):

@@ -21,5 +21,11 @@ __device__ __forceinline__ uint32_t tile_index_3bit(const uint8_t* tile, int g, 
   return ((base[0] >> sh) & 1u) | (((base[64] >> sh) & 1u) << 1) | (((base[128] >> sh) & 1u) << 2);
 }
 
+// Index of column kk (0..255) of row g (0..7) inside one 1024-byte 4-bit tile.
+__device__ __forceinline__ uint32_t tile_index_4bit(const uint8_t* tile, int g, int kk) {
+  const int h = kk >> 7, r = kk & 127, t = r >> 5, m = r & 31;
+  return (tile[512 * h + 16 * (4 * g + t) + (m >> 1)] >> (4 * (m & 1))) & 15u;
+}
+
 }  // namespace lcd
 #endif

@@ -17,7 +17,7 @@ static inline uint32_t payload_checksum(const uint8_t* p, size_t n) {
 bool parse_header(const void* header_host, Header* h) {
   std::memcpy(h, header_host, sizeof(Header));
   if (h->magic != kMagic || h->version != kVersion || h->layout != kLayoutPair16x256) return false;
-  if (h->bits != 2 && h->bits != 3) return false;
+  if (h->bits != 2 && h->bits != 3 && h->bits != 4) return false;
   if (h->C < 1 || h->C > (1u << h->bits)) return false;
   if (h->N < 1 || h->K < 1) return false;
   if (h->K_pad != round_up_u64(h->K, kTileK)) return false;
@@ -46,6 +46,13 @@ static inline void locate2(int g, int kk, int* byte, int* shift) {
   *shift = 2 * (r & 3);
 }
 
+// Position of column kk (0..255) of tile row g inside a 4-bit tile (two 512-byte planes, one per k-block).
+static inline void locate4(int g, int kk, int* byte, int* shift) {
+  const int h = kk >> 7, r = kk & 127, t = r >> 5, m = r & 31;
+  *byte = 512 * h + 16 * (4 * g + t) + (m >> 1);
+  *shift = 4 * (m & 1);
+}
+
 // 3-bit: the (up to three) places the bits of column kk of tile row g go to.
 static inline void locate3(int g, int kk, int byte[3], int shift[3], int* contiguous) {
   const int h = kk >> 7, r = kk & 127, t = r >> 5, m = r & 31, lane = 4 * g + t;
@@ -70,7 +77,7 @@ using namespace lcd;
 
 extern "C" lcd_status lcd_packed_weights_bytes(int64_t N, int64_t K, int bits, size_t* bytes) {
   if (!bytes || N < 1 || K < 1) return LCD_ERR_INVALID_ARG;
-  if (bits != 2 && bits != 3) return LCD_ERR_UNSUPPORTED;
+  if (bits != 2 && bits != 3 && bits != 4) return LCD_ERR_UNSUPPORTED;
   *bytes = blob_bytes((uint64_t)N, (uint64_t)K, bits);
   return LCD_OK;
 }
@@ -79,7 +86,7 @@ extern "C" lcd_status lcd_pack_weights(const uint8_t* idx, const uint16_t* codeb
                                        int bits, int C, void* out, size_t out_bytes, int64_t* bad_n,
                                        int64_t* bad_k) {
   if (!idx || !codebook_fp16 || !out || N < 1 || K < 1) return LCD_ERR_INVALID_ARG;
-  if (bits != 2 && bits != 3) return LCD_ERR_UNSUPPORTED;
+  if (bits != 2 && bits != 3 && bits != 4) return LCD_ERR_UNSUPPORTED;
   if (C < 1 || C > (1 << bits)) return LCD_ERR_INVALID_ARG;
   const size_t total = blob_bytes((uint64_t)N, (uint64_t)K, bits);
   if (out_bytes < total) return LCD_ERR_BUFFER_TOO_SMALL;
@@ -109,6 +116,10 @@ extern "C" lcd_status lcd_pack_weights(const uint8_t* idx, const uint16_t* codeb
           if (bits == 2) {
             int byte, shift;
             locate2(g, kk, &byte, &shift);
+            tile[byte] |= (uint8_t)(v << shift);
+          } else if (bits == 4) {
+            int byte, shift;
+            locate4(g, kk, &byte, &shift);
             tile[byte] |= (uint8_t)(v << shift);
           } else {
             int byte[3], shift[3], contiguous;
@@ -173,6 +184,10 @@ extern "C" lcd_status lcd_unpack_weights(const void* blob_v, size_t blob_bytes_i
           int byte, shift;
           locate2(g, kk, &byte, &shift);
           v = (tile[byte] >> shift) & 3u;
+        } else if (h.bits == 4) {
+          int byte, shift;
+          locate4(g, kk, &byte, &shift);
+          v = (tile[byte] >> shift) & 15u;
         } else {
           int byte[3], shift[3], contiguous;
           locate3(g, kk, byte, shift, &contiguous);

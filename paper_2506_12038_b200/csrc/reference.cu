@@ -1,6 +1,6 @@
 // Reference-grade lookup-and-accumulate kernel (Section 4.2 of the LCD paper, plain form): for every weight,
 // read its centroid index from the tiled blob, look the centroid up in the row codebook, multiply by the
-// token's activation level and accumulate in fp32.  Works for every M, N, K and both index widths; it is the
+// token's activation level and accumulate in fp32.  Works for every M, N, K and every index width; it is the
 // library's correctness anchor, not a fast path.
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -16,7 +16,7 @@ reference_kernel(const uint8_t* __restrict__ tiles, const uint16_t* __restrict__
                  int64_t K_pad, int bits, int act_bits, const uint8_t* __restrict__ act_idx,
                  const float* __restrict__ act_scale,
                  int64_t M, float* __restrict__ y, int64_t ldy) {
-  __shared__ float s_cb[8][8];
+  __shared__ float s_cb[8][16];
   const int g = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int64_t rg = blockIdx.x;
   const int64_t n = rg * 8 + g;
@@ -30,7 +30,8 @@ reference_kernel(const uint8_t* __restrict__ tiles, const uint16_t* __restrict__
   float acc = 0.0f;
   for (int64_t k = 0; k < K; ++k) {
     const uint8_t* tile = tiles + (((rg >> 1) * n_kt + k / kTileK) * 2 + (rg & 1)) * tile_bytes;
-    const uint32_t w = bits == 2 ? tile_index_2bit(tile, g, (int)(k % kTileK)) : tile_index_3bit(tile, g, (int)(k % kTileK));
+    const int kk = (int)(k % kTileK);
+    const uint32_t w = bits == 2 ? tile_index_2bit(tile, g, kk) : bits == 3 ? tile_index_3bit(tile, g, kk) : tile_index_4bit(tile, g, kk);
     int q;
     if (act_bits == 8) {
       q = (int)(int8_t)act_row[k];

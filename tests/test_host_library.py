@@ -30,7 +30,7 @@ def test_library_exports_every_declared_symbol():
 
 
 @pytest.mark.parametrize("bits,C,N,K", [(2, 4, 19, 700), (3, 8, 19, 700), (3, 5, 8, 256), (2, 3, 1, 1), (2, 4, 64, 1024),
-                                       (3, 8, 33, 513)])
+                                       (3, 8, 33, 513), (4, 16, 19, 700), (4, 10, 33, 513), (4, 9, 1, 1)])
 def test_packer_matches_oracle_bit_for_bit(bits, C, N, K):
     rng = np.random.default_rng(N * 1000 + K + bits)
     idx = rng.integers(0, C, size=(N, K), dtype=np.uint8)
@@ -46,7 +46,7 @@ def test_packer_matches_oracle_bit_for_bit(bits, C, N, K):
 
 
 def test_packer_edge_patterns():
-    for bits in (2, 3):
+    for bits in (2, 3, 4):
         C = 1 << bits
         cb = np.zeros((8, C), dtype=np.float16)
         for fill in (0, C - 1):
@@ -62,8 +62,8 @@ def test_packer_error_codes():
         lcd.pack_weights(idx, cb, 2, 3)
     assert e.value.status == 4 and "n=2 k=5" in str(e.value)
     with pytest.raises(lcd.LcdError) as e:
-        lcd.pack_weights(np.zeros((4, 8), dtype=np.uint8), np.zeros((4, 16), dtype=np.float16), 4, 16)
-    assert e.value.status == 2
+        lcd.pack_weights(np.zeros((4, 8), dtype=np.uint8), np.zeros((4, 32), dtype=np.float16), 5, 32)
+    assert e.value.status == 2        # five-bit indices: no kernel
     lib = binding.lib
     out = ctypes.c_size_t()
     assert lib.lcd_packed_weights_bytes(0, 8, 2, ctypes.byref(out)) == 1

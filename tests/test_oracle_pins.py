@@ -199,7 +199,7 @@ def test_act_pack_roundtrip_and_padding():
 
 
 # ---------------------------------------------------------------- packing
-@pytest.mark.parametrize("bits,C", [(2, 4), (3, 8), (3, 5), (2, 3)])
+@pytest.mark.parametrize("bits,C", [(2, 4), (3, 8), (3, 5), (2, 3), (4, 16), (4, 10)])
 def test_pack_roundtrip_random(bits, C):
     rng = np.random.default_rng(bits * 10 + C)
     N, K = 19, 300
@@ -213,7 +213,7 @@ def test_pack_roundtrip_random(bits, C):
     assert np.array_equal(i2, idx) and np.array_equal(c2.view(np.uint16), cb.view(np.uint16)) and (b2, C2) == (bits, C)
 
 
-@pytest.mark.parametrize("bits", [2, 3])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 def test_pack_one_hot_positions_hit_distinct_bits(bits):
     # each (row, column) of one tile maps to its own bit field: one-hot inputs give disjoint blobs whose
     # union is the all-ones blob, and every payload bit is covered exactly once (exactly `bits` bits/weight)
@@ -285,6 +285,29 @@ def test_pack_3bit_layout_spot_bytes():
     expect[512 + 0] = 0x08
     expect[8 * 14 + 4 + 3] = 0x80
     assert np.array_equal(body, expect)
+
+
+def test_pack_4bit_layout_spot_bytes():
+    # by hand from the layout text: a 4-bit tile is two 512-byte planes (k-block h = 0, 1); in plane h lane l = 4g+t
+    # has 16 bytes at 16*l, byte p = the columns 128h + 32t + 2p (low nibble) and 2p + 1 (high nibble); an item is
+    # the tile of rows 0-7 (1024 bytes) followed by the tile of rows 8-15
+    N, K = 16, 256
+    idx = np.zeros((N, K), dtype=np.uint8)
+    idx[0, 0] = 9            # g=0,t=0,h=0,m=0            -> plane 0, byte 0, low nibble
+    idx[0, 1] = 12           # m=1                        -> the same byte, high nibble
+    idx[2, 37] = 15          # g=2,h=0,t=1,m=5: p=2,i=1   -> byte 16*(8+1) + 2, high nibble
+    idx[7, 255] = 10         # g=7,h=1,t=3,m=31: p=15,i=1 -> byte 512 + 16*31 + 15, high nibble
+    idx[9, 130] = 3          # second tile, g=1,h=1,t=0,m=2: p=1,i=0 -> byte 1024 + 512 + 16*4 + 1, low nibble
+    blob = O.pack_weights(idx, np.zeros((N, 16), dtype=np.float16), 4)
+    body = blob[256:256 + 2048]
+    expect = np.zeros(2048, dtype=np.uint8)
+    expect[0] = 9 | (12 << 4)
+    expect[16 * 9 + 2] = 15 << 4
+    expect[512 + 16 * 31 + 15] = 10 << 4
+    expect[1024 + 512 + 16 * 4 + 1] = 3
+    assert np.array_equal(body, expect)
+    # the codebook area follows the index area: 16 rows of 16 fp16 values, 256-byte aligned
+    assert blob.size == 256 + 2048 + 512
 
 
 def test_pack_rejects_bad_indices_and_corruption():
