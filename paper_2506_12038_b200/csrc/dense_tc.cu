@@ -892,6 +892,7 @@ lcd_status launch_dense_tc(const Problem& p, bool fp16_operands, void* workspace
                            int32_t* status_word, void* stream) {
   if (!workspace || workspace_bytes < dense_tc_workspace_bytes(p.M, p.K_pad)) return LCD_ERR_BUFFER_TOO_SMALL;
   if (p.M > 0x7fffffffLL / 2 || p.N > 0x7fffffffLL / 2) return LCD_ERR_UNSUPPORTED;
+  if (p.bits != 2 && p.bits != 3) return LCD_ERR_UNSUPPORTED;      // 4-bit indices: not decoded by this kernel
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int64_t n_quarters = p.M * (p.K_pad / 32);
   const unsigned blocks = (unsigned)((n_quarters + 255) / 256);

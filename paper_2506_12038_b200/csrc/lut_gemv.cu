@@ -39,7 +39,8 @@ namespace {
 constexpr int kWarps = 16;
 constexpr int kThreads = kWarps * 32;
 // ring slots per warp: three, or two where 16 tokens need the shared memory for their activation levels
-__host__ __device__ constexpr int ring_depth(int mg) { return mg == 2 ? 2 : 3; }
+// (4-bit indices: items are 2 KB, three slots per warp would not leave room for the activation windows)
+__host__ __device__ constexpr int ring_depth(int mg, int bits) { return (mg == 2 || bits == 4) ? 2 : 3; }
 constexpr int kMaxDepth = 3;
 constexpr int kStageItems = 2;       // items per slot
 constexpr int kBarBytes = 512;       // mbarriers: kWarps * kMaxDepth * 8 = 384 bytes, padded
@@ -124,13 +125,14 @@ struct Planes {
 template <int BITS, int KIND>
 struct RowTables {
   uint32_t lo[KIND == kFixed16 ? 2 : 1], hi[KIND == kFixed16 ? 2 : 1];   // [plane]
+  uint32_t lo2[KIND == kFixed16 ? 2 : 1], hi2[KIND == kFixed16 ? 2 : 1]; // 4 bit: entries 8..11 and 12..15
   float scale;                                                          // kFixed16: 2^(e-15)
   float c[KIND == kBuckets ? (1 << BITS) : 1];                           // kBuckets: centroid values
 };
 
 template <int BITS>
 struct RawCodebook {
-  uint32_t w[BITS == 2 ? 2 : 4];
+  uint32_t w[BITS == 2 ? 2 : BITS == 3 ? 4 : 8];
 };
 
 template <int BITS>
@@ -142,6 +144,10 @@ __device__ __forceinline__ RawCodebook<BITS> load_codebook(const uint16_t* cb_ro
   } else {
     const uint4 v = __ldg(reinterpret_cast<const uint4*>(cb_row));
     r.w[0] = v.x; r.w[1] = v.y; r.w[2] = v.z; r.w[3] = v.w;
+    if (BITS == 4) {
+      const uint4 u = __ldg(reinterpret_cast<const uint4*>(cb_row) + 1);
+      r.w[BITS == 4 ? 4 : 0] = u.x; r.w[BITS == 4 ? 5 : 0] = u.y; r.w[BITS == 4 ? 6 : 0] = u.z; r.w[BITS == 4 ? 7 : 0] = u.w;
+    }
   }
   return r;
 }
@@ -160,7 +166,7 @@ __device__ __forceinline__ RowTables<BITS, KIND> build_tables(const RawCodebook<
 #pragma unroll
     for (int i = 0; i < C; ++i) T.c[i] = v[i];
     T.scale = 1.0f;
-    T.lo[0] = T.hi[0] = 0;
+    T.lo[0] = T.hi[0] = T.lo2[0] = T.hi2[0] = 0;
   } else {
     float mx = 0.0f;
 #pragma unroll
@@ -170,7 +176,7 @@ __device__ __forceinline__ RowTables<BITS, KIND> build_tables(const RawCodebook<
     ex = ex < -30 ? -30 : ex;
     const float up = __uint_as_float((uint32_t)(15 - ex + 127) << 23);   // 2^(15-ex): |v| * up < 32768
     T.scale = __uint_as_float((uint32_t)(ex - 15 + 127) << 23);          // 2^(ex-15)
-    uint32_t hb[2] = {0, 0}, lb[2] = {0, 0};
+    uint32_t hb[4] = {0, 0, 0, 0}, lb[4] = {0, 0, 0, 0};
 #pragma unroll
     for (int i = 0; i < C; ++i) {
       const int f = __float2int_rn(v[i] * up);
@@ -178,7 +184,8 @@ __device__ __forceinline__ RowTables<BITS, KIND> build_tables(const RawCodebook<
       lb[i >> 2] |= ((uint32_t)f & 0xffu) << (8 * (i & 3));
     }
     T.lo[0] = hb[0]; T.lo[1] = lb[0];
-    if (BITS == 3) { T.hi[0] = hb[1]; T.hi[1] = lb[1]; } else { T.hi[0] = hb[0]; T.hi[1] = lb[0]; }
+    if (BITS >= 3) { T.hi[0] = hb[1]; T.hi[1] = lb[1]; } else { T.hi[0] = hb[0]; T.hi[1] = lb[0]; }
+    T.lo2[0] = hb[2]; T.lo2[1] = lb[2]; T.hi2[0] = hb[3]; T.hi2[1] = lb[3];
   }
   return T;
 }
@@ -186,8 +193,11 @@ __device__ __forceinline__ RowTables<BITS, KIND> build_tables(const RawCodebook<
 // Four weights (selector nibbles of sel, low 16 bits) looked up in plane p of a row's tables.  p is a constant
 // after unrolling.  kBuckets: plane p < C - 1 is the one-hot table of centroid p + 1 (byte w is 1 iff
 // w == p + 1), the last plane is all ones.
+// 4 bit: sel holds the low three bits of four indices, pick the byte choice 0x3210 + 4 * (bit 3 of each index)
+// between the looked-up entries 0..7 and 8..15.
 template <int BITS, int KIND>
-__device__ __forceinline__ uint32_t pick_lookup(const RowTables<BITS, KIND>& T, uint32_t sel, int p) {
+__device__ __forceinline__ uint32_t pick_lookup(const RowTables<BITS, KIND>& T, uint32_t sel, int p, uint32_t pick = 0) {
+  if (KIND == kFixed16 && BITS == 4) return prmt(prmt(T.lo[p], T.hi[p], sel), prmt(T.lo2[p], T.hi2[p], sel), pick);
   if (KIND == kFixed16) return prmt(T.lo[p], T.hi[p], sel);
   if (p == (1 << BITS) - 1) return 0x01010101u;
   const int w = p + 1;
@@ -371,6 +381,16 @@ __device__ __forceinline__ void process_item(const uint8_t* item, const uint8_t*
     const uint4 wb = *reinterpret_cast<const uint4*>(item + HALF + 16 * lane);
     raw_a[0] = wa.x; raw_a[1] = wa.y; raw_a[2] = wa.z; raw_a[3] = wa.w;
     raw_b[0] = wb.x; raw_b[1] = wb.y; raw_b[2] = wb.z; raw_b[3] = wb.w;
+  } else if (BITS == 4) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {       // one 512-byte plane per k-block
+      const uint4 wa = *reinterpret_cast<const uint4*>(item + 512 * h + 16 * lane);
+      const uint4 wb = *reinterpret_cast<const uint4*>(item + HALF + 512 * h + 16 * lane);
+      raw_a[(BITS == 4 ? 4 : 0) * h] = wa.x; raw_a[(BITS == 4 ? 4 : 0) * h + 1] = wa.y;
+      raw_a[(BITS == 4 ? 4 : 0) * h + 2] = wa.z; raw_a[(BITS == 4 ? 4 : 0) * h + (BITS == 4 ? 3 : 0)] = wa.w;
+      raw_b[(BITS == 4 ? 4 : 0) * h] = wb.x; raw_b[(BITS == 4 ? 4 : 0) * h + 1] = wb.y;
+      raw_b[(BITS == 4 ? 4 : 0) * h + 2] = wb.z; raw_b[(BITS == 4 ? 4 : 0) * h + (BITS == 4 ? 3 : 0)] = wb.w;
+    }
   } else {
 #pragma unroll
     for (int b = 0; b < 3; ++b) {
@@ -391,7 +411,17 @@ __device__ __forceinline__ void process_item(const uint8_t* item, const uint8_t*
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
     uint32_t sel_a[8], sel_b[8];    // selector words of rows g and g + 8: lookup l uses the low 16 bits of sel[l]
-    if (BITS == 2) {
+    uint32_t pick_a[8] = {0, 0, 0, 0, 0, 0, 0, 0}, pick_b[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (BITS == 4) {
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {     // word w: eight indices in natural order
+        const uint32_t ua = raw_a[(BITS == 4 ? 4 : 0) * h + (BITS == 4 ? w : 0)], ub = raw_b[(BITS == 4 ? 4 : 0) * h + (BITS == 4 ? w : 0)];
+        const uint32_t a7 = ua & 0x77777777u, b7 = ub & 0x77777777u;
+        const uint32_t ap = ((ua >> 1) & 0x44444444u) | 0x32103210u, bp = ((ub >> 1) & 0x44444444u) | 0x32103210u;
+        sel_a[2 * w] = a7; sel_a[2 * w + 1] = a7 >> 16; pick_a[2 * w] = ap; pick_a[2 * w + 1] = ap >> 16;
+        sel_b[2 * w] = b7; sel_b[2 * w + 1] = b7 >> 16; pick_b[2 * w] = bp; pick_b[2 * w + 1] = bp >> 16;
+      }
+    } else if (BITS == 2) {
 #pragma unroll
       for (int w = 0; w < 2; ++w) {
         const uint32_t ua = raw_a[2 * h + w], ub = raw_b[2 * h + w];
@@ -421,10 +451,10 @@ __device__ __forceinline__ void process_item(const uint8_t* item, const uint8_t*
 #pragma unroll
       for (int p = 0; p < PL; ++p) {
         uint32_t a[4];
-        a[0] = pick_lookup<BITS, KIND>(Ta, sel_a[2 * j], p);
-        a[1] = pick_lookup<BITS, KIND>(Tb, sel_b[2 * j], p);
-        a[2] = pick_lookup<BITS, KIND>(Ta, sel_a[2 * j + 1], p);
-        a[3] = pick_lookup<BITS, KIND>(Tb, sel_b[2 * j + 1], p);
+        a[0] = pick_lookup<BITS, KIND>(Ta, sel_a[2 * j], p, pick_a[2 * j]);
+        a[1] = pick_lookup<BITS, KIND>(Tb, sel_b[2 * j], p, pick_b[2 * j]);
+        a[2] = pick_lookup<BITS, KIND>(Ta, sel_a[2 * j + 1], p, pick_a[2 * j + 1]);
+        a[3] = pick_lookup<BITS, KIND>(Tb, sel_b[2 * j + 1], p, pick_b[2 * j + 1]);
 #pragma unroll
         for (int G = 0; G < MG; ++G) {
           const uint4& qq = qv[h][j >> 1][G];
@@ -441,7 +471,7 @@ template <int BITS, int KIND, int MG>
 __global__ void __launch_bounds__(kThreads, 1)
 lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ status) {
   extern __shared__ __align__(128) uint8_t smem[];
-  constexpr int kDepth = ring_depth(MG);
+  constexpr int kDepth = ring_depth(MG, BITS);
   constexpr int ITEM = 512 * BITS;
   constexpr int SLOT = kStageItems * ITEM;
   constexpr int PL = Planes<BITS, KIND>::value;
@@ -1002,7 +1032,7 @@ lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void*
   if (workspace_bytes < lut_gemv_workspace_bytes(probs, count, algo) || !workspace) return LCD_ERR_BUFFER_TOO_SMALL;
 
   const int item_bytes = 512 * bits;
-  const size_t ring_bytes = (size_t)kWarps * ring_depth(MG) * kStageItems * item_bytes;
+  const size_t ring_bytes = (size_t)kWarps * ring_depth(MG, bits) * kStageItems * item_bytes;
   const size_t combine_bytes = kind == kFixed16 ? (size_t)kWarps * MG * planes * 128 * sizeof(int) : 0;
   const size_t act_budget = (size_t)kMaxSmem - kBarBytes - combine_bytes - ring_bytes;
 
@@ -1098,6 +1128,11 @@ lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void*
                                          : launch_t<2, kFixed16, 2>(batch, grid, smem, status_word, s);
     return MG == 1 ? launch_t<2, kBuckets, 1>(batch, grid, smem, status_word, s)
                    : launch_t<2, kBuckets, 2>(batch, grid, smem, status_word, s);
+  }
+  if (bits == 4) {      // 16-entry tables; the one-hot bucket tables would need sixteen planes
+    if (kind != kFixed16) return LCD_ERR_UNSUPPORTED;
+    return MG == 1 ? launch_t<4, kFixed16, 1>(batch, grid, smem, status_word, s)
+                   : launch_t<4, kFixed16, 2>(batch, grid, smem, status_word, s);
   }
   if (kind == kFixed16) return MG == 1 ? launch_t<3, kFixed16, 1>(batch, grid, smem, status_word, s)
                                        : launch_t<3, kFixed16, 2>(batch, grid, smem, status_word, s);

@@ -653,6 +653,7 @@ lcd_status launch_lut_gemv_tc(const Problem* probs, int count, void* workspace, 
   if (workspace_bytes < lut_gemv_tc_workspace_bytes(probs, count)) return LCD_ERR_BUFFER_TOO_SMALL;
   if (workspace == nullptr) return LCD_ERR_INVALID_ARG;
   const int bits = probs[0].bits;
+  if (bits != 2 && bits != 3) return LCD_ERR_UNSUPPORTED;
   TcBatch batch;
   batch.count = count;
   size_t off = 0;

@@ -86,7 +86,7 @@ def run_case(L, algo, tight=True):
 SHAPES = [(8, 256), (200, 1000), (1031, 520), (64, 4096), (24, 11008), (520, 2304)]
 
 
-@pytest.mark.parametrize("bits", [2, 3])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 @pytest.mark.parametrize("N,K", SHAPES)
 @pytest.mark.parametrize("M", [1, 2, 3, 5, 16])
 def test_register_lut_matches_oracle(bits, N, K, M):
@@ -269,6 +269,36 @@ def test_between_17_and_32_tokens_library_choice_matches_oracle(bits, N, K, M):
     check_y(y, O.lut_linear_dequant(L.idx, L.codebook, q_ref, s_ref))
 
 
+@pytest.mark.parametrize("N,K,M", [(200, 1000, 1), (4096, 4096, 1), (1031, 520, 8), (40, 11008, 16), (300, 28672, 4),
+                                   (64, 2304, 20), (520, 768, 70), (24, 700, 300)])
+def test_four_bit_indices_library_choice_and_fused_launch(N, K, M):
+    # 9 to 16 centroids per row (the paper's 3.3-bit point is 10): the register tables hold sixteen entries (two
+    # eight-entry lookups and a byte choice); above 16 tokens the library runs 16-token chunks (up to 32 tokens) or
+    # the plain kernel.  Ten centroids, library's choice of kernel, and the one-launch form for up to 16 tokens.
+    L = gen.random_case(seed=N + K + M + 4, N=N, K=K, bits=4, M=M, C=10)
+    w = lcd.PackedWeights(lcd.pack_weights(L.idx, L.codebook, 4, 10))
+    x, inv_s = torch.from_numpy(L.x).cuda(), torch.from_numpy(L.inv_s).cuda()
+    a, s = lcd.smooth_quantize_act(x, inv_s)
+    q_ref, s_ref = O.smooth_quantize(L.x, L.inv_s)
+    y_ref = O.lut_linear_dequant(L.idx, L.codebook, q_ref, s_ref)
+    word = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    ws = torch.zeros((max(lcd.lut_linear_workspace_bytes(w, M), 256),), dtype=torch.uint8, device="cuda")
+    y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    for _ in range(2):
+        lcd.lut_linear(w, a, s, y=y, workspace=ws, status_word=word)
+    torch.cuda.synchronize()
+    assert int(word.item()) == 0 and not ws.any()
+    check_y(y, y_ref, tight=M <= 32)
+    if M <= 16:
+        y2 = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        fb = lcd.FusedBatch([(w, x, inv_s, y2)], status_word=word)
+        fb.run()
+        torch.cuda.synchronize()
+        assert int(word.item()) == 0 and torch.equal(y2, y)
+    with pytest.raises(lcd.LcdError):                 # no one-hot bucket tables and no tensor-core decoders at this width
+        lcd.lut_linear(w, a, s, algo=lcd.ALGO_BUCKET_LUT if M <= 16 else lcd.ALGO_DENSE_TC)
+
+
 def test_status_word_untouched_on_success():
     L = gen.random_case(seed=3, N=100, K=600, bits=2, M=2)
     w = lcd.PackedWeights(lcd.pack_weights(L.idx, L.codebook, 2))
@@ -279,13 +309,13 @@ def test_status_word_untouched_on_success():
     assert int(word.item()) == 12345
 
 
-@pytest.mark.parametrize("bits", [2, 3])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 @pytest.mark.parametrize("N,K,M", [(8, 256, 1), (200, 1000, 3), (1031, 520, 17), (64, 4096, 40), (24, 700, 33)])
 def test_reference_kernel_matches_oracle(bits, N, K, M):
     run_case(gen.random_case(seed=N + K + M + bits, N=N, K=K, bits=bits, M=M), lcd.ALGO_REFERENCE)
 
 
-@pytest.mark.parametrize("bits,C", [(3, 5), (3, 6), (2, 3), (2, 1), (3, 1)])
+@pytest.mark.parametrize("bits,C", [(3, 5), (3, 6), (2, 3), (2, 1), (3, 1), (4, 10), (4, 9), (4, 16), (4, 1)])
 def test_fewer_centroids_than_index_width(bits, C):
     L = gen.random_case(seed=77 + C, N=40, K=777, bits=bits, M=2, C=C)
     run_case(L, lcd.ALGO_AUTO)
