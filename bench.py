@@ -77,7 +77,8 @@ def build_layers(cfg_id, M):
     cfg = gen.CONFIGS[cfg_id]
     layers = []
     for mi, (name, N, K) in enumerate(cfg["shapes"]):
-        L = gen.make_layer(cfg_id, mi, N, K, cfg["bits"], M, outlier_frac=cfg["frac"], outlier_scale=cfg["scale"])
+        L = gen.make_layer(cfg_id, mi, N, K, cfg["bits"], M, C=cfg.get("C"), outlier_frac=cfg["frac"],
+                           outlier_scale=cfg["scale"])
         layers.append((name, L))
     return cfg, layers
 
@@ -263,7 +264,7 @@ def measure_config(args, cfg_id, M, dev, world, local, primary):
 
     mats = []
     for name, L in layers:
-        blob = lcd.pack_weights(L.idx, L.codebook, bits)
+        blob = lcd.pack_weights(L.idx, L.codebook, bits, L.C)
         ws = [lcd.PackedWeights(blob, dev) for _ in range(copies)]
         x = torch.from_numpy(L.x).to(dev)
         inv_s = torch.from_numpy(L.inv_s).to(dev)

@@ -18,7 +18,6 @@ static bool aligned(const void* p, size_t a) { return reinterpret_cast<uintptr_t
 static lcd_algo resolve_algo(const Problem& p, lcd_algo algo) {
   if (algo != LCD_ALGO_AUTO) return algo;
   if (p.M <= 16) return resolve_small_m(&p, 1, algo);
-  if (p.bits == 4) return LCD_ALGO_REFERENCE;      // no tensor-core decoder for 4-bit indices: the plain kernel
   return kHaveDenseTc ? LCD_ALGO_DENSE_TC : LCD_ALGO_REFERENCE;
 }
 
@@ -28,8 +27,7 @@ static lcd_algo resolve_algo(const Problem& p, lcd_algo algo) {
 // 49 and 39 vs 49 with 3-bit ones; on rows of 4096 columns the two are within 5 % at M = 17 and the tensor-core
 // kernel wins from M = 24 on; from M = 64 it wins everywhere by 2 to 8 times).
 static bool two_chunks(const Problem& p, lcd_algo algo) {
-  // (4-bit indices have no tensor-core decoder: chunks of 16 tokens up to 64 tokens, the plain kernel above)
-  return algo == LCD_ALGO_AUTO && p.act_bits == 4 && p.M > 16 && p.M <= 32 && (p.K_pad >= 8192 || p.bits == 4);
+  return algo == LCD_ALGO_AUTO && p.act_bits == 4 && p.M > 16 && p.M <= 32 && p.K_pad >= 8192;
 }
 
 static bool small_m_family(lcd_algo a) {

@@ -131,7 +131,7 @@ __global__ void __launch_bounds__(256) expand_levels_kernel(const uint8_t* __res
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
       const int p = 2 * v + e;
-      const int col = BITS == 3 ? p : 16 * (p >> 4) + 8 * ((p >> 2) & 1) + 2 * (p & 3) + ((p >> 3) & 1);
+      const int col = BITS != 2 ? p : 16 * (p >> 4) + 8 * ((p >> 2) & 1) + 2 * (p & 3) + ((p >> 3) & 1);
       const uint32_t nib = (src[col >> 3] >> (4 * (col & 7))) & 15u;
       pair |= (0x6400u | nib) << (16 * e);        // fp16 bits of 1024 + a
     }
@@ -445,7 +445,7 @@ __global__ void __launch_bounds__(256) expand_levels_i8_kernel(const uint8_t* __
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const int p = 4 * v + e;
-      const int col = BITS == 3 ? p : 16 * (p >> 4) + 8 * ((p >> 2) & 1) + 2 * (p & 3) + ((p >> 3) & 1);
+      const int col = BITS != 2 ? p : 16 * (p >> 4) + 8 * ((p >> 2) & 1) + 2 * (p & 3) + ((p >> 3) & 1);
       const uint32_t nib = (src[col >> 3] >> (4 * (col & 7))) & 15u;
       word |= ((nib - 8u) & 0xffu) << (8 * e);       // q = a - 8 as a signed byte
     }
@@ -653,7 +653,7 @@ dense_i8_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
       int rp = (tile / P.n_tiles_m) * (kBM / 16) + dw;
       rp = rp < P.n_rp ? rp : P.n_rp - 1;          // rows past the matrix repeat the last group; never stored
       // byte tables of this thread's row: 16-bit fixed point, high (signed) and low (unsigned) bytes
-      uint32_t TH[2] = {0, 0}, TL[2] = {0, 0};
+      uint32_t TH[4] = {0, 0, 0, 0}, TL[4] = {0, 0, 0, 0};     // entries 4i .. 4i + 3 in word i (4 bit: all four words)
       {
         const uint16_t* cb = P.codebook + ((size_t)rp * 16 + 8 * u + g) * (1 << BITS);
         float up;
@@ -667,8 +667,9 @@ dense_i8_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
         if (BITS == 2) { TH[1] = TH[0]; TL[1] = TL[0]; }
       }
       const uint8_t* row_items = P.items + (size_t)rp * P.n_kt * ITEM + u * HALF;
-      uint32_t cur[2][BITS == 2 ? 2 : 3], nxt[2][BITS == 2 ? 2 : 3];      // [quarter][word]
-      auto load_stage = [&](uint32_t (&dst)[2][BITS == 2 ? 2 : 3], int kt) {
+      constexpr int NW = BITS == 2 ? 2 : BITS == 3 ? 3 : 4;      // index words of a quarter of one k-block
+      uint32_t cur[2][NW], nxt[2][NW];      // [quarter][word]
+      auto load_stage = [&](uint32_t (&dst)[2][NW], int kt) {
         const uint8_t* item = row_items + (size_t)kt * ITEM;
 #pragma unroll
         for (int xq = 0; xq < 2; ++xq) {
@@ -676,6 +677,9 @@ dense_i8_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
           if (BITS == 2) {
             const uint2 w = __ldg(reinterpret_cast<const uint2*>(item + 16 * l + 8 * grp));
             dst[xq][0] = w.x; dst[xq][1] = w.y;
+          } else if (BITS == 4) {           // one 512-byte plane per k-block, 16 bytes per lane
+            const uint4 w = __ldg(reinterpret_cast<const uint4*>(item + 512 * grp + 16 * l));
+            dst[xq][0] = w.x; dst[xq][1] = w.y; dst[xq][NW > 2 ? 2 : 0] = w.z; dst[xq][NW > 3 ? 3 : 0] = w.w;
           } else {
 #pragma unroll
             for (int b = 0; b < 3; ++b)
@@ -693,8 +697,15 @@ dense_i8_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
         uint32_t hw[2][2][4], lw[2][2][4];          // [quarter][chunk][word]
 #pragma unroll
         for (int xq = 0; xq < 2; ++xq) {
-          uint32_t sel[8];
-          if (BITS == 2) {
+          uint32_t sel[8], pick[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+          if (BITS == 4) {                  // natural order; pick = byte choice between entries 0..7 and 8..15
+#pragma unroll
+            for (int wd = 0; wd < 4; ++wd) {
+              const uint32_t raw = cur[xq][NW > 3 ? wd : 0];
+              const uint32_t s7 = raw & 0x77777777u, pk = ((raw >> 1) & 0x44444444u) | 0x32103210u;
+              sel[2 * wd] = s7; sel[2 * wd + 1] = s7 >> 16; pick[2 * wd] = pk; pick[2 * wd + 1] = pk >> 16;
+            }
+          } else if (BITS == 2) {
 #pragma unroll
             for (int wd = 0; wd < 2; ++wd) {
               const uint32_t raw = cur[xq][wd];
@@ -712,8 +723,13 @@ dense_i8_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
           for (int c = 0; c < 2; ++c)
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-              hw[xq][c][i] = prmt_b(TH[0], TH[1], sel[4 * c + i]);
-              lw[xq][c][i] = prmt_b(TL[0], TL[1], sel[4 * c + i]);
+              if (BITS == 4) {
+                hw[xq][c][i] = prmt_b(prmt_b(TH[0], TH[1], sel[4 * c + i]), prmt_b(TH[2], TH[3], sel[4 * c + i]), pick[4 * c + i]);
+                lw[xq][c][i] = prmt_b(prmt_b(TL[0], TL[1], sel[4 * c + i]), prmt_b(TL[2], TL[3], sel[4 * c + i]), pick[4 * c + i]);
+              } else {
+                hw[xq][c][i] = prmt_b(TH[0], TH[1], sel[4 * c + i]);
+                lw[xq][c][i] = prmt_b(TL[0], TL[1], sel[4 * c + i]);
+              }
             }
         }
         if (!bar_wait(empty(slot), ((it / kStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
@@ -732,7 +748,7 @@ dense_i8_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
 #pragma unroll
         for (int xq = 0; xq < 2; ++xq)
 #pragma unroll
-          for (int b = 0; b < (BITS == 2 ? 2 : 3); ++b) cur[xq][b] = nxt[xq][b];
+          for (int b = 0; b < NW; ++b) cur[xq][b] = nxt[xq][b];
       }
     }
   }
@@ -892,7 +908,7 @@ lcd_status launch_dense_tc(const Problem& p, bool fp16_operands, void* workspace
                            int32_t* status_word, void* stream) {
   if (!workspace || workspace_bytes < dense_tc_workspace_bytes(p.M, p.K_pad)) return LCD_ERR_BUFFER_TOO_SMALL;
   if (p.M > 0x7fffffffLL / 2 || p.N > 0x7fffffffLL / 2) return LCD_ERR_UNSUPPORTED;
-  if (p.bits != 2 && p.bits != 3) return LCD_ERR_UNSUPPORTED;      // 4-bit indices: not decoded by this kernel
+  if (p.bits == 4 && fp16_operands) return LCD_ERR_UNSUPPORTED;    // 4-bit indices: the int8 kernel only
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int64_t n_quarters = p.M * (p.K_pad / 32);
   const unsigned blocks = (unsigned)((n_quarters + 255) / 256);
@@ -911,6 +927,9 @@ lcd_status launch_dense_tc(const Problem& p, bool fp16_operands, void* workspace
     if (p.bits == 2) return bn == 128 ? launch_dense_i8<2, 128>(p, levels, status_word, s)
                           : bn == 192 ? launch_dense_i8<2, 192>(p, levels, status_word, s)
                                       : launch_dense_i8<2, 256>(p, levels, status_word, s);
+    if (p.bits == 4) return bn == 128 ? launch_dense_i8<4, 128>(p, levels, status_word, s)
+                          : bn == 192 ? launch_dense_i8<4, 192>(p, levels, status_word, s)
+                                      : launch_dense_i8<4, 256>(p, levels, status_word, s);
     return bn == 128 ? launch_dense_i8<3, 128>(p, levels, status_word, s)
          : bn == 192 ? launch_dense_i8<3, 192>(p, levels, status_word, s)
                      : launch_dense_i8<3, 256>(p, levels, status_word, s);

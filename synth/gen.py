@@ -167,4 +167,6 @@ CONFIGS = {
     2: dict(name="llama7b-3bit-M4-16", shapes=LLAMA7B, bits=3, Ms=[4, 16], frac=0.01, scale=50.0),
     3: dict(name="llama13b-2bit-M2048", shapes=LLAMA13B, bits=2, Ms=[2048], frac=0.01, scale=50.0),
     4: dict(name="llama70b-mlp-2bit-M1-8", shapes=LLAMA70B_MLP, bits=2, Ms=[1, 8], frac=0.005, scale=100.0),
+    # ten centroids per row in 4-bit indices: the paper's 3.3-bit operating point
+    5: dict(name="llama7b-4bit-10centroids-M1-16", shapes=LLAMA7B, bits=4, C=10, Ms=[1, 16], frac=0.01, scale=50.0),
 }
