@@ -34,7 +34,7 @@ from synth import gen  # noqa: E402
 # since reports traffic = null.  Keys: (kernel source, configuration, M).
 NCU_TRAFFIC = {
     # one launch (input transformation + lookup) of the LLaMA-7B-shaped 2-bit layer at M = 1
-    ("lut_smem.cu", 1, 1): {"sha256": "", "bytes_per_launch": 51875584 + 48640},
+    ("lut_smem.cu", 1, 1): {"sha256": "f14795184ea2befb46a489352d144b95f89ea0e2f26f8c36bad69d4a05436a55", "bytes_per_launch": 51871232 + 122368},
     # the seven launches of the LLaMA-13B-shaped layer at M = 2048: q captured (17.11 + 0.44 MB, taken four times for
     # q/k/v/o), gate captured (28.37 + 56.32 MB, twice for gate/up), down scaled from q by its 2.7 times longer rows
     # (same tiles, traffic in proportion to K)
