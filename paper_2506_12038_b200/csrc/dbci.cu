@@ -81,9 +81,21 @@ __global__ void __launch_bounds__(256) dbci_core_kernel(const float* __restrict_
   if (i >= m) { fwd[i] = -1; rev[i] = -1; return; }
   const float* y = x + L;
   const double v = (double)y[i], eps = P->eps;
-  const long long lo = lower_bound_d(y, 0, m, v - eps);
-  const long long hi = upper_bound_d(y, 0, m, v + eps);
-  const bool core = hi - lo >= P->min_pts;
+  const long long min_pts = P->min_pts;
+  bool core;
+  if (min_pts <= 64) {
+    // Only "at least MinPts neighbours" matters: count outwards over the sorted neighbours and stop at MinPts (the
+    // same two comparisons as the searches below; MinPts is the size of the smaller outlier cluster, usually a few).
+    const double a = v - eps, b = v + eps;
+    long long cnt = 1;
+    for (long long j = i - 1; j >= 0 && cnt < min_pts && !((double)y[j] < a); --j) ++cnt;
+    for (long long j = i + 1; j < m && cnt < min_pts && (double)y[j] <= b; ++j) ++cnt;
+    core = cnt >= min_pts;
+  } else {
+    const long long lo = lower_bound_d(y, 0, m, v - eps);
+    const long long hi = upper_bound_d(y, 0, m, v + eps);
+    core = hi - lo >= min_pts;
+  }
   fwd[i] = core ? (int)i : -1;
   rev[m - 1 - i] = core ? (int)(m - 1 - i) : -1;
 }
@@ -115,30 +127,41 @@ __global__ void __launch_bounds__(256) dbci_label_kernel(const float* __restrict
                                                          int* __restrict__ first, int* __restrict__ last, int max_clusters) {
   const long long L = P->L, R = P->R, m = R - L;
   const long long g = (long long)blockIdx.x * 256 + threadIdx.x;
-  if (g >= n) return;
   const int n_mid = m > 0 ? cid1[m - 1] : 0;
-  int lab;
-  if (g < L) lab = 0;
-  else if (g >= R) lab = n_mid + 1;
-  else {
-    const long long i = g - L;
-    const int pc = prev_core[i];
-    const int nr = next_rev[m - 1 - i];
-    const int nx = nr < 0 ? -1 : (int)(m - 1 - nr);
-    if (pc == (int)i) {
-      lab = cid1[i];
-    } else {
-      const double v = (double)x[g], eps = P->eps;
-      const double dl = pc >= 0 ? v - (double)x[L + pc] : 1e300;
-      const double dr = nx >= 0 ? (double)x[L + nx] - v : 1e300;
-      if (dl <= eps && dl <= dr) lab = cid1[pc];
-      else if (dr <= eps) lab = cid1[nx];
-      else lab = -1;
+  int lab = -2;                                  // -2: past the end of the array
+  if (g < n) {
+    if (g < L) lab = 0;
+    else if (g >= R) lab = n_mid + 1;
+    else {
+      const long long i = g - L;
+      const int pc = prev_core[i];
+      const int nr = next_rev[m - 1 - i];
+      const int nx = nr < 0 ? -1 : (int)(m - 1 - nr);
+      if (pc == (int)i) {
+        lab = cid1[i];
+      } else {
+        const double v = (double)x[g], eps = P->eps;
+        const double dl = pc >= 0 ? v - (double)x[L + pc] : 1e300;
+        const double dr = nx >= 0 ? (double)x[L + nx] - v : 1e300;
+        if (dl <= eps && dl <= dr) lab = cid1[pc];
+        else if (dr <= eps) lab = cid1[nx];
+        else lab = -1;
+      }
     }
+    if (labels) labels[g] = lab;
   }
-  if (labels) labels[g] = lab;
-  if (lab < 0) atomicAdd(&P->n_noise, 1);
-  else if (lab < max_clusters) {
+  // First and last member of every cluster, and the noise count.  Neighbours in the sorted array almost always share a
+  // label, and millions of atomics on a handful of addresses serialise: a warp whose lanes agree sends one pair.
+  const int lane = threadIdx.x & 31;
+  const unsigned noise = __ballot_sync(0xffffffffu, lab == -1);
+  if (lane == 0 && noise) atomicAdd(&P->n_noise, __popc(noise));
+  const int lab0 = __shfl_sync(0xffffffffu, lab, 0);
+  if (__all_sync(0xffffffffu, lab == lab0)) {
+    if (lab0 >= 0 && lab0 < max_clusters) {
+      if (lane == 0) atomicMin(first + lab0, (int)g);
+      if (lane == 31) atomicMax(last + lab0, (int)g);
+    }
+  } else if (lab >= 0 && lab < max_clusters) {
     atomicMin(first + lab, (int)g);
     atomicMax(last + lab, (int)g);
   }
