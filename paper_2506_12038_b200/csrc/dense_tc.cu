@@ -420,12 +420,19 @@ __device__ __forceinline__ void mma_i8(uint32_t tmem_d, uint64_t adesc, uint64_t
       "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}"
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-      : "r"(taddr) : "memory");
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&v)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+               : "r"(taddr) : "memory");
+}
+
+// Waits for the tensor-memory loads in flight.  The loaded registers are operands: nothing that reads them can be
+// scheduled before the wait.
+__device__ __forceinline__ void tmem_wait8(uint32_t (&a)[8], uint32_t (&b)[8]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]),
+                 "+r"(b[0]), "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(b[4]), "+r"(b[5]), "+r"(b[6]), "+r"(b[7])
+               :: "memory");
 }
 
 // Activation levels as int8 in the decoder's column order (see expand_levels_kernel): one thread per (token,
@@ -618,24 +625,64 @@ dense_i8_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
       // this thread's row: 2^(e-15) of its fixed-point tables (rows past the matrix are never stored)
       const int n_cb = n < P.n_rp * 16 ? n : P.n_rp * 16 - 1;
       const float row_scale = row_exponent_scale<BITS>(P.codebook + (size_t)n_cb * (1 << BITS), nullptr);
+      // The token scales of a pair of this warp's chunks live in one register: lane l holds the scale of token
+      // l & 15 of chunk 2r + (l >> 4).  The first pair is asked for before the wait for the accumulators, the next
+      // one while the current pair is drained.  (The chunk loop is not unrolled: measured no faster unrolled.)
+      constexpr int kMyChunks = BN / 16 / (kI8EpiWarps / 4);
+      static_assert(kMyChunks % 2 == 0, "an even number of 16-token chunks per epilogue warp");
+      auto pair_scales = [&](int r) {
+        const int m = m0 + 16 * (half + (kI8EpiWarps / 4) * (2 * r + (lane >> 4))) + (lane & 15);
+        return m < P.M ? __ldg(P.act_scale + m) : 0.0f;
+      };
+      float sc_cur = pair_scales(0), sc_next = 0.0f;
       ok = __all_sync(0xffffffffu, bar_wait(tmem_full(buf), (tl / NBUF) & 1u, abort_flag));
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll 1
-      for (int c = half; c < BN / 16; c += kI8EpiWarps / 4) {
-        uint32_t hi[16], lo[16];
-        const uint32_t t_hi = tmem_base + ((uint32_t)(32 * quad) << 16) + buf * (2 * BN) + 16 * c;
-        tmem_ld16(t_hi, hi);
-        tmem_ld16(t_hi + BN, lo);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        const int mc = m0 + 16 * c;
-        const float my_scale = (lane < 16 && mc + lane < P.M) ? __ldg(P.act_scale + mc + lane) : 0.0f;
+      float* y_row = P.y + (size_t)(m0 + 16 * half) * P.ldy + n;
+      const bool row_ok = n < P.N;
+      // Eight tokens at a time (sixteen accumulator registers leave room to overlap the tokens' dependent chains), two
+      // register sets: the loads of the next eight are in flight while these are converted and stored.
+      const uint32_t t_tile = tmem_base + ((uint32_t)(32 * quad) << 16) + buf * (2 * BN) + 16 * half;
+      uint32_t hiA[8], loA[8], hiB[8], loB[8];
+      tmem_ld8(t_tile, hiA);
+      tmem_ld8(t_tile + BN, loA);
+      auto drain8 = [&](const uint32_t (&hi)[8], const uint32_t (&lo)[8], float sc, int src0, int m_first, float* y8) {
+        float s[8], v[8];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float s = __shfl_sync(0xffffffffu, my_scale, j) * row_scale;
-          if (mc + j < P.M && n < P.N)
-            P.y[(size_t)(mc + j) * P.ldy + n] = ((float)(int)hi[j] * 256.0f + (float)(int)lo[j]) * s;
+        for (int j = 0; j < 8; ++j) s[j] = __shfl_sync(0xffffffffu, sc, src0 + j) * row_scale;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = (float)(int)hi[j] * 256.0f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = (v[j] + (float)(int)lo[j]) * s[j];
+        if (m_first + 8 <= P.M) {          // (uniform) all eight tokens are inside: no test per token
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (row_ok) y8[(size_t)j * P.ldy] = v[j];
+        } else {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (m_first + j < P.M && row_ok) y8[(size_t)j * P.ldy] = v[j];
         }
+      };
+#pragma unroll 1
+      for (int i = 0; i < kMyChunks; ++i) {
+        if ((i & 1) == 0) {
+          if (i) sc_cur = sc_next;
+          if (i + 2 < kMyChunks) sc_next = pair_scales((i >> 1) + 1);
+        }
+        const uint32_t t_chunk = t_tile + 16 * (kI8EpiWarps / 4) * i;
+        const int mc = m0 + 16 * (half + (kI8EpiWarps / 4) * i);
+        tmem_wait8(hiA, loA);
+        tmem_ld8(t_chunk + 8, hiB);
+        tmem_ld8(t_chunk + 8 + BN, loB);
+        drain8(hiA, loA, sc_cur, 16 * (i & 1), mc, y_row);
+        tmem_wait8(hiB, loB);
+        if (i + 1 < kMyChunks) {
+          tmem_ld8(t_chunk + 16 * (kI8EpiWarps / 4), hiA);
+          tmem_ld8(t_chunk + 16 * (kI8EpiWarps / 4) + BN, loA);
+        }
+        drain8(hiB, loB, sc_cur, 16 * (i & 1) + 8, mc + 8, y_row + (size_t)8 * P.ldy);
+        y_row += (size_t)(16 * (kI8EpiWarps / 4)) * P.ldy;
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       bar_arrive(tmem_empty(buf));
