@@ -932,7 +932,7 @@ lcd_status launch_dense_i8(const Problem& p, int8_t* levels, int32_t* status_wor
 // (the epilogue of the widths with one accumulator buffer)}, measured on the LLaMA-13B shapes at about 1.7 GHz.
 // The launcher takes the width with the smallest waves x (columns x stage + fixed).
 struct TileShape { int bn, stage_clks, epilogue_clks; };
-constexpr TileShape kShapes[3] = {{128, 425, 0}, {192, 400, 13000}, {256, 535, 13000}};
+constexpr TileShape kShapes[3] = {{128, 425, 0}, {192, 400, 6500}, {256, 535, 7500}};
 
 int pick_shape(int64_t M, int64_t N_pad, int64_t n_ks) {
   const int n_sm = dense_sm_count();
