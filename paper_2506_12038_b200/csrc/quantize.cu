@@ -5,6 +5,8 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
+
 #include "common.h"
 
 namespace lcd {
@@ -13,11 +15,12 @@ constexpr int kQThreads = 1024;   // few tokens: one large CTA per token, everyt
 constexpr int kQThreadsMany = 256; // many tokens: small CTAs, latency hidden by the number of CTAs
 constexpr int kQChunks = 4;    // register-resident path: K <= 8 * kQThreads * kQChunks columns
 
-__device__ __forceinline__ int quant_level(float v) {
-  // round half to even, then clip to the 4-bit symmetric range
-  float r = rintf(v);
-  r = fminf(fmaxf(r, -8.0f), 7.0f);
-  return (int)r;
+// a = q + 8 with q = round half to even of v, clipped to the 4-bit symmetric range.  Clipping first gives the same
+// level (the bounds are integers), and adding 1.5 * 2^23 + 8 rounds the clipped value to an integer, ties to even,
+// in one binary32 addition and leaves q + 8 in the low four bits of the sum: no conversion instructions.
+__device__ __forceinline__ uint32_t quant_nibble(float v) {
+  const float u = fminf(fmaxf(v, -8.0f), 7.0f);
+  return __float_as_uint(__fadd_rn(u, 12582920.0f)) & 0xfu;
 }
 
 // One token per CTA.  VEC: rows are 16-byte aligned and K is a multiple of 8, so each thread handles 8
@@ -108,7 +111,7 @@ __device__ __forceinline__ void smooth_quantize_token(const __half* __restrict__
           const float2 v = __half22float2(h[i]);
           float t0 = __fmul_rn(v.x, f[2 * i]), t1 = __fmul_rn(v.y, f[2 * i + 1]);
           if (!is_static) { t0 = __fmul_rn(t0, r); t1 = __fmul_rn(t1, r); }
-          const uint32_t a0 = (uint32_t)(quant_level(t0) + 8), a1 = (uint32_t)(quant_level(t1) + 8);
+          const uint32_t a0 = quant_nibble(t0), a1 = quant_nibble(t1);
           packed |= (a0 | (a1 << 4)) << (8 * i);
         }
       }
@@ -123,7 +126,7 @@ __device__ __forceinline__ void smooth_quantize_token(const __half* __restrict__
         if (k < K) {
           float t = __fmul_rn(__half2float(xr[k]), inv_smooth ? inv_smooth[k] : 1.0f);
           if (!is_static) t = __fmul_rn(t, r);
-          a[i] = (uint32_t)(quant_level(t) + 8);
+          a[i] = quant_nibble(t);
         }
       }
       out[j] = (uint8_t)(a[0] | (a[1] << 4));
@@ -131,26 +134,27 @@ __device__ __forceinline__ void smooth_quantize_token(const __half* __restrict__
   }
 }
 
-// Same result as smooth_quantize_token<true>, for rows of at most 8 * kQThreads * kQChunks columns: every thread
+// Same result as smooth_quantize_token<true>, for rows of at most 8 * THREADS * CHUNKS columns: every thread
 // keeps its products t_k = x_k * inv_smooth_k in registers between the maximum search and the rounding, so x
 // and inv_smooth are read once and all loads are in flight together.
+template <int THREADS, int CHUNKS>
 __device__ __forceinline__ void smooth_quantize_token_cached(const __half* __restrict__ x, int64_t m, int64_t K,
                                                              int64_t K_pad, int64_t ldx,
                                                              const float* __restrict__ inv_smooth,
                                                              const float* __restrict__ static_scale,
                                                              uint8_t* __restrict__ act_idx,
                                                              float* __restrict__ act_scale) {
-  __shared__ float s_red[kQThreads / 32];
+  __shared__ float s_red[THREADS / 32];
   __shared__ float s_mult;
   const __half* xr = x + m * ldx;
   uint8_t* out = act_idx + m * (K_pad / 2);
   const int tid = threadIdx.x;
   const bool is_static = static_scale != nullptr;
-  float t[kQChunks][8];
+  float t[CHUNKS][8];
   float amax = 0.0f;
 #pragma unroll
-  for (int c = 0; c < kQChunks; ++c) {
-    const int64_t k = ((int64_t)c * kQThreads + tid) * 8;
+  for (int c = 0; c < CHUNKS; ++c) {
+    const int64_t k = ((int64_t)c * THREADS + tid) * 8;
     if (k < K) {
       const uint4 raw = *reinterpret_cast<const uint4*>(xr + k);
       const __half2* h = reinterpret_cast<const __half2*>(&raw);
@@ -182,7 +186,7 @@ __device__ __forceinline__ void smooth_quantize_token_cached(const __half* __res
     if ((tid & 31) == 0) s_red[tid >> 5] = amax;
     __syncthreads();
     if (tid < 32) {
-      float v = tid < kQThreads / 32 ? s_red[tid] : 0.0f;
+      float v = tid < THREADS / 32 ? s_red[tid] : 0.0f;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
       if (tid == 0) {
@@ -201,8 +205,8 @@ __device__ __forceinline__ void smooth_quantize_token_cached(const __half* __res
     act_scale[m] = *static_scale;
   }
 #pragma unroll
-  for (int c = 0; c < kQChunks; ++c) {
-    const int64_t k = ((int64_t)c * kQThreads + tid) * 8;
+  for (int c = 0; c < CHUNKS; ++c) {
+    const int64_t k = ((int64_t)c * THREADS + tid) * 8;
     if (k < K_pad) {
       uint32_t packed = 0x88888888u;
       if (k < K) {
@@ -210,7 +214,104 @@ __device__ __forceinline__ void smooth_quantize_token_cached(const __half* __res
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const float u = is_static ? t[c][i] : __fmul_rn(t[c][i], r);
-          packed |= (uint32_t)(quant_level(u) + 8) << (4 * i);
+          packed |= quant_nibble(u) << (4 * i);
+        }
+      }
+      *reinterpret_cast<uint32_t*>(out + k / 2) = packed;
+    }
+  }
+}
+
+// The same for many tokens (small CTAs, several per SM): a thread keeps its columns of x as the 16-byte words it
+// loaded (four registers per eight columns, so that enough CTAs fit an SM to keep the memory system busy) and forms
+// the products x_k * inv_smooth_k twice, with the same single operations, once for the maximum and once for the
+// levels; inv_smooth comes from L1 the second time.  Rows of at most 8 * THREADS * CHUNKS columns.
+template <int THREADS, int CHUNKS>
+__device__ __forceinline__ void smooth_quantize_token_words(const __half* __restrict__ x, int64_t m, int64_t K,
+                                                            int64_t K_pad, int64_t ldx,
+                                                            const float* __restrict__ inv_smooth,
+                                                            const float* __restrict__ static_scale,
+                                                            uint8_t* __restrict__ act_idx,
+                                                            float* __restrict__ act_scale) {
+  __shared__ float s_red[THREADS / 32];
+  __shared__ float s_mult;
+  const __half* xr = x + m * ldx;
+  uint8_t* out = act_idx + m * (K_pad / 2);
+  const int tid = threadIdx.x;
+  const bool is_static = static_scale != nullptr;
+  uint4 raw[CHUNKS];
+#pragma unroll
+  for (int c = 0; c < CHUNKS; ++c) {
+    const int64_t k = ((int64_t)c * THREADS + tid) * 8;
+    raw[c] = k < K ? *reinterpret_cast<const uint4*>(xr + k) : make_uint4(0u, 0u, 0u, 0u);
+  }
+  auto products = [&](int c, int64_t k, float (&t)[8]) {
+    const __half2* h = reinterpret_cast<const __half2*>(&raw[c]);
+    float f[8];
+    if (inv_smooth) {
+      const float4 a = __ldg(reinterpret_cast<const float4*>(inv_smooth + k));
+      const float4 b = __ldg(reinterpret_cast<const float4*>(inv_smooth + k + 4));
+      f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) f[i] = 1.0f;
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 v = __half22float2(h[i]);
+      t[2 * i] = __fmul_rn(v.x, f[2 * i]);
+      t[2 * i + 1] = __fmul_rn(v.y, f[2 * i + 1]);
+    }
+  };
+  float r = 1.0f;
+  if (!is_static) {
+    float amax = 0.0f;
+#pragma unroll
+    for (int c = 0; c < CHUNKS; ++c) {
+      const int64_t k = ((int64_t)c * THREADS + tid) * 8;
+      if (k < K) {
+        float t[8];
+        products(c, k, t);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(t[i]));
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if ((tid & 31) == 0) s_red[tid >> 5] = amax;
+    __syncthreads();
+    if (tid < 32) {
+      float v = tid < THREADS / 32 ? s_red[tid] : 0.0f;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+      if (tid == 0) {
+        float sq = 1.0f, rr = 0.0f;
+        if (v > 0.0f) {
+          sq = __fdiv_rn(v, 7.0f);
+          rr = __fdiv_rn(7.0f, v);
+        }
+        s_mult = rr;
+        act_scale[m] = sq;
+      }
+    }
+    __syncthreads();
+    r = s_mult;
+  } else if (tid == 0) {
+    act_scale[m] = *static_scale;
+  }
+#pragma unroll
+  for (int c = 0; c < CHUNKS; ++c) {
+    const int64_t k = ((int64_t)c * THREADS + tid) * 8;
+    if (k < K_pad) {
+      uint32_t packed = 0x88888888u;
+      if (k < K) {
+        float t[8];
+        products(c, k, t);
+        packed = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float u = is_static ? t[i] : __fmul_rn(t[i], r);
+          packed |= quant_nibble(u) << (4 * i);
         }
       }
       *reinterpret_cast<uint32_t*>(out + k / 2) = packed;
@@ -233,8 +334,10 @@ struct QuantBatch {
   QuantProblem p[LCD_MAX_BATCH];
 };
 
-// One CTA per token of every problem of the batch.
-template <int THREADS>
+// One CTA per token of every problem of the batch.  CHUNKS > 0: rows of at most 8 * THREADS * CHUNKS columns take the
+// register-resident path (the launcher picks the smallest instance that covers the batch's longest row, so that the
+// instance's register count, and with it the number of CTAs per SM, fits the rows at hand).
+template <int THREADS, int CHUNKS>
 __global__ void __launch_bounds__(THREADS) smooth_quantize_kernel(const __grid_constant__ QuantBatch batch) {
   // This kernel may itself have been started early (programmatic stream serialization): wait for the kernel
   // before it, then let the next one start its own prologue; that one still waits for this grid to finish
@@ -247,9 +350,18 @@ __global__ void __launch_bounds__(THREADS) smooth_quantize_kernel(const __grid_c
     if ((int)blockIdx.x >= batch.p[i].cta0) pi = i;
   const QuantProblem& q = batch.p[pi];
   const int64_t m = (int64_t)blockIdx.x - q.cta0;
-  if (THREADS == kQThreads && q.vec && q.K <= (long long)8 * kQThreads * kQChunks)
-    smooth_quantize_token_cached(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx, q.act_scale);
-  else if (q.vec)
+  if constexpr (CHUNKS > 0) {
+    if (q.vec && q.K_pad <= (long long)8 * THREADS * CHUNKS) {
+      if constexpr (THREADS == kQThreads)
+        smooth_quantize_token_cached<THREADS, CHUNKS>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx,
+                                                      q.act_scale);
+      else
+        smooth_quantize_token_words<THREADS, CHUNKS>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx,
+                                                     q.act_scale);
+      return;
+    }
+  }
+  if (q.vec)
     smooth_quantize_token<true, THREADS>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx, q.act_scale);
   else
     smooth_quantize_token<false, THREADS>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx, q.act_scale);
@@ -288,8 +400,21 @@ lcd_status launch_smooth_quantize_batch(const lcd_act_problem* probs, int count,
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  const cudaError_t e = many ? cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany>, batch)
-                             : cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreads>, batch);
+  // register-resident instance that covers the longest vectorisable row (0: none does)
+  long long chunks = 0;
+  const int threads = many ? kQThreadsMany : kQThreads;
+  for (int i = 0; i < count; ++i)
+    if (batch.p[i].vec) chunks = std::max(chunks, (batch.p[i].K_pad + 8 * threads - 1) / (8 * threads));
+  cudaError_t e;
+  if (!many)
+    e = chunks >= 1 && chunks <= kQChunks ? cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreads, kQChunks>, batch)
+                                          : cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreads, 0>, batch);
+  else if (chunks < 1 || chunks > 8) e = cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany, 0>, batch);
+  else if (chunks <= 2) e = cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany, 2>, batch);
+  else if (chunks <= 3) e = cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany, 3>, batch);
+  else if (chunks <= 4) e = cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany, 4>, batch);
+  else if (chunks <= 6) e = cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany, 6>, batch);
+  else e = cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany, 8>, batch);
   if (e != cudaSuccess) {
     set_cuda_error((int)e);
     return LCD_ERR_CUDA;

@@ -10,10 +10,12 @@ namespace lcd {
 
 namespace {
 
+// The signed byte of round-half-to-even(v) clipped to [-128, 127].  Clipping first gives the same level (integer
+// bounds); adding 1.5 * 2^23 rounds to an integer, ties to even, in one binary32 addition and leaves the level's
+// two's complement in the low byte of the sum.
 __device__ __forceinline__ uint32_t level8(float v) {
-  float r = rintf(v);                              // round half to even
-  r = fminf(fmaxf(r, -128.0f), 127.0f);
-  return (uint32_t)(int)r & 0xffu;
+  const float u = fminf(fmaxf(v, -128.0f), 127.0f);
+  return __float_as_uint(__fadd_rn(u, 12582912.0f)) & 0xffu;
 }
 
 // One token per CTA.  vec: rows are 16-byte aligned and K is a multiple of 8: 8 columns per thread and step.
