@@ -211,30 +211,56 @@ __device__ __forceinline__ uint32_t pick_lookup(const RowTables<BITS, KIND>& T, 
 //   2 bit: staged words [E(w0) E(w1) O(w0) O(w1) E(w2) E(w3) O(w2) O(w3)], E/O = even/odd columns of a word;
 //   3 bit: natural column order.
 // With 8-bit levels a group of 8 columns is two source words of signed bytes and only the order changes.
+// One source word (act8: a pair) of a token's levels into its place j of the staged window.
 template <int BITS>
-__device__ __forceinline__ void stage_window(uint32_t* dst, const uint32_t* src, int n_words, int tid, bool act8) {
+__device__ __forceinline__ void stage_word(uint32_t* dst, int j, uint32_t a_lo, uint32_t a_hi, bool act8) {
+  uint32_t e, o;
+  if (act8) {
+    if (BITS == 2) { e = prmt(a_lo, a_hi, 0x6420u); o = prmt(a_lo, a_hi, 0x7531u); }
+    else { e = a_lo; o = a_hi; }
+  } else {
+    e = a_lo & 0x0f0f0f0fu; o = (a_lo >> 4) & 0x0f0f0f0fu;
+    e = (e + 0x78787878u) ^ 0x80808080u;   // per byte a - 8, no carry between bytes
+    o = (o + 0x78787878u) ^ 0x80808080u;
+  }
+  const int quarter = j >> 2, w = j & 3;
+  if (BITS == 2) {
+    dst[quarter * 8 + (w & 1) + 4 * (w >> 1)] = e;
+    dst[quarter * 8 + 2 + (w & 1) + 4 * (w >> 1)] = o;
+  } else if (act8) {
+    dst[quarter * 8 + 2 * w] = e;
+    dst[quarter * 8 + 2 * w + 1] = o;
+  } else {
+    dst[quarter * 8 + 2 * w] = prmt(e, o, 0x5140u);
+    dst[quarter * 8 + 2 * w + 1] = prmt(e, o, 0x7362u);
+  }
+}
+// The windows of n_tok tokens.  src: the first token's levels of the window's columns, the next token's
+// src_stride words on (act8: pairs of words); dst likewise, dst_stride bytes apart.  The loads of eight tokens are
+// issued together: one after the other they would cost a trip to L2 per token.
+template <int BITS>
+__device__ __forceinline__ void stage_window(uint8_t* dst, int dst_stride, const uint32_t* src, size_t src_stride,
+                                             int n_tok, int n_words, int tid, bool act8) {
   for (int j = tid; j < n_words; j += kThreads) {
-    uint32_t e, o;
-    if (act8) {
-      const uint2 a = __ldcg(reinterpret_cast<const uint2*>(src) + j);
-      if (BITS == 2) { e = prmt(a.x, a.y, 0x6420u); o = prmt(a.x, a.y, 0x7531u); }
-      else { e = a.x; o = a.y; }
-    } else {
-      const uint32_t a = __ldcg(src + j);
-      e = a & 0x0f0f0f0fu; o = (a >> 4) & 0x0f0f0f0fu;
-      e = (e + 0x78787878u) ^ 0x80808080u;   // per byte a - 8, no carry between bytes
-      o = (o + 0x78787878u) ^ 0x80808080u;
-    }
-    const int quarter = j >> 2, w = j & 3;
-    if (BITS == 2) {
-      dst[quarter * 8 + (w & 1) + 4 * (w >> 1)] = e;
-      dst[quarter * 8 + 2 + (w & 1) + 4 * (w >> 1)] = o;
-    } else if (act8) {
-      dst[quarter * 8 + 2 * w] = e;
-      dst[quarter * 8 + 2 * w + 1] = o;
-    } else {
-      dst[quarter * 8 + 2 * w] = prmt(e, o, 0x5140u);
-      dst[quarter * 8 + 2 * w + 1] = prmt(e, o, 0x7362u);
+#pragma unroll 1
+    for (int m0 = 0; m0 < n_tok; m0 += 8) {
+      uint32_t lo[8], hi[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        lo[u] = hi[u] = 0u;
+        if (m0 + u < n_tok) {
+          if (act8) {
+            const uint2 a = __ldcg(reinterpret_cast<const uint2*>(src + (size_t)(m0 + u) * src_stride * 2) + j);
+            lo[u] = a.x; hi[u] = a.y;
+          } else {
+            lo[u] = __ldcg(src + (size_t)(m0 + u) * src_stride + j);
+          }
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (m0 + u < n_tok)
+          stage_word<BITS>(reinterpret_cast<uint32_t*>(dst + (size_t)(m0 + u) * dst_stride), j, lo[u], hi[u], act8);
     }
   }
 }
@@ -718,6 +744,24 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
 #pragma unroll
   for (int G = 0; G < MG; ++G) tok_off[G] = (uint32_t)((8 * G + g < P.M ? 8 * G + g : P.M - 1) * P.tstride + t * 32);
 
+  // s_q of this lane's tokens 8G + 2t and 8G + 2t + 1 (asked for once: a load per output would put a trip to L2 into
+  // every finished row group)
+  float sq_tok[MG][2];
+#pragma unroll
+  for (int G = 0; G < MG; ++G)
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int m = 8 * G + 2 * t + e;
+      sq_tok[G][e] = 1.0f;
+      if (m < P.M) {
+        if (fused) {
+          const float A = s_amax[m];
+          sq_tok[G][e] = A > 0.0f ? __fdiv_rn(A, 7.0f) : 1.0f;
+        } else {
+          sq_tok[G][e] = __ldg(P.act_scale + m);
+        }
+      }
+    }
   // y of the 16-row group rp from complete sums
   auto write_y = [&](uint32_t rp) {
 #pragma unroll
@@ -740,14 +784,7 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
 #pragma unroll
             for (int p = 0; p < PL - 1; ++p) v = fmaf(T.c[p + 1], (float)acc[G][p][r], v);
           }
-          float sq;
-          if (fused) {
-            const float A = s_amax[m];
-            sq = A > 0.0f ? __fdiv_rn(A, 7.0f) : 1.0f;
-          } else {
-            sq = __ldg(P.act_scale + m);
-          }
-          P.y[(size_t)m * P.ldy + n] = v * sq;
+          P.y[(size_t)m * P.ldy + n] = v * sq_tok[G][r & 1];
         }
       }
   };
@@ -786,8 +823,19 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
     if (kSmemCombine) {
       bool run_done = whole;
       if (!whole) {
-        uint32_t first = 0;
-        const uint32_t n_contrib = geo.contributors(pn, rp, &first);
+        uint32_t first = 0, n_contrib;
+        if (nw == (uint32_t)kWarps) {
+          // the run belongs to this CTA and this warp works on it: the other warps on it are its neighbours, found by
+          // walking the warps' first items (shares are a CTA's items split evenly, see wx0) down and up from here
+          const uint32_t xs = geo.run_start(pn * geo.n_rp + rp) - cx0, xe = xs + pw_n - 1;
+          uint32_t wf = (uint32_t)warp, wl = (uint32_t)warp;
+          while (wf > 0 && part_begin(wf, c_items, nw) > xs) --wf;
+          while (wl + 1 < nw && part_begin(wl + 1, c_items, nw) <= xe) ++wl;
+          first = wf;
+          n_contrib = wl - wf + 1;
+        } else {
+          n_contrib = geo.contributors(pn, rp, &first);
+        }
         int* a = s_acc + first * ACC_INTS + lane;
 #pragma unroll
         for (int G = 0; G < MG; ++G)
@@ -853,17 +901,18 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
     for (uint32_t wdw = 0; wdw < 2 && pbase + wdw <= pB; ++wdw) {
       const uint32_t pn = pbase + wdw;
       const int n_words = (int)geo.panel_width(pn) * 32;
-      for (int m = 0; m < n_tok && !fast_stage; ++m) {
-        uint32_t* dst = reinterpret_cast<uint32_t*>(act_s + wdw * win_bytes + m * P.tstride);
-        if (fused) {
+      if (fused) {
+        for (int m = 0; m < n_tok && !fast_stage; ++m) {
+          uint32_t* dst = reinterpret_cast<uint32_t*>(act_s + wdw * win_bytes + m * P.tstride);
           const float A = s_amax[m];
           stage_window_from_x<BITS>(dst, P.x + (size_t)m * P.ldx, P.inv_smooth, (int)(pn * P.pw) * 256, P.K,
                                     P.x_vec != 0, A > 0.0f ? __fdiv_rn(7.0f, A) : 0.0f, n_words, tid);
-        } else {
-          stage_window<BITS>(dst, reinterpret_cast<const uint32_t*>(P.act_idx + ((size_t)m * P.n_kt * 128 +
-                                                                                 (size_t)pn * P.pw * 128) * (P.act_bits == 8 ? 2 : 1)),
-                             n_words, tid, P.act_bits == 8);
         }
+      } else {
+        const bool act8 = P.act_bits == 8;
+        stage_window<BITS>(act_s + wdw * win_bytes, P.tstride,
+                           reinterpret_cast<const uint32_t*>(P.act_idx + (size_t)pn * P.pw * 128 * (act8 ? 2 : 1)),
+                           (size_t)P.n_kt * 32, n_tok, n_words, tid, act8);
       }
     }
     if (!ring_primed) {            // first pass: the staging loads above are queued, now the rest of the ring
