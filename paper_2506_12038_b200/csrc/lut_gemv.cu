@@ -71,6 +71,8 @@ struct GemvProblem {
 
 struct GemvBatch {
   int count;
+  int first_cta[LCD_MAX_BATCH];   // p[i].cta0 once more, side by side: a CTA finds its problem from one line of the
+                                  // parameter block (entries from `count` on are INT_MAX)
   GemvProblem p[LCD_MAX_BATCH];
 };
 
@@ -508,9 +510,8 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
 
   // which problem this CTA works on
   int pi = 0;
-#pragma unroll 1
-  for (int i = 1; i < batch.count; ++i)
-    if ((int)blockIdx.x >= batch.p[i].cta0) pi = i;
+#pragma unroll
+  for (int i = 1; i < LCD_MAX_BATCH; ++i) pi = (int)blockIdx.x >= batch.first_cta[i] ? i : pi;
   const GemvProblem& P = batch.p[pi];
   RunGeometry geo;
   geo.n_rp = (uint32_t)P.n_rp; geo.n_kt = (uint32_t)P.n_kt; geo.pw = (uint32_t)P.pw;
@@ -1170,6 +1171,7 @@ lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void*
     }
   }
   for (int i = count; i < LCD_MAX_BATCH; ++i) batch.p[i] = batch.p[0];
+  for (int i = 0; i < LCD_MAX_BATCH; ++i) batch.first_cta[i] = i < count ? batch.p[i].cta0 : 0x7fffffff;
   const size_t smem = kBarBytes + combine_bytes + ring_bytes + act_bytes;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (bits == 2) {
