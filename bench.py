@@ -423,6 +423,7 @@ def measure_config(args, cfg_id, M, dev, world, local, primary):
             for hb in hbatch:
                 for i, mt in enumerate(mats):
                     hb.x_view(i).copy_(torch.from_numpy(mt["L"].x))
+                hb.capture()       # copy in, launches, copy out recorded once; every step replays them and waits
             h2d, d2h = hbatch[0].x_host.numel(), hbatch[0].y_host.numel()
 
             def e2e_step(c):

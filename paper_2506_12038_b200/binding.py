@@ -459,7 +459,28 @@ class HostBatch:
         w, _, M = self._keep[i]
         return self.y_host[self._y_off[i]:self._y_off[i] + M * w.N * 4].view(torch.float32).view(M, w.N)
 
+    def capture(self):
+        """Records one call (copy in, launches, copy out) as a CUDA graph; run() without a stream replays it
+        from then on: one graph launch instead of two copies and the kernel launches.  The buffers are owned
+        here and keep their addresses, so the recording stays valid."""
+        import torch
+        self.run()                                   # first-use set-up (function attributes) outside the capture
+        torch.cuda.current_stream().synchronize()
+        side = torch.cuda.Stream(device=self.scratch.device)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                self._enqueue(None)
+        self._graph = graph
+        return self
+
     def run(self, stream=None):
+        if stream is None and getattr(self, "_graph", None) is not None:
+            self._graph.replay()
+            return
+        self._enqueue(stream)
+
+    def _enqueue(self, stream):
         _check(lib.lcd_linear_host_batch(self.arr, self.count, c_void_p(self.x_host.data_ptr()),
                                          c_void_p(self.y_host.data_ptr()), c_void_p(self.scratch.data_ptr()),
                                          self.scratch.numel(),

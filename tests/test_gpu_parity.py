@@ -373,6 +373,17 @@ def test_grouped_host_buffer_entry_point():
         for i, L in enumerate(cases):
             q_ref, s_ref = O.smooth_quantize(L.x, L.inv_s)
             check_y(hb.y_view(i), O.lut_linear_dequant(L.idx, L.codebook, q_ref, s_ref))
+    # the recorded form (what the benchmark's end-to-end leg replays): new inputs in the same pinned buffers
+    hb.capture()
+    for rep in range(2):
+        for i, L in enumerate(cases):
+            hb.x_view(i).copy_(torch.from_numpy(L.x) * (0.5 + rep))
+        hb.y_host.fill_(255)
+        hb.run()
+        torch.cuda.synchronize()
+        for i, L in enumerate(cases):
+            q_ref, s_ref = O.smooth_quantize((L.x.astype(np.float32) * np.float32(0.5 + rep)).astype(np.float16), L.inv_s)
+            check_y(hb.y_view(i), O.lut_linear_dequant(L.idx, L.codebook, q_ref, s_ref))
 
 
 # ------------------------------------------------------------------------------- full sizes, bench launch shape
