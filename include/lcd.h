@@ -375,7 +375,8 @@ lcd_status lcd_linear_host(const void* packed_weights_dev, const void* header_ho
 /* The same for up to LCD_MAX_BATCH independent problems with M <= 16 and equal index width (the projections of
  * a decoder layer): ONE host-to-device copy of all inputs, one grouped quantise launch, one grouped lookup
  * launch (a single launch that does both when every problem has one token), ONE device-to-host copy of all
- * outputs.  The host staging buffers are laid out by the library:
+ * outputs (none when the outputs total at most 512 KB and y_host_all is pinned memory the device can address: the
+ * kernels then store y into it directly).  The host staging buffers are laid out by the library:
  * problem i's x (fp16 [M][K], dense) starts at the sum of the earlier problems' M*K*2 bytes rounded up to 16,
  * its y (fp32 [M][N], dense) at the sum of the earlier problems' M*N*4 bytes rounded up to 16;
  * lcd_linear_host_batch_sizes returns the total sizes (any of the three outputs may be NULL).  x_host_all and
