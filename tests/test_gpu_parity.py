@@ -38,7 +38,11 @@ def check_y(y_gpu, y_ref, tight=True):
 # ------------------------------------------------------------------------------- input transformation
 @pytest.mark.parametrize("M,K,ld_extra,use_inv", [(1, 4096, 0, True), (5, 1000, 0, True), (3, 999, 0, True),
                                                   (4, 264, 8, True), (2, 250, 3, False), (1, 1, 0, True),
-                                                  (7, 11008, 0, True), (33, 520, 0, False)])
+                                                  (7, 11008, 0, True), (33, 520, 0, False),
+                                                  # more than 296 tokens: the small-CTA instances, one per row-length bracket
+                                                  (300, 520, 0, False), (300, 4096, 0, True), (301, 7000, 8, True),
+                                                  (300, 11008, 0, True), (297, 13824, 0, True), (300, 17000, 0, True),
+                                                  (300, 999, 0, True)])
 def test_smooth_quantize_bit_exact(M, K, ld_extra, use_inv):
     ch = gen.outlier_channels(11, K, 0.01)
     x = gen.activations(100 + M + K, M, K, ch, 50.0)
