@@ -62,7 +62,7 @@ def parse_args():
                          "'reclassify' = the Section 3.2 reclassification and centroid offsets, 'dbci' = the Section 3.1 "
                          "centroid initialisation")
     ap.add_argument("--two-call", action="store_true",
-                    help="M <= 16: quantise and look up in two launches per layer instead of the fused one")
+                    help="quantise and look up in separate calls instead of the fused one")
     ap.add_argument("--algo", default="auto", choices=["auto", "register", "bucket", "tensor", "shared"],
                     help="lookup kernel for M <= 16 (default: the library's choice)")
     return ap.parse_args()
@@ -315,7 +315,20 @@ def measure_config(args, cfg_id, M, dev, world, local, primary):
         def lookup_only(mi, c):
             single[mi][c].run()
     else:
+        # many tokens, 4-bit levels: the library's one-call form, which transforms the inputs of all matrices in one
+        # launch straight into the tensor-core kernel's operand bytes and then runs that kernel per matrix;
+        # --two-call, 8-bit levels and 17..32 tokens: per matrix quantise, (expand,) lookup
+        fused = (not args.two_call) and args.act_bits == 4 and args.algo == "auto" and M > 32 and len(mats) <= lcd.MAX_BATCH
+        if fused:
+            fbatch = [lcd.FusedBatch([(mt["w"][c], mt["x"], mt["inv_s"], mt["y"]) for mt in mats], status_word=status)
+                      for c in range(copies)]
+            for mt in mats:       # the stored levels of the per-matrix timings and of the parity check
+                lcd.smooth_quantize_act(mt["x"], mt["inv_s"], act_idx=mt["a"], act_scale=mt["s"])
+
         def step(c):
+            if fused:
+                fbatch[c].run()
+                return
             for mt in mats:
                 lcd.smooth_quantize_act(mt["x"], mt["inv_s"], act_idx=mt["a"], act_scale=mt["s"],
                                         act_bits=args.act_bits)
@@ -325,7 +338,8 @@ def measure_config(args, cfg_id, M, dev, world, local, primary):
             mt = mats[mi]
             lcd.lut_linear(mt["w"][c], mt["a"], mt["s"], y=mt["y"], workspace=mt["work"], status_word=status)
 
-    launches_per_step = (1 if fused else 2) if grouped else 2 * len(mats)
+    # kernels per step: grouped 1 (fused) or 2; many tokens 1 + one per matrix (fused) or quantise, expand, lookup per matrix
+    launches_per_step = (1 if fused else 2) if grouped else (1 + len(mats) if fused else 3 * len(mats))
     stream = torch.cuda.Stream(device=dev)
     with torch.cuda.stream(stream):
         for c in range(copies):
@@ -519,6 +533,7 @@ def measure_config(args, cfg_id, M, dev, world, local, primary):
                                                 graphs=f"steps replayed as CUDA graphs of {copies} consecutive steps",
                                                 launches=("1 launch per layer: quantise + lookup fused" if grouped and fused
                                                           else "1 grouped quantise + 1 grouped lookup per layer" if grouped
+                                                          else "1 quantise launch for the layer + 1 tensor-core launch per matrix (one library call)" if fused
                                                           else "per matrix: quantise + lookup")),
             "timing": {"repeats": len(rep_ms), "steps_per_repeat": steps, "timed_ms_total": sum(rep_ms),
                        "us_per_step_median": statistics.median(rep_ms) / steps * 1e3 / world,

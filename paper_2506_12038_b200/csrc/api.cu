@@ -329,17 +329,30 @@ extern "C" lcd_status lcd_lut_linear_act8(const void* packed_weights_dev, const 
   }
 }
 
+// Levels and scales of the many-token form of the fused call inside its workspace: per problem M x K_pad signed
+// bytes, then M scales, each rounded up to 256 bytes.
+static size_t fused_dense_levels_bytes(const Problem& p) { return (size_t)round_up_u64((uint64_t)p.M * p.K_pad, 256); }
+static size_t fused_dense_bytes(const Problem& p) {
+  return fused_dense_levels_bytes(p) + (size_t)round_up_u64((uint64_t)p.M * sizeof(float), 256);
+}
+
 static lcd_status fused_problems(const lcd_fused_problem* problems, int count, lcd_algo algo, bool pointers,
                                  Problem* p, lcd_algo* resolved) {
   if (!problems || count < 1 || count > LCD_MAX_BATCH) return LCD_ERR_INVALID_ARG;
   if (algo != LCD_ALGO_AUTO && algo != LCD_ALGO_REGISTER_LUT && algo != LCD_ALGO_BUCKET_LUT &&
-      algo != LCD_ALGO_SHARED_BUCKET)
+      algo != LCD_ALGO_SHARED_BUCKET && algo != LCD_ALGO_DENSE_TC)
     return LCD_ERR_UNSUPPORTED;
+  // either every problem has at most 16 tokens (one lookup launch that transforms its inputs itself) or every
+  // problem has more than 32 (one transformation launch, then the tensor-core kernel per problem)
+  bool many = false;
+  for (int i = 0; i < count; ++i) many = many || (problems[i].M > 16);
   for (int i = 0; i < count; ++i) {
     const lcd_fused_problem& q = problems[i];
     if (q.M < 1 || !q.header_host) return LCD_ERR_INVALID_ARG;
-    if (q.M > 16) return LCD_ERR_UNSUPPORTED;
+    if (many ? (q.M <= 32 || (algo != LCD_ALGO_AUTO && algo != LCD_ALGO_DENSE_TC)) : algo == LCD_ALGO_DENSE_TC)
+      return LCD_ERR_UNSUPPORTED;
     if (!shape_problem(q.header_host, q.M, &p[i])) return LCD_ERR_BAD_BLOB;
+    if (many && p[i].K_pad >= (1 << 21)) return LCD_ERR_UNSUPPORTED;      // the int32 sums of the planes could overflow
     if (p[i].bits != p[0].bits) return LCD_ERR_UNSUPPORTED;
     p[i].act_bits = 16;
     if (!pointers) continue;
@@ -358,6 +371,10 @@ static lcd_status fused_problems(const lcd_fused_problem* problems, int count, l
     p[i].y = q.y;
     p[i].ldy = q.ldy;
   }
+  if (many) {
+    *resolved = LCD_ALGO_DENSE_TC;
+    return LCD_OK;
+  }
   return batch_family(p, count, algo, resolved);
 }
 
@@ -368,6 +385,12 @@ extern "C" lcd_status lcd_linear_fused_batch_workspace_bytes(const lcd_fused_pro
   const lcd_status st = fused_problems(problems, count, algo, false, p, &resolved);
   if (st != LCD_OK) return st;
   if (!bytes) return LCD_ERR_INVALID_ARG;
+  if (resolved == LCD_ALGO_DENSE_TC) {
+    size_t total = 0;
+    for (int i = 0; i < count; ++i) total += fused_dense_bytes(p[i]);
+    *bytes = total;
+    return LCD_OK;
+  }
   *bytes = lut_gemv_workspace_bytes(p, count, resolved);
   return LCD_OK;
 }
@@ -377,8 +400,41 @@ extern "C" lcd_status lcd_linear_fused_batch(const lcd_fused_problem* problems, 
                                              void* cuda_stream) {
   Problem p[LCD_MAX_BATCH];
   lcd_algo resolved;
-  const lcd_status st = fused_problems(problems, count, algo, true, p, &resolved);
+  lcd_status st = fused_problems(problems, count, algo, true, p, &resolved);
   if (st != LCD_OK) return st;
+  if (resolved == LCD_ALGO_DENSE_TC) {
+    // Many tokens: ONE launch transforms the inputs of all problems (Section 4.1, the operation sequence of
+    // lcd_smooth_quantize_act) and writes the levels as the signed bytes the tensor-core kernel reads, in its order:
+    // no packed 4-bit copy, no expansion pass.  Then that kernel, once per problem.
+    size_t need = 0;
+    for (int i = 0; i < count; ++i) need += fused_dense_bytes(p[i]);
+    if (!workspace || workspace_bytes < need) return LCD_ERR_BUFFER_TOO_SMALL;
+    if (!aligned(workspace, 256)) return LCD_ERR_INVALID_ARG;
+    lcd_act_problem acts[LCD_MAX_BATCH];
+    uint8_t* at = static_cast<uint8_t*>(workspace);
+    for (int i = 0; i < count; ++i) {
+      acts[i].x_fp16 = p[i].x_fp16;
+      acts[i].M = p[i].M;
+      acts[i].K = p[i].K;
+      acts[i].ldx = p[i].ldx;
+      acts[i].inv_smooth = p[i].inv_smooth;
+      acts[i].static_scale = nullptr;
+      acts[i].act_idx = at;
+      acts[i].act_scale = reinterpret_cast<float*>(at + fused_dense_levels_bytes(p[i]));
+      at += fused_dense_bytes(p[i]);
+    }
+    st = launch_smooth_quantize_dense_levels(acts, count, p[0].bits, cuda_stream);
+    if (st != LCD_OK) return st;
+    for (int i = 0; i < count; ++i) {
+      p[i].act_bits = 4;
+      p[i].act_idx = acts[i].act_idx;
+      p[i].act_scale = acts[i].act_scale;
+      p[i].dense_levels = true;
+      st = launch_dense_tc(p[i], false, nullptr, 0, status_word_dev, cuda_stream);
+      if (st != LCD_OK) return st;
+    }
+    return LCD_OK;
+  }
   const size_t need = lut_gemv_workspace_bytes(p, count, resolved);
   if (!workspace || workspace_bytes < need) return LCD_ERR_BUFFER_TOO_SMALL;
   if (!aligned(workspace, 256)) return LCD_ERR_INVALID_ARG;

@@ -42,6 +42,7 @@ struct Problem {
   int bits, C;
   const uint8_t* act_idx;   // device [M][K_pad/2] (4-bit levels + 8) or [M][K_pad] signed bytes (act_bits == 8)
   int act_bits = 4;         // 4 or 8; 16 = not quantised yet: the lookup kernel does Section 4.1 itself from x
+  bool dense_levels = false;          // act_idx already holds the signed bytes the int8 tensor-core kernel reads
   const void* x_fp16 = nullptr;       // act_bits == 16: device fp16 [M][ldx]
   int64_t ldx = 0;
   const float* inv_smooth = nullptr;  // act_bits == 16: device fp32 [K] or null
@@ -69,6 +70,9 @@ lcd_status launch_dbci(const float* weights, int64_t n, void* workspace, float* 
                        int32_t* labels, float* sorted_out, lcd_dbci_result* result, void* stream);
 lcd_status launch_reference(const Problem& p, void* stream);
 lcd_status launch_smooth_quantize_batch(const lcd_act_problem* probs, int count, void* stream);
+// The same transformation with the levels written as signed bytes [M][K_pad] in the order the int8 tensor-core kernel
+// reads them for this index width (act_idx of the problems points to that buffer)
+lcd_status launch_smooth_quantize_dense_levels(const lcd_act_problem* probs, int count, int bits, void* stream);
 // LCD_ALGO_REGISTER_LUT / LCD_ALGO_BUCKET_LUT for up to LCD_MAX_BATCH problems of equal index width in one launch
 size_t lut_gemv_workspace_bytes(const Problem* probs, int count, lcd_algo algo);
 lcd_status launch_lut_gemv(const Problem* probs, int count, lcd_algo algo, void* workspace, size_t workspace_bytes,

@@ -618,6 +618,7 @@ dense_i8_kernel(const __grid_constant__ CUtensorMap tmap_act, const DenseParams 
     const int quad = warp & 3, half = (warp - kFirstEpiWarp) >> 2;
     uint32_t tl = 0;
     bool ok = true;
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // the token scales may come from the kernel before this one
     for (int tile = blockIdx.x; tile < P.n_tiles && ok; tile += gridDim.x, ++tl) {
       const uint32_t buf = tl % NBUF;
       const int n = (tile / P.n_tiles_m) * kBM + 32 * quad + lane;
@@ -953,7 +954,7 @@ size_t dense_tc_workspace_bytes(int64_t M, int64_t K_pad) { return (size_t)round
 
 lcd_status launch_dense_tc(const Problem& p, bool fp16_operands, void* workspace, size_t workspace_bytes,
                            int32_t* status_word, void* stream) {
-  if (!workspace || workspace_bytes < dense_tc_workspace_bytes(p.M, p.K_pad)) return LCD_ERR_BUFFER_TOO_SMALL;
+  if (!p.dense_levels && (!workspace || workspace_bytes < dense_tc_workspace_bytes(p.M, p.K_pad))) return LCD_ERR_BUFFER_TOO_SMALL;
   if (p.M > 0x7fffffffLL / 2 || p.N > 0x7fffffffLL / 2) return LCD_ERR_UNSUPPORTED;
   if (p.bits == 4 && fp16_operands) return LCD_ERR_UNSUPPORTED;    // 4-bit indices: the int8 kernel only
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -962,7 +963,10 @@ lcd_status launch_dense_tc(const Problem& p, bool fp16_operands, void* workspace
   if (p.act_bits == 8 && fp16_operands) return LCD_ERR_UNSUPPORTED;
   if (!fp16_operands) {
     int8_t* levels = static_cast<int8_t*>(workspace);
-    if (p.act_bits == 8) {
+    if (p.dense_levels) {
+      // the input transformation of this call has already written the signed bytes in this kernel's order
+      levels = const_cast<int8_t*>(reinterpret_cast<const int8_t*>(p.act_idx));
+    } else if (p.act_bits == 8) {
       // signed bytes already: the 3-bit decoder's order is the natural one, the 2-bit one needs the permutation
       if (p.bits == 2) permute_levels_i8_kernel<<<blocks, 256, 0, s>>>(p.act_idx, n_quarters, levels);
       else levels = const_cast<int8_t*>(reinterpret_cast<const int8_t*>(p.act_idx));

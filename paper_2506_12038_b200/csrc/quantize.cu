@@ -23,9 +23,52 @@ __device__ __forceinline__ uint32_t quant_nibble(float v) {
   return __float_as_uint(__fadd_rn(u, 12582920.0f)) & 0xfu;
 }
 
+// Output forms.  kOutNibbles: the levels a = q + 8 packed two per byte, [K_pad / 2] bytes per token (what
+// lcd_smooth_quantize_act returns).  kOutBytes / kOutBytes2: the levels q as signed bytes, [K_pad] per token, for
+// the tensor-core kernel that follows in the same call: in column order, or in the order in which the 2-bit
+// decoder lists the weights of a 32-column quarter (position 16*(c>>4) + 8*(c&1) + 4*((c>>3)&1) + ((c>>1)&3)
+// holds column c).
+constexpr int kOutNibbles = 0, kOutBytes = 1, kOutBytes2 = 2;
+
+__device__ __forceinline__ uint32_t prmt_q(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+  return d;
+}
+// Eight levels (nibble i of `packed` = a of column k + i, k a multiple of 8) into a token's output row.
+template <int OUT>
+__device__ __forceinline__ void store_levels8(uint8_t* row, int64_t k, uint32_t packed) {
+  if (OUT == kOutNibbles) {
+    *reinterpret_cast<uint32_t*>(row + k / 2) = packed;
+    return;
+  }
+  uint32_t e = packed & 0x0f0f0f0fu, o = (packed >> 4) & 0x0f0f0f0fu;     // columns k, k+2, .. / k+1, k+3, ..
+  e = (e + 0x78787878u) ^ 0x80808080u;      // per byte a - 8, no carry between bytes
+  o = (o + 0x78787878u) ^ 0x80808080u;
+  if (OUT == kOutBytes) {
+    *reinterpret_cast<uint2*>(row + k) = make_uint2(prmt_q(e, o, 0x5140u), prmt_q(e, o, 0x7362u));
+  } else {
+    const int64_t quarter = k & ~(int64_t)31;
+    const int c8 = (int)(k & 31) >> 3;                  // which eight columns of the quarter
+    uint8_t* dst = row + quarter + 16 * (c8 >> 1) + 4 * (c8 & 1);
+    *reinterpret_cast<uint32_t*>(dst) = e;
+    *reinterpret_cast<uint32_t*>(dst + 8) = o;
+  }
+}
+// One level (a = q + 8 of column k).
+template <int OUT>
+__device__ __forceinline__ void store_level1(uint8_t* row, int64_t k, uint32_t a) {
+  const uint8_t q = (uint8_t)((a - 8u) & 0xffu);
+  if (OUT == kOutBytes) row[k] = q;
+  else {
+    const int c = (int)(k & 31);
+    row[(k & ~(int64_t)31) + 16 * (c >> 4) + 8 * (c & 1) + 4 * ((c >> 3) & 1) + ((c >> 1) & 3)] = q;
+  }
+}
+
 // One token per CTA.  VEC: rows are 16-byte aligned and K is a multiple of 8, so each thread handles 8
 // consecutive columns per step (one 16-byte load of x, two of inv_smooth, one 4-byte store).
-template <bool VEC, int THREADS>
+template <bool VEC, int THREADS, int OUT = kOutNibbles>
 __device__ __forceinline__ void smooth_quantize_token(const __half* __restrict__ x, int64_t m, int64_t K,
                                                       int64_t K_pad, int64_t ldx,
                                                       const float* __restrict__ inv_smooth,
@@ -34,7 +77,7 @@ __device__ __forceinline__ void smooth_quantize_token(const __half* __restrict__
   __shared__ float s_red[THREADS / 32];
   __shared__ float s_mult;
   const __half* xr = x + m * ldx;
-  uint8_t* out = act_idx + m * (K_pad / 2);
+  uint8_t* out = act_idx + m * (OUT == kOutNibbles ? K_pad / 2 : K_pad);
   const int tid = threadIdx.x;
   const bool is_static = static_scale != nullptr;
 
@@ -115,7 +158,7 @@ __device__ __forceinline__ void smooth_quantize_token(const __half* __restrict__
           packed |= (a0 | (a1 << 4)) << (8 * i);
         }
       }
-      *reinterpret_cast<uint32_t*>(out + k / 2) = packed;
+      store_levels8<OUT>(out, k, packed);
     }
   } else {
     for (int64_t j = tid; j < K_pad / 2; j += THREADS) {
@@ -129,7 +172,8 @@ __device__ __forceinline__ void smooth_quantize_token(const __half* __restrict__
           a[i] = quant_nibble(t);
         }
       }
-      out[j] = (uint8_t)(a[0] | (a[1] << 4));
+      if (OUT == kOutNibbles) out[j] = (uint8_t)(a[0] | (a[1] << 4));
+      else { store_level1<OUT>(out, 2 * j, a[0]); store_level1<OUT>(out, 2 * j + 1, a[1]); }
     }
   }
 }
@@ -226,7 +270,7 @@ __device__ __forceinline__ void smooth_quantize_token_cached(const __half* __res
 // loaded (four registers per eight columns, so that enough CTAs fit an SM to keep the memory system busy) and forms
 // the products x_k * inv_smooth_k twice, with the same single operations, once for the maximum and once for the
 // levels; inv_smooth comes from L1 the second time.  Rows of at most 8 * THREADS * CHUNKS columns.
-template <int THREADS, int CHUNKS>
+template <int THREADS, int CHUNKS, int OUT = kOutNibbles>
 __device__ __forceinline__ void smooth_quantize_token_words(const __half* __restrict__ x, int64_t m, int64_t K,
                                                             int64_t K_pad, int64_t ldx,
                                                             const float* __restrict__ inv_smooth,
@@ -236,7 +280,7 @@ __device__ __forceinline__ void smooth_quantize_token_words(const __half* __rest
   __shared__ float s_red[THREADS / 32];
   __shared__ float s_mult;
   const __half* xr = x + m * ldx;
-  uint8_t* out = act_idx + m * (K_pad / 2);
+  uint8_t* out = act_idx + m * (OUT == kOutNibbles ? K_pad / 2 : K_pad);
   const int tid = threadIdx.x;
   const bool is_static = static_scale != nullptr;
   uint4 raw[CHUNKS];
@@ -314,7 +358,7 @@ __device__ __forceinline__ void smooth_quantize_token_words(const __half* __rest
           packed |= quant_nibble(u) << (4 * i);
         }
       }
-      *reinterpret_cast<uint32_t*>(out + k / 2) = packed;
+      store_levels8<OUT>(out, k, packed);
     }
   }
 }
@@ -337,7 +381,7 @@ struct QuantBatch {
 // One CTA per token of every problem of the batch.  CHUNKS > 0: rows of at most 8 * THREADS * CHUNKS columns take the
 // register-resident path (the launcher picks the smallest instance that covers the batch's longest row, so that the
 // instance's register count, and with it the number of CTAs per SM, fits the rows at hand).
-template <int THREADS, int CHUNKS>
+template <int THREADS, int CHUNKS, int OUT = kOutNibbles>
 __global__ void __launch_bounds__(THREADS) smooth_quantize_kernel(const __grid_constant__ QuantBatch batch) {
   // This kernel may itself have been started early (programmatic stream serialization): wait for the kernel
   // before it, then let the next one start its own prologue; that one still waits for this grid to finish
@@ -356,18 +400,32 @@ __global__ void __launch_bounds__(THREADS) smooth_quantize_kernel(const __grid_c
         smooth_quantize_token_cached<THREADS, CHUNKS>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx,
                                                       q.act_scale);
       else
-        smooth_quantize_token_words<THREADS, CHUNKS>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx,
-                                                     q.act_scale);
+        smooth_quantize_token_words<THREADS, CHUNKS, OUT>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale,
+                                                          q.act_idx, q.act_scale);
       return;
     }
   }
   if (q.vec)
-    smooth_quantize_token<true, THREADS>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx, q.act_scale);
+    smooth_quantize_token<true, THREADS, OUT>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx, q.act_scale);
   else
-    smooth_quantize_token<false, THREADS>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx, q.act_scale);
+    smooth_quantize_token<false, THREADS, OUT>(q.x, m, q.K, q.K_pad, q.ldx, q.inv_smooth, q.static_scale, q.act_idx, q.act_scale);
 }
 
-lcd_status launch_smooth_quantize_batch(const lcd_act_problem* probs, int count, void* stream) {
+namespace {
+
+template <int OUT>
+cudaError_t launch_small_ctas(const cudaLaunchConfig_t& cfg, long long chunks, const QuantBatch& batch) {
+  if (chunks < 1 || chunks > 8) return cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany, 0, OUT>, batch);
+  if (chunks <= 2) return cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany, 2, OUT>, batch);
+  if (chunks <= 3) return cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany, 3, OUT>, batch);
+  if (chunks <= 4) return cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany, 4, OUT>, batch);
+  if (chunks <= 6) return cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany, 6, OUT>, batch);
+  return cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany, 8, OUT>, batch);
+}
+
+// out_form: kOutNibbles (act_idx = [M][K_pad / 2]) or signed bytes for the tensor-core kernel (act_idx = [M][K_pad],
+// kOutBytes in column order, kOutBytes2 in the 2-bit decoder's order).
+lcd_status launch_quantize_form(const lcd_act_problem* probs, int count, int out_form, void* stream) {
   QuantBatch batch;
   batch.count = count;
   long long grid = 0;
@@ -385,14 +443,14 @@ lcd_status launch_smooth_quantize_batch(const lcd_act_problem* probs, int count,
     q.cta0 = (int)grid;
     q.vec = (reinterpret_cast<uintptr_t>(a.x_fp16) % 16 == 0) && (a.ldx % 8 == 0) && (a.K % 8 == 0) &&
             (a.inv_smooth == nullptr || reinterpret_cast<uintptr_t>(a.inv_smooth) % 16 == 0) &&
-            (reinterpret_cast<uintptr_t>(a.act_idx) % 4 == 0);
+            (reinterpret_cast<uintptr_t>(a.act_idx) % (out_form == kOutNibbles ? 4 : 8) == 0);
     grid += a.M;
     if (grid > 0x7fffffffLL) return LCD_ERR_INVALID_ARG;
   }
   for (int i = count; i < LCD_MAX_BATCH; ++i) batch.p[i] = batch.p[0];
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
-  const bool many = grid > 296;
+  const bool many = grid > 296 || out_form != kOutNibbles;      // the byte forms exist for the small CTAs only
   cfg.blockDim = dim3(many ? kQThreadsMany : kQThreads);
   cfg.stream = static_cast<cudaStream_t>(stream);
   cudaLaunchAttribute attr[1];
@@ -409,17 +467,24 @@ lcd_status launch_smooth_quantize_batch(const lcd_act_problem* probs, int count,
   if (!many)
     e = chunks >= 1 && chunks <= kQChunks ? cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreads, kQChunks>, batch)
                                           : cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreads, 0>, batch);
-  else if (chunks < 1 || chunks > 8) e = cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany, 0>, batch);
-  else if (chunks <= 2) e = cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany, 2>, batch);
-  else if (chunks <= 3) e = cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany, 3>, batch);
-  else if (chunks <= 4) e = cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany, 4>, batch);
-  else if (chunks <= 6) e = cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany, 6>, batch);
-  else e = cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreadsMany, 8>, batch);
+  else if (out_form == kOutBytes) e = launch_small_ctas<kOutBytes>(cfg, chunks, batch);
+  else if (out_form == kOutBytes2) e = launch_small_ctas<kOutBytes2>(cfg, chunks, batch);
+  else e = launch_small_ctas<kOutNibbles>(cfg, chunks, batch);
   if (e != cudaSuccess) {
     set_cuda_error((int)e);
     return LCD_ERR_CUDA;
   }
   return LCD_OK;
+}
+
+}  // namespace
+
+lcd_status launch_smooth_quantize_batch(const lcd_act_problem* probs, int count, void* stream) {
+  return launch_quantize_form(probs, count, kOutNibbles, stream);
+}
+
+lcd_status launch_smooth_quantize_dense_levels(const lcd_act_problem* probs, int count, int bits, void* stream) {
+  return launch_quantize_form(probs, count, bits == 2 ? kOutBytes2 : kOutBytes, stream);
 }
 
 lcd_status launch_smooth_quantize(const void* x, int64_t M, int64_t K, int64_t ldx, const float* inv_smooth,

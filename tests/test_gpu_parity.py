@@ -647,6 +647,41 @@ def test_fused_launch_equals_two_call_path_and_oracle(bits, algo):
     assert torch.equal(y, lcd.lut_linear(w, a, s, algo=algo))
 
 
+@pytest.mark.parametrize("bits", [2, 3, 4])
+def test_fused_call_with_many_tokens_equals_two_call_path_and_oracle(bits):
+    # more than 32 tokens: one transformation launch for all problems writes the tensor-core kernel's signed bytes
+    # directly; the levels are the same, so y equals the two-call result bit for bit
+    shapes = [(200, 1000, 33), (130, 520, 64), (24, 11008, 300), (257, 250, 40), (1031, 4096, 130)]   # 250: unaligned rows
+    C = 10 if bits == 4 else None
+    cases = [gen.random_case(seed=71 * i + bits, N=N, K=K, bits=bits, M=M, C=C) for i, (N, K, M) in enumerate(shapes)]
+    cases[1].x[3, :] = 0                                    # an all-zero token: scale 1, levels 0
+    items, two_call, refs = [], [], []
+    for L in cases:
+        w = lcd.PackedWeights(lcd.pack_weights(L.idx, L.codebook, bits, C) if C else lcd.pack_weights(L.idx, L.codebook, bits))
+        x, inv_s = torch.from_numpy(L.x).cuda(), torch.from_numpy(L.inv_s).cuda()
+        y = torch.full((L.M, L.N), float("nan"), dtype=torch.float32, device="cuda")
+        items.append((w, x, inv_s, y))
+        a, s = lcd.smooth_quantize_act(x, inv_s)
+        two_call.append(lcd.lut_linear(w, a, s, algo=lcd.ALGO_DENSE_TC))
+        q_ref, s_ref = O.smooth_quantize(L.x, L.inv_s)
+        refs.append(O.lut_linear_dequant(L.idx, L.codebook, q_ref, s_ref))
+    word = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    fb = lcd.FusedBatch(items, status_word=word)
+    for _ in range(2):
+        fb.run()
+    torch.cuda.synchronize()
+    assert int(word.item()) == 0
+    for (w, x, inv_s, y), y2, y_ref in zip(items, two_call, refs):
+        assert torch.equal(y, y2)
+        check_y(y, y_ref)
+    # a mix of few and many tokens, and 17 to 32 tokens, are refused before anything is launched
+    for bad in ([items[0], (items[0][0], items[0][1][:4], items[0][2], items[0][3][:4])],
+                [(items[0][0], items[0][1][:20], items[0][2], items[0][3][:20])]):
+        with pytest.raises(lcd.LcdError) as err:
+            lcd.FusedBatch(bad)
+        assert err.value.status == 2
+
+
 # ------------------------------------------------------------------------------- adaptive smoothing search (offline)
 @pytest.mark.parametrize("T,K,ld_extra", [(128, 4096, 0), (64, 1000, 8), (5, 250, 3), (1, 256, 0)])
 def test_smoothing_search_matches_oracle(T, K, ld_extra):
