@@ -36,8 +36,8 @@ __device__ __forceinline__ uint32_t prmt_q(uint32_t a, uint32_t b, uint32_t sel)
   return d;
 }
 // Eight levels (nibble i of `packed` = a of column k + i, k a multiple of 8) into a token's output row.
-template <int OUT>
-__device__ __forceinline__ void store_levels8(uint8_t* row, int64_t k, uint32_t packed) {
+template <int OUT, typename Index>
+__device__ __forceinline__ void store_levels8(uint8_t* row, Index k, uint32_t packed) {
   if (OUT == kOutNibbles) {
     *reinterpret_cast<uint32_t*>(row + k / 2) = packed;
     return;
@@ -48,7 +48,7 @@ __device__ __forceinline__ void store_levels8(uint8_t* row, int64_t k, uint32_t 
   if (OUT == kOutBytes) {
     *reinterpret_cast<uint2*>(row + k) = make_uint2(prmt_q(e, o, 0x5140u), prmt_q(e, o, 0x7362u));
   } else {
-    const int64_t quarter = k & ~(int64_t)31;
+    const Index quarter = k & ~(Index)31;
     const int c8 = (int)(k & 31) >> 3;                  // which eight columns of the quarter
     uint8_t* dst = row + quarter + 16 * (c8 >> 1) + 4 * (c8 & 1);
     *reinterpret_cast<uint32_t*>(dst) = e;
@@ -271,8 +271,8 @@ __device__ __forceinline__ void smooth_quantize_token_cached(const __half* __res
 // the products x_k * inv_smooth_k twice, with the same single operations, once for the maximum and once for the
 // levels; inv_smooth comes from L1 the second time.  Rows of at most 8 * THREADS * CHUNKS columns.
 template <int THREADS, int CHUNKS, int OUT = kOutNibbles>
-__device__ __forceinline__ void smooth_quantize_token_words(const __half* __restrict__ x, int64_t m, int64_t K,
-                                                            int64_t K_pad, int64_t ldx,
+__device__ __forceinline__ void smooth_quantize_token_words(const __half* __restrict__ x, int64_t m, int64_t K64,
+                                                            int64_t K_pad64, int64_t ldx,
                                                             const float* __restrict__ inv_smooth,
                                                             const float* __restrict__ static_scale,
                                                             uint8_t* __restrict__ act_idx,
@@ -280,16 +280,17 @@ __device__ __forceinline__ void smooth_quantize_token_words(const __half* __rest
   __shared__ float s_red[THREADS / 32];
   __shared__ float s_mult;
   const __half* xr = x + m * ldx;
-  uint8_t* out = act_idx + m * (OUT == kOutNibbles ? K_pad / 2 : K_pad);
+  uint8_t* out = act_idx + m * (OUT == kOutNibbles ? K_pad64 / 2 : K_pad64);
   const int tid = threadIdx.x;
   const bool is_static = static_scale != nullptr;
+  const int K = (int)K64, K_pad = (int)K_pad64;        // at most 8 * THREADS * CHUNKS columns: 32-bit column arithmetic
   uint4 raw[CHUNKS];
 #pragma unroll
   for (int c = 0; c < CHUNKS; ++c) {
-    const int64_t k = ((int64_t)c * THREADS + tid) * 8;
+    const int k = (c * THREADS + tid) * 8;
     raw[c] = k < K ? *reinterpret_cast<const uint4*>(xr + k) : make_uint4(0u, 0u, 0u, 0u);
   }
-  auto products = [&](int c, int64_t k, float (&t)[8]) {
+  auto products = [&](int c, int k, float (&t)[8]) {
     const __half2* h = reinterpret_cast<const __half2*>(&raw[c]);
     float f[8];
     if (inv_smooth) {
@@ -312,7 +313,7 @@ __device__ __forceinline__ void smooth_quantize_token_words(const __half* __rest
     float amax = 0.0f;
 #pragma unroll
     for (int c = 0; c < CHUNKS; ++c) {
-      const int64_t k = ((int64_t)c * THREADS + tid) * 8;
+      const int k = (c * THREADS + tid) * 8;
       if (k < K) {
         float t[8];
         products(c, k, t);
@@ -343,22 +344,38 @@ __device__ __forceinline__ void smooth_quantize_token_words(const __half* __rest
   } else if (tid == 0) {
     act_scale[m] = *static_scale;
   }
+  // static mode: the caller's factors already hold the scale, so the second multiplication is by exactly 1
+  const float r_eff = is_static ? 1.0f : r;
 #pragma unroll
   for (int c = 0; c < CHUNKS; ++c) {
-    const int64_t k = ((int64_t)c * THREADS + tid) * 8;
+    const int k = (c * THREADS + tid) * 8;
     if (k < K_pad) {
-      uint32_t packed = 0x88888888u;
+      // e / o: the levels of columns k, k+2, k+4, k+6 / k+1, k+3, k+5, k+7, one per byte (a = q + 8 for the packed
+      // form, q as a signed byte otherwise); padding columns hold level 0
+      uint32_t e = OUT == kOutNibbles ? 0x08080808u : 0u, o = e;
       if (k < K) {
         float t[8];
         products(c, k, t);
-        packed = 0;
+        uint32_t b[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          const float u = is_static ? t[i] : __fmul_rn(t[i], r);
-          packed |= quant_nibble(u) << (4 * i);
+          const float u = fminf(fmaxf(is_static ? t[i] : __fmul_rn(t[i], r_eff), -8.0f), 7.0f);
+          // clipped, then rounded to an integer (ties to even) by one addition: the low byte of the sum is the level
+          b[i] = __float_as_uint(__fadd_rn(u, OUT == kOutNibbles ? 12582920.0f : 12582912.0f));
         }
+        e = prmt_q(prmt_q(b[0], b[2], 0x0040u), prmt_q(b[4], b[6], 0x0040u), 0x5410u);
+        o = prmt_q(prmt_q(b[1], b[3], 0x0040u), prmt_q(b[5], b[7], 0x0040u), 0x5410u);
       }
-      store_levels8<OUT>(out, k, packed);
+      if (OUT == kOutNibbles) {
+        *reinterpret_cast<uint32_t*>(out + k / 2) = (e & 0x0f0f0f0fu) | ((o & 0x0f0f0f0fu) << 4);
+      } else if (OUT == kOutBytes) {
+        *reinterpret_cast<uint2*>(out + k) = make_uint2(prmt_q(e, o, 0x5140u), prmt_q(e, o, 0x7362u));
+      } else {
+        const int c8 = (k & 31) >> 3;                  // which eight columns of the 32-column quarter
+        uint8_t* dst = out + (k & ~31) + 16 * (c8 >> 1) + 4 * (c8 & 1);
+        *reinterpret_cast<uint32_t*>(dst) = e;
+        *reinterpret_cast<uint32_t*>(dst + 8) = o;
+      }
     }
   }
 }
@@ -426,12 +443,11 @@ cudaError_t launch_small_ctas(const cudaLaunchConfig_t& cfg, long long chunks, c
 // out_form: kOutNibbles (act_idx = [M][K_pad / 2]) or signed bytes for the tensor-core kernel (act_idx = [M][K_pad],
 // kOutBytes in column order, kOutBytes2 in the 2-bit decoder's order).
 lcd_status launch_quantize_form(const lcd_act_problem* probs, int count, int out_form, void* stream) {
-  QuantBatch batch;
-  batch.count = count;
-  long long grid = 0;
+  QuantProblem all[LCD_MAX_BATCH];
+  long long tokens = 0;
   for (int i = 0; i < count; ++i) {
     const lcd_act_problem& a = probs[i];
-    QuantProblem& q = batch.p[i];
+    QuantProblem& q = all[i];
     q.x = static_cast<const __half*>(a.x_fp16);
     q.inv_smooth = a.inv_smooth;
     q.static_scale = a.static_scale;
@@ -440,39 +456,63 @@ lcd_status launch_quantize_form(const lcd_act_problem* probs, int count, int out
     q.K = a.K;
     q.K_pad = (long long)round_up_u64((uint64_t)a.K, kTileK);
     q.ldx = a.ldx;
-    q.cta0 = (int)grid;
+    q.cta0 = (int)a.M;          // (the token count until the launches are formed below)
     q.vec = (reinterpret_cast<uintptr_t>(a.x_fp16) % 16 == 0) && (a.ldx % 8 == 0) && (a.K % 8 == 0) &&
             (a.inv_smooth == nullptr || reinterpret_cast<uintptr_t>(a.inv_smooth) % 16 == 0) &&
             (reinterpret_cast<uintptr_t>(a.act_idx) % (out_form == kOutNibbles ? 4 : 8) == 0);
-    grid += a.M;
-    if (grid > 0x7fffffffLL) return LCD_ERR_INVALID_ARG;
+    tokens += a.M;
+    if (tokens > 0x7fffffffLL) return LCD_ERR_INVALID_ARG;
   }
-  for (int i = count; i < LCD_MAX_BATCH; ++i) batch.p[i] = batch.p[0];
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)grid);
-  const bool many = grid > 296 || out_form != kOutNibbles;      // the byte forms exist for the small CTAs only
-  cfg.blockDim = dim3(many ? kQThreadsMany : kQThreads);
-  cfg.stream = static_cast<cudaStream_t>(stream);
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  // register-resident instance that covers the longest vectorisable row (0: none does)
-  long long chunks = 0;
+  const bool many = tokens > 296 || out_form != kOutNibbles;      // the byte forms exist for the small CTAs only
   const int threads = many ? kQThreadsMany : kQThreads;
-  for (int i = 0; i < count; ++i)
-    if (batch.p[i].vec) chunks = std::max(chunks, (batch.p[i].K_pad + 8 * threads - 1) / (8 * threads));
-  cudaError_t e;
-  if (!many)
-    e = chunks >= 1 && chunks <= kQChunks ? cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreads, kQChunks>, batch)
-                                          : cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreads, 0>, batch);
-  else if (out_form == kOutBytes) e = launch_small_ctas<kOutBytes>(cfg, chunks, batch);
-  else if (out_form == kOutBytes2) e = launch_small_ctas<kOutBytes2>(cfg, chunks, batch);
-  else e = launch_small_ctas<kOutNibbles>(cfg, chunks, batch);
-  if (e != cudaSuccess) {
-    set_cuda_error((int)e);
-    return LCD_ERR_CUDA;
+  // register-resident instance a problem's rows fit (0: none, the two-pass instance)
+  auto instance_of = [&](const QuantProblem& q) -> int {
+    if (!q.vec) return 0;
+    const long long chunks = (q.K_pad + 8 * threads - 1) / (8 * threads);
+    if (!many) return chunks <= kQChunks ? kQChunks : 0;
+    return chunks <= 2 ? 2 : chunks <= 3 ? 3 : chunks <= 4 ? 4 : chunks <= 6 ? 6 : chunks <= 8 ? 8 : 0;
+  };
+  // Few tokens: one launch, the instance of the longest row.  Many tokens: one launch per instance that occurs, so
+  // that short rows are not run through the loops and registers of the longest one.
+  bool done[LCD_MAX_BATCH] = {};
+  for (int first = 0; first < count; ++first) {
+    if (done[first]) continue;
+    int inst = instance_of(all[first]);
+    QuantBatch batch;
+    batch.count = 0;
+    long long grid = 0;
+    for (int i = first; i < count; ++i) {
+      if (done[i]) continue;
+      const int mine = instance_of(all[i]);
+      if (many && mine != inst) continue;
+      if (!many && mine != 0) inst = mine;       // one launch: the kernel itself sends a row that does not fit the two-pass way
+      QuantProblem& q = batch.p[batch.count++];
+      q = all[i];
+      q.cta0 = (int)grid;
+      grid += all[i].cta0;
+      done[i] = true;
+    }
+    for (int i = batch.count; i < LCD_MAX_BATCH; ++i) batch.p[i] = batch.p[0];
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(threads);
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e;
+    if (!many)
+      e = inst ? cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreads, kQChunks>, batch)
+               : cudaLaunchKernelEx(&cfg, smooth_quantize_kernel<kQThreads, 0>, batch);
+    else if (out_form == kOutBytes) e = launch_small_ctas<kOutBytes>(cfg, inst, batch);
+    else if (out_form == kOutBytes2) e = launch_small_ctas<kOutBytes2>(cfg, inst, batch);
+    else e = launch_small_ctas<kOutNibbles>(cfg, inst, batch);
+    if (e != cudaSuccess) {
+      set_cuda_error((int)e);
+      return LCD_ERR_CUDA;
+    }
   }
   return LCD_OK;
 }
