@@ -306,13 +306,13 @@ lcd_status lcd_reclassify(const uint8_t* idx, const uint16_t* codebook_fp16, con
  *   algo:       LCD_ALGO_AUTO, REGISTER_LUT or BUCKET_LUT;
  *   workspace:  as lcd_lut_linear_batch (same size: lcd_linear_fused_batch_workspace_bytes; zero-filled
  *               before first use, left zero-filled).
- * Many tokens (prefill): when EVERY problem has more than 32 tokens, algo is
+ * Many tokens (prefill): when EVERY problem has more than 16 tokens, algo is
  * LCD_ALGO_AUTO or LCD_ALGO_DENSE_TC and the call is: one launch that transforms the inputs of all problems (same
  * operation sequence, same levels) and writes them as the signed bytes the int8 tensor-core kernel reads, in its
  * order, into the workspace (per problem M * K_pad bytes and M scales; no zero-fill contract, the contents are
  * scratch), then that kernel once per problem: no packed 4-bit copy and no expansion pass in between.  y equals
- * the two-call result bit for bit.  A mix of problems with at most 16 and more than 16 tokens, and problems with
- * 17 to 32 tokens, give LCD_ERR_UNSUPPORTED (use the two calls).
+ * the two-call result of LCD_ALGO_DENSE_TC bit for bit.  A mix of problems with at most 16 and more than 16 tokens
+ * gives LCD_ERR_UNSUPPORTED (use the two calls).
  * -------------------------------------------------------------------------------------------- */
 typedef struct {
   const void* packed_weights_dev; /* device, 256-byte aligned */

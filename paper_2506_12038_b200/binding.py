@@ -364,7 +364,7 @@ def resolve_batch_algo(weights_and_tokens, algo: int = ALGO_AUTO) -> int:
 class FusedBatch:
     """Up to MAX_BATCH independent problems from x to y in one call: items are (PackedWeights, x fp16 [M,K] CUDA,
     inv_smooth or None, y fp32 [M,N] CUDA).  Every M <= 16: ONE launch that quantises the activations and runs the
-    lookup.  Every M > 32: one launch that quantises all inputs, then the tensor-core kernel per problem."""
+    lookup.  Every M > 16: one launch that quantises all inputs, then the tensor-core kernel per problem."""
 
     def __init__(self, items, algo: int = ALGO_AUTO, status_word=None):
         import torch

@@ -343,13 +343,13 @@ static lcd_status fused_problems(const lcd_fused_problem* problems, int count, l
       algo != LCD_ALGO_SHARED_BUCKET && algo != LCD_ALGO_DENSE_TC)
     return LCD_ERR_UNSUPPORTED;
   // either every problem has at most 16 tokens (one lookup launch that transforms its inputs itself) or every
-  // problem has more than 32 (one transformation launch, then the tensor-core kernel per problem)
+  // problem has more than 16 (one transformation launch, then the tensor-core kernel per problem)
   bool many = false;
   for (int i = 0; i < count; ++i) many = many || (problems[i].M > 16);
   for (int i = 0; i < count; ++i) {
     const lcd_fused_problem& q = problems[i];
     if (q.M < 1 || !q.header_host) return LCD_ERR_INVALID_ARG;
-    if (many ? (q.M <= 32 || (algo != LCD_ALGO_AUTO && algo != LCD_ALGO_DENSE_TC)) : algo == LCD_ALGO_DENSE_TC)
+    if (many ? (q.M <= 16 || (algo != LCD_ALGO_AUTO && algo != LCD_ALGO_DENSE_TC)) : algo == LCD_ALGO_DENSE_TC)
       return LCD_ERR_UNSUPPORTED;
     if (!shape_problem(q.header_host, q.M, &p[i])) return LCD_ERR_BAD_BLOB;
     if (many && p[i].K_pad >= (1 << 21)) return LCD_ERR_UNSUPPORTED;      // the int32 sums of the planes could overflow
