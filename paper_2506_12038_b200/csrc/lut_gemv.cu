@@ -340,12 +340,6 @@ __device__ __forceinline__ void cursor_set(Cursor& c, uint32_t x, const GemvProb
   c.rp = r / c.pw;
   c.kk = r - c.rp * c.pw;
 }
-__device__ __forceinline__ uint32_t stage_len(const Cursor& c, uint32_t x_end) {
-  uint32_t n = x_end - c.x;
-  n = n < (uint32_t)kStageItems ? n : (uint32_t)kStageItems;
-  const uint32_t row_left = c.pw - c.kk;
-  return n < row_left ? n : row_left;
-}
 __device__ __forceinline__ void cursor_advance(Cursor& c, uint32_t n, const GemvProblem& P) {
   c.x += n;
   c.kk += n;
@@ -557,7 +551,7 @@ lut_gemv_kernel(const __grid_constant__ GemvBatch batch, int32_t* __restrict__ s
   const uint8_t* f_src = P.items;
   const uint32_t ring_u32 = smem_u32(ring);
   bool aborted = false;
-  Cursor fc, cc;
+  Cursor fc = {0, 0, 0, 0, 1}, cc = fc;      // set for real before the first fetch (cursor_set below)
 
   uint64_t stream_policy;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_policy));
